@@ -1,0 +1,170 @@
+"""Pins for the integer side of the oracle: the chunk-granular state machine (Sect. 3.4-3.6),
+against closed forms from the span analysis (Sect. 3.8), conservation laws, and a second,
+independent set-based simulator written here."""
+import numpy as np
+import pytest
+
+import oracle
+import taurus_gen as tg
+from helpers import random_multigraph
+
+
+def second_simulator(V, row_ptr, col, prop, m, is_hub, chunk, pool):
+    """Independent restatement with Python sets; victims by a full sort of (pending, id)."""
+    pend = {v: int(m[v]) + 1 for v in range(V)}
+    in_pool, evicted, done, started_hubs = set(), set(), set(), set()
+    ev = rl = 0
+    reload_count = {v: 0 for v in range(V)}
+    complete_chunk = {}
+    per_chunk = []
+    peak = 0
+    for c, s in enumerate(range(0, V, chunk)):
+        e = min(s + chunk, V)
+        msgs = [int(col[k]) for u in range(s, e) for k in range(row_ptr[u], row_ptr[u + 1]) if prop is None or prop[k]]
+        touched = set(msgs) | set(range(s, e))
+        T = {v for v in touched if not is_hub[v]}
+        hs = len(T & in_pool)
+        evs = T & evicted
+        ns = T - in_pool - evicted
+        need = len(evs) + len(ns)
+        if need > pool:
+            return None
+        deficit = need - (pool - len(in_pool))
+        n_ev = 0
+        if deficit > 0:
+            order = sorted((pend[v], v) for v in in_pool - T)
+            if len(order) < deficit:
+                return None
+            for _, v in order[:deficit]:
+                in_pool.remove(v); evicted.add(v); ev += 1; n_ev += 1
+        for v in evs:
+            evicted.remove(v); in_pool.add(v); rl += 1; reload_count[v] += 1
+        in_pool |= ns
+        started_hubs |= {v for v in touched if is_hub[v]}
+        peak = max(peak, len(in_pool))
+        for v in msgs:
+            pend[v] -= 1
+        for v in range(s, e):
+            pend[v] -= 1
+        fin = {v for v in touched if pend[v] == 0}
+        for v in fin:
+            complete_chunk[v] = c
+            in_pool.discard(v)
+        done |= fin
+        per_chunk.append(dict(hs=hs, ns=len(ns), ev=len(evs), gs=len(touched) - len(T), need=need, evicted=n_ev,
+                              reloaded=len(evs), completed=len(fin), occupancy=len(in_pool)))
+    return dict(evictions=ev, reloads=rl, peak=peak, complete_chunk=complete_chunk, reload_count=reload_count,
+                per_chunk=per_chunk, completed=len(done), left=len(in_pool) + len(evicted))
+
+
+def _setup(V, E, seed, fanout=0, hub_count=0):
+    row_ptr, col = random_multigraph(V, E, seed)
+    inl = oracle.build_in_lists(V, row_ptr, col)
+    ms = oracle.message_sets(inl, fanout, seed, 0)
+    hub = oracle.hub_set(np.diff(inl.ptr).astype(np.int32), hub_count)
+    return row_ptr, col, inl, ms, hub
+
+
+@pytest.mark.parametrize("pool", [2, 3, 5, 8, 30])
+@pytest.mark.parametrize("fanout,hub_count", [(0, 0), (0, 3), (2, 2)])
+def test_matches_the_second_simulator_on_tiny_graphs(pool, fanout, hub_count):
+    V, E, chunk = 40, 70, 1
+    agree = 0
+    for seed in range(10):
+        row_ptr, col, inl, ms, hub = _setup(V, E, seed, fanout, hub_count)
+        a = oracle.simulate(V, row_ptr, col, ms, hub, chunk, pool)
+        b = second_simulator(V, row_ptr, col, ms.prop, ms.m, hub, chunk, pool)
+        if b is None:
+            assert a.rc in (-2, -3)
+            continue
+        agree += 1
+        assert a.rc == 0
+        assert a.stats["evictions"] == b["evictions"] and a.stats["reloads"] == b["reloads"]
+        assert a.stats["peak_occupancy"] == b["peak"] and a.stats["completed"] == b["completed"] == V
+        assert b["left"] == 0
+        assert all(a.complete_chunk[v] == b["complete_chunk"][v] for v in range(V))
+        assert all(a.reload_count[v] == b["reload_count"][v] for v in range(V))
+        for c, rec in enumerate(b["per_chunk"]):
+            for k, val in rec.items():
+                assert a.per_chunk[k][c] == val, (k, c)
+    assert agree >= 2 or pool < 5
+
+
+@pytest.mark.parametrize("chunk", [1, 7, 64])
+@pytest.mark.parametrize("fanout", [0, 3])
+def test_completion_chunk_closed_form(chunk, fanout):
+    """c(v) = max rank of the in-neighbours (Sect. 3.8), with the self message: chunk of max(v, max M(v))."""
+    V, E = 500, 4000
+    row_ptr, col, inl, ms, hub = _setup(V, E, 3, fanout, 5)
+    sim = oracle.simulate(V, row_ptr, col, ms, hub, chunk, V)
+    cf = oracle.complete_chunk_closed_form(ms, chunk)
+    # the closed form written out with loops, independent of the vectorised helper
+    for v in range(0, V, 37):
+        last = max([v] + ms.src[ms.ptr[v]:ms.ptr[v + 1]].tolist())
+        assert cf[v] == last // chunk
+    assert (sim.complete_chunk == cf).all()
+    assert sim.stats["completed"] == V and sim.per_chunk["completed"].sum() == V
+    assert (np.bincount(cf, minlength=sim.per_chunk["completed"].size) == sim.per_chunk["completed"]).all()
+
+
+@pytest.mark.parametrize("hub_count", [0, 10])
+def test_active_set_identity_with_unbounded_pool(hub_count):
+    """A(t) = #{v : a(v) <= t < c(v)} and sum_t A(t) = sum_v L(v) (Sect. 3.8), in chunk units, non-hub vertices."""
+    V, E, chunk = 800, 6000, 16
+    row_ptr, col, inl, ms, hub = _setup(V, E, 4, 0, hub_count)
+    sim = oracle.simulate(V, row_ptr, col, ms, hub, chunk, V)
+    a = oracle.first_touch_chunk(ms, chunk).astype(np.int64)
+    c = oracle.complete_chunk_closed_form(ms, chunk).astype(np.int64)
+    nh = hub == 0
+    for t in range(sim.per_chunk["occupancy"].size):
+        assert sim.per_chunk["occupancy"][t] == int(((a <= t) & (t < c) & nh).sum())
+    assert sim.per_chunk["occupancy"].sum() == int((c - a)[nh].sum())
+    assert sim.stats["evictions"] == 0 and sim.stats["reloads"] == 0
+
+
+def test_pool_at_peak_needs_no_eviction_and_one_less_does():
+    V, E, chunk = 600, 5000, 8
+    row_ptr, col, inl, ms, hub = _setup(V, E, 5)
+    free_run = oracle.simulate(V, row_ptr, col, ms, hub, chunk, V)
+    peak = free_run.stats["peak_occupancy"]
+    at_peak = oracle.simulate(V, row_ptr, col, ms, hub, chunk, peak)
+    assert at_peak.rc == 0 and at_peak.stats["evictions"] == 0
+    below = oracle.simulate(V, row_ptr, col, ms, hub, chunk, peak - 1)
+    assert below.rc == 0 and below.stats["evictions"] >= 1
+
+
+@pytest.mark.parametrize("pool_frac", [0.9, 0.6, 0.4])
+def test_conservation_laws_under_eviction(pool_frac):
+    w = tg.scaled(tg.WORKLOADS["large"], 20_000, chunk=256)
+    g = tg.make_graph(w)
+    inl = oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
+    ms = oracle.message_sets(inl, 0, 1, 0)
+    hub = oracle.hub_set(g.in_degree, w.hub_count)
+    peak = oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, g.V).stats["peak_occupancy"]
+    pool = int(peak * pool_frac)
+    sim = oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, pool)
+    assert sim.rc == 0
+    st = sim.stats
+    assert st["evictions"] == st["reloads"] > 0          # every victim has pending >= 1, so it must come back
+    assert st["free_end"] == pool and st["completed"] == g.V and st["bad_transitions"] == 0
+    assert st["peak_occupancy"] <= pool
+    assert st["total_messages"] == g.E and st["hub_vertices"] == w.hub_count
+    assert st["hub_messages"] == int(g.in_degree[hub == 1].sum())
+    assert sim.reload_count.sum() == st["reloads"] and sim.reload_count.max() == st["max_reload_count"]
+    assert (sim.reload_count[hub == 1] == 0).all()       # pinned: never evicted
+    assert (sim.per_chunk["occupancy"] <= pool).all()
+    # the completion chunk does not depend on the pool size
+    assert (sim.complete_chunk == oracle.complete_chunk_closed_form(ms, w.chunk)).all()
+
+
+def test_pool_too_small_is_reported():
+    V, E = 100, 2000
+    row_ptr, col, inl, ms, hub = _setup(V, E, 6)
+    assert oracle.simulate(V, row_ptr, col, ms, hub, 50, 10).rc == -2
+
+
+def test_hub_set_takes_largest_in_degree_ties_by_smaller_id():
+    din = np.array([5, 9, 9, 1, 9, 0], np.int32)
+    assert oracle.hub_set(din, 2).tolist() == [0, 1, 1, 0, 0, 0]
+    assert oracle.hub_set(din, 4).tolist() == [1, 1, 1, 0, 1, 0]
+    assert oracle.hub_set(din, 0).sum() == 0
