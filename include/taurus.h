@@ -1,0 +1,220 @@
+/*
+ * libtaurus: source-centric, layer-wise broadcast step of out-of-core GNN
+ * inference on one NVIDIA B200 (sm_100a).  C ABI, no C++ or framework types.
+ *
+ * One layer pass streams the vertices once in id order (Sect. 3.1): the caller
+ * pushes chunks of contiguous source vertices with their feature rows
+ * (Sect. 3.3, "chunk"); the library projects the rows through the layer's
+ * weights, pushes each projected row along the chunk's CSR out-edges
+ * (Sect. 3.2) into per-destination accumulators, counts down each
+ * destination's pending messages (Sect. 3.4), and finalises destinations whose
+ * count reached zero into a graduation buffer (Sect. 3.6) that the caller
+ * drains.  Accumulators of the highest in-degree vertices are pinned in a
+ * GPU-resident hub store (Sect. 3.5.1); all others live in a bounded slot pool
+ * (Sect. 3.5.2) whose fewest-pending rows are evicted to pinned host memory
+ * when the pool is full (Sect. 3.5.3-3.5.4) and reloaded before they receive
+ * further messages.  Per-layer fanout sampling suppresses all but `fanout`
+ * hashed in-edges per destination (Sect. 3.9, sampling paragraph).
+ *
+ * Layer formula (Eq. 1-2 with the SAGEConv split of Sect. 3.9):
+ *   out_v = act( c_in(v) * sum_{u in M(v)} c_out(u) * (h_u W_neigh)
+ *                + c_self(v) * (h_v W_self) + b )
+ *   SAGE-mean: c_out = 1, c_in = 1 / max(|M(v)|, 1), c_self = 1
+ *   GCN-sym  : c_out(u) = (dout(u)+1)^-1/2, c_in(v) = (din(v)+1)^-1/2,
+ *              c_self = c_out * c_in, W_self = W_neigh
+ * M(v) is the multiset of propagated in-edges of v (all of them, or the
+ * sampled ones); every CSR entry is one message, duplicates and self-loops
+ * included.
+ *
+ * General rules.  Every function returns TAURUS_OK (0) or a negative
+ * TAURUS_ERR_* code; nothing throws, aborts or traps.  Unless stated
+ * otherwise a pointer argument may point to host or device memory (the
+ * library asks the CUDA runtime which).  The caller owns every buffer it
+ * passes and may free it as soon as the call that took it has returned, with
+ * the exceptions stated at taurus_push_chunk.  The library owns all state
+ * behind taurus_ctx.  A context is bound to the device current at
+ * taurus_graph_init and is not thread-safe.  Errors found on the device
+ * (pool too small, host store full, index out of bounds in a checked build)
+ * are sticky: the chunk that hit one is not applied and every later call
+ * on the context returns the code.
+ */
+#ifndef TAURUS_H
+#define TAURUS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  TAURUS_OK = 0,
+  TAURUS_ERR_INVALID_ARG = -1,     /* null / misaligned pointer, size out of range, inconsistent graph        */
+  TAURUS_ERR_ORDER = -2,           /* chunk not contiguous / ascending, or no layer begun, or layer not drained */
+  TAURUS_ERR_POOL_TOO_SMALL = -3,  /* one chunk needs more slots than pool_slots, or too few eligible victims  */
+  TAURUS_ERR_HOST_STORE_FULL = -4, /* more rows evicted at once than host_evict_rows                            */
+  TAURUS_ERR_DRAIN_FULL = -5,      /* the chunk could overflow the graduation buffer: drain, then push again    */
+  TAURUS_ERR_CUDA = -6,            /* a CUDA runtime call failed (see taurus_last_cuda_error)                   */
+  TAURUS_ERR_INTERNAL = -7,        /* a device-side consistency check failed                                    */
+  TAURUS_ERR_NOMEM = -8,           /* host or device allocation failed                                          */
+  TAURUS_ERR_UNSUPPORTED = -9      /* shape or size outside what the kernels were built for                     */
+};
+
+enum { TAURUS_SAGE_MEAN = 0, TAURUS_GCN_SYM = 1 };
+enum { TAURUS_GEMM_FP32 = 0, TAURUS_GEMM_BF16 = 1 };
+/* vertex states of Sect. 3.4 */
+enum { TAURUS_NOT_STARTED = 0, TAURUS_IN_BUFFER = 1, TAURUS_EVICTED = 2, TAURUS_ON_GPU = 3, TAURUS_COMPLETED = 4 };
+
+typedef struct taurus_ctx taurus_ctx;
+
+/* CSR out-edge topology (Sect. 3.2).  Copied at init. */
+typedef struct {
+  int64_t V, E;              /* V < 2^31, E < 2^32                                             */
+  const int64_t* row_ptr;    /* [V+1] offsets, row_ptr[0] = 0, row_ptr[V] = E, non-decreasing  */
+  const int32_t* col_idx;    /* [E] destinations in [0, V); multi-edges and self-loops allowed */
+  const int32_t* in_degree;  /* [V] with multiplicity; must equal the histogram of col_idx     */
+} taurus_graph;
+
+/* Layer weights.  Copied at init.  dims[l] -> dims[l+1]; matrices are row-major dims[l] x dims[l+1] fp32. */
+typedef struct {
+  int32_t mode;                /* TAURUS_SAGE_MEAN or TAURUS_GCN_SYM                          */
+  int32_t L;                   /* number of layers, 1..16                                     */
+  const int32_t* dims;         /* [L+1], each in 1..1024 (host pointer)                       */
+  const float* const* W_neigh; /* [L] (host array of pointers)                                */
+  const float* const* W_self;  /* [L]; ignored for GCN (the self term uses W_neigh)           */
+  const float* const* bias;    /* [L] each dims[l+1]; an entry may be NULL for zero bias      */
+  const int32_t* act;          /* [L] 0 = identity, 1 = ReLU (host pointer)                   */
+  int32_t gemm_mode;           /* TAURUS_GEMM_FP32: fp32-accurate projection; TAURUS_GEMM_BF16: bf16 operands, fp32 accumulate */
+} taurus_model;
+
+typedef struct {
+  int64_t chunk_sources;    /* largest number of sources one push may carry (Sect. 3.3)                    */
+  int64_t pool_slots;       /* capacity of the accumulator slot pool (hot store, Sect. 3.5.2)              */
+  int64_t hub_count;        /* vertices pinned in the hub store: the largest by (in_degree desc, id asc)   */
+  const int32_t* fanout;    /* [L] per-layer fanout, 0 = exact; NULL = all exact; at most 64 (host pointer) */
+  uint64_t seed;            /* seed of the neighbour-sampling hash                                         */
+  int64_t host_evict_rows;  /* capacity (rows) of the pinned host store for evicted accumulators; 0 = none */
+  int64_t drain_rows;       /* capacity (rows) of the graduation buffer                                    */
+  int32_t flags;            /* TAURUS_FLAG_*                                                               */
+} taurus_run;
+
+enum {
+  TAURUS_FLAG_CHECKED = 1,      /* bounds-check every slot / vertex index on the device (slower; sets ERR_INTERNAL) */
+  TAURUS_FLAG_SIMT_GEMM = 2     /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */
+};
+
+/* Integer accounting of one layer pass (Sect. 4.4-4.7 report these quantities). */
+typedef struct {
+  int64_t evictions;           /* IN_BUFFER -> EVICTED transitions                               */
+  int64_t reloads;             /* EVICTED -> IN_BUFFER transitions                               */
+  int64_t max_reload_count;    /* most reloads of one vertex                                     */
+  int64_t reload_histogram[17];/* vertices by reload count 0..15, last bin = 16 or more          */
+  int64_t peak_occupancy;      /* most pool slots in use at once                                 */
+  int64_t hub_messages;        /* propagated messages delivered to hub-store vertices            */
+  int64_t total_messages;      /* propagated messages, self messages not counted                 */
+  int64_t hub_vertices;
+  int64_t completed;           /* vertices finalised                                             */
+  int64_t sum_hs, sum_ns, sum_ev, sum_gs; /* per-chunk touched vertices by state at the start of the chunk, summed over chunks:
+                                  IN_BUFFER, NOT_STARTED, EVICTED (non-hub) and hub vertices    */
+  int64_t free_slots;          /* free pool slots now                                            */
+  int64_t chunks;              /* chunks pushed                                                  */
+} taurus_stats;
+
+/* Columns of one per-chunk record returned by taurus_get_chunk_log. */
+enum {
+  TAURUS_CK_HS = 0, TAURUS_CK_NS, TAURUS_CK_EV, TAURUS_CK_GS, TAURUS_CK_NEED, TAURUS_CK_EVICTED,
+  TAURUS_CK_RELOADED, TAURUS_CK_COMPLETED, TAURUS_CK_OCCUPANCY, TAURUS_CK_COLUMNS
+};
+
+/*
+ * Creates a context on the current device: copies topology, degrees and weights, selects the hub set,
+ * allocates the slot pool, the hub store, the pinned host store and the graduation buffer.  When any
+ * fanout is non-zero it also builds the in-edge order (ascending source id, equal sources in CSR order)
+ * that the sampler indexes (Sect. 3.9).  Blocking.  On failure *out is NULL.
+ */
+int taurus_graph_init(taurus_ctx** out, const taurus_graph* graph, const taurus_model* model, const taurus_run* run);
+
+/*
+ * Starts layer `layer` (0-based): every vertex NOT_STARTED, pending count |M(v)| + 1 (the +1 is the
+ * vertex's own self message, delivered with its chunk), pool empty; builds the layer's edge mask when
+ * fanout[layer] > 0 (Sect. 3.9).  Blocking (synchronises `cuda_stream`).  A layer may be begun again.
+ */
+int taurus_layer_begin(taurus_ctx* ctx, int32_t layer, void* cuda_stream);
+
+/*
+ * Pushes sources [src_begin, src_end): Sect. 3.1 broadcast of one chunk.  `features` is
+ * [src_end - src_begin] x dims[layer] fp32 row-major, rows contiguous, in device memory or in host
+ * memory (pinned host memory makes the copy asynchronous).  Chunks must arrive in ascending, contiguous
+ * order starting at 0, at most chunk_sources per push.  All work is enqueued on `cuda_stream`
+ * (a cudaStream_t, NULL = default stream) and the call returns without waiting; `features` must stay
+ * valid and unchanged until that work has run (synchronise the stream, or drain).  Returns
+ * TAURUS_ERR_DRAIN_FULL, before changing any state, when the vertices this chunk completes might not
+ * fit the graduation buffer: drain and push the same chunk again.
+ */
+int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream);
+
+/*
+ * Copies out the vertices finalised since the last drain (Sect. 3.6): out_ids[i] and the dims[layer+1]
+ * floats out_rows[i * dims[layer+1] ...], in no particular order, and empties the graduation buffer.
+ * Blocking (synchronises the stream of the last push).  Fails with TAURUS_ERR_INVALID_ARG and drains
+ * nothing when more than capacity_rows rows are waiting (*out_count then holds that number).
+ */
+int taurus_drain_completed(taurus_ctx* ctx, int64_t* out_ids, float* out_rows, int64_t capacity_rows, int64_t* out_count);
+
+/*
+ * Same as taurus_drain_completed, but row i is written to dense_rows[out_id * ld ...] (ld in floats,
+ * ld >= dims[layer+1]): the vertex-ordered matrix the next layer streams (Sect. 3.7 keeps outputs
+ * sorted by vertex id for this reason).  dense_rows may be device memory or pinned host memory.
+ * out_ids may be NULL.
+ */
+int taurus_drain_dense(taurus_ctx* ctx, float* dense_rows, int64_t ld, int64_t* out_ids, int64_t capacity_rows,
+                       int64_t* out_count);
+
+/* Ends the layer: blocking; checks that every vertex completed and every slot is free (else
+ * TAURUS_ERR_ORDER), and fills *stats (may be NULL). */
+int taurus_layer_end(taurus_ctx* ctx, taurus_stats* stats);
+
+/* Accounting so far in the current layer (blocking). */
+int taurus_get_stats(taurus_ctx* ctx, taurus_stats* stats);
+
+/* Per-chunk records of the current layer: out[c * TAURUS_CK_COLUMNS + k], host memory, at most
+ * capacity_chunks records; *out_chunks = records written. */
+int taurus_get_chunk_log(taurus_ctx* ctx, int64_t* out, int64_t capacity_chunks, int64_t* out_chunks);
+
+/* Per-vertex arrays of the current layer copied to host memory (blocking): which = 0 state (uint8 [V]),
+ * 1 pending count (int32 [V]), 2 reload count (int32 [V]), 3 hub flag (uint8 [V]). */
+int taurus_get_vertex_array(taurus_ctx* ctx, int32_t which, void* out_host);
+
+/*
+ * Sampled in-edges of one destination in layer `layer` (Sect. 3.9): the CSR edge indices kept, ascending,
+ * and their sources; n = min(in_degree, fanout) (all in-edges when fanout is 0).  Host outputs.
+ */
+int taurus_get_sampled_edges(taurus_ctx* ctx, int32_t layer, int64_t dst, int64_t* out_edge_ids, int32_t* out_sources,
+                             int32_t capacity, int32_t* n);
+
+/* The propagated-edge mask of the current layer as one bit per CSR edge (bit e & 31 of word e >> 5),
+ * host output of ceil(E / 32) words; all ones in exact mode. */
+int taurus_get_edge_mask(taurus_ctx* ctx, uint32_t* out_words);
+
+/* Upper bound on the vertices that sources [src_begin, src_end) complete in the current layer
+ * (exact when both ends are multiples of 64 or the ends of the graph). */
+int taurus_completion_bound(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, int64_t* out_bound);
+
+/* Kernels launched by this context since init (for launch accounting in benchmarks). */
+int64_t taurus_launch_count(const taurus_ctx* ctx);
+
+/* Device time of the last push's phases in milliseconds, measured with CUDA events when
+ * taurus_set_timing(ctx, 1) is on: out[0] copy-in, out[1] projection, out[2] classify..reload,
+ * out[3] scatter, out[4] finalise.  Blocking. */
+int taurus_set_timing(taurus_ctx* ctx, int32_t on);
+int taurus_get_phase_ms(taurus_ctx* ctx, float* out5);
+
+void taurus_destroy(taurus_ctx* ctx);
+const char* taurus_strerror(int code);
+/* Text of the last CUDA runtime error seen by this library on this thread ("" if none). */
+const char* taurus_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TAURUS_H */

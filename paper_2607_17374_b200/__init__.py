@@ -1,0 +1,10 @@
+"""B200-native source-centric broadcast step for layer-wise GNN inference (libtaurus).
+
+The product is the CUDA library behind include/taurus.h; this package is its thin ctypes binding.
+There is no CPU fallback: importing the binding works anywhere, but every call needs the compiled
+library (python -m paper_2607_17374_b200.build) and a CUDA device.
+"""
+from .binding import (  # noqa: F401
+    Context, TaurusError, Stats, library_path, load_library,
+    SAGE_MEAN, GCN_SYM, GEMM_FP32, GEMM_BF16, FLAG_CHECKED, FLAG_SIMT_GEMM, CHUNK_LOG_COLUMNS, ERROR_CODES,
+)

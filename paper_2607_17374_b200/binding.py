@@ -1,0 +1,257 @@
+"""ctypes binding of libtaurus: argument marshalling only.  Method names follow the C entry points
+(taurus_graph_init -> Context(...), taurus_push_chunk -> Context.push_chunk, ...)."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+SAGE_MEAN, GCN_SYM = 0, 1
+GEMM_FP32, GEMM_BF16 = 0, 1
+FLAG_CHECKED, FLAG_SIMT_GEMM = 1, 2
+CHUNK_LOG_COLUMNS = ["hs", "ns", "ev", "gs", "need", "evicted", "reloaded", "completed", "occupancy"]
+ERROR_CODES = {
+    "OK": 0, "INVALID_ARG": -1, "ORDER": -2, "POOL_TOO_SMALL": -3, "HOST_STORE_FULL": -4, "DRAIN_FULL": -5,
+    "CUDA": -6, "INTERNAL": -7, "NOMEM": -8, "UNSUPPORTED": -9,
+}
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_lib = None
+
+
+def library_path() -> str:
+    return os.path.join(_PKG, "libtaurus.so")
+
+
+class TaurusError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        msg = "%s failed: %d" % (where, code)
+        if _lib is not None:
+            msg += " (%s)" % _lib.taurus_strerror(code).decode()
+        if detail:
+            msg += ": " + detail
+        super().__init__(msg)
+
+
+class _Graph(ctypes.Structure):
+    _fields_ = [("V", ctypes.c_int64), ("E", ctypes.c_int64), ("row_ptr", ctypes.c_void_p),
+                ("col_idx", ctypes.c_void_p), ("in_degree", ctypes.c_void_p)]
+
+
+class _Model(ctypes.Structure):
+    _fields_ = [("mode", ctypes.c_int32), ("L", ctypes.c_int32), ("dims", ctypes.POINTER(ctypes.c_int32)),
+                ("W_neigh", ctypes.POINTER(ctypes.c_void_p)), ("W_self", ctypes.POINTER(ctypes.c_void_p)),
+                ("bias", ctypes.POINTER(ctypes.c_void_p)), ("act", ctypes.POINTER(ctypes.c_int32)),
+                ("gemm_mode", ctypes.c_int32)]
+
+
+class _Run(ctypes.Structure):
+    _fields_ = [("chunk_sources", ctypes.c_int64), ("pool_slots", ctypes.c_int64), ("hub_count", ctypes.c_int64),
+                ("fanout", ctypes.POINTER(ctypes.c_int32)), ("seed", ctypes.c_uint64),
+                ("host_evict_rows", ctypes.c_int64), ("drain_rows", ctypes.c_int64), ("flags", ctypes.c_int32)]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("evictions", ctypes.c_int64), ("reloads", ctypes.c_int64), ("max_reload_count", ctypes.c_int64),
+                ("reload_histogram", ctypes.c_int64 * 17), ("peak_occupancy", ctypes.c_int64),
+                ("hub_messages", ctypes.c_int64), ("total_messages", ctypes.c_int64), ("hub_vertices", ctypes.c_int64),
+                ("completed", ctypes.c_int64), ("sum_hs", ctypes.c_int64), ("sum_ns", ctypes.c_int64),
+                ("sum_ev", ctypes.c_int64), ("sum_gs", ctypes.c_int64), ("free_slots", ctypes.c_int64),
+                ("chunks", ctypes.c_int64)]
+
+    def as_dict(self) -> dict:
+        d = {}
+        for name, _ in self._fields_:
+            v = getattr(self, name)
+            d[name] = list(v) if name == "reload_histogram" else int(v)
+        return d
+
+
+EXPORTS = [
+    "taurus_graph_init", "taurus_layer_begin", "taurus_push_chunk", "taurus_drain_completed", "taurus_drain_dense",
+    "taurus_layer_end", "taurus_get_stats", "taurus_get_chunk_log", "taurus_get_vertex_array",
+    "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count",
+    "taurus_set_timing", "taurus_get_phase_ms", "taurus_destroy", "taurus_strerror", "taurus_last_cuda_error",
+]
+
+
+def load_library():
+    """Loads libtaurus.so.  Fails loudly when it has not been built: there is no fallback path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise RuntimeError("libtaurus.so is missing at %s: build it with `python -m paper_2607_17374_b200.build` "
+                           "(needs nvcc); this package has no CPU fallback" % path)
+    lib = ctypes.CDLL(path)
+    vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+    lib.taurus_graph_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_Graph), ctypes.POINTER(_Model), ctypes.POINTER(_Run)]
+    lib.taurus_layer_begin.argtypes = [vp, i32, vp]
+    lib.taurus_push_chunk.argtypes = [vp, i64, i64, vp, vp]
+    lib.taurus_drain_completed.argtypes = [vp, vp, vp, i64, ctypes.POINTER(i64)]
+    lib.taurus_drain_dense.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(i64)]
+    lib.taurus_layer_end.argtypes = [vp, ctypes.POINTER(Stats)]
+    lib.taurus_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
+    lib.taurus_get_chunk_log.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
+    lib.taurus_get_vertex_array.argtypes = [vp, i32, vp]
+    lib.taurus_get_sampled_edges.argtypes = [vp, i32, i64, vp, vp, i32, ctypes.POINTER(i32)]
+    lib.taurus_get_edge_mask.argtypes = [vp, vp]
+    lib.taurus_completion_bound.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
+    lib.taurus_launch_count.argtypes = [vp]
+    lib.taurus_launch_count.restype = i64
+    lib.taurus_set_timing.argtypes = [vp, i32]
+    lib.taurus_get_phase_ms.argtypes = [vp, vp]
+    lib.taurus_destroy.argtypes = [vp]
+    lib.taurus_destroy.restype = None
+    lib.taurus_strerror.argtypes = [ctypes.c_int]
+    lib.taurus_strerror.restype = ctypes.c_char_p
+    lib.taurus_last_cuda_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _ptr(x) -> Optional[int]:
+    """Address of a torch tensor, a numpy array, or a raw integer address."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        if not x.flags.c_contiguous:
+            raise ValueError("array must be C-contiguous")
+        return x.ctypes.data
+    if hasattr(x, "data_ptr"):
+        if not x.is_contiguous():
+            raise ValueError("tensor must be contiguous")
+        return x.data_ptr()
+    raise TypeError("expected a torch tensor, a numpy array or an address, got %r" % type(x))
+
+
+def _stream(s) -> Optional[int]:
+    if s is None:
+        return None
+    return s if isinstance(s, int) else s.cuda_stream
+
+
+class Context:
+    """One taurus_ctx.  Every method is one C call; see include/taurus.h for the semantics."""
+
+    def __init__(self, V: int, E: int, row_ptr, col_idx, in_degree, mode: int, dims: Sequence[int], W_neigh, W_self,
+                 bias, act: Sequence[int], chunk_sources: int, pool_slots: int, hub_count: int = 0,
+                 fanout: Optional[Sequence[int]] = None, seed: int = 1, host_evict_rows: int = 0, drain_rows: int = 0,
+                 gemm_mode: int = GEMM_FP32, flags: int = 0):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        L = len(dims) - 1
+        self.V, self.E, self.L, self.dims = V, E, L, tuple(int(d) for d in dims)
+        keep = [row_ptr, col_idx, in_degree, W_neigh, W_self, bias]
+        g = _Graph(V, E, _ptr(row_ptr), _ptr(col_idx), _ptr(in_degree))
+        c_dims = (ctypes.c_int32 * (L + 1))(*self.dims)
+        c_act = (ctypes.c_int32 * L)(*[int(a) for a in act])
+        c_wn = (ctypes.c_void_p * L)(*[_ptr(w) for w in W_neigh])
+        c_ws = (ctypes.c_void_p * L)(*[_ptr(w) for w in W_self]) if W_self is not None else None
+        c_b = (ctypes.c_void_p * L)(*[_ptr(b) for b in bias]) if bias is not None else None
+        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode)
+        c_f = (ctypes.c_int32 * L)(*[int(f) for f in fanout]) if fanout is not None else None
+        r = _Run(chunk_sources, pool_slots, hub_count, c_f, seed, host_evict_rows, drain_rows or chunk_sources, flags)
+        rc = self._lib.taurus_graph_init(ctypes.byref(self._h), ctypes.byref(g), ctypes.byref(m), ctypes.byref(r))
+        del keep
+        if rc != 0:
+            self._h = ctypes.c_void_p()
+            raise TaurusError(rc, "taurus_graph_init", self._lib.taurus_last_cuda_error().decode())
+        self.layer = -1
+
+    def _check(self, rc: int, where: str):
+        if rc != 0:
+            raise TaurusError(rc, where, self._lib.taurus_last_cuda_error().decode() if rc == ERROR_CODES["CUDA"] else "")
+
+    def layer_begin(self, layer: int, stream=None):
+        self._check(self._lib.taurus_layer_begin(self._h, layer, _stream(stream)), "taurus_layer_begin")
+        self.layer = layer
+
+    def push_chunk(self, src_begin: int, src_end: int, features, stream=None, raise_on_drain_full: bool = True) -> int:
+        rc = self._lib.taurus_push_chunk(self._h, src_begin, src_end, _ptr(features), _stream(stream))
+        if rc == ERROR_CODES["DRAIN_FULL"] and not raise_on_drain_full:
+            return rc
+        self._check(rc, "taurus_push_chunk")
+        return rc
+
+    def drain_completed(self, out_ids, out_rows, capacity_rows: int) -> int:
+        n = ctypes.c_int64(0)
+        self._check(self._lib.taurus_drain_completed(self._h, _ptr(out_ids), _ptr(out_rows), capacity_rows, ctypes.byref(n)),
+                    "taurus_drain_completed")
+        return int(n.value)
+
+    def drain_dense(self, dense_rows, ld: int, capacity_rows: int, out_ids=None) -> int:
+        n = ctypes.c_int64(0)
+        self._check(self._lib.taurus_drain_dense(self._h, _ptr(dense_rows), ld, _ptr(out_ids), capacity_rows, ctypes.byref(n)),
+                    "taurus_drain_dense")
+        return int(n.value)
+
+    def layer_end(self) -> dict:
+        s = Stats()
+        self._check(self._lib.taurus_layer_end(self._h, ctypes.byref(s)), "taurus_layer_end")
+        return s.as_dict()
+
+    def get_stats(self) -> dict:
+        s = Stats()
+        self._check(self._lib.taurus_get_stats(self._h, ctypes.byref(s)), "taurus_get_stats")
+        return s.as_dict()
+
+    def get_chunk_log(self, capacity_chunks: int = 1 << 20) -> dict:
+        out = np.zeros((capacity_chunks, len(CHUNK_LOG_COLUMNS)), np.int64)
+        n = ctypes.c_int64(0)
+        self._check(self._lib.taurus_get_chunk_log(self._h, out.ctypes.data, capacity_chunks, ctypes.byref(n)),
+                    "taurus_get_chunk_log")
+        return {k: out[:n.value, i].copy() for i, k in enumerate(CHUNK_LOG_COLUMNS)}
+
+    def get_vertex_array(self, which: str) -> np.ndarray:
+        idx = {"state": 0, "pending": 1, "reload_count": 2, "hub": 3}[which]
+        out = np.empty(self.V, np.uint8 if idx in (0, 3) else np.int32)
+        self._check(self._lib.taurus_get_vertex_array(self._h, idx, out.ctypes.data), "taurus_get_vertex_array")
+        return out
+
+    def get_sampled_edges(self, layer: int, dst: int, capacity: int = 1 << 16):
+        eids = np.empty(capacity, np.int64)
+        srcs = np.empty(capacity, np.int32)
+        n = ctypes.c_int32(0)
+        self._check(self._lib.taurus_get_sampled_edges(self._h, layer, dst, eids.ctypes.data, srcs.ctypes.data, capacity,
+                                                       ctypes.byref(n)), "taurus_get_sampled_edges")
+        k = min(n.value, capacity)
+        return eids[:k].copy(), srcs[:k].copy(), int(n.value)
+
+    def get_edge_mask(self) -> np.ndarray:
+        words = np.empty((self.E + 31) // 32, np.uint32)
+        self._check(self._lib.taurus_get_edge_mask(self._h, words.ctypes.data), "taurus_get_edge_mask")
+        return words
+
+    def completion_bound(self, src_begin: int, src_end: int) -> int:
+        n = ctypes.c_int64(0)
+        self._check(self._lib.taurus_completion_bound(self._h, src_begin, src_end, ctypes.byref(n)), "taurus_completion_bound")
+        return int(n.value)
+
+    def launch_count(self) -> int:
+        return int(self._lib.taurus_launch_count(self._h))
+
+    def set_timing(self, on: bool):
+        self._check(self._lib.taurus_set_timing(self._h, 1 if on else 0), "taurus_set_timing")
+
+    def get_phase_ms(self):
+        out = (ctypes.c_float * 5)()
+        self._check(self._lib.taurus_get_phase_ms(self._h, out), "taurus_get_phase_ms")
+        return [float(x) for x in out]
+
+    def destroy(self):
+        if self._h:
+            self._lib.taurus_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -1,0 +1,517 @@
+// Per-vertex state machine on the device (Sect. 3.4-3.6): classify the destinations a chunk touches,
+// make room in the slot pool (fewest-pending eviction, Sect. 3.5.3), allocate / reload slots,
+// finalise completed vertices into the graduation buffer.  All decisions are taken from integer state
+// at chunk granularity, so the accounting is deterministic although the scatter is not ordered.
+//
+// Every kernel reads the counts it depends on from the device control block and is launched with a
+// fixed grid, so a push never waits for the host.  A kernel that finds ctl->error set returns at once.
+#include "taurus_internal.h"
+
+#define FULL 0xffffffffu
+
+static __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
+
+static __device__ __forceinline__ bool edge_propagated(const uint32_t* mask, long long e) {
+  return mask == nullptr || ((mask[e >> 5] >> (e & 31)) & 1u);
+}
+
+static __device__ __forceinline__ int messages_of(int din, int fanout) {
+  return (fanout > 0 && din > fanout) ? fanout : din;
+}
+
+// ------------------------------------------------------------------------------------------------ layer reset
+__global__ void reset_vertices_kernel(long long V, const int32_t* din, int fanout, int32_t* pend, uint8_t* state,
+                                      int32_t* loc, int32_t* touch, int32_t* reload) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
+    pend[v] = messages_of(din[v], fanout) + 1;
+    state[v] = TAURUS_NOT_STARTED;
+    loc[v] = -1;
+    touch[v] = 0;
+    reload[v] = 0;
+  }
+}
+
+__global__ void reset_pool_kernel(long long pool_slots, long long host_rows, long long hub_count, const int32_t* hub_ids,
+                                  int32_t* loc, int32_t* owner, int32_t* free_stack, int32_t* host_free, DevCtl* ctl) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (long long i = tid; i < pool_slots; i += stride) {
+    owner[i] = -1;
+    free_stack[i] = (int32_t)(pool_slots - 1 - i);   // slot 0 is handed out first
+  }
+  for (long long i = tid; i < host_rows; i += stride) host_free[i] = (int32_t)(host_rows - 1 - i);
+  for (long long i = tid; i < hub_count; i += stride) loc[hub_ids[i]] = (int32_t)(pool_slots + i);
+  if (tid == 0) {
+    ctl->free_top = pool_slots;
+    ctl->host_free_top = host_rows;
+  }
+}
+
+void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st) {
+  int blocks = c->sm_count * 8;
+  cudaMemsetAsync(c->d_ctl, 0, sizeof(DevCtl), st);
+  reset_vertices_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_din, c->fanout[layer], c->d_pend, c->d_state, c->d_loc,
+                                                c->d_touch, c->d_reload);
+  reset_pool_kernel<<<blocks, 256, 0, st>>>(c->pool_slots, c->host_rows, c->hub_count, c->d_hub_ids, c->d_loc, c->d_owner,
+                                            c->d_free_stack, c->d_host_free, c->d_ctl);
+  int Hp = taurus_round_up(c->dims[layer + 1], 4);
+  if (c->hub_count > 0)
+    cudaMemsetAsync(c->d_acc + (size_t)c->pool_slots * Hp, 0, (size_t)c->hub_count * Hp * sizeof(float), st);
+  c->launches += 2;
+}
+
+// ------------------------------------------------------------------------------------------------ classify (S3)
+// One item per CSR edge of the chunk and one per chunk vertex (its self message).  The first item that
+// touches a vertex in this chunk (atomicMax on the epoch stamp) classifies it by its state at chunk start.
+// loc encoding: -1 none, [0, pool_slots) pool slot, >= pool_slots hub row, <= -2 host row (-2 - loc).
+__global__ void classify_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const long long e0 = a.row_ptr[a.src_begin], e1 = a.row_ptr[a.src_end];
+  const long long ne = e1 - e0, total = ne + (a.src_end - a.src_begin);
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  int hs = 0, ns = 0, ev = 0, gs = 0, bad = 0;
+  for (long long base = warp0 * 32; base < total; base += warps * 32) {
+    long long i = base + lane_id();
+    int v = -1;
+    if (i < ne) {
+      long long e = e0 + i;
+      if (edge_propagated(a.mask, e)) v = a.col[e];
+    } else if (i < total) {
+      v = (int)(a.src_begin + (i - ne));
+    }
+    bool need = false;
+    if (v >= a.V) { bad = 1; v = -1; }
+    if (v >= 0) {
+      int old = atomicMax(&a.touch[v], a.epoch);
+      if (old != a.epoch) {   // first touch in this chunk
+        int l = a.loc[v];
+        int s = a.state[v];
+        if (l >= a.pool_slots) {          // hub store: pinned, never takes a pool slot
+          gs++;
+          if (s == TAURUS_NOT_STARTED) a.state[v] = TAURUS_ON_GPU;
+        } else if (s == TAURUS_IN_BUFFER) {
+          hs++;
+        } else if (s == TAURUS_NOT_STARTED) {
+          ns++; need = true;
+        } else if (s == TAURUS_EVICTED) {
+          ev++; need = true;
+        } else {
+          bad = 1;                        // a completed vertex cannot receive a message
+        }
+      }
+    }
+    unsigned m = __ballot_sync(FULL, need);
+    if (m) {
+      int leader = __ffs(m) - 1, idx = 0;
+      if (lane_id() == leader) idx = atomicAdd(&ctl->need_count, __popc(m));
+      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
+      if (need && idx < a.pool_slots) a.need_list[idx] = v;
+    }
+  }
+  for (int o = 16; o; o >>= 1) {
+    hs += __shfl_xor_sync(FULL, hs, o); ns += __shfl_xor_sync(FULL, ns, o);
+    ev += __shfl_xor_sync(FULL, ev, o); gs += __shfl_xor_sync(FULL, gs, o);
+    bad |= __shfl_xor_sync(FULL, bad, o);
+  }
+  if (lane_id() == 0) {
+    if (hs) atomicAdd(&ctl->hs, hs);
+    if (ns) atomicAdd(&ctl->ns, ns);
+    if (ev) atomicAdd(&ctl->ev, ev);
+    if (gs) atomicAdd(&ctl->gs, gs);
+    if (bad) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+  }
+}
+
+void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  classify_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
+  c->launches += 1;
+}
+
+// ------------------------------------------------------------------------------------------------ make room (S4)
+// plan: need, deficit, capacity checks, peak occupancy.
+__global__ void plan_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (threadIdx.x != 0 || ctl->error) return;
+  long long need = ctl->need_count;
+  if (need > a.pool_slots) { ctl->error = TAURUS_ERR_POOL_TOO_SMALL; return; }
+  long long deficit = need - ctl->free_top;
+  if (deficit < 0) deficit = 0;
+  if (deficit > ctl->host_free_top) { ctl->error = TAURUS_ERR_HOST_STORE_FULL; return; }
+  ctl->deficit = (int32_t)deficit;
+  ctl->sel_prefix = 0ull;
+  ctl->sel_k = deficit;
+  ctl->victim_count = 0;
+  long long occ = a.pool_slots - (ctl->free_top + deficit - need);
+  if (occ > ctl->peak_occupancy) ctl->peak_occupancy = occ;
+}
+
+// Victims are the `deficit` smallest keys (pending << 31 | id) among IN_BUFFER vertices the chunk does not
+// touch.  Keys are unique, so an MSB-first radix select over 6 digits of 11 bits finds the exact
+// threshold key; every key <= threshold is a victim.
+static __device__ __forceinline__ int sel_shift(int pass) { return TAURUS_SEL_BITS * (TAURUS_SEL_PASSES - 1 - pass); }
+
+__global__ void select_keys_kernel(ChunkArgs a) {   // pass 0: gather keys, histogram of the top digit
+  DevCtl* ctl = a.ctl;
+  if (ctl->error || ctl->deficit == 0) return;
+  __shared__ unsigned int sh[TAURUS_SEL_BINS];
+  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < a.pool_slots; s += stride) {
+    int v = a.owner[s];
+    unsigned long long key = ~0ull;
+    if (v >= 0 && a.touch[v] != a.epoch) key = ((unsigned long long)(unsigned)a.pend[v] << 31) | (unsigned long long)v;
+    a.keys[s] = key;
+    if (key != ~0ull) atomicAdd(&sh[(unsigned)(key >> sel_shift(0)) & (TAURUS_SEL_BINS - 1)], 1u);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x)
+    if (sh[i]) atomicAdd(&ctl->hist[i], sh[i]);
+}
+
+__global__ void select_hist_kernel(ChunkArgs a, int pass) {   // passes 1..5
+  DevCtl* ctl = a.ctl;
+  if (ctl->error || ctl->deficit == 0) return;
+  __shared__ unsigned int sh[TAURUS_SEL_BINS];
+  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  const int shift = sel_shift(pass);
+  const unsigned long long prefix = ctl->sel_prefix;
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < a.pool_slots; s += stride) {
+    unsigned long long key = a.keys[s];
+    if (key != ~0ull && (key >> (shift + TAURUS_SEL_BITS)) == prefix)
+      atomicAdd(&sh[(unsigned)(key >> shift) & (TAURUS_SEL_BINS - 1)], 1u);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x)
+    if (sh[i]) atomicAdd(&ctl->hist[i], sh[i]);
+}
+
+__global__ void select_resolve_kernel(ChunkArgs a, int pass) {   // one block: pick the digit that holds rank k
+  DevCtl* ctl = a.ctl;
+  if (ctl->error || ctl->deficit == 0) return;
+  __shared__ unsigned int sh[TAURUS_SEL_BINS];
+  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) { sh[i] = ctl->hist[i]; ctl->hist[i] = 0; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long k = ctl->sel_k, cum = 0;
+    int b = 0;
+    for (; b < TAURUS_SEL_BINS; ++b) {
+      if (cum + sh[b] >= k) break;
+      cum += sh[b];
+    }
+    if (b == TAURUS_SEL_BINS) { ctl->error = TAURUS_ERR_POOL_TOO_SMALL; return; }   // fewer eligible victims than needed
+    ctl->sel_prefix = (ctl->sel_prefix << TAURUS_SEL_BITS) | (unsigned long long)b;
+    ctl->sel_k = k - cum;
+  }
+}
+
+__global__ void evict_list_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error || ctl->deficit == 0) return;
+  const unsigned long long thr = ctl->sel_prefix;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  for (long long base = warp0 * 32; base < a.pool_slots; base += warps * 32) {
+    long long s = base + lane_id();
+    bool hit = s < a.pool_slots && a.keys[s] <= thr;   // ~0 (ineligible) is never <= a real key
+    unsigned m = __ballot_sync(FULL, hit);
+    if (m) {
+      int leader = __ffs(m) - 1, idx = 0;
+      if (lane_id() == leader) idx = atomicAdd(&ctl->victim_count, __popc(m));
+      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
+      if (hit && idx < a.pool_slots) a.victims[idx] = (int32_t)s;
+    }
+  }
+}
+
+// One warp per victim: accumulator row -> pinned host row, IN_BUFFER -> EVICTED, slot back on the free stack.
+__global__ void evict_copy_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error || ctl->deficit == 0) return;
+  const int n = ctl->deficit;
+  if (ctl->victim_count != n) {   // the select must have produced exactly `deficit` victims
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+    return;
+  }
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int vec = a.Hp >> 2;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    int slot = a.victims[i];
+    int v = a.owner[slot];
+    int hrow = 0;
+    if (lane_id() == 0) {
+      long long h = atomicAdd((unsigned long long*)&ctl->host_free_top, (unsigned long long)-1ll) - 1;
+      hrow = a.host_free[h];
+    }
+    hrow = __shfl_sync(FULL, hrow, 0);
+    const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)slot * a.Hp);
+    float4* dst = reinterpret_cast<float4*>(a.host_store + (size_t)hrow * a.Hp);
+    for (int k = lane_id(); k < vec; k += 32) dst[k] = src[k];
+    if (lane_id() == 0) {
+      a.loc[v] = -2 - hrow;
+      a.state[v] = TAURUS_EVICTED;
+      a.owner[slot] = -1;
+      long long f = atomicAdd((unsigned long long*)&ctl->free_top, 1ull);
+      a.free_stack[f] = slot;
+    }
+  }
+}
+
+// One warp per vertex that needs a slot: pop a slot; EVICTED -> copy the host row back (a reload),
+// NOT_STARTED -> zero the row; either way the vertex is IN_BUFFER afterwards.
+__global__ void alloc_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const int n = ctl->need_count;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int vec = a.Hp >> 2;
+  int reloaded = 0;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    int v = a.need_list[i];
+    int slot = -1, st = 0, l = 0;
+    if (lane_id() == 0) {
+      long long f = atomicAdd((unsigned long long*)&ctl->free_top, (unsigned long long)-1ll) - 1;
+      slot = f >= 0 ? a.free_stack[f] : -1;
+      st = a.state[v];
+      l = a.loc[v];
+    }
+    slot = __shfl_sync(FULL, slot, 0);
+    st = __shfl_sync(FULL, st, 0);
+    l = __shfl_sync(FULL, l, 0);
+    if (slot < 0) {
+      if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+      continue;
+    }
+    float4* dst = reinterpret_cast<float4*>(a.acc + (size_t)slot * a.Hp);
+    if (st == TAURUS_EVICTED) {
+      int hrow = -2 - l;
+      const float4* src = reinterpret_cast<const float4*>(a.host_store + (size_t)hrow * a.Hp);
+      for (int k = lane_id(); k < vec; k += 32) dst[k] = src[k];
+      if (lane_id() == 0) {
+        long long h = atomicAdd((unsigned long long*)&ctl->host_free_top, 1ull);
+        a.host_free[h] = hrow;
+        a.reload_count[v] += 1;
+        reloaded++;
+      }
+    } else {
+      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int k = lane_id(); k < vec; k += 32) dst[k] = z;
+    }
+    if (lane_id() == 0) {
+      a.loc[v] = slot;
+      a.owner[slot] = v;
+      a.state[v] = TAURUS_IN_BUFFER;
+    }
+  }
+  if (lane_id() == 0 && reloaded) atomicAdd(&ctl->reloaded, reloaded);
+}
+
+void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  const int blocks = c->sm_count * 8;
+  plan_kernel<<<1, 32, 0, st>>>(a);
+  c->launches += 1;
+  if (c->pool_slots < c->V - c->hub_count) {   // eviction is impossible when every non-hub vertex has a slot
+    select_keys_kernel<<<blocks, 256, 0, st>>>(a);
+    select_resolve_kernel<<<1, 1024, 0, st>>>(a, 0);
+    for (int p = 1; p < TAURUS_SEL_PASSES; ++p) {
+      select_hist_kernel<<<blocks, 256, 0, st>>>(a, p);
+      select_resolve_kernel<<<1, 1024, 0, st>>>(a, p);
+    }
+    evict_list_kernel<<<blocks, 256, 0, st>>>(a);
+    evict_copy_kernel<<<blocks, 256, 0, st>>>(a);
+    c->launches += 2 * TAURUS_SEL_PASSES + 2;
+  }
+  alloc_kernel<<<blocks, 256, 0, st>>>(a);
+  c->launches += 1;
+}
+
+// ------------------------------------------------------------------------------------------------ finalise (S6 tail, S7)
+// One warp per completed vertex (listed by the scatter kernel when its pending count reached zero):
+// out = act(c_in(v) * acc) into the graduation buffer (Sect. 3.6); the slot is released.
+__global__ void finalise_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const int n = ctl->done_count;
+  const long long base = ctl->grad_count;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int vec = a.Hp >> 2;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    if (base + i >= a.drain_rows) {
+      if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+      continue;
+    }
+    int v = a.done_list[i];
+    int l = a.loc[v];
+    float scale;
+    if (a.mode == TAURUS_SAGE_MEAN) {
+      int m = messages_of(a.din[v], a.fanout);
+      scale = 1.0f / (float)(m > 1 ? m : 1);
+    } else {
+      scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+    }
+    const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
+    float4* dst = reinterpret_cast<float4*>(a.grad_rows + (size_t)(base + i) * a.Hp);
+    for (int k = lane_id(); k < vec; k += 32) {
+      float4 x = src[k];
+      x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
+      if (a.act) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
+      dst[k] = x;
+    }
+    if (lane_id() == 0) {
+      a.grad_ids[base + i] = v;
+      a.state[v] = TAURUS_COMPLETED;
+      if (l < a.pool_slots) {
+        a.owner[l] = -1;
+        long long f = atomicAdd((unsigned long long*)&ctl->free_top, 1ull);
+        a.free_stack[f] = l;
+      }
+    }
+  }
+}
+
+// One thread: fold the chunk's counters into the layer totals, write the chunk record, reset.
+__global__ void commit_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (threadIdx.x != 0 || ctl->error) return;
+  long long c = ctl->chunks;
+  if (c < a.log_capacity) {
+    long long* r = a.chunk_log + c * TAURUS_CK_COLUMNS;
+    r[TAURUS_CK_HS] = ctl->hs; r[TAURUS_CK_NS] = ctl->ns; r[TAURUS_CK_EV] = ctl->ev; r[TAURUS_CK_GS] = ctl->gs;
+    r[TAURUS_CK_NEED] = ctl->need_count; r[TAURUS_CK_EVICTED] = ctl->deficit; r[TAURUS_CK_RELOADED] = ctl->reloaded;
+    r[TAURUS_CK_COMPLETED] = ctl->done_count; r[TAURUS_CK_OCCUPANCY] = a.pool_slots - ctl->free_top;
+  }
+  ctl->sum_hs += ctl->hs; ctl->sum_ns += ctl->ns; ctl->sum_ev += ctl->ev; ctl->sum_gs += ctl->gs;
+  ctl->evictions += ctl->deficit;
+  ctl->reloads += ctl->reloaded;
+  ctl->completed += ctl->done_count;
+  ctl->grad_count += ctl->done_count;
+  ctl->chunks = c + 1;
+  ctl->hs = ctl->ns = ctl->ev = ctl->gs = 0;
+  ctl->need_count = 0; ctl->done_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;
+}
+
+void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  finalise_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
+  commit_kernel<<<1, 32, 0, st>>>(a);
+  c->launches += 2;
+}
+
+// ------------------------------------------------------------------------------------------------ drain helpers
+// Row i of the graduation buffer goes to dense[id * ld ...]: the vertex-ordered matrix the next layer streams.
+__global__ void place_rows_kernel(const long long* ids, const float* rows, int Hp, int d_out, float* dense, long long ld,
+                                  long long count) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const bool vec_ok = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(dense) & 15) == 0);
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < count; i += warps) {
+    long long id = ids[i];
+    const float* src = rows + (size_t)i * Hp;
+    float* dst = dense + (size_t)id * ld;
+    if (vec_ok) {
+      int full = d_out >> 2;
+      for (int k = lane_id(); k < full; k += 32)
+        reinterpret_cast<float4*>(dst)[k] = reinterpret_cast<const float4*>(src)[k];
+      for (int k = (full << 2) + lane_id(); k < d_out; k += 32) dst[k] = src[k];
+    } else {
+      for (int k = lane_id(); k < d_out; k += 32) dst[k] = src[k];
+    }
+  }
+}
+
+void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st) {
+  if (count <= 0) return;
+  long long blocks = (count + 7) / 8;
+  if (blocks > c->sm_count * 16) blocks = c->sm_count * 16;
+  place_rows_kernel<<<(int)blocks, 256, 0, st>>>(c->d_grad_ids, c->d_grad_rows, Hp, d_out, dense, ld, count);
+  c->launches += 1;
+}
+
+__global__ void reload_histogram_kernel(long long V, const int32_t* reload, long long* hist18) {
+  __shared__ unsigned int sh[17];
+  __shared__ int shmax;
+  if (threadIdx.x < 17) sh[threadIdx.x] = 0;
+  if (threadIdx.x == 0) shmax = 0;
+  __syncthreads();
+  long long stride = (long long)gridDim.x * blockDim.x;
+  int mx = 0;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
+    int r = reload[v];
+    if (r > mx) mx = r;
+    if (r > 0) atomicAdd(&sh[r < 16 ? r : 16], 1u);   // bin 0 is derived on the host from V
+  }
+  if (mx) atomicMax(&shmax, mx);
+  __syncthreads();
+  if (threadIdx.x < 17 && sh[threadIdx.x]) atomicAdd((unsigned long long*)&hist18[threadIdx.x], (unsigned long long)sh[threadIdx.x]);
+  if (threadIdx.x == 0 && shmax) atomicMax(&hist18[17], (long long)shmax);
+}
+
+void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st) {
+  cudaMemsetAsync(d_hist18, 0, 18 * sizeof(long long), st);
+  reload_histogram_kernel<<<c->sm_count * 4, 256, 0, st>>>(c->V, c->d_reload, d_hist18);
+  c->launches += 1;
+}
+
+// ------------------------------------------------------------------------------------------------ completion ranks
+// Completion rank of v = max(v, largest source among its propagated in-edges): the chunk holding that
+// rank is the one in which v completes (Sect. 3.8, c(v)).  A histogram over blocks of 64 ranks lets the
+// host bound, without a device round trip, how many rows a pushed range can add to the graduation buffer.
+__global__ void rank_init_kernel(long long V, int32_t* last) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) last[v] = (int32_t)v;
+}
+__global__ void rank_max_kernel(long long V, const long long* row_ptr, const int32_t* col, const uint32_t* mask, int32_t* last) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    long long b = row_ptr[u], e = row_ptr[u + 1];
+    for (long long k = b + lane_id(); k < e; k += 32)
+      if (edge_propagated(mask, k)) atomicMax(&last[col[k]], (int32_t)u);
+  }
+}
+__global__ void rank_hist_kernel(long long V, const int32_t* last, int32_t* hist) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) atomicAdd(&hist[last[v] >> 6], 1);
+}
+
+void launch_completion_ranks(taurus_ctx* c, cudaStream_t st) {
+  int blocks = c->sm_count * 8;
+  long long nb = (c->V + 63) / 64;
+  cudaMemsetAsync(c->d_rank_hist, 0, (size_t)nb * sizeof(int32_t), st);
+  rank_init_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_vtmp);
+  rank_max_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_vtmp);
+  rank_hist_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_vtmp, c->d_rank_hist);
+  c->launches += 3;
+}
+
+// ------------------------------------------------------------------------------------------------ init check
+__global__ void degree_hist_kernel(long long E, const int32_t* col, long long V, int32_t* hist, int* flag) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < E; e += stride) {
+    int v = col[e];
+    if (v < 0 || v >= V) *flag = 1; else atomicAdd(&hist[v], 1);
+  }
+}
+__global__ void degree_compare_kernel(long long V, const int32_t* hist, const int32_t* din, const long long* row_ptr, int* flag) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride)
+    if (hist[v] != din[v] || row_ptr[v + 1] < row_ptr[v]) *flag = 1;
+}
+
+int check_in_degrees(taurus_ctx* c, cudaStream_t st) {
+  int* d_flag = nullptr;
+  if (cudaMalloc(&d_flag, sizeof(int)) != cudaSuccess) return -1;
+  cudaMemsetAsync(d_flag, 0, sizeof(int), st);
+  cudaMemsetAsync(c->d_vtmp, 0, (size_t)c->V * sizeof(int32_t), st);
+  int blocks = c->sm_count * 8;
+  degree_hist_kernel<<<blocks, 256, 0, st>>>(c->E, c->d_col, c->V, c->d_vtmp, d_flag);
+  degree_compare_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_vtmp, c->d_din, c->d_row_ptr, d_flag);
+  int flag = 0;
+  cudaMemcpyAsync(&flag, d_flag, sizeof(int), cudaMemcpyDeviceToHost, st);
+  cudaStreamSynchronize(st);
+  cudaFree(d_flag);
+  c->launches += 2;
+  return flag;
+}

@@ -1,0 +1,497 @@
+// Host side of libtaurus: the C ABI of include/taurus.h.  Validation, allocation, per-layer set-up and the
+// launch sequence of a push.  No arithmetic of the method happens on the host: a push enqueues kernels
+// and returns.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "taurus_internal.h"
+
+static thread_local char g_cuda_err[256] = "";
+
+static bool cuda_ok(cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return true;
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+  cudaGetLastError();
+  return false;
+}
+#define CU(call) do { if (!cuda_ok((call), #call)) return TAURUS_ERR_CUDA; } while (0)
+
+template <class T>
+static int dev_alloc(T** p, size_t count) {
+  *p = nullptr;
+  cudaError_t e = cudaMalloc((void**)p, (count > 0 ? count : 1) * sizeof(T));
+  if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); snprintf(g_cuda_err, sizeof(g_cuda_err), "cudaMalloc of %zu bytes failed", count * sizeof(T)); return TAURUS_ERR_NOMEM; }
+  return cuda_ok(e, "cudaMalloc") ? TAURUS_OK : TAURUS_ERR_CUDA;
+}
+#define ALLOC(p, n) do { int rc_ = dev_alloc(&(p), (size_t)(n)); if (rc_) return rc_; } while (0)
+
+enum { PK_HOST_PAGEABLE = 0, PK_HOST_PINNED = 1, PK_DEVICE = 2 };
+static int pointer_kind(const void* p) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return PK_HOST_PAGEABLE; }
+  if (at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged) return PK_DEVICE;
+  if (at.type == cudaMemoryTypeHost) return PK_HOST_PINNED;
+  return PK_HOST_PAGEABLE;
+}
+
+extern "C" const char* taurus_last_cuda_error(void) { return g_cuda_err; }
+
+extern "C" const char* taurus_strerror(int code) {
+  switch (code) {
+    case TAURUS_OK: return "ok";
+    case TAURUS_ERR_INVALID_ARG: return "invalid argument";
+    case TAURUS_ERR_ORDER: return "call out of order (chunk order, layer not begun, or layer incomplete)";
+    case TAURUS_ERR_POOL_TOO_SMALL: return "accumulator pool too small for one chunk";
+    case TAURUS_ERR_HOST_STORE_FULL: return "pinned host store for evicted rows is full";
+    case TAURUS_ERR_DRAIN_FULL: return "graduation buffer could overflow: drain first";
+    case TAURUS_ERR_CUDA: return "CUDA runtime error";
+    case TAURUS_ERR_INTERNAL: return "device-side consistency check failed";
+    case TAURUS_ERR_NOMEM: return "out of memory";
+    case TAURUS_ERR_UNSUPPORTED: return "unsupported shape or size";
+    default: return "unknown error";
+  }
+}
+
+extern "C" void taurus_destroy(taurus_ctx* c) {
+  if (!c) return;
+  int prev = 0;
+  cudaGetDevice(&prev);
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  cudaFree(c->d_row_ptr); cudaFree(c->d_col); cudaFree(c->d_din);
+  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) { cudaFree(c->d_Wcat[l]); cudaFree(c->d_bias[l]); cudaFree(c->d_Wtc[l]); }
+  cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
+  cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
+  cudaFree(c->d_need_list); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
+  if (c->h_store) cudaFreeHost(c->h_store);
+  cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X); cudaFree(c->d_PT);
+  cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
+  cudaFree(c->d_ctl); cudaFree(c->d_chunk_log);
+  if (c->h_ctl) cudaFreeHost(c->h_ctl);
+  if (c->order_event) cudaEventDestroy(c->order_event);
+  for (auto& e : c->phase_ev) if (e) cudaEventDestroy(e);
+  cudaGetLastError();
+  cudaSetDevice(prev);
+  delete c;
+}
+
+static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m, const taurus_run* r) {
+  cudaDeviceProp prop;
+  CU(cudaGetDevice(&c->device));
+  CU(cudaGetDeviceProperties(&prop, c->device));
+  c->sm_count = prop.multiProcessorCount;
+  c->V = g->V; c->E = g->E; c->L = m->L; c->mode = m->mode; c->gemm_mode = m->gemm_mode; c->flags = r->flags;
+  c->seed = r->seed;
+  c->chunk_sources = r->chunk_sources; c->pool_slots = r->pool_slots; c->hub_count = r->hub_count;
+  c->host_rows = r->host_evict_rows; c->drain_rows = r->drain_rows;
+  bool any_sampled = false;
+  for (int l = 0; l <= m->L; ++l) c->dims[l] = m->dims[l];
+  for (int l = 0; l < m->L; ++l) {
+    c->act[l] = m->act ? m->act[l] : 0;
+    c->fanout[l] = r->fanout ? r->fanout[l] : 0;
+    any_sampled |= c->fanout[l] > 0;
+    c->Hmax = std::max(c->Hmax, taurus_round_up(c->dims[l + 1], 4));
+    c->Kmax = std::max(c->Kmax, taurus_round_up(c->dims[l], 4));
+  }
+  const long long V = c->V, E = c->E;
+
+  // graph
+  ALLOC(c->d_row_ptr, V + 1); ALLOC(c->d_col, E); ALLOC(c->d_din, V); ALLOC(c->d_vtmp, V);
+  CU(cudaMemcpy(c->d_row_ptr, g->row_ptr, (size_t)(V + 1) * sizeof(long long), cudaMemcpyDefault));
+  if (E > 0) CU(cudaMemcpy(c->d_col, g->col_idx, (size_t)E * sizeof(int32_t), cudaMemcpyDefault));
+  CU(cudaMemcpy(c->d_din, g->in_degree, (size_t)V * sizeof(int32_t), cudaMemcpyDefault));
+  long long ends[2] = {-1, -1};
+  CU(cudaMemcpy(&ends[0], c->d_row_ptr, sizeof(long long), cudaMemcpyDeviceToHost));
+  CU(cudaMemcpy(&ends[1], c->d_row_ptr + V, sizeof(long long), cudaMemcpyDeviceToHost));
+  if (ends[0] != 0 || ends[1] != E) return TAURUS_ERR_INVALID_ARG;
+  int bad = check_in_degrees(c, nullptr);
+  if (bad < 0) return TAURUS_ERR_NOMEM;
+  if (bad) return TAURUS_ERR_INVALID_ARG;
+  CU(cudaGetLastError());
+
+  // hub set: the hub_count largest by (in_degree descending, id ascending)
+  ALLOC(c->d_hub, V); ALLOC(c->d_hub_ids, c->hub_count);
+  CU(cudaMemset(c->d_hub, 0, (size_t)V));
+  if (c->hub_count > 0) {
+    std::vector<int32_t> din((size_t)V);
+    CU(cudaMemcpy(din.data(), c->d_din, (size_t)V * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    std::vector<unsigned long long> key((size_t)V);
+    for (long long v = 0; v < V; ++v)
+      key[(size_t)v] = ((unsigned long long)(0x7fffffffu - (unsigned)din[(size_t)v]) << 32) | (unsigned long long)v;
+    std::nth_element(key.begin(), key.begin() + (c->hub_count - 1), key.end());
+    std::sort(key.begin(), key.begin() + c->hub_count);
+    std::vector<int32_t> ids((size_t)c->hub_count);
+    std::vector<uint8_t> flag((size_t)V, 0);
+    for (long long i = 0; i < c->hub_count; ++i) { ids[(size_t)i] = (int32_t)(key[(size_t)i] & 0xffffffffu); flag[(size_t)ids[(size_t)i]] = 1; }
+    CU(cudaMemcpy(c->d_hub_ids, ids.data(), ids.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->d_hub, flag.data(), flag.size(), cudaMemcpyHostToDevice));
+  }
+
+  // weights: Wcat = [W_neigh | W_self] with both halves padded to Hp columns
+  for (int l = 0; l < c->L; ++l) {
+    const int K = c->dims[l], d_out = c->dims[l + 1], Hp = taurus_round_up(d_out, 4);
+    const int N = c->mode == TAURUS_SAGE_MEAN ? 2 * Hp : Hp;
+    std::vector<float> wn((size_t)K * d_out), ws, b((size_t)Hp, 0.f), cat((size_t)K * N, 0.f);
+    CU(cudaMemcpy(wn.data(), m->W_neigh[l], wn.size() * sizeof(float), cudaMemcpyDefault));
+    if (c->mode == TAURUS_SAGE_MEAN) {
+      ws.resize((size_t)K * d_out);
+      CU(cudaMemcpy(ws.data(), m->W_self[l], ws.size() * sizeof(float), cudaMemcpyDefault));
+    }
+    if (m->bias && m->bias[l]) CU(cudaMemcpy(b.data(), m->bias[l], (size_t)d_out * sizeof(float), cudaMemcpyDefault));
+    for (int k = 0; k < K; ++k)
+      for (int j = 0; j < d_out; ++j) {
+        cat[(size_t)k * N + j] = wn[(size_t)k * d_out + j];
+        if (c->mode == TAURUS_SAGE_MEAN) cat[(size_t)k * N + Hp + j] = ws[(size_t)k * d_out + j];
+      }
+    ALLOC(c->d_Wcat[l], cat.size()); ALLOC(c->d_bias[l], b.size());
+    CU(cudaMemcpy(c->d_Wcat[l], cat.data(), cat.size() * sizeof(float), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->d_bias[l], b.data(), b.size() * sizeof(float), cudaMemcpyHostToDevice));
+  }
+
+  // per-vertex state
+  ALLOC(c->d_pend, V); ALLOC(c->d_state, V); ALLOC(c->d_loc, V); ALLOC(c->d_touch, V); ALLOC(c->d_reload, V);
+  ALLOC(c->d_rank_hist, (V + 63) / 64);
+  // pool, hub store
+  ALLOC(c->d_acc, (size_t)(c->pool_slots + c->hub_count) * c->Hmax);
+  ALLOC(c->d_owner, c->pool_slots); ALLOC(c->d_free_stack, c->pool_slots); ALLOC(c->d_need_list, c->pool_slots);
+  if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); }
+  ALLOC(c->d_host_free, c->host_rows);
+  if (c->host_rows > 0) {
+    cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->host_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
+    if (e != cudaSuccess) { cuda_ok(e, "cudaHostAlloc(evicted-row store)"); c->h_store = nullptr; return TAURUS_ERR_NOMEM; }
+    CU(cudaHostGetDevicePointer((void**)&c->d_store_alias, c->h_store, 0));
+  }
+  // graduation buffer, chunk buffers
+  ALLOC(c->d_grad_ids, c->drain_rows); ALLOC(c->d_grad_rows, (size_t)c->drain_rows * c->Hmax); ALLOC(c->d_done_list, c->drain_rows);
+  ALLOC(c->d_X, (size_t)c->chunk_sources * c->Kmax);
+  ALLOC(c->d_PT, (size_t)c->chunk_sources * 2 * c->Hmax);
+  // sampling
+  if (any_sampled) {
+    int rc = build_in_edge_order(c);
+    if (rc) { cuda_ok(cudaGetLastError(), "build_in_edge_order"); return rc; }
+    ALLOC(c->d_mask, (E + 31) / 32);
+  }
+  // control
+  ALLOC(c->d_ctl, 1);
+  CU(cudaMemset(c->d_ctl, 0, sizeof(DevCtl)));
+  CU(cudaHostAlloc((void**)&c->h_ctl, sizeof(DevCtl), cudaHostAllocDefault));
+  memset(c->h_ctl, 0, sizeof(DevCtl));
+  c->log_capacity = std::max<long long>(1024, 4 * ((V + c->chunk_sources - 1) / c->chunk_sources));
+  ALLOC(c->d_chunk_log, (size_t)c->log_capacity * TAURUS_CK_COLUMNS);
+  CU(cudaEventCreateWithFlags(&c->order_event, cudaEventDisableTiming));
+  for (auto& e : c->phase_ev) CU(cudaEventCreate(&e));
+  CU(cudaDeviceSynchronize());
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const taurus_model* m, const taurus_run* r) {
+  if (!out) return TAURUS_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!g || !m || !r || !g->row_ptr || !g->in_degree || (g->E > 0 && !g->col_idx)) return TAURUS_ERR_INVALID_ARG;
+  if (g->V < 1 || g->V >= (1ll << 31) || g->E < 0 || g->E >= (1ll << 32)) return TAURUS_ERR_INVALID_ARG;
+  if (m->L < 1 || m->L > TAURUS_MAX_LAYERS || !m->dims || !m->W_neigh) return TAURUS_ERR_INVALID_ARG;
+  if (m->mode != TAURUS_SAGE_MEAN && m->mode != TAURUS_GCN_SYM) return TAURUS_ERR_INVALID_ARG;
+  if (m->gemm_mode != TAURUS_GEMM_FP32 && m->gemm_mode != TAURUS_GEMM_BF16) return TAURUS_ERR_INVALID_ARG;
+  if (m->mode == TAURUS_SAGE_MEAN && !m->W_self) return TAURUS_ERR_INVALID_ARG;
+  for (int l = 0; l <= m->L; ++l)
+    if (m->dims[l] < 1 || m->dims[l] > TAURUS_MAX_DIM) return TAURUS_ERR_INVALID_ARG;
+  for (int l = 0; l < m->L; ++l) {
+    if (!m->W_neigh[l] || (m->mode == TAURUS_SAGE_MEAN && !m->W_self[l])) return TAURUS_ERR_INVALID_ARG;
+    if (r->fanout && (r->fanout[l] < 0 || r->fanout[l] > TAURUS_MAX_FANOUT)) return TAURUS_ERR_INVALID_ARG;
+  }
+  if (r->chunk_sources < 1 || r->chunk_sources > (1 << 24) || r->pool_slots < 1 || r->pool_slots >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
+  if (r->hub_count < 0 || r->hub_count > g->V || r->host_evict_rows < 0 || r->host_evict_rows >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
+  if (r->drain_rows < 1 || r->drain_rows >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
+  if (r->pool_slots + r->hub_count >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
+  taurus_ctx* c = new (std::nothrow) taurus_ctx();
+  if (!c) return TAURUS_ERR_NOMEM;
+  int rc;
+  try { rc = init_impl(c, g, m, r); } catch (const std::bad_alloc&) { rc = TAURUS_ERR_NOMEM; }
+  if (rc != TAURUS_OK) { taurus_destroy(c); return rc; }
+  *out = c;
+  return TAURUS_OK;
+}
+
+// Reads the device control block (after synchronising `st`) and returns its sticky error.
+static int read_ctl(taurus_ctx* c, cudaStream_t st) {
+  CU(cudaStreamSynchronize(st));
+  CU(cudaMemcpy(c->h_ctl, c->d_ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost));
+  return c->h_ctl->error;
+}
+
+extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_stream) {
+  if (!c || layer < 0 || layer >= c->L) return TAURUS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CU(cudaSetDevice(c->device));
+  if (c->last_stream != st) CU(cudaStreamSynchronize(c->last_stream));
+  c->layer = layer;
+  memset(c->h_ctl, 0, sizeof(DevCtl));
+  c->next_src = 0; c->chunk_seq = 0; c->ub_since_drain = 0; c->last_stream = st;
+  launch_layer_reset(c, layer, st);
+  c->d_mask_cur = nullptr;
+  if (c->fanout[layer] > 0) {
+    launch_sample_mask(c, layer, st);
+    c->d_mask_cur = c->d_mask;
+  }
+  launch_completion_ranks(c, st);
+  CU(cudaGetLastError());
+  const long long nb = (c->V + 63) / 64;
+  std::vector<int32_t> hist((size_t)nb);
+  CU(cudaMemcpyAsync(hist.data(), c->d_rank_hist, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  c->rank_cum.assign((size_t)nb + 1, 0);
+  for (long long i = 0; i < nb; ++i) c->rank_cum[(size_t)i + 1] = c->rank_cum[(size_t)i] + hist[(size_t)i];
+  return TAURUS_OK;
+}
+
+static long long completion_bound(const taurus_ctx* c, long long s, long long e) {
+  const long long nb = (long long)c->rank_cum.size() - 1;
+  long long b0 = s / 64, b1 = std::min(nb, (e + 63) / 64);
+  return c->rank_cum[(size_t)b1] - c->rank_cum[(size_t)b0];
+}
+
+extern "C" int taurus_completion_bound(taurus_ctx* c, int64_t src_begin, int64_t src_end, int64_t* out_bound) {
+  if (!c || !out_bound || src_begin < 0 || src_end > c->V || src_begin > src_end) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  *out_bound = completion_bound(c, src_begin, src_end);
+  return TAURUS_OK;
+}
+
+static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
+  ChunkArgs a;
+  const int l = c->layer;
+  a.row_ptr = c->d_row_ptr; a.col = c->d_col; a.din = c->d_din; a.mask = c->d_mask_cur;
+  a.pend = c->d_pend; a.state = c->d_state; a.loc = c->d_loc; a.touch = c->d_touch; a.reload_count = c->d_reload;
+  a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list;
+  a.victims = c->d_victims; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
+  a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
+  a.Hp = taurus_round_up(c->dims[l + 1], 4);
+  a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;
+  a.bias = c->d_bias[l];
+  a.ctl = c->d_ctl; a.chunk_log = c->d_chunk_log; a.log_capacity = c->log_capacity;
+  a.V = c->V; a.pool_slots = c->pool_slots; a.hub_count = c->hub_count; a.host_rows = c->host_rows; a.drain_rows = c->drain_rows;
+  a.src_begin = s; a.src_end = e;
+  a.epoch = (int32_t)(c->chunk_seq + 1);
+  a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.checked = (c->flags & TAURUS_FLAG_CHECKED) ? 1 : 0;
+  return a;
+}
+
+extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream) {
+  if (!c || !features) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  if (src_begin != c->next_src) return TAURUS_ERR_ORDER;
+  if (src_end <= src_begin || src_end > c->V || src_end - src_begin > c->chunk_sources) return TAURUS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(features) & 3) != 0) return TAURUS_ERR_INVALID_ARG;
+  if (c->h_ctl->error) return c->h_ctl->error;
+  const long long bound = completion_bound(c, src_begin, src_end);
+  if (c->ub_since_drain + bound > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CU(cudaSetDevice(c->device));
+  if (st != c->last_stream) {   // keep chunk order across streams
+    CU(cudaEventRecord(c->order_event, c->last_stream));
+    CU(cudaStreamWaitEvent(st, c->order_event, 0));
+    c->last_stream = st;
+  }
+  const int l = c->layer;
+  const int K = c->dims[l];
+  const int n = (int)(src_end - src_begin);
+  const bool timing = c->timing != 0;
+  if (timing) cudaEventRecord(c->phase_ev[0], st);
+  // S1: features to the device
+  const float* X = features;
+  int ldx = K;
+  if (pointer_kind(features) != PK_DEVICE) {
+    CU(cudaMemcpyAsync(c->d_X, features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, st));
+    X = c->d_X;
+  }
+  if (timing) cudaEventRecord(c->phase_ev[1], st);
+  ChunkArgs a = make_args(c, src_begin, src_end);
+  // S2: projection
+  launch_project_simt(c, l, X, ldx, src_begin, n, st);
+  if (timing) cudaEventRecord(c->phase_ev[2], st);
+  // S3, S4
+  launch_classify(c, a, st);
+  launch_make_room(c, a, st);
+  if (timing) cudaEventRecord(c->phase_ev[3], st);
+  // S5, S5', S6
+  launch_scatter(c, a, st);
+  if (timing) cudaEventRecord(c->phase_ev[4], st);
+  // S7
+  launch_finalise(c, a, st);
+  if (timing) cudaEventRecord(c->phase_ev[5], st);
+  CU(cudaGetLastError());
+  c->next_src = src_end;
+  c->chunk_seq += 1;
+  c->ub_since_drain += bound;
+  return TAURUS_OK;
+}
+
+static int drain_common(taurus_ctx* c, long long capacity, long long* out_count, long long* count) {
+  if (!c || !out_count || capacity < 0) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  int err = read_ctl(c, c->last_stream);
+  if (err) return err;
+  *count = c->h_ctl->grad_count;
+  *out_count = *count;
+  if (*count > capacity) return TAURUS_ERR_INVALID_ARG;
+  return TAURUS_OK;
+}
+
+static int drain_reset(taurus_ctx* c) {
+  CU(cudaMemsetAsync(reinterpret_cast<char*>(c->d_ctl) + offsetof(DevCtl, grad_count), 0, sizeof(long long), c->last_stream));
+  CU(cudaStreamSynchronize(c->last_stream));
+  c->ub_since_drain = 0;
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_drain_completed(taurus_ctx* c, int64_t* out_ids, float* out_rows, int64_t capacity_rows, int64_t* out_count) {
+  long long count = 0, oc = 0;
+  int rc = drain_common(c, capacity_rows, &oc, &count);
+  if (out_count) *out_count = oc;
+  if (rc) return rc;
+  if (count > 0) {
+    if (!out_ids || !out_rows) return TAURUS_ERR_INVALID_ARG;
+    const int d_out = c->dims[c->layer + 1], Hp = taurus_round_up(d_out, 4);
+    cudaStream_t st = c->last_stream;
+    CU(cudaMemcpyAsync(out_ids, c->d_grad_ids, (size_t)count * sizeof(long long), cudaMemcpyDefault, st));
+    CU(cudaMemcpy2DAsync(out_rows, (size_t)d_out * sizeof(float), c->d_grad_rows, (size_t)Hp * sizeof(float),
+                         (size_t)d_out * sizeof(float), (size_t)count, cudaMemcpyDefault, st));
+  }
+  return drain_reset(c);
+}
+
+extern "C" int taurus_drain_dense(taurus_ctx* c, float* dense_rows, int64_t ld, int64_t* out_ids, int64_t capacity_rows,
+                                  int64_t* out_count) {
+  if (!c || !dense_rows) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer >= 0 && ld < c->dims[c->layer + 1]) return TAURUS_ERR_INVALID_ARG;
+  float* dense_dev = dense_rows;
+  int kind = pointer_kind(dense_rows);
+  if (kind == PK_HOST_PAGEABLE) return TAURUS_ERR_INVALID_ARG;
+  if (kind == PK_HOST_PINNED) {
+    if (!cuda_ok(cudaHostGetDevicePointer((void**)&dense_dev, dense_rows, 0), "cudaHostGetDevicePointer")) return TAURUS_ERR_INVALID_ARG;
+  }
+  long long count = 0, oc = 0;
+  int rc = drain_common(c, capacity_rows, &oc, &count);
+  if (out_count) *out_count = oc;
+  if (rc) return rc;
+  if (count > 0) {
+    const int d_out = c->dims[c->layer + 1], Hp = taurus_round_up(d_out, 4);
+    cudaStream_t st = c->last_stream;
+    launch_place_rows(c, dense_dev, ld, d_out, Hp, count, st);
+    if (out_ids) CU(cudaMemcpyAsync(out_ids, c->d_grad_ids, (size_t)count * sizeof(long long), cudaMemcpyDefault, st));
+    CU(cudaGetLastError());
+  }
+  return drain_reset(c);
+}
+
+static int fill_stats(taurus_ctx* c, taurus_stats* s) {
+  const DevCtl* h = c->h_ctl;
+  memset(s, 0, sizeof(*s));
+  long long* d_hist = nullptr;
+  ALLOC(d_hist, 18);
+  launch_reload_histogram(c, d_hist, c->last_stream);
+  long long hist[18];
+  cudaError_t e = cudaMemcpy(hist, d_hist, sizeof(hist), cudaMemcpyDeviceToHost);
+  cudaFree(d_hist);
+  CU(e);
+  long long nonzero = 0;
+  for (int i = 1; i < 17; ++i) { s->reload_histogram[i] = hist[i]; nonzero += hist[i]; }
+  s->reload_histogram[0] = c->V - nonzero;
+  s->max_reload_count = hist[17];
+  s->evictions = h->evictions; s->reloads = h->reloads; s->peak_occupancy = h->peak_occupancy;
+  s->hub_messages = h->hub_messages; s->total_messages = h->total_messages; s->hub_vertices = c->hub_count;
+  s->completed = h->completed; s->sum_hs = h->sum_hs; s->sum_ns = h->sum_ns; s->sum_ev = h->sum_ev; s->sum_gs = h->sum_gs;
+  s->free_slots = h->free_top; s->chunks = h->chunks;
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_get_stats(taurus_ctx* c, taurus_stats* stats) {
+  if (!c || !stats) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  int err = read_ctl(c, c->last_stream);
+  if (err) return err;
+  return fill_stats(c, stats);
+}
+
+extern "C" int taurus_layer_end(taurus_ctx* c, taurus_stats* stats) {
+  if (!c) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  int err = read_ctl(c, c->last_stream);
+  if (err) return err;
+  if (stats) { int rc = fill_stats(c, stats); if (rc) return rc; }
+  if (c->next_src != c->V || c->h_ctl->completed != c->V || c->h_ctl->free_top != c->pool_slots) return TAURUS_ERR_ORDER;
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_get_chunk_log(taurus_ctx* c, int64_t* out, int64_t capacity_chunks, int64_t* out_chunks) {
+  if (!c || !out || !out_chunks || capacity_chunks < 0) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  int err = read_ctl(c, c->last_stream);
+  if (err) return err;
+  long long n = std::min<long long>(std::min<long long>(c->h_ctl->chunks, c->log_capacity), capacity_chunks);
+  if (n > 0) CU(cudaMemcpy(out, c->d_chunk_log, (size_t)n * TAURUS_CK_COLUMNS * sizeof(long long), cudaMemcpyDeviceToHost));
+  *out_chunks = n;
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_get_vertex_array(taurus_ctx* c, int32_t which, void* out_host) {
+  if (!c || !out_host || which < 0 || which > 3) return TAURUS_ERR_INVALID_ARG;
+  CU(cudaSetDevice(c->device));
+  CU(cudaStreamSynchronize(c->last_stream));
+  const void* src = which == 0 ? (const void*)c->d_state : which == 1 ? (const void*)c->d_pend
+                    : which == 2 ? (const void*)c->d_reload : (const void*)c->d_hub;
+  size_t bytes = (size_t)c->V * ((which == 0 || which == 3) ? 1 : 4);
+  CU(cudaMemcpy(out_host, src, bytes, cudaMemcpyDeviceToHost));
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_get_sampled_edges(taurus_ctx* c, int32_t layer, int64_t dst, int64_t* out_edge_ids, int32_t* out_sources,
+                                        int32_t capacity, int32_t* n) {
+  if (!c || !n || layer < 0 || layer >= c->L || dst < 0 || dst >= c->V || capacity < 0) return TAURUS_ERR_INVALID_ARG;
+  if (capacity > 0 && (!out_edge_ids || !out_sources)) return TAURUS_ERR_INVALID_ARG;
+  if (!c->d_csc_eid) return TAURUS_ERR_ORDER;   // built only when some layer is sampled
+  CU(cudaSetDevice(c->device));
+  CU(cudaStreamSynchronize(c->last_stream));
+  int rc = sampled_edges_of(c, layer, dst, (long long*)out_edge_ids, out_sources, capacity, n);
+  if (rc == TAURUS_ERR_CUDA) cuda_ok(cudaGetLastError(), "sampled_edges_of");
+  return rc;
+}
+
+extern "C" int taurus_get_edge_mask(taurus_ctx* c, uint32_t* out_words) {
+  if (!c || !out_words) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  CU(cudaStreamSynchronize(c->last_stream));
+  size_t words = (size_t)((c->E + 31) / 32);
+  if (c->d_mask_cur) CU(cudaMemcpy(out_words, c->d_mask_cur, words * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+  else {
+    memset(out_words, 0xff, words * sizeof(uint32_t));
+    if (c->E & 31) out_words[words - 1] = (1u << (c->E & 31)) - 1u;
+  }
+  return TAURUS_OK;
+}
+
+extern "C" int64_t taurus_launch_count(const taurus_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int taurus_set_timing(taurus_ctx* c, int32_t on) {
+  if (!c) return TAURUS_ERR_INVALID_ARG;
+  c->timing = on ? 1 : 0;
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out5) {
+  if (!c || !out5) return TAURUS_ERR_INVALID_ARG;
+  if (!c->timing || c->chunk_seq == 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  CU(cudaStreamSynchronize(c->last_stream));
+  for (int i = 0; i < 5; ++i) CU(cudaEventElapsedTime(&out5[i], c->phase_ev[i], c->phase_ev[i + 1]));
+  return TAURUS_OK;
+}

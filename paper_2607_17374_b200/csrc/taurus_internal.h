@@ -1,0 +1,164 @@
+// Internal declarations shared by the translation units of libtaurus.
+// Host control lives in taurus_host.cu; each kernels_*.cu file holds kernels and their launchers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "taurus.h"
+
+#define TAURUS_MAX_LAYERS 16
+#define TAURUS_MAX_DIM 1024
+#define TAURUS_MAX_FANOUT 64
+#define TAURUS_SEL_BITS 11                      // radix-select digit width
+#define TAURUS_SEL_BINS (1 << TAURUS_SEL_BITS)
+#define TAURUS_SEL_PASSES 6                     // 6 x 11 = 66 bits >= the 62-bit (pending, id) key
+
+// Device-resident control block: counters the kernels of one chunk hand to one another, so that
+// no step of a push needs the host.  One per context.
+struct DevCtl {
+  int32_t error;          // sticky TAURUS_ERR_* found on the device
+  int32_t need_count;     // touched vertices that need a slot (NOT_STARTED or EVICTED), this chunk
+  int32_t done_count;     // vertices whose pending count reached zero, this chunk
+  int32_t deficit;        // slots to free by eviction, this chunk
+  int32_t victim_count;   // victims listed so far, this chunk
+  int32_t hs, ns, ev, gs; // touched vertices by state at chunk start
+  int32_t reloaded;       // reloads this chunk
+  int32_t pad0;
+  long long free_top;       // entries on the free-slot stack
+  long long host_free_top;  // entries on the free-host-row stack
+  long long grad_count;     // rows waiting in the graduation buffer
+  unsigned long long sel_prefix;  // radix select: digits fixed so far (high bits)
+  long long sel_k;                // radix select: rank still to resolve inside the prefix bucket
+  unsigned int hist[TAURUS_SEL_BINS];
+  // layer totals
+  long long evictions, reloads, peak_occupancy, hub_messages, total_messages, completed;
+  long long sum_hs, sum_ns, sum_ev, sum_gs, chunks;
+  long long bad_index;      // first out-of-range index seen by a checked kernel (debug aid)
+};
+
+// Everything the per-chunk kernels need, passed by value.
+struct ChunkArgs {
+  // graph
+  const long long* row_ptr;
+  const int32_t* col;
+  const int32_t* din;
+  const uint32_t* mask;     // NULL = every edge propagated
+  // per-vertex state
+  int32_t* pend;
+  uint8_t* state;
+  int32_t* loc;             // pool slot / hub row (>= pool_slots) / host row while EVICTED; -1 = none
+  int32_t* touch;           // chunk epoch of the last touch
+  int32_t* reload_count;
+  // pool
+  float* acc;               // [(pool_slots + hub_count) x Hp]
+  int32_t* owner;           // [pool_slots] vertex in the slot, -1 = free
+  int32_t* free_stack;      // [pool_slots]
+  int32_t* need_list;       // [pool_slots]
+  int32_t* victims;         // [pool_slots]
+  unsigned long long* keys; // [pool_slots]
+  float* host_store;        // device alias of the pinned host rows [host_evict_rows x Hp]
+  int32_t* host_free;       // [host_evict_rows]
+  // graduation buffer
+  long long* grad_ids;
+  float* grad_rows;         // [drain_rows x Hp]
+  int32_t* done_list;       // [drain_rows]
+  // projected rows of this chunk: P at column 0, T at column Hp (SAGE only)
+  const float* PT;
+  int32_t ldpt;
+  const float* bias;        // [Hp]
+  DevCtl* ctl;
+  long long* chunk_log;     // [log_capacity x TAURUS_CK_COLUMNS]
+  long long log_capacity;
+  long long V, pool_slots, hub_count, host_rows, drain_rows;
+  long long src_begin, src_end;
+  int32_t epoch;            // chunk sequence number + 1 within the layer
+  int32_t Hp;               // padded accumulator width (multiple of 4)
+  int32_t mode, act, fanout, checked;
+};
+
+struct taurus_ctx {
+  int device = 0;
+  long long V = 0, E = 0;
+  int L = 0, mode = 0, gemm_mode = 0, flags = 0;
+  int dims[TAURUS_MAX_LAYERS + 1] = {0};
+  int act[TAURUS_MAX_LAYERS] = {0};
+  int fanout[TAURUS_MAX_LAYERS] = {0};
+  int Hmax = 0, Kmax = 0;   // padded maxima over layers
+  unsigned long long seed = 0;
+  long long chunk_sources = 0, pool_slots = 0, hub_count = 0, host_rows = 0, drain_rows = 0;
+  // device graph
+  long long* d_row_ptr = nullptr;
+  int32_t* d_col = nullptr;
+  int32_t* d_din = nullptr;
+  // weights per layer: Wcat is [Kp x Ncat] row-major fp32 (P columns then T columns), bias [Hp]
+  float* d_Wcat[TAURUS_MAX_LAYERS] = {nullptr};
+  float* d_bias[TAURUS_MAX_LAYERS] = {nullptr};
+  void* d_Wtc[TAURUS_MAX_LAYERS] = {nullptr};   // tensor-core operand images of Wcat (layout owned by kernels_gemm_tc.cu)
+  // state
+  int32_t* d_pend = nullptr;
+  uint8_t* d_state = nullptr;
+  int32_t* d_loc = nullptr;
+  int32_t* d_touch = nullptr;
+  int32_t* d_reload = nullptr;
+  uint8_t* d_hub = nullptr;
+  int32_t* d_hub_ids = nullptr;
+  float* d_acc = nullptr;
+  int32_t* d_owner = nullptr;
+  int32_t* d_free_stack = nullptr;
+  int32_t* d_need_list = nullptr;
+  int32_t* d_victims = nullptr;
+  unsigned long long* d_keys = nullptr;
+  float* h_store = nullptr;      // pinned, mapped
+  float* d_store_alias = nullptr;
+  int32_t* d_host_free = nullptr;
+  long long* d_grad_ids = nullptr;
+  float* d_grad_rows = nullptr;
+  int32_t* d_done_list = nullptr;
+  float* d_X = nullptr;          // staged feature chunk [chunk_sources x Kmax]
+  float* d_PT = nullptr;         // projected chunk [chunk_sources x 2 Hmax]
+  long long* d_csc_ptr = nullptr;
+  uint32_t* d_csc_eid = nullptr;
+  uint32_t* d_mask = nullptr;
+  uint32_t* d_mask_cur = nullptr; // d_mask when the current layer is sampled, else NULL (every edge propagated)
+  int32_t* d_vtmp = nullptr;     // [V] scratch for layer_begin
+  int32_t* d_rank_hist = nullptr;
+  DevCtl* d_ctl = nullptr;
+  DevCtl* h_ctl = nullptr;       // pinned
+  long long* d_chunk_log = nullptr;
+  long long log_capacity = 0;
+  // host bookkeeping
+  int layer = -1;
+  long long next_src = 0;
+  long long chunk_seq = 0;
+  std::vector<long long> rank_cum;   // completions by block of 64 completion ranks, prefix sums
+  long long ub_since_drain = 0;      // upper bound on rows in the graduation buffer
+  cudaStream_t last_stream = nullptr;
+  cudaEvent_t order_event = nullptr;
+  long long launches = 0;
+  int timing = 0;
+  cudaEvent_t phase_ev[6] = {nullptr};
+  int sm_count = 148;
+};
+
+static inline int taurus_round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// ---- kernels_state.cu
+void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st);
+void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
+void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);   // plan, select, evict, alloc/reload
+void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // finalise + commit
+void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st);
+void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st);
+void launch_completion_ranks(taurus_ctx* c, cudaStream_t st);                // fills d_rank_hist
+int check_in_degrees(taurus_ctx* c, cudaStream_t st);                        // 0 ok, 1 mismatch
+// ---- kernels_scatter.cu
+void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
+// ---- kernels_gemm_simt.cu
+void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
+// ---- kernels_sample.cu
+int build_in_edge_order(taurus_ctx* c);                                      // csc_ptr, csc_eid
+void launch_sample_mask(taurus_ctx* c, int layer, cudaStream_t st);
+int sampled_edges_of(taurus_ctx* c, int layer, long long dst, long long* out_eids, int32_t* out_src, int cap, int* n);

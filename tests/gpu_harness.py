@@ -1,0 +1,102 @@
+"""Drives libtaurus through its binding for the GPU parity tests and compares with the oracle."""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle
+import taurus_gen as tg
+
+
+def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_features=False, drain_rows=None,
+                host_evict_rows=None, chunk_plan=None, gemm_mode=None):
+    """Runs every layer of workload w on the GPU.  Returns per-layer outputs (float32 [V, d_out]), the ids each
+    chunk completed, stats and chunk logs.  Layer l+1 streams layer l's drained output."""
+    import torch
+    import paper_2607_17374_b200 as tb
+
+    dev = torch.device("cuda:0")
+    V, L = g.V, w.L
+    host_evict = host_evict_rows if host_evict_rows is not None else max(0, V - w.hub_count - w.pool_slots)
+    ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
+                     model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
+                     drain_rows or V, w.gemm_mode if gemm_mode is None else gemm_mode, flags)
+    res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
+    if host_features:
+        feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
+    else:
+        feat = torch.from_numpy(np.ascontiguousarray(x0)).to(dev)
+    stream = torch.cuda.current_stream()
+    for l in range(L):
+        d_out = w.dims[l + 1]
+        dense = torch.zeros((V, d_out), dtype=torch.float32, device=dev)
+        ids_buf = torch.empty(V, dtype=torch.int64, device=dev)
+        ctx.layer_begin(l, stream)
+        if w.fanout[l] > 0:
+            res["masks"].append(ctx.get_edge_mask())
+        else:
+            res["masks"].append(None)
+        per_chunk = []
+        plan = chunk_plan or [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
+        for (s, e) in plan:
+            rc = ctx.push_chunk(s, e, feat[s:e], stream, raise_on_drain_full=False)
+            if rc != 0:   # graduation buffer could overflow: drain, then push again
+                n = ctx.drain_dense(dense, d_out, V, ids_buf)
+                per_chunk.append(("drain", ids_buf[:n].cpu().numpy().copy()))
+                ctx.push_chunk(s, e, feat[s:e], stream)
+            if drain_each_chunk:
+                n = ctx.drain_dense(dense, d_out, V, ids_buf)
+                per_chunk.append(ids_buf[:n].cpu().numpy().copy())
+        n = ctx.drain_dense(dense, d_out, V, ids_buf)
+        if n or not drain_each_chunk:
+            per_chunk.append(("tail", ids_buf[:n].cpu().numpy().copy()))
+        res["stats"].append(ctx.layer_end())
+        res["chunk_log"].append(ctx.get_chunk_log())
+        res["reload_count"].append(ctx.get_vertex_array("reload_count"))
+        res["completed"].append(per_chunk)
+        res["outs"].append(dense.cpu().numpy())
+        feat = dense.cpu().pin_memory() if host_features else dense
+    return res
+
+
+def run_oracle(w, g, model, x0):
+    """Oracle outputs for every layer plus the integer simulation per layer."""
+    inl = oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
+    din, dout = np.diff(inl.ptr), np.diff(g.row_ptr)
+    hub = oracle.hub_set(g.in_degree, w.hub_count)
+    h = x0.astype(np.float64)
+    out = dict(outs=[], sims=[], msets=[], hub=hub)
+    for l in range(w.L):
+        ms = oracle.message_sets(inl, w.fanout[l], w.seed, l)
+        h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l])
+        out["outs"].append(h)
+        out["sims"].append(oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, w.pool_slots))
+        out["msets"].append(ms)
+    return out
+
+
+def row_error(got, ref):
+    """max over rows of ||g_v - r_v||_inf / (||r_v||_inf + 1e-6), and the element-wise figures."""
+    got = got.astype(np.float64)
+    diff = np.abs(got - ref)
+    row = diff.max(axis=1) / (np.abs(ref).max(axis=1) + 1e-6)
+    elem = diff / (np.abs(ref) + 1e-6)
+    return float(row.max()), float(elem.max()), elem
+
+
+def check_accounting(lib_stats, lib_log, lib_reload, sim, completed_chunks=None):
+    st = sim.stats
+    for k_lib, k_or in [("evictions", "evictions"), ("reloads", "reloads"), ("max_reload_count", "max_reload_count"),
+                        ("peak_occupancy", "peak_occupancy"), ("hub_messages", "hub_messages"),
+                        ("total_messages", "total_messages"), ("hub_vertices", "hub_vertices"), ("completed", "completed"),
+                        ("sum_hs", "sum_hs"), ("sum_ns", "sum_ns"), ("sum_ev", "sum_ev"), ("sum_gs", "sum_gs"),
+                        ("free_slots", "free_end")]:
+        assert lib_stats[k_lib] == st[k_or], (k_lib, lib_stats[k_lib], st[k_or])
+    for k in ["hs", "ns", "ev", "gs", "need", "evicted", "reloaded", "completed", "occupancy"]:
+        assert (lib_log[k] == sim.per_chunk[k]).all(), k
+    assert (lib_reload == sim.reload_count).all()
+    hist = np.bincount(np.minimum(sim.reload_count, 16), minlength=17)
+    assert lib_stats["reload_histogram"] == hist.tolist()
+    if completed_chunks is not None:
+        for c, ids in enumerate(completed_chunks):
+            want = np.flatnonzero(sim.complete_chunk == c)
+            assert ids.size == want.size and (np.sort(ids) == want).all(), c
