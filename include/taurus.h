@@ -93,8 +93,11 @@ typedef struct {
   int64_t hub_count;        /* vertices pinned in the hub store: the largest by (in_degree desc, id asc)   */
   const int32_t* fanout;    /* [L] per-layer fanout, 0 = exact; NULL = all exact; at most 64 (host pointer) */
   uint64_t seed;            /* seed of the neighbour-sampling hash                                         */
-  int64_t host_evict_rows;  /* capacity (rows) of the pinned host store for evicted accumulators; 0 = none */
-  int64_t drain_rows;       /* capacity (rows) of the graduation buffer                                    */
+  int64_t host_evict_rows;  /* capacity (rows) of the pinned host store for evicted accumulators; 0 = none.
+                               Must cover the rows evicted at once plus one chunk's victims (a chunk's victims
+                               leave before its reloads hand their host rows back); V - hub_count always suffices */
+  int64_t drain_rows;       /* capacity (rows) of the graduation buffer; must hold the completions of any one
+                               pushed range as bounded by taurus_completion_bound (64-source granularity)  */
   int32_t flags;            /* TAURUS_FLAG_*                                                               */
 } taurus_run;
 

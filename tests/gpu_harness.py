@@ -16,7 +16,9 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
 
     dev = torch.device("cuda:0")
     V, L = g.V, w.L
-    host_evict = host_evict_rows if host_evict_rows is not None else max(0, V - w.hub_count - w.pool_slots)
+    # rows evicted at once, plus the transient of one chunk (victims leave before that chunk's reloads return rows)
+    host_evict = host_evict_rows if host_evict_rows is not None else (
+        0 if w.pool_slots >= V - w.hub_count else V - w.hub_count)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
                      drain_rows or V, w.gemm_mode if gemm_mode is None else gemm_mode, flags)

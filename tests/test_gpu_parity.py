@@ -30,3 +30,166 @@ def test_tiny_config_two_layers_exact():
     _compare_layers(lib, orc, FP32_TOL)
     for l in range(w.L):
         check_accounting(lib["stats"][l], lib["chunk_log"][l], lib["reload_count"][l], orc["sims"][l], lib["completed"][l])
+
+
+def _full_check(w, g=None, bias_scale=0.3, tol=FP32_TOL, **kw):
+    g = g or tg.make_graph(w)
+    model = tg.make_model(w, bias_scale=bias_scale)
+    x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
+    lib = run_library(w, g, model, x0, **kw)
+    orc = run_oracle(w, g, model, x0)
+    _compare_layers(lib, orc, tol)
+    for l in range(w.L):
+        assert orc["sims"][l].rc == 0
+        check_accounting(lib["stats"][l], lib["chunk_log"][l], lib["reload_count"][l], orc["sims"][l], lib["completed"][l])
+    return lib, orc
+
+
+def test_eviction_and_hub_store_small_pool():
+    """Scaled 'large' shape: pool well below the peak active set, hubs pinned; accounting bit-exact."""
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 60_000, chunk=1024)
+    w = replace(w, dims=(128, 256, 64), fanout=(0, 0), pool_slots=16_000, hub_count=60)
+    lib, orc = _full_check(w)
+    assert lib["stats"][0]["evictions"] > 1000 and lib["stats"][0]["max_reload_count"] >= 1
+    assert lib["stats"][0]["hub_messages"] > 0
+
+
+def test_sampled_inference_masks_and_outputs():
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["sampled"], 50_000, chunk=2048)
+    w = replace(w, dims=(128, 256, 256, 47), pool_slots=28_000, hub_count=50)
+    g = tg.make_graph(w)
+    lib, orc = _full_check(w, g)
+    for l in range(w.L):
+        want = np.packbits(orc["msets"][l].prop, bitorder="little")
+        got = lib["masks"][l].view(np.uint8)[:want.size]
+        assert (got == want).all(), l
+    # kept edge lists of single destinations, hubs included
+    ctx = lib["ctx"]
+    order = np.argsort(-g.in_degree)
+    for dst in list(order[:8]) + list(range(0, g.V, 4999)):
+        for l in range(w.L):
+            eids, srcs, n = ctx.get_sampled_edges(l, int(dst))
+            ms = orc["msets"][l]
+            assert n == ms.m[dst]
+            assert (eids == ms.eid[ms.ptr[dst]:ms.ptr[dst + 1]]).all()
+            assert (srcs == ms.src[ms.ptr[dst]:ms.ptr[dst + 1]]).all()
+
+
+def test_gcn_sym_mode_with_eviction():
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["stress"], 40_000, chunk=1024)
+    w = replace(w, dims=(96, 128, 32), gemm_mode=tg.GEMM_FP32, pool_slots=20_000)
+    _full_check(w)
+
+
+def test_mid_shape_ragged_widths_and_tail():
+    """Symmetric graph, F = 100 and out = 47 (padded rows), V not a multiple of the chunk, host-pinned features."""
+    w = tg.scaled(tg.WORKLOADS["mid"], 30_011, chunk=4096)
+    _full_check(w, host_features=True, drain_each_chunk=True)
+
+
+def test_no_drain_until_layer_end_and_uneven_chunks():
+    from dataclasses import replace
+    w = replace(tg.WORKLOADS["tiny"], dims=(64, 32, 8))
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
+    plan, s = [], 0
+    sizes = [1, 1024, 7, 333, 1000, 64]
+    i = 0
+    while s < g.V:
+        e = min(g.V, s + sizes[i % len(sizes)]); plan.append((s, e)); s = e; i += 1
+    lib = run_library(w, g, model, x0, drain_each_chunk=False, chunk_plan=plan)
+    orc = run_oracle(w, g, model, x0)
+    _compare_layers(lib, orc, FP32_TOL)
+    for l in range(w.L):
+        assert lib["stats"][l]["completed"] == g.V
+        ids = np.concatenate([x[1] if isinstance(x, tuple) else x for x in lib["completed"][l]])
+        assert ids.size == g.V and np.unique(ids).size == g.V      # every vertex completes exactly once
+
+
+def test_graph_with_empty_rows_isolated_vertices_and_one_hub():
+    """Degenerate structure: many zero-out-degree sources in a row, isolated vertices, one destination of everything."""
+    from helpers import csr_from_edges
+    from dataclasses import replace
+    V = 3000
+    rng = np.random.default_rng(0)
+    edges = [(int(u), 7) for u in range(0, V, 3)]                        # star into vertex 7
+    edges += [(int(u), int(rng.integers(0, V))) for u in rng.integers(0, V, 4000) if u % 5 == 0]
+    edges += [(100, int(v)) for v in rng.integers(0, V, 2500)]           # one heavy source
+    row_ptr, col = csr_from_edges(V, edges)
+    g = tg.Graph(V, len(edges), row_ptr, col, np.bincount(col, minlength=V).astype(np.int32))
+    for hub_count in (0, 1):
+        w = replace(tg.WORKLOADS["tiny"], V=V, E=g.E, dims=(20, 36, 5), chunk=256, pool_slots=V, hub_count=hub_count)
+        _full_check(w, g)
+
+
+def test_error_paths():
+    import paper_2607_17374_b200 as tb
+    import torch
+    from dataclasses import replace
+    w = replace(tg.WORKLOADS["tiny"], dims=(64, 32))
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    x = torch.from_numpy(tg.features(1, 0, 0, g.V, 64)).cuda()
+    mk = lambda **kw: tb.Context(g.V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self,
+                                 model.bias, model.act, kw.pop("chunk", 1024), kw.pop("pool", g.V), 0, None, 1, 0,
+                                 kw.pop("drain", g.V), 0, 0)
+    # inconsistent in-degrees are rejected at init
+    bad = g.in_degree.copy(); bad[0] += 1
+    with pytest.raises(tb.TaurusError) as ei:
+        tb.Context(g.V, g.E, g.row_ptr, g.col_idx, bad, w.mode, w.dims, model.W_neigh, model.W_self, model.bias, model.act,
+                   1024, g.V, 0, None, 1, 0, g.V, 0, 0)
+    assert ei.value.code == tb.ERROR_CODES["INVALID_ARG"]
+    ctx = mk()
+    with pytest.raises(tb.TaurusError) as ei:      # no layer begun
+        ctx.push_chunk(0, 1024, x[:1024])
+    assert ei.value.code == tb.ERROR_CODES["ORDER"]
+    ctx.layer_begin(0)
+    with pytest.raises(tb.TaurusError) as ei:      # not contiguous
+        ctx.push_chunk(1024, 2048, x[1024:2048])
+    assert ei.value.code == tb.ERROR_CODES["ORDER"]
+    with pytest.raises(tb.TaurusError) as ei:      # too many sources
+        ctx.push_chunk(0, 2048, x[:2048])
+    assert ei.value.code == tb.ERROR_CODES["INVALID_ARG"]
+    ctx.push_chunk(0, 1024, x[:1024])
+    with pytest.raises(tb.TaurusError) as ei:      # layer not finished
+        ctx.layer_end()
+    assert ei.value.code == tb.ERROR_CODES["ORDER"]
+    ctx.destroy()
+    # graduation buffer too small for a chunk: reported before any state change, then drain and retry works
+    ctx = mk(drain=4000)
+    ctx.layer_begin(0)
+    ids = torch.empty(g.V, dtype=torch.int64, device="cuda"); rows = torch.empty((g.V, 32), device="cuda")
+    done, saw_full = 0, False
+    todo = [(s, min(s + 1024, g.V)) for s in range(0, g.V, 1024)]
+    while todo:
+        s, e = todo.pop(0)
+        rc = ctx.push_chunk(s, e, x[s:e], raise_on_drain_full=False)
+        if rc == tb.ERROR_CODES["DRAIN_FULL"]:
+            saw_full = True
+            n = ctx.drain_completed(ids, rows, g.V)
+            done += n
+            if n == 0:          # even an empty buffer cannot take this range: split it
+                assert ctx.completion_bound(s, e) > 4000 and e - s > 64
+                mid = (s + e) // 2
+                todo[:0] = [(s, mid), (mid, e)]
+            else:
+                todo.insert(0, (s, e))
+    done += ctx.drain_completed(ids, rows, g.V)
+    assert saw_full and done == g.V
+    ctx.layer_end()
+    ctx.destroy()
+    # pool too small for one chunk: sticky device-side error
+    ctx = mk(pool=64)
+    ctx.layer_begin(0)
+    ctx.push_chunk(0, 1024, x[:1024])
+    with pytest.raises(tb.TaurusError) as ei:
+        ctx.drain_completed(ids, rows, g.V)
+    assert ei.value.code == tb.ERROR_CODES["POOL_TOO_SMALL"]
+    with pytest.raises(tb.TaurusError) as ei:
+        ctx.push_chunk(1024, 2048, x[1024:2048])
+    assert ei.value.code == tb.ERROR_CODES["POOL_TOO_SMALL"]
+    ctx.destroy()
