@@ -1,0 +1,315 @@
+"""Benchmark of the source-centric broadcast step (libtaurus) on synthetic graphs.
+
+A step is one full pass of the hot path over the workload: every layer, every chunk (copy-in, projection,
+classify, make-room, scatter, finalise, drain).  The metric is propagated edges per second (GTEPS,
+self messages not counted) over the whole step.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mid] [--impl ours|reference]
+
+N > 1 (under torchrun): the path has no exchange step, so every rank runs an independent replica of the
+workload on its own GPU ("replicas only", weak scaling); the value is the sum over ranks / max time.
+--impl reference times the CPU oracle (a deliberately plain program) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import taurus_gen as tg  # noqa: E402
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=3)
+    p.add_argument("--warmup", type=int, default=3)
+    p.add_argument("--workload", default="mid")
+    p.add_argument("--vertices", type=int, default=0, help="scale the workload to this many vertices (0 = full size)")
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--no-e2e", action="store_true")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--simt-gemm", action="store_true", help="use the plain FFMA projection kernel")
+    return p.parse_args()
+
+
+def workload_of(args):
+    w = tg.WORKLOADS[args.workload]
+    if args.vertices:
+        w = tg.scaled(w, args.vertices)
+    return w
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.samples = index, threading.Event(), []
+
+    def run(self):
+        while not self.stop_flag.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                f = [x.strip() for x in out.strip().split(",")]
+                if len(f) >= 6:
+                    self.samples.append(f)
+            except Exception:
+                pass
+            self.stop_flag.wait(0.2)
+
+    def summary(self):
+        if not self.samples:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        mhz = sorted(float(s[0]) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return dict(sm_mhz=mhz[len(mhz) // 2], sm_max_mhz=float(self.samples[0][1]), reasons=reasons, samples=len(mhz))
+
+
+# ----------------------------------------------------------------------------------------------- reference arm / CPU baseline
+
+def oracle_sample(w, g, budget_s=12.0, inl=None):
+    """Times the oracle (as it stands) on a bounded destination sample of layer 0.  Returns (edges/s, info)."""
+    import oracle
+    t0 = time.time()
+    inl = inl or oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
+    t_inl = time.time() - t0
+    ms = oracle.message_sets(inl, w.fanout[0], w.seed, 0)
+    model = tg.make_model(w)
+    rng = np.random.default_rng(0)
+    n_dst = min(g.V, 4096)
+    rate, used, edges, total_t = 0.0, 0, 0, 0.0
+    x = tg.features(w.seed, 0, 0, g.V, w.dims[0]).astype(np.float64)
+    din, dout = np.diff(inl.ptr), np.diff(g.row_ptr)
+    while True:
+        dst = np.sort(rng.choice(g.V, size=n_dst, replace=False)).astype(np.int64)
+        t1 = time.time()
+        oracle.layer_forward(ms, w.mode, din, dout, x, model.W_neigh[0], model.W_self[0], model.bias[0], model.act[0], dst)
+        dt = time.time() - t1
+        e = int(ms.m[dst].sum())
+        edges += e; total_t += dt; used += n_dst
+        rate = e / dt
+        if total_t >= budget_s or n_dst >= g.V:
+            break
+        n_dst = int(min(g.V, max(n_dst * 2, n_dst * (budget_s - total_t) / max(dt, 1e-3) * 0.7)))
+    info = dict(cores=oracle.cores_used(), kind="oracle",
+                sample="layer 0 (%d -> %d), %d sampled destinations, %d in-edges pulled in %.1f s; in-list build %.1f s not counted"
+                       % (w.dims[0], w.dims[1], used, edges, total_t, t_inl))
+    return edges / total_t, info, inl
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workload_of(args)
+    g = tg.make_graph(w)
+    inl = None
+    for _ in range(max(args.warmup, 0) and 1):
+        _, _, inl = oracle_sample(w, g, 2.0, inl)
+    vals, info = [], None
+    t0 = time.time()
+    for _ in range(args.steps):
+        v, info, inl = oracle_sample(w, g, 8.0, inl)
+        vals.append(v)
+    value = float(np.mean(vals)) / 1e9
+    line = dict(impl="reference", metric="edges/sec per GNN layer (GTEPS)", value=value, unit="GTEPS", n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=(time.time() - t0) * 1e3 / max(args.steps, 1),
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=w.name, V=g.V, E=g.E, dims=list(w.dims), l2="inputs larger than L2"),
+                cpu_baseline=dict(value=value, unit="GTEPS", **info),
+                e2e=dict(value=value, unit="GTEPS", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2607_17374_b200 as tb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = workload_of(args)
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    V, L = g.V, w.L
+    chunks = [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
+    drain_rows = V   # badly ordered graphs complete a large share of V in the last chunks
+    host_evict = 0 if w.pool_slots >= V - w.hub_count else V - w.hub_count
+    flags = tb.FLAG_SIMT_GEMM if args.simt_gemm else 0
+    ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
+                     model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags)
+    x_host = torch.empty((V, w.dims[0]), dtype=torch.float32).pin_memory()
+    tg.features(w.seed, 0, 0, V, w.dims[0], out=x_host.numpy())
+    x_dev = x_host.to(dev)
+    dmax = max(w.dims[1:])
+    dense_dev = [torch.zeros(V * dmax, dtype=torch.float32, device=dev) for _ in range(2)]
+    stream = torch.cuda.current_stream()
+    edges_per_layer = []
+
+    def step(feat0, flat, collect_stats=False):
+        """One pass over all layers.  feat0 and the two flat ping-pong buffers live on the device (value) or in
+        pinned host memory (e2e); layer l's output [V, dims[l+1]] is the next layer's feature matrix."""
+        feat = feat0
+        out = None
+        for l in range(L):
+            d_out = w.dims[l + 1]
+            out = flat[l % 2][:V * d_out].view(V, d_out)
+            ctx.layer_begin(l, stream)
+            for (s, e) in chunks:
+                rc = ctx.push_chunk(s, e, feat[s:e], stream, raise_on_drain_full=False)
+                if rc != 0:
+                    ctx.drain_dense(out, d_out, V)
+                    ctx.push_chunk(s, e, feat[s:e], stream)
+            ctx.drain_dense(out, d_out, V)
+            st = ctx.layer_end()
+            if collect_stats:
+                edges_per_layer.append(st["total_messages"])
+            feat = out
+        return out
+
+    # warm-up (also collects the per-layer message counts)
+    barrier()
+    for i in range(max(args.warmup, 1)):
+        step(x_dev, dense_dev, collect_stats=(i == 0))
+    torch.cuda.synchronize()
+    msgs_per_step = int(sum(edges_per_layer))
+
+    # ---- device-resident timing
+    sampler = ClockSampler(local)
+    sampler.start()
+    ctx.set_timing(True)
+    launches0 = ctx.launch_count()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(x_dev, dense_dev)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    ctx.set_timing(False)
+    launches = ctx.launch_count() - launches0
+    sampler.stop_flag.set()
+    sampler.join()
+    phases = ctx.get_phase_ms()   # [pushes, 5]
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+    value = world * msgs_per_step * args.steps / (ms_max * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (the scatter), from the events recorded inside the timed region
+    n_push = len(chunks) * L * args.steps
+    ph = phases[:n_push].reshape(args.steps, L, len(chunks), 5)
+    scatter_ms = ph[..., 3]
+    layer_bytes = []
+    n_src = V
+    for l in range(L):
+        Hp = (w.dims[l + 1] + 3) // 4 * 4
+        layer_bytes.append(edges_per_layer[l] * (12 + 2 * 4 * Hp) + n_src * (4 * Hp + 8))
+    alg_bytes_step = float(sum(layer_bytes))
+    scatter_total_ms = float(scatter_ms.sum()) / args.steps
+    pk = peaks()
+    achieved = alg_bytes_step / (scatter_total_ms * 1e-3) / 1e9
+    roofline = dict(bound="hbm", kernel="scatter_kernel", achieved=achieved, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=achieved / pk["hbm_gbs"], peak_source=pk["source"], traffic=None,
+                    launches_per_step=len(chunks) * L, avg_launch_ms=scatter_total_ms / (len(chunks) * L),
+                    algorithmic_bytes_per_launch=alg_bytes_step / (len(chunks) * L),
+                    per_layer=[dict(layer=l, scatter_ms=float(scatter_ms[:, l].sum()) / args.steps,
+                                    gbs=layer_bytes[l] / (float(scatter_ms[:, l].sum()) / args.steps * 1e-3) / 1e9,
+                                    gteps_scatter_only=edges_per_layer[l] / (float(scatter_ms[:, l].sum()) / args.steps * 1e-3) / 1e9)
+                               for l in range(L)])
+    phase_ms = dict(zip(["copy_in", "projection", "classify_make_room", "scatter", "finalise"],
+                        [float(x) / args.steps for x in ph.sum(axis=(0, 1, 2))]))
+
+    # ---- end to end: host-pinned features in, host-pinned layer outputs out, every step
+    e2e = None
+    if not args.no_e2e:
+        dense_host = [torch.zeros(V * dmax, dtype=torch.float32).pin_memory() for _ in range(2)]
+        step(x_host, dense_host)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step(x_host, dense_host)
+        e1.record(stream)
+        barrier()
+        wall = (time.time() - t0) * 1e3
+        t = torch.tensor([max(e0.elapsed_time(e1), wall)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+        e2e = dict(value=world * msgs_per_step * args.steps / (e2e_ms * 1e-3) / 1e9, unit="GTEPS",
+                   ms_per_step=e2e_ms / args.steps,
+                   h2d_bytes_per_step=int(sum(4 * V * w.dims[l] for l in range(L))),
+                   d2h_bytes_per_step=int(sum(4 * V * w.dims[l + 1] for l in range(L))))
+        del dense_host
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, info, _ = oracle_sample(w, g, 12.0)
+        cpu = dict(value=v / 1e9, unit="GTEPS", **info)
+
+    if rank == 0:
+        line = dict(metric="edges/sec per GNN layer (GTEPS)", value=value, unit="GTEPS", n_gpus=world, steps=args.steps,
+                    warmup=args.warmup, ms_per_step=ms_max / args.steps, higher_is_better=True, scaling="weak",
+                    vs_baseline=None, dtype="f32", data="synthetic",
+                    config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=w.chunk, chunks_per_layer=len(chunks),
+                                pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
+                                mode="sage_mean" if w.mode == 0 else "gcn_sym", messages_per_step=msgs_per_step,
+                                l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
+                                parallelism="replicas only" if world > 1 else "1 gpu",
+                                layer_ms=[float(ph[:, l].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
+                    clocks=sampler.summary(), roofline=roofline, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
+        print(json.dumps(line))
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -206,11 +206,12 @@ int taurus_completion_bound(taurus_ctx* ctx, int64_t src_begin, int64_t src_end,
 /* Kernels launched by this context since init (for launch accounting in benchmarks). */
 int64_t taurus_launch_count(const taurus_ctx* ctx);
 
-/* Device time of the last push's phases in milliseconds, measured with CUDA events when
- * taurus_set_timing(ctx, 1) is on: out[0] copy-in, out[1] projection, out[2] classify..reload,
- * out[3] scatter, out[4] finalise.  Blocking. */
+/* Per-push device times.  taurus_set_timing(ctx, 1) starts a recording window: every later push (up to
+ * 16384) brackets its phases with CUDA events on the push's stream.  taurus_get_phase_ms (blocking) returns,
+ * for each recorded push p, out[p * 5 + k] in milliseconds: k = 0 copy-in, 1 projection, 2 classify..reload,
+ * 3 scatter, 4 finalise; *out_pushes = pushes written (at most capacity_pushes). */
 int taurus_set_timing(taurus_ctx* ctx, int32_t on);
-int taurus_get_phase_ms(taurus_ctx* ctx, float* out5);
+int taurus_get_phase_ms(taurus_ctx* ctx, float* out, int64_t capacity_pushes, int64_t* out_pushes);
 
 void taurus_destroy(taurus_ctx* ctx);
 const char* taurus_strerror(int code);

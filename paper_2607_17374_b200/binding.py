@@ -104,7 +104,7 @@ def load_library():
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
-    lib.taurus_get_phase_ms.argtypes = [vp, vp]
+    lib.taurus_get_phase_ms.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
     lib.taurus_destroy.argtypes = [vp]
     lib.taurus_destroy.restype = None
     lib.taurus_strerror.argtypes = [ctypes.c_int]
@@ -240,10 +240,13 @@ class Context:
     def set_timing(self, on: bool):
         self._check(self._lib.taurus_set_timing(self._h, 1 if on else 0), "taurus_set_timing")
 
-    def get_phase_ms(self):
-        out = (ctypes.c_float * 5)()
-        self._check(self._lib.taurus_get_phase_ms(self._h, out), "taurus_get_phase_ms")
-        return [float(x) for x in out]
+    def get_phase_ms(self, capacity_pushes: int = 16384) -> np.ndarray:
+        """float32 [pushes, 5]: copy-in, projection, classify..reload, scatter, finalise (ms) per recorded push."""
+        out = np.zeros((capacity_pushes, 5), np.float32)
+        n = ctypes.c_int64(0)
+        self._check(self._lib.taurus_get_phase_ms(self._h, out.ctypes.data, capacity_pushes, ctypes.byref(n)),
+                    "taurus_get_phase_ms")
+        return out[:n.value].copy()
 
     def destroy(self):
         if self._h:

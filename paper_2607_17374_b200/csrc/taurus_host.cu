@@ -183,7 +183,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   c->log_capacity = std::max<long long>(1024, 4 * ((V + c->chunk_sources - 1) / c->chunk_sources));
   ALLOC(c->d_chunk_log, (size_t)c->log_capacity * TAURUS_CK_COLUMNS);
   CU(cudaEventCreateWithFlags(&c->order_event, cudaEventDisableTiming));
-  for (auto& e : c->phase_ev) CU(cudaEventCreate(&e));
+  c->rank_cum_cache.assign((size_t)c->L, std::vector<long long>());
   CU(cudaDeviceSynchronize());
   return TAURUS_OK;
 }
@@ -237,21 +237,29 @@ extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_strea
     launch_sample_mask(c, layer, st);
     c->d_mask_cur = c->d_mask;
   }
-  launch_completion_ranks(c, st);
+  if (c->rank_cum_cache[(size_t)layer].empty()) {
+    // completion ranks depend only on the topology and the layer's edge mask: computed once per layer
+    launch_completion_ranks(c, st);
+    CU(cudaGetLastError());
+    const long long nb = (c->V + 63) / 64;
+    std::vector<int32_t> hist((size_t)nb);
+    CU(cudaMemcpyAsync(hist.data(), c->d_rank_hist, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    std::vector<long long>& cum = c->rank_cum_cache[(size_t)layer];
+    cum.assign((size_t)nb + 1, 0);
+    for (long long i = 0; i < nb; ++i) cum[(size_t)i + 1] = cum[(size_t)i] + hist[(size_t)i];
+  }
+  c->rank_cum = &c->rank_cum_cache[(size_t)layer];
   CU(cudaGetLastError());
-  const long long nb = (c->V + 63) / 64;
-  std::vector<int32_t> hist((size_t)nb);
-  CU(cudaMemcpyAsync(hist.data(), c->d_rank_hist, (size_t)nb * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
-  c->rank_cum.assign((size_t)nb + 1, 0);
-  for (long long i = 0; i < nb; ++i) c->rank_cum[(size_t)i + 1] = c->rank_cum[(size_t)i] + hist[(size_t)i];
   return TAURUS_OK;
 }
 
 static long long completion_bound(const taurus_ctx* c, long long s, long long e) {
-  const long long nb = (long long)c->rank_cum.size() - 1;
+  const std::vector<long long>& cum = *c->rank_cum;
+  const long long nb = (long long)cum.size() - 1;
   long long b0 = s / 64, b1 = std::min(nb, (e + 63) / 64);
-  return c->rank_cum[(size_t)b1] - c->rank_cum[(size_t)b0];
+  return cum[(size_t)b1] - cum[(size_t)b0];
 }
 
 extern "C" int taurus_completion_bound(taurus_ctx* c, int64_t src_begin, int64_t src_end, int64_t* out_bound) {
@@ -299,8 +307,15 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   const int l = c->layer;
   const int K = c->dims[l];
   const int n = (int)(src_end - src_begin);
-  const bool timing = c->timing != 0;
-  if (timing) cudaEventRecord(c->phase_ev[0], st);
+  cudaEvent_t* pev = nullptr;
+  if (c->timing && c->timed_pushes < TAURUS_MAX_TIMED_PUSHES) {
+    const size_t need = (size_t)(c->timed_pushes + 1) * 6;
+    while (c->phase_ev.size() < need) { cudaEvent_t e; CU(cudaEventCreate(&e)); c->phase_ev.push_back(e); }
+    pev = &c->phase_ev[(size_t)c->timed_pushes * 6];
+    c->timed_pushes += 1;
+  }
+  const bool timing = pev != nullptr;
+  if (timing) cudaEventRecord(pev[0], st);
   // S1: features to the device
   const float* X = features;
   int ldx = K;
@@ -308,21 +323,21 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
     CU(cudaMemcpyAsync(c->d_X, features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, st));
     X = c->d_X;
   }
-  if (timing) cudaEventRecord(c->phase_ev[1], st);
+  if (timing) cudaEventRecord(pev[1], st);
   ChunkArgs a = make_args(c, src_begin, src_end);
   // S2: projection
   launch_project_simt(c, l, X, ldx, src_begin, n, st);
-  if (timing) cudaEventRecord(c->phase_ev[2], st);
+  if (timing) cudaEventRecord(pev[2], st);
   // S3, S4
   launch_classify(c, a, st);
   launch_make_room(c, a, st);
-  if (timing) cudaEventRecord(c->phase_ev[3], st);
+  if (timing) cudaEventRecord(pev[3], st);
   // S5, S5', S6
   launch_scatter(c, a, st);
-  if (timing) cudaEventRecord(c->phase_ev[4], st);
+  if (timing) cudaEventRecord(pev[4], st);
   // S7
   launch_finalise(c, a, st);
-  if (timing) cudaEventRecord(c->phase_ev[5], st);
+  if (timing) cudaEventRecord(pev[5], st);
   CU(cudaGetLastError());
   c->next_src = src_end;
   c->chunk_seq += 1;
@@ -484,14 +499,18 @@ extern "C" int64_t taurus_launch_count(const taurus_ctx* c) { return c ? c->laun
 extern "C" int taurus_set_timing(taurus_ctx* c, int32_t on) {
   if (!c) return TAURUS_ERR_INVALID_ARG;
   c->timing = on ? 1 : 0;
+  if (on) c->timed_pushes = 0;
   return TAURUS_OK;
 }
 
-extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out5) {
-  if (!c || !out5) return TAURUS_ERR_INVALID_ARG;
-  if (!c->timing || c->chunk_seq == 0) return TAURUS_ERR_ORDER;
+extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out, int64_t capacity_pushes, int64_t* out_pushes) {
+  if (!c || !out || !out_pushes || capacity_pushes < 0) return TAURUS_ERR_INVALID_ARG;
   CU(cudaSetDevice(c->device));
   CU(cudaStreamSynchronize(c->last_stream));
-  for (int i = 0; i < 5; ++i) CU(cudaEventElapsedTime(&out5[i], c->phase_ev[i], c->phase_ev[i + 1]));
+  long long n = std::min<long long>(c->timed_pushes, capacity_pushes);
+  for (long long p = 0; p < n; ++p)
+    for (int i = 0; i < 5; ++i)
+      CU(cudaEventElapsedTime(&out[p * 5 + i], c->phase_ev[(size_t)p * 6 + i], c->phase_ev[(size_t)p * 6 + i + 1]));
+  *out_pushes = n;
   return TAURUS_OK;
 }

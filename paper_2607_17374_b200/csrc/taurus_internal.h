@@ -12,6 +12,7 @@
 #define TAURUS_MAX_LAYERS 16
 #define TAURUS_MAX_DIM 1024
 #define TAURUS_MAX_FANOUT 64
+#define TAURUS_MAX_TIMED_PUSHES 16384
 #define TAURUS_SEL_BITS 11                      // radix-select digit width
 #define TAURUS_SEL_BINS (1 << TAURUS_SEL_BITS)
 #define TAURUS_SEL_PASSES 6                     // 6 x 11 = 66 bits >= the 62-bit (pending, id) key
@@ -133,13 +134,15 @@ struct taurus_ctx {
   int layer = -1;
   long long next_src = 0;
   long long chunk_seq = 0;
-  std::vector<long long> rank_cum;   // completions by block of 64 completion ranks, prefix sums
+  const std::vector<long long>* rank_cum = nullptr;   // current layer: completions by block of 64 completion ranks, prefix sums
   long long ub_since_drain = 0;      // upper bound on rows in the graduation buffer
   cudaStream_t last_stream = nullptr;
   cudaEvent_t order_event = nullptr;
   long long launches = 0;
   int timing = 0;
-  cudaEvent_t phase_ev[6] = {nullptr};
+  std::vector<cudaEvent_t> phase_ev;   // 6 events per timed push, created on demand
+  long long timed_pushes = 0;          // pushes recorded since timing was switched on
+  std::vector<std::vector<long long>> rank_cum_cache;   // per layer: rank_cum computed at the first layer_begin
   int sm_count = 148;
 };
 
