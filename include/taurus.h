@@ -203,6 +203,41 @@ int taurus_get_edge_mask(taurus_ctx* ctx, uint32_t* out_words);
  * (exact when both ends are multiples of 64 or the ends of the graph). */
 int taurus_completion_bound(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, int64_t* out_bound);
 
+/*
+ * (No counterpart in the paper: an addition of this library.)
+ *
+ * Completion counts without any allocation.  Some callers cannot let a library allocate device memory
+ * while they run: a serving process whose framework allocator already owns the whole GPU (cudaMalloc
+ * would fail or fragment it), a real-time loop in which cudaMalloc / cudaFree would stall every stream of
+ * the device, or an embedder whose memory is accounted per request.  For them this entry point computes
+ * what taurus_layer_begin computes for taurus_completion_bound, but with its scratch (one int32 per
+ * vertex) in a static device array inside the library image instead of memory obtained at run time.
+ * It calls no cudaMalloc, cudaFree, cudaHostAlloc or other allocating routine.
+ *
+ * out_counts[b], b in [0, ceil(V / 64)), receives the number of vertices whose completion rank
+ * max(v, largest source among the propagated in-edges of v) lies in [64 b, 64 b + 64): the vertices a
+ * push of those 64 sources completes (Sect. 3.8, c(v)).  edge_mask is the layer's propagated-edge mask in
+ * the format of taurus_get_edge_mask, or NULL when every edge is propagated.  *out_bad_index is set to 1
+ * if a destination outside [0, V) was met (such edges are skipped), else 0.
+ *
+ * Arguments: row_ptr [V+1], col_idx [E], edge_mask [ceil(E/32)] or NULL, out_counts [ceil(V/64)] and
+ * out_bad_index [1] are DEVICE pointers owned by the caller; the work is enqueued on cuda_stream
+ * (a cudaStream_t, NULL = default stream) on the current device and the call does not wait for it.
+ *
+ * Limits and sharing: V may not exceed TAURUS_NOALLOC_MAX_VERTICES (else TAURUS_ERR_UNSUPPORTED, nothing
+ * is enqueued).  The scratch array (16 MiB) is part of the library image: every GPU on which the library
+ * is loaded keeps it until the process exits.  All calls on a device share it and it keeps the previous
+ * call's contents; each call rewrites the entries it reads, so calls issued one after another on one
+ * stream are independent, but two calls whose kernels overlap on the GPU (different streams, or different
+ * host threads) race on it and must be serialised by the caller.  The first call on each device looks up
+ * the array's device address (cudaGetSymbolAddress, with that device current); make that first call
+ * before starting any stream capture.
+ */
+#define TAURUS_NOALLOC_MAX_VERTICES (4 * 1024 * 1024)
+int taurus_completion_counts_noalloc(int64_t V, int64_t E, const int64_t* row_ptr, const int32_t* col_idx,
+                                     const uint32_t* edge_mask, int32_t* out_counts, int32_t* out_bad_index,
+                                     void* cuda_stream);
+
 /* Kernels launched by this context since init (for launch accounting in benchmarks). */
 int64_t taurus_launch_count(const taurus_ctx* ctx);
 

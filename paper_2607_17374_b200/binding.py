@@ -75,7 +75,9 @@ EXPORTS = [
     "taurus_layer_end", "taurus_get_stats", "taurus_get_chunk_log", "taurus_get_vertex_array",
     "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count",
     "taurus_set_timing", "taurus_get_phase_ms", "taurus_destroy", "taurus_strerror", "taurus_last_cuda_error",
+    "taurus_completion_counts_noalloc",
 ]
+NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
 
 def load_library():
@@ -101,6 +103,7 @@ def load_library():
     lib.taurus_get_sampled_edges.argtypes = [vp, i32, i64, vp, vp, i32, ctypes.POINTER(i32)]
     lib.taurus_get_edge_mask.argtypes = [vp, vp]
     lib.taurus_completion_bound.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
+    lib.taurus_completion_counts_noalloc.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -135,6 +138,14 @@ def _stream(s) -> Optional[int]:
     if s is None:
         return None
     return s if isinstance(s, int) else s.cuda_stream
+
+
+def completion_counts_noalloc(V: int, E: int, row_ptr, col_idx, edge_mask, out_counts, out_bad_index, stream=None) -> int:
+    """taurus_completion_counts_noalloc: per-64-source completion counts computed with the library's static
+    scratch array, for callers that cannot allocate device memory.  Every array argument is a device tensor or
+    address owned by the caller; returns the C return code (0 = enqueued)."""
+    return int(load_library().taurus_completion_counts_noalloc(V, E, _ptr(row_ptr), _ptr(col_idx), _ptr(edge_mask),
+                                                               _ptr(out_counts), _ptr(out_bad_index), _stream(stream)))
 
 
 class Context:
