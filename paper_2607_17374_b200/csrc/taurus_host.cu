@@ -63,7 +63,8 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaSetDevice(c->device);
   cudaDeviceSynchronize();
   cudaFree(c->d_row_ptr); cudaFree(c->d_col); cudaFree(c->d_din);
-  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) { cudaFree(c->d_Wcat[l]); cudaFree(c->d_bias[l]); cudaFree(c->d_Wtc[l]); }
+  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) { cudaFree(c->d_Wcat[l]); cudaFree(c->d_bias[l]); }
+  free_tc_weights(c);
   cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
   cudaFree(c->d_need_list); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
@@ -150,6 +151,11 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     ALLOC(c->d_Wcat[l], cat.size()); ALLOC(c->d_bias[l], b.size());
     CU(cudaMemcpy(c->d_Wcat[l], cat.data(), cat.size() * sizeof(float), cudaMemcpyHostToDevice));
     CU(cudaMemcpy(c->d_bias[l], b.data(), b.size() * sizeof(float), cudaMemcpyHostToDevice));
+    if (!(c->flags & TAURUS_FLAG_SIMT_GEMM)) {
+      int rc = prepare_tc_weights(c, l, cat, K, N);
+      if (rc == TAURUS_ERR_NOMEM) return rc;
+      if (rc != TAURUS_OK) { cudaGetLastError(); free_tc_weights(c); }   // no tensor-map support: the FFMA kernel is used
+    }
   }
 
   // per-vertex state
@@ -326,7 +332,12 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   if (timing) cudaEventRecord(pev[1], st);
   ChunkArgs a = make_args(c, src_begin, src_end);
   // S2: projection
-  launch_project_simt(c, l, X, ldx, src_begin, n, st);
+  if (project_tc_usable(c, l, X, ldx)) {
+    int rc = launch_project_tc(c, l, X, ldx, src_begin, n, st);
+    if (rc) return rc;
+  } else {
+    launch_project_simt(c, l, X, ldx, src_begin, n, st);
+  }
   if (timing) cudaEventRecord(pev[2], st);
   // S3, S4
   launch_classify(c, a, st);

@@ -97,7 +97,7 @@ struct taurus_ctx {
   // weights per layer: Wcat is [Kp x Ncat] row-major fp32 (P columns then T columns), bias [Hp]
   float* d_Wcat[TAURUS_MAX_LAYERS] = {nullptr};
   float* d_bias[TAURUS_MAX_LAYERS] = {nullptr};
-  void* d_Wtc[TAURUS_MAX_LAYERS] = {nullptr};   // tensor-core operand images of Wcat (layout owned by kernels_gemm_tc.cu)
+  void* tc_image[TAURUS_MAX_LAYERS] = {nullptr};   // tensor-core operand images of Wcat (owned by kernels_gemm_tc.cu)
   // state
   int32_t* d_pend = nullptr;
   uint8_t* d_state = nullptr;
@@ -161,6 +161,11 @@ int check_in_degrees(taurus_ctx* c, cudaStream_t st);                        // 
 void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_gemm_simt.cu
 void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
+// ---- kernels_gemm_tc.cu
+int prepare_tc_weights(taurus_ctx* c, int layer, const std::vector<float>& cat, int K, int N);
+void free_tc_weights(taurus_ctx* c);
+bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);
+int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
 // ---- kernels_sample.cu
 int build_in_edge_order(taurus_ctx* c);                                      // csc_ptr, csc_eid
 void launch_sample_mask(taurus_ctx* c, int layer, cudaStream_t st);
