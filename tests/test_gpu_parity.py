@@ -193,3 +193,29 @@ def test_error_paths():
         ctx.push_chunk(1024, 2048, x[1024:2048])
     assert ei.value.code == tb.ERROR_CODES["POOL_TOO_SMALL"]
     ctx.destroy()
+
+
+@pytest.mark.parametrize("dims", [(64, 64, 16), (100, 256, 47), (512, 256, 256), (36, 20, 12)])
+def test_projection_kernels_agree_with_the_oracle(dims):
+    """The three projection paths on the same chunk stream: fp32 tensor-core (3 x TF32), bf16 tensor-core, FFMA."""
+    import paper_2607_17374_b200 as tb
+    from dataclasses import replace
+    w = replace(tg.scaled(tg.WORKLOADS["mid"], 9_000, chunk=1000), dims=dims, fanout=(0,) * (len(dims) - 1))
+    g = tg.make_graph(w)
+    model = tg.make_model(w, bias_scale=0.3)
+    x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
+    orc = run_oracle(w, g, model, x0)
+    for name, kw, tol in [("fp32 tensor core", dict(), FP32_TOL), ("ffma", dict(flags=tb.FLAG_SIMT_GEMM), FP32_TOL),
+                          # bf16 operands: the 2e-2 bound is stated for the configs' widths; a 12-20 wide output row has
+                          # too small an infinity norm for it, so the narrow case only guards against gross errors
+                          ("bf16 tensor core", dict(gemm_mode=tg.GEMM_BF16), BF16_TOL if min(dims[1:]) >= 16 else 0.1)]:
+        lib = run_library(w, g, model, x0, drain_each_chunk=False, **kw)
+        print(name)
+        _compare_layers(lib, orc, tol)
+
+
+def test_gcn_bf16_mode():
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["stress"], 30_000, chunk=2048)
+    w = replace(w, dims=(512, 256, 256), pool_slots=30_000)
+    _full_check(w, tol=BF16_TOL)
