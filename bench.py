@@ -39,6 +39,7 @@ def parse_args():
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--simt-gemm", action="store_true", help="use the plain FFMA projection kernel")
+    p.add_argument("--no-grouping", action="store_true", help="CSR-order scatter for every chunk")
     return p.parse_args()
 
 
@@ -170,7 +171,7 @@ def run_ours(args):
     chunks = [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
     drain_rows = V   # badly ordered graphs complete a large share of V in the last chunks
     host_evict = 0 if w.pool_slots >= V - w.hub_count else V - w.hub_count
-    flags = tb.FLAG_SIMT_GEMM if args.simt_gemm else 0
+    flags = (tb.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (tb.FLAG_NO_GROUPING if args.no_grouping else 0)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags)
     x_host = torch.empty((V, w.dims[0]), dtype=torch.float32).pin_memory()

@@ -103,7 +103,8 @@ typedef struct {
 
 enum {
   TAURUS_FLAG_CHECKED = 1,      /* bounds-check every slot / vertex index on the device (slower; sets ERR_INTERNAL) */
-  TAURUS_FLAG_SIMT_GEMM = 2     /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */
+  TAURUS_FLAG_SIMT_GEMM = 2,    /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */
+  TAURUS_FLAG_NO_GROUPING = 4   /* do not build the destination-grouped edge order: every chunk takes the CSR-order kernels */
 };
 
 /* Integer accounting of one layer pass (Sect. 4.4-4.7 report these quantities). */

@@ -1,6 +1,7 @@
-// Scatter step (S5, S5', head of S6): push each projected source row along the chunk's propagated
-// CSR out-edges into the destination's accumulator row with vector fp32 reductions, count down the
-// destination's pending messages, and list the destinations whose count reached zero
+// Scatter step (S5, S5'): push each projected source row along the chunk's propagated CSR out-edges into
+// the destination's accumulator row with vector fp32 reductions and count down the destination's pending
+// messages with integer reductions (no atomic returns a value; completed destinations are compacted by the
+// next kernel)
 // (Sect. 3.1 broadcast; Sect. 3.4 pending counts; Sect. 3.6 graduation trigger).
 //
 // Work is cut by EDGES, not by sources: a warp owns a run of consecutive 32-edge tiles of the chunk's CSR
@@ -98,23 +99,13 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
       }
       // pending count and slot of this lane's destination
       int l = -1;
-      bool done = false;
       if (v >= 0) {
         l = a.loc[v];
         if (l < 0 || l >= loc_limit) { bad = 1; l = -1; }
         else {
-          int old = atomicSub(&a.pend[v], 1);
-          done = old == 1;
-          if (old < 1) bad = 1;
+          atomicAdd(&a.pend[v], -1);   // result unused: a reduction; completion is read after the kernel
           if (!self_run) { msgs++; if (l >= a.pool_slots) hub_msgs++; }
         }
-      }
-      unsigned dm = __ballot_sync(FULL, done);
-      if (dm) {
-        int leader = __ffs(dm) - 1, idx = 0;
-        if (lane == leader) idx = atomicAdd(&ctl->done_count, __popc(dm));
-        idx = __shfl_sync(FULL, idx, leader) + __popc(dm & ((1u << lane) - 1));
-        if (done) { if (idx < a.drain_rows) a.done_list[idx] = v; else bad = 1; }
       }
       const unsigned live = __ballot_sync(FULL, l >= 0);
       // accumulate: EPS items per step, LPE lanes per item

@@ -82,11 +82,12 @@ __global__ void classify_kernel(ChunkArgs a) {
     } else if (i < total) {
       v = (int)(a.src_begin + (i - ne));
     }
-    bool need = false;
+    bool need = false, first = false;
     if (v >= a.V) { bad = 1; v = -1; }
     if (v >= 0) {
       int old = atomicMax(&a.touch[v], a.epoch);
       if (old != a.epoch) {   // first touch in this chunk
+        first = true;
         int l = a.loc[v];
         int s = a.state[v];
         if (l >= a.pool_slots) {          // hub store: pinned, never takes a pool slot
@@ -109,6 +110,13 @@ __global__ void classify_kernel(ChunkArgs a) {
       if (lane_id() == leader) idx = atomicAdd(&ctl->need_count, __popc(m));
       idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
       if (need && idx < a.pool_slots) a.need_list[idx] = v;
+    }
+    m = __ballot_sync(FULL, first);
+    if (m) {
+      int leader = __ffs(m) - 1, idx = 0;
+      if (lane_id() == leader) idx = atomicAdd(&ctl->touched_count, __popc(m));
+      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
+      if (first) { if (idx < a.touched_capacity) a.touched_list[idx] = v; else bad = 1; }
     }
   }
   for (int o = 16; o; o >>= 1) {
@@ -331,7 +339,38 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
 }
 
 // ------------------------------------------------------------------------------------------------ finalise (S6 tail, S7)
-// One warp per completed vertex (listed by the scatter kernel when its pending count reached zero):
+// S6: compact the touched vertices whose pending count reached zero (warp ballot + prefix) into done_list.
+// The scatter only decrements the counts with fire-and-forget reductions; completion is read here, after
+// the kernel boundary, when every reduction of the chunk has landed.
+__global__ void compact_done_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const int n = ctl->touched_count;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  int bad = 0;
+  for (long long base = warp0 * 32; base < n; base += warps * 32) {
+    long long i = base + lane_id();
+    int v = -1;
+    bool done = false;
+    if (i < n) {
+      v = a.touched_list[i];
+      int p = a.pend[v];
+      done = p == 0;
+      if (p < 0) bad = 1;
+    }
+    unsigned m = __ballot_sync(FULL, done);
+    if (m) {
+      int leader = __ffs(m) - 1, idx = 0;
+      if (lane_id() == leader) idx = atomicAdd(&ctl->done_count, __popc(m));
+      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
+      if (done) { if (idx < a.drain_rows) a.done_list[idx] = v; else bad = 1; }
+    }
+  }
+  if (__any_sync(FULL, bad) && lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+}
+
+// One warp per completed vertex (listed by compact_done_kernel):
 // out = act(c_in(v) * acc) into the graduation buffer (Sect. 3.6); the slot is released.
 __global__ void finalise_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
@@ -392,13 +431,14 @@ __global__ void commit_kernel(ChunkArgs a) {
   ctl->grad_count += ctl->done_count;
   ctl->chunks = c + 1;
   ctl->hs = ctl->ns = ctl->ev = ctl->gs = 0;
-  ctl->need_count = 0; ctl->done_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;
+  ctl->need_count = 0; ctl->done_count = 0; ctl->touched_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;
 }
 
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  compact_done_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
   finalise_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
   commit_kernel<<<1, 32, 0, st>>>(a);
-  c->launches += 2;
+  c->launches += 3;
 }
 
 // ------------------------------------------------------------------------------------------------ drain helpers
@@ -514,4 +554,29 @@ int check_in_degrees(taurus_ctx* c, cudaStream_t st) {
   cudaFree(d_flag);
   c->launches += 2;
   return flag;
+}
+
+// ------------------------------------------------------------------------------------------------ sizing
+__global__ void window_edges_kernel(long long V, long long window, const long long* row_ptr, unsigned long long* out_max) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  unsigned long long mx = 0;
+  for (long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x; u < V; u += stride) {
+    long long e = u + window < V ? u + window : V;
+    unsigned long long n = (unsigned long long)(row_ptr[e] - row_ptr[u]);
+    if (n > mx) mx = n;
+  }
+  for (int o = 16; o; o >>= 1) { unsigned long long t = __shfl_xor_sync(FULL, mx, o); if (t > mx) mx = t; }
+  if (lane_id() == 0 && mx) atomicMax(out_max, mx);
+}
+
+long long max_window_edges(taurus_ctx* c) {
+  unsigned long long* d = nullptr;
+  if (cudaMalloc(&d, sizeof(unsigned long long)) != cudaSuccess) return -1;
+  cudaMemset(d, 0, sizeof(unsigned long long));
+  window_edges_kernel<<<c->sm_count * 8, 256>>>(c->V, c->chunk_sources, c->d_row_ptr, d);
+  unsigned long long h = 0;
+  cudaError_t e = cudaMemcpy(&h, d, sizeof(h), cudaMemcpyDeviceToHost);
+  cudaFree(d);
+  c->launches += 1;
+  return e == cudaSuccess ? (long long)h : -1;
 }

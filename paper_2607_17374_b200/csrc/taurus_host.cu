@@ -67,10 +67,11 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   free_tc_weights(c);
   cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
-  cudaFree(c->d_need_list); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
+  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X); cudaFree(c->d_PT);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
+  cudaFree(c->d_gdst); cudaFree(c->d_gsrc); cudaFree(c->d_geid); cudaFree(c->d_gmask);
   cudaFree(c->d_ctl); cudaFree(c->d_chunk_log);
   if (c->h_ctl) cudaFreeHost(c->h_ctl);
   if (c->order_event) cudaEventDestroy(c->order_event);
@@ -163,6 +164,13 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   ALLOC(c->d_rank_hist, (V + 63) / 64);
   // pool, hub store
   ALLOC(c->d_acc, (size_t)(c->pool_slots + c->hub_count) * c->Hmax);
+  {
+    // a push of at most chunk_sources sources touches at most its edges plus its own vertices
+    long long max_edges = max_window_edges(c);
+    if (max_edges < 0) return TAURUS_ERR_CUDA;
+    c->touched_capacity = std::min<long long>(V, max_edges + c->chunk_sources);
+    ALLOC(c->d_touched_list, c->touched_capacity);
+  }
   ALLOC(c->d_owner, c->pool_slots); ALLOC(c->d_free_stack, c->pool_slots); ALLOC(c->d_need_list, c->pool_slots);
   if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); }
   ALLOC(c->d_host_free, c->host_rows);
@@ -180,6 +188,12 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     int rc = build_in_edge_order(c);
     if (rc) { cuda_ok(cudaGetLastError(), "build_in_edge_order"); return rc; }
     ALLOC(c->d_mask, (E + 31) / 32);
+  }
+  // destination-grouped edge order of the chunk grid
+  if (!(c->flags & TAURUS_FLAG_NO_GROUPING)) {
+    int rc = build_grouped_order(c, any_sampled);
+    if (rc) { cuda_ok(cudaGetLastError(), "build_grouped_order"); return rc; }
+    if (any_sampled) ALLOC(c->d_gmask, (E + 31) / 32);
   }
   // control
   ALLOC(c->d_ctl, 1);
@@ -242,6 +256,7 @@ extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_strea
   if (c->fanout[layer] > 0) {
     launch_sample_mask(c, layer, st);
     c->d_mask_cur = c->d_mask;
+    if (c->d_gdst) launch_group_mask(c, st);
   }
   if (c->rank_cum_cache[(size_t)layer].empty()) {
     // completion ranks depend only on the topology and the layer's edge mask: computed once per layer
@@ -281,6 +296,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.row_ptr = c->d_row_ptr; a.col = c->d_col; a.din = c->d_din; a.mask = c->d_mask_cur;
   a.pend = c->d_pend; a.state = c->d_state; a.loc = c->d_loc; a.touch = c->d_touch; a.reload_count = c->d_reload;
   a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list;
+  a.touched_list = c->d_touched_list; a.touched_capacity = c->touched_capacity;
   a.victims = c->d_victims; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
   a.Hp = taurus_round_up(c->dims[l + 1], 4);
@@ -340,11 +356,13 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   }
   if (timing) cudaEventRecord(pev[2], st);
   // S3, S4
-  launch_classify(c, a, st);
+  const bool grouped = c->d_gdst != nullptr && src_begin % c->chunk_sources == 0 &&
+                       src_end == std::min<long long>(c->V, src_begin + c->chunk_sources);
+  if (grouped) launch_classify_grouped(c, a, st); else launch_classify(c, a, st);
   launch_make_room(c, a, st);
   if (timing) cudaEventRecord(pev[3], st);
   // S5, S5', S6
-  launch_scatter(c, a, st);
+  if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
   if (timing) cudaEventRecord(pev[4], st);
   // S7
   launch_finalise(c, a, st);

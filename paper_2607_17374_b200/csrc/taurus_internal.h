@@ -23,11 +23,11 @@ struct DevCtl {
   int32_t error;          // sticky TAURUS_ERR_* found on the device
   int32_t need_count;     // touched vertices that need a slot (NOT_STARTED or EVICTED), this chunk
   int32_t done_count;     // vertices whose pending count reached zero, this chunk
+  int32_t touched_count;  // vertices touched by this chunk (first touches), this chunk
   int32_t deficit;        // slots to free by eviction, this chunk
   int32_t victim_count;   // victims listed so far, this chunk
   int32_t hs, ns, ev, gs; // touched vertices by state at chunk start
   int32_t reloaded;       // reloads this chunk
-  int32_t pad0;
   long long free_top;       // entries on the free-slot stack
   long long host_free_top;  // entries on the free-host-row stack
   long long grad_count;     // rows waiting in the graduation buffer
@@ -58,6 +58,8 @@ struct ChunkArgs {
   int32_t* owner;           // [pool_slots] vertex in the slot, -1 = free
   int32_t* free_stack;      // [pool_slots]
   int32_t* need_list;       // [pool_slots]
+  int32_t* touched_list;    // [touched_capacity] every vertex the chunk touches, listed at its first touch
+  long long touched_capacity;
   int32_t* victims;         // [pool_slots]
   unsigned long long* keys; // [pool_slots]
   float* host_store;        // device alias of the pinned host rows [host_evict_rows x Hp]
@@ -110,6 +112,8 @@ struct taurus_ctx {
   int32_t* d_owner = nullptr;
   int32_t* d_free_stack = nullptr;
   int32_t* d_need_list = nullptr;
+  int32_t* d_touched_list = nullptr;
+  long long touched_capacity = 0;
   int32_t* d_victims = nullptr;
   unsigned long long* d_keys = nullptr;
   float* h_store = nullptr;      // pinned, mapped
@@ -123,6 +127,10 @@ struct taurus_ctx {
   long long* d_csc_ptr = nullptr;
   uint32_t* d_csc_eid = nullptr;
   uint32_t* d_mask = nullptr;
+  int32_t* d_gdst = nullptr;      // grouped order (per grid chunk, edges sorted by destination): destinations
+  int32_t* d_gsrc = nullptr;      //   sources
+  uint32_t* d_geid = nullptr;     //   CSR edge indices (kept only when some layer is sampled)
+  uint32_t* d_gmask = nullptr;    // current layer's edge mask in grouped order
   uint32_t* d_mask_cur = nullptr; // d_mask when the current layer is sampled, else NULL (every edge propagated)
   int32_t* d_vtmp = nullptr;     // [V] scratch for layer_begin
   int32_t* d_rank_hist = nullptr;
@@ -156,6 +164,7 @@ void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // 
 void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st);
 void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st);
 void launch_completion_ranks(taurus_ctx* c, cudaStream_t st);                // fills d_rank_hist
+long long max_window_edges(taurus_ctx* c);                                  // most edges of any chunk_sources consecutive sources
 int check_in_degrees(taurus_ctx* c, cudaStream_t st);                        // 0 ok, 1 mismatch
 // ---- kernels_scatter.cu
 void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
@@ -166,6 +175,11 @@ int prepare_tc_weights(taurus_ctx* c, int layer, const std::vector<float>& cat, 
 void free_tc_weights(taurus_ctx* c);
 bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);
 int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
+// ---- kernels_group.cu
+int build_grouped_order(taurus_ctx* c, bool keep_edge_ids);
+void launch_group_mask(taurus_ctx* c, cudaStream_t st);
+void launch_classify_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
+void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_sample.cu
 int build_in_edge_order(taurus_ctx* c);                                      // csc_ptr, csc_eid
 void launch_sample_mask(taurus_ctx* c, int layer, cudaStream_t st);
