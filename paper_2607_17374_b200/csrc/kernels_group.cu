@@ -105,22 +105,28 @@ void launch_group_mask(taurus_ctx* c, cudaStream_t st) {
 // ------------------------------------------------------------------------------------------------ classify (S3)
 // Same decisions as the CSR-order classify; adjacent duplicates of a destination are skipped before the
 // epoch stamp is touched (exact layers), and the stamp is tested before the atomic.
-__global__ void classify_grouped_kernel(ChunkArgs a, const int32_t* __restrict__ g_dst, const uint32_t* __restrict__ gmask) {
+__global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, const int32_t* __restrict__ g_dst, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
+  // list appends are aggregated per block: single-address atomics are the throughput limit of this kernel
+  __shared__ int s_cnt[2][2][8];   // [parity][need / touched][warp]
+  __shared__ int s_base[2][2];
   const long long e0 = a.row_ptr[a.src_begin], e1 = a.row_ptr[a.src_end];
   const long long ne = e1 - e0, total = ne + (a.src_end - a.src_begin);
-  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  int hs = 0, ns = 0, ev = 0, gs = 0, bad = 0;
-  for (long long base = warp0 * 32; base < total; base += warps * 32) {
-    long long i = base + lane_id();
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const int warp = threadIdx.x >> 5;
+  int hs = 0, ns = 0, ev = 0, gs = 0, bad = 0, par = 0;
+  for (long long base = (long long)blockIdx.x * blockDim.x; base < total; base += stride, par ^= 1) {
+    long long i = base + threadIdx.x;
     int v = -1;
+    bool sole = false;   // this item is the only one that can touch v in this chunk: no atomic needed
     if (i < ne) {
       long long e = e0 + i;
       if (gmask == nullptr) {
         v = g_dst[e];
-        if (i > 0 && g_dst[e - 1] == v) v = -1;   // same destination as the previous edge: already handled
+        if (i > 0 && g_dst[e - 1] == v) v = -1;   // not the first edge of its destination group
+        // only a vertex of the chunk's own range can also be touched by its self item
+        sole = v < a.src_begin || v >= a.src_end;
       } else if ((gmask[e >> 5] >> (e & 31)) & 1u) {
         v = g_dst[e];
       }
@@ -129,8 +135,10 @@ __global__ void classify_grouped_kernel(ChunkArgs a, const int32_t* __restrict__
     }
     bool need = false, first = false;
     if (v >= a.V) { bad = 1; v = -1; }
-    if (v >= 0 && a.touch[v] != a.epoch) {
-      int old = atomicMax(&a.touch[v], a.epoch);
+    if (v >= 0 && (sole || a.touch[v] != a.epoch)) {
+      int old;
+      if (sole) { old = 0; a.touch[v] = a.epoch; }
+      else old = atomicMax(&a.touch[v], a.epoch);
       if (old != a.epoch) {
         first = true;
         int l = a.loc[v];
@@ -149,19 +157,22 @@ __global__ void classify_grouped_kernel(ChunkArgs a, const int32_t* __restrict__
         }
       }
     }
-    unsigned m = __ballot_sync(FULL, need);
-    if (m) {
-      int leader = __ffs(m) - 1, idx = 0;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->need_count, __popc(m));
-      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (need && idx < a.pool_slots) a.need_list[idx] = v;
+    const unsigned mn = __ballot_sync(FULL, need), mt = __ballot_sync(FULL, first);
+    if (lane_id() == 0) { s_cnt[par][0][warp] = __popc(mn); s_cnt[par][1][warp] = __popc(mt); }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+      int sum = 0;
+      for (int w = 0; w < 8; ++w) { int c = s_cnt[par][threadIdx.x][w]; s_cnt[par][threadIdx.x][w] = sum; sum += c; }
+      s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &ctl->need_count : &ctl->touched_count, sum) : 0;
     }
-    m = __ballot_sync(FULL, first);
-    if (m) {
-      int leader = __ffs(m) - 1, idx = 0;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->touched_count, __popc(m));
-      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (first) { if (idx < a.touched_capacity) a.touched_list[idx] = v; else bad = 1; }
+    __syncthreads();
+    if (need) {
+      int idx = s_base[par][0] + s_cnt[par][0][warp] + __popc(mn & ((1u << lane_id()) - 1));
+      if (idx < a.pool_slots) a.need_list[idx] = v;
+    }
+    if (first) {
+      int idx = s_base[par][1] + s_cnt[par][1][warp] + __popc(mt & ((1u << lane_id()) - 1));
+      if (idx < a.touched_capacity) a.touched_list[idx] = v; else bad = 1;
     }
   }
   for (int o = 16; o; o >>= 1) {

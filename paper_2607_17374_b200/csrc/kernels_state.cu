@@ -21,12 +21,12 @@ static __device__ __forceinline__ int messages_of(int din, int fanout) {
 
 // ------------------------------------------------------------------------------------------------ layer reset
 __global__ void reset_vertices_kernel(long long V, const int32_t* din, int fanout, int32_t* pend, uint8_t* state,
-                                      int32_t* loc, int32_t* touch, int32_t* reload) {
+                                      int32_t* loc, int32_t* touch, int32_t* reload, int direct) {
   long long stride = (long long)gridDim.x * blockDim.x;
   for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
     pend[v] = messages_of(din[v], fanout) + 1;
     state[v] = TAURUS_NOT_STARTED;
-    loc[v] = -1;
+    loc[v] = direct ? (int32_t)v : -1;
     touch[v] = 0;
     reload[v] = 0;
   }
@@ -52,7 +52,7 @@ void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st) {
   int blocks = c->sm_count * 8;
   cudaMemsetAsync(c->d_ctl, 0, sizeof(DevCtl), st);
   reset_vertices_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_din, c->fanout[layer], c->d_pend, c->d_state, c->d_loc,
-                                                c->d_touch, c->d_reload);
+                                                c->d_touch, c->d_reload, c->pool_slots >= c->V ? 1 : 0);
   reset_pool_kernel<<<blocks, 256, 0, st>>>(c->pool_slots, c->host_rows, c->hub_count, c->d_hub_ids, c->d_loc, c->d_owner,
                                             c->d_free_stack, c->d_host_free, c->d_ctl);
   int Hp = taurus_round_up(c->dims[layer + 1], 4);
@@ -65,16 +65,19 @@ void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st) {
 // One item per CSR edge of the chunk and one per chunk vertex (its self message).  The first item that
 // touches a vertex in this chunk (atomicMax on the epoch stamp) classifies it by its state at chunk start.
 // loc encoding: -1 none, [0, pool_slots) pool slot, >= pool_slots hub row, <= -2 host row (-2 - loc).
-__global__ void classify_kernel(ChunkArgs a) {
+__global__ void __launch_bounds__(256) classify_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
+  // list appends are aggregated per block: single-address atomics are the throughput limit of this kernel
+  __shared__ int s_cnt[2][2][8];   // [parity][need / touched][warp]
+  __shared__ int s_base[2][2];
   const long long e0 = a.row_ptr[a.src_begin], e1 = a.row_ptr[a.src_end];
   const long long ne = e1 - e0, total = ne + (a.src_end - a.src_begin);
-  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  int hs = 0, ns = 0, ev = 0, gs = 0, bad = 0;
-  for (long long base = warp0 * 32; base < total; base += warps * 32) {
-    long long i = base + lane_id();
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const int warp = threadIdx.x >> 5;
+  int hs = 0, ns = 0, ev = 0, gs = 0, bad = 0, par = 0;
+  for (long long base = (long long)blockIdx.x * blockDim.x; base < total; base += stride, par ^= 1) {
+    long long i = base + threadIdx.x;
     int v = -1;
     if (i < ne) {
       long long e = e0 + i;
@@ -84,7 +87,7 @@ __global__ void classify_kernel(ChunkArgs a) {
     }
     bool need = false, first = false;
     if (v >= a.V) { bad = 1; v = -1; }
-    if (v >= 0) {
+    if (v >= 0 && a.touch[v] != a.epoch) {
       int old = atomicMax(&a.touch[v], a.epoch);
       if (old != a.epoch) {   // first touch in this chunk
         first = true;
@@ -104,19 +107,22 @@ __global__ void classify_kernel(ChunkArgs a) {
         }
       }
     }
-    unsigned m = __ballot_sync(FULL, need);
-    if (m) {
-      int leader = __ffs(m) - 1, idx = 0;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->need_count, __popc(m));
-      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (need && idx < a.pool_slots) a.need_list[idx] = v;
+    const unsigned mn = __ballot_sync(FULL, need), mt = __ballot_sync(FULL, first);
+    if (lane_id() == 0) { s_cnt[par][0][warp] = __popc(mn); s_cnt[par][1][warp] = __popc(mt); }
+    __syncthreads();
+    if (threadIdx.x < 2) {
+      int sum = 0;
+      for (int w = 0; w < 8; ++w) { int c = s_cnt[par][threadIdx.x][w]; s_cnt[par][threadIdx.x][w] = sum; sum += c; }
+      s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &ctl->need_count : &ctl->touched_count, sum) : 0;
     }
-    m = __ballot_sync(FULL, first);
-    if (m) {
-      int leader = __ffs(m) - 1, idx = 0;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->touched_count, __popc(m));
-      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (first) { if (idx < a.touched_capacity) a.touched_list[idx] = v; else bad = 1; }
+    __syncthreads();
+    if (need) {
+      int idx = s_base[par][0] + s_cnt[par][0][warp] + __popc(mn & ((1u << lane_id()) - 1));
+      if (idx < a.pool_slots) a.need_list[idx] = v;
+    }
+    if (first) {
+      int idx = s_base[par][1] + s_cnt[par][1][warp] + __popc(mt & ((1u << lane_id()) - 1));
+      if (idx < a.touched_capacity) a.touched_list[idx] = v; else bad = 1;
     }
   }
   for (int o = 16; o; o >>= 1) {
@@ -152,7 +158,16 @@ __global__ void plan_kernel(ChunkArgs a) {
   ctl->sel_prefix = 0ull;
   ctl->sel_k = deficit;
   ctl->victim_count = 0;
-  long long occ = a.pool_slots - (ctl->free_top + deficit - need);
+  // Stack positions are handed out by list index, not by per-item atomics: victim i frees into
+  // free_stack[F + i] and takes host row host_free[H - 1 - i]; need-list entry i takes
+  // free_stack[F + deficit - 1 - i].  The counters are brought to their end-of-chunk values here.
+  const long long F = ctl->free_top, H = ctl->host_free_top;
+  ctl->evict_push_base = F;
+  ctl->host_pop_base = H;
+  ctl->alloc_base = F + deficit;
+  ctl->free_top = F + deficit - need;
+  ctl->host_free_top = H - deficit;      // reloads of this chunk push on top of this
+  long long occ = a.pool_slots - ctl->free_top;
   if (occ > ctl->peak_occupancy) ctl->peak_occupancy = occ;
 }
 
@@ -251,12 +266,7 @@ __global__ void evict_copy_kernel(ChunkArgs a) {
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
     int slot = a.victims[i];
     int v = a.owner[slot];
-    int hrow = 0;
-    if (lane_id() == 0) {
-      long long h = atomicAdd((unsigned long long*)&ctl->host_free_top, (unsigned long long)-1ll) - 1;
-      hrow = a.host_free[h];
-    }
-    hrow = __shfl_sync(FULL, hrow, 0);
+    const int hrow = a.host_free[ctl->host_pop_base - 1 - i];
     const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)slot * a.Hp);
     float4* dst = reinterpret_cast<float4*>(a.host_store + (size_t)hrow * a.Hp);
     for (int k = lane_id(); k < vec; k += 32) dst[k] = src[k];
@@ -264,8 +274,7 @@ __global__ void evict_copy_kernel(ChunkArgs a) {
       a.loc[v] = -2 - hrow;
       a.state[v] = TAURUS_EVICTED;
       a.owner[slot] = -1;
-      long long f = atomicAdd((unsigned long long*)&ctl->free_top, 1ull);
-      a.free_stack[f] = slot;
+      a.free_stack[ctl->evict_push_base + i] = slot;
     }
   }
 }
@@ -283,8 +292,8 @@ __global__ void alloc_kernel(ChunkArgs a) {
     int v = a.need_list[i];
     int slot = -1, st = 0, l = 0;
     if (lane_id() == 0) {
-      long long f = atomicAdd((unsigned long long*)&ctl->free_top, (unsigned long long)-1ll) - 1;
-      slot = f >= 0 ? a.free_stack[f] : -1;
+      if (a.direct) slot = v;
+      else { long long f = ctl->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
       st = a.state[v];
       l = a.loc[v];
     }
@@ -311,8 +320,7 @@ __global__ void alloc_kernel(ChunkArgs a) {
       for (int k = lane_id(); k < vec; k += 32) dst[k] = z;
     }
     if (lane_id() == 0) {
-      a.loc[v] = slot;
-      a.owner[slot] = v;
+      if (!a.direct) { a.loc[v] = slot; a.owner[slot] = v; }
       a.state[v] = TAURUS_IN_BUFFER;
     }
   }
@@ -366,6 +374,18 @@ __global__ void compact_done_kernel(ChunkArgs a) {
       idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
       if (done) { if (idx < a.drain_rows) a.done_list[idx] = v; else bad = 1; }
     }
+    // the slots of the completed non-hub vertices go back on the free stack (finalise still reads the rows:
+    // nothing allocates before the next chunk)
+    const int l = done ? a.loc[v] : 0x7fffffff;
+    const bool rel = done && l < a.pool_slots;
+    m = __ballot_sync(FULL, rel);
+    if (m) {
+      int leader = __ffs(m) - 1;
+      long long f = 0;
+      if (lane_id() == leader) f = (long long)atomicAdd((unsigned long long*)&ctl->free_top, (unsigned long long)__popc(m));
+      f = __shfl_sync(FULL, f, leader) + __popc(m & ((1u << lane_id()) - 1));
+      if (rel && !a.direct) { a.free_stack[f] = l; a.owner[l] = -1; }
+    }
   }
   if (__any_sync(FULL, bad) && lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
 }
@@ -404,11 +424,6 @@ __global__ void finalise_kernel(ChunkArgs a) {
     if (lane_id() == 0) {
       a.grad_ids[base + i] = v;
       a.state[v] = TAURUS_COMPLETED;
-      if (l < a.pool_slots) {
-        a.owner[l] = -1;
-        long long f = atomicAdd((unsigned long long*)&ctl->free_top, 1ull);
-        a.free_stack[f] = l;
-      }
     }
   }
 }

@@ -307,6 +307,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.src_begin = s; a.src_end = e;
   a.epoch = (int32_t)(c->chunk_seq + 1);
   a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.checked = (c->flags & TAURUS_FLAG_CHECKED) ? 1 : 0;
+  a.direct = c->pool_slots >= c->V ? 1 : 0;
   return a;
 }
 

@@ -31,6 +31,9 @@ struct DevCtl {
   long long free_top;       // entries on the free-slot stack
   long long host_free_top;  // entries on the free-host-row stack
   long long grad_count;     // rows waiting in the graduation buffer
+  long long alloc_base;       // this chunk: need-list entry i takes free_stack[alloc_base - 1 - i]
+  long long evict_push_base;  // this chunk: victim i's slot goes to free_stack[evict_push_base + i]
+  long long host_pop_base;    // this chunk: victim i's row goes to host row host_free[host_pop_base - 1 - i]
   unsigned long long sel_prefix;  // radix select: digits fixed so far (high bits)
   long long sel_k;                // radix select: rank still to resolve inside the prefix bucket
   unsigned int hist[TAURUS_SEL_BINS];
@@ -80,6 +83,7 @@ struct ChunkArgs {
   int32_t epoch;            // chunk sequence number + 1 within the layer
   int32_t Hp;               // padded accumulator width (multiple of 4)
   int32_t mode, act, fanout, checked;
+  int32_t direct;           // pool_slots >= V: vertex v owns slot v, no free stack, no eviction
 };
 
 struct taurus_ctx {
