@@ -28,6 +28,11 @@ sys.path.insert(0, ROOT)
 import taurus_gen as tg  # noqa: E402
 
 
+# DRAM bytes (read + write) per accumulator-row reduction of scatter_grouped_kernel<32,2>, from the ncu capture
+# summarised in profiles/scatter_grouped_kernel_mid_1200k.md (2.70 GB per launch / 1.486 M groups).
+SCATTER_TRAFFIC_PER_GROUP_BYTES = 1817.0
+
+
 def parse_args():
     p = argparse.ArgumentParser()
     p.add_argument("--gpus", type=int, default=1)
@@ -181,6 +186,7 @@ def run_ours(args):
     dense_dev = [torch.zeros(V * dmax, dtype=torch.float32, device=dev) for _ in range(2)]
     stream = torch.cuda.current_stream()
     edges_per_layer = []
+    groups_per_layer = []
 
     def step(feat0, flat, collect_stats=False):
         """One pass over all layers.  feat0 and the two flat ping-pong buffers live on the device (value) or in
@@ -200,6 +206,7 @@ def run_ours(args):
             st = ctx.layer_end()
             if collect_stats:
                 edges_per_layer.append(st["total_messages"])
+                groups_per_layer.append(st["scatter_groups"])
             feat = out
         return out
 
@@ -238,21 +245,33 @@ def run_ours(args):
     n_push = len(chunks) * L * args.steps
     ph = phases[:n_push].reshape(args.steps, L, len(chunks), 5)
     scatter_ms = ph[..., 3]
-    layer_bytes = []
+    # Algorithmic bytes of the scatter ("Kernels"): per accumulator-row reduction a read-modify-write of
+    # the row (2 * 4 Hp) plus slot and pending-count words (8); per propagated edge its (destination, source)
+    # words (8); per source its projected row read once (4 Hp) and its self message (row read 4 Hp + RMW 2 * 4 Hp + 8).
+    # In CSR order a "group" is one edge.  The per-edge cold-miss model (12 + 2 * 4 Hp per edge) is kept beside it.
+    layer_bytes, edge_model_bytes = [], []
     n_src = V
     for l in range(L):
         Hp = (w.dims[l + 1] + 3) // 4 * 4
-        layer_bytes.append(edges_per_layer[l] * (12 + 2 * 4 * Hp) + n_src * (4 * Hp + 8))
+        layer_bytes.append(groups_per_layer[l] * (8 * Hp + 8) + edges_per_layer[l] * 8 + n_src * (4 * Hp + 12 * Hp + 8))
+        edge_model_bytes.append(edges_per_layer[l] * (12 + 8 * Hp) + n_src * (4 * Hp + 8))
     alg_bytes_step = float(sum(layer_bytes))
     scatter_total_ms = float(scatter_ms.sum()) / args.steps
     pk = peaks()
     achieved = alg_bytes_step / (scatter_total_ms * 1e-3) / 1e9
-    roofline = dict(bound="hbm", kernel="scatter_kernel", achieved=achieved, peak=pk["hbm_gbs"], unit="GB/s",
-                    frac=achieved / pk["hbm_gbs"], peak_source=pk["source"], traffic=None,
+    grouped = not args.no_grouping
+    roofline = dict(bound="hbm", kernel="scatter_grouped_kernel" if grouped else "scatter_kernel", achieved=achieved,
+                    peak=pk["hbm_gbs"], unit="GB/s", frac=achieved / pk["hbm_gbs"], peak_source=pk["source"],
+                    traffic=SCATTER_TRAFFIC_PER_GROUP_BYTES * sum(groups_per_layer[l] for l in range(L) if w.dims[l + 1] > 128)
+                    / max(1, sum(1 for l in range(L) if w.dims[l + 1] > 128) * len(chunks)) if grouped else None,
+                    traffic_note="ncu dram read+write per launch of the H=256 kernel, scaled by groups per launch "
+                                 "(profiles/scatter_grouped_kernel_mid_1200k.md)" if grouped else None,
                     launches_per_step=len(chunks) * L, avg_launch_ms=scatter_total_ms / (len(chunks) * L),
                     algorithmic_bytes_per_launch=alg_bytes_step / (len(chunks) * L),
+                    edge_model_gbs=float(sum(edge_model_bytes)) / (scatter_total_ms * 1e-3) / 1e9,
                     per_layer=[dict(layer=l, scatter_ms=float(scatter_ms[:, l].sum()) / args.steps,
                                     gbs=layer_bytes[l] / (float(scatter_ms[:, l].sum()) / args.steps * 1e-3) / 1e9,
+                                    groups=int(groups_per_layer[l]),
                                     gteps_scatter_only=edges_per_layer[l] / (float(scatter_ms[:, l].sum()) / args.steps * 1e-3) / 1e9)
                                for l in range(L)])
     phase_ms = dict(zip(["copy_in", "projection", "classify_make_room", "scatter", "finalise"],

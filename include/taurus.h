@@ -122,6 +122,8 @@ typedef struct {
                                   IN_BUFFER, NOT_STARTED, EVICTED (non-hub) and hub vertices    */
   int64_t free_slots;          /* free pool slots now                                            */
   int64_t chunks;              /* chunks pushed                                                  */
+  int64_t scatter_groups;      /* accumulator-row reductions the scatter issued for propagated messages: one per
+                                  message in CSR order, one per (chunk, destination) group in grouped order    */
 } taurus_stats;
 
 /* Columns of one per-chunk record returned by taurus_get_chunk_log. */

@@ -60,7 +60,7 @@ class Stats(ctypes.Structure):
                 ("hub_messages", ctypes.c_int64), ("total_messages", ctypes.c_int64), ("hub_vertices", ctypes.c_int64),
                 ("completed", ctypes.c_int64), ("sum_hs", ctypes.c_int64), ("sum_ns", ctypes.c_int64),
                 ("sum_ev", ctypes.c_int64), ("sum_gs", ctypes.c_int64), ("free_slots", ctypes.c_int64),
-                ("chunks", ctypes.c_int64)]
+                ("chunks", ctypes.c_int64), ("scatter_groups", ctypes.c_int64)]
 
     def as_dict(self) -> dict:
         d = {}

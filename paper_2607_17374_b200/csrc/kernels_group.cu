@@ -14,7 +14,6 @@
 #include "taurus_internal.h"
 
 #define FULL 0xffffffffu
-#define SPAN_TILES 4   // 32-edge tiles per warp span
 
 static __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
 
@@ -31,16 +30,18 @@ __global__ void group_values_kernel(long long s, long long e, const long long* r
     for (long long k = b + lane_id(); k < t; k += 32) vals[k - e0] = ((unsigned long long)u << 32) | (unsigned long long)k;
   }
 }
-__global__ void group_split_kernel(long long n, const unsigned long long* vals, int32_t* g_src, uint32_t* g_eid) {
+__global__ void group_split_kernel(long long n, long long chunk_begin, const int32_t* dst_sorted, const unsigned long long* vals,
+                                   int2* g_edge, uint32_t* g_eid) {
   long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
     unsigned long long v = vals[i];
-    g_src[i] = (int32_t)(v >> 32);
+    g_edge[i] = make_int2(dst_sorted[i], (int32_t)((long long)(v >> 32) - chunk_begin));   // (destination, source - chunk start)
     if (g_eid) g_eid[i] = (uint32_t)v;
   }
 }
 
-// g_dst / g_src (/ g_eid): per grid chunk, the chunk's CSR edges stably sorted by destination.
+// g_dst, g_edge = (destination, source - chunk start) (/ g_eid): per grid chunk, the chunk's CSR edges stably
+// sorted by destination.
 int build_grouped_order(taurus_ctx* c, bool keep_edge_ids) {
   const long long V = c->V, E = c->E, cs = c->chunk_sources;
   const long long n_chunks = (V + cs - 1) / cs;
@@ -56,7 +57,7 @@ int build_grouped_order(taurus_ctx* c, bool keep_edge_ids) {
   long long max_edges = 1;
   for (long long k = 0; k < n_chunks; ++k) max_edges = std::max(max_edges, bounds[(size_t)k + 1] - bounds[(size_t)k]);
   if (cudaMalloc(&c->d_gdst, (size_t)(E > 0 ? E : 1) * sizeof(int32_t)) != cudaSuccess) return TAURUS_ERR_NOMEM;
-  if (cudaMalloc(&c->d_gsrc, (size_t)(E > 0 ? E : 1) * sizeof(int32_t)) != cudaSuccess) return TAURUS_ERR_NOMEM;
+  if (cudaMalloc(&c->d_gedge, (size_t)(E > 0 ? E : 1) * sizeof(int2)) != cudaSuccess) return TAURUS_ERR_NOMEM;
   if (keep_edge_ids && cudaMalloc(&c->d_geid, (size_t)(E > 0 ? E : 1) * sizeof(uint32_t)) != cudaSuccess) return TAURUS_ERR_NOMEM;
   unsigned long long *vals_in = nullptr, *vals_out = nullptr;
   void* tmp = nullptr;
@@ -75,7 +76,7 @@ int build_grouped_order(taurus_ctx* c, bool keep_edge_ids) {
       group_values_kernel<<<c->sm_count * 4, 256>>>(s, e, c->d_row_ptr, e0, vals_in);
       size_t b = tmp_bytes;
       if (cub::DeviceRadixSort::SortPairs(tmp, b, c->d_col + e0, c->d_gdst + e0, vals_in, vals_out, ne, 0, end_bit) != cudaSuccess) { rc = TAURUS_ERR_CUDA; break; }
-      group_split_kernel<<<c->sm_count * 4, 256>>>(ne, vals_out, c->d_gsrc + e0, c->d_geid ? c->d_geid + e0 : nullptr);
+      group_split_kernel<<<c->sm_count * 4, 256>>>(ne, s, c->d_gdst + e0, vals_out, c->d_gedge + e0, c->d_geid ? c->d_geid + e0 : nullptr);
     }
     if (rc == TAURUS_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAURUS_ERR_CUDA;
   } while (0);
@@ -194,54 +195,66 @@ void launch_classify_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st)
   c->launches += 1;
 }
 
-// ------------------------------------------------------------------------------------------------ scatter (S5, S5', S6 head)
-// Lanes are grouped LPE to an edge; sub-group `sub` of a warp walks its own part of each 32-edge tile.
-template <int LPE, int VPL>
-__global__ void __launch_bounds__(256) scatter_grouped_kernel(ChunkArgs a, const int32_t* __restrict__ g_dst,
-                                                              const int32_t* __restrict__ g_src,
-                                                              const uint32_t* __restrict__ gmask) {
+// ------------------------------------------------------------------------------------------------ scatter (S5, S5')
+// Lanes are grouped LPE to an edge (VPL float4 of the row each); sub-group `sub` of a warp walks its own
+// contiguous stretch of the sorted edge list, four edges per step: the four edge records are read with
+// sub-group-uniform loads (L1 hits), the four projected rows are requested together, then the rows are
+// added to the running group sum or, at a destination change, the sum is flushed with one vector reduction
+// per lane and one integer reduction on the pending count.  The loop body is kept to a few tens of
+// instructions per edge: an earlier version with lane-parallel edge loads and shuffles was issue-bound.
+#define SPAN_EDGES 128   // edges per warp span (all sub-groups together)
+
+template <int LPE, int VPL, bool SAMPLED, bool DIRECT>
+__global__ void __launch_bounds__(256, (VPL <= 2 ? 3 : 1))
+scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
   constexpr int EPS = 32 / LPE;                 // sub-groups per warp
+  constexpr int STRETCH = SPAN_EDGES / EPS;     // edges one sub-group walks per span
   const int lane = lane_id();
   const int sub = lane / LPE;
   const int c4 = lane % LPE;
   const int nvec = a.Hp >> 2;
   const long long e0 = a.row_ptr[a.src_begin], e1 = a.row_ptr[a.src_end];
   const long long n_src = a.src_end - a.src_begin;
-  const long long edge_tiles = (e1 - e0 + 31) >> 5;
-  const long long spans = (edge_tiles + SPAN_TILES - 1) / SPAN_TILES;
+  const long long spans = (e1 - e0 + SPAN_EDGES - 1) / SPAN_EDGES;
   const long long self_tiles = (n_src + 31) >> 5;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const long long loc_limit = a.pool_slots + a.hub_count;
-  unsigned long long msgs = 0, hub_msgs = 0;
+  const int loc_limit = (int)(a.pool_slots + a.hub_count);
+  const int pool = (int)a.pool_slots;
+  const int ld4 = a.ldpt >> 2;                  // row pitch of the projected rows in float4
+  const float4* __restrict__ Pbase = reinterpret_cast<const float4*>(a.PT) + c4;
+  unsigned msgs = 0, hub_msgs = 0, groups = 0;
   int bad = 0;
 
-  // state of the group this sub-group is summing; its slot is requested when the group starts so that the
-  // load has landed by the time the group is flushed
   int cur = -1, cnt = 0, cur_loc = -1;
   float4 sum[VPL];
+  // byte addressing with 32-bit x 32-bit -> 64-bit products keeps the address arithmetic to one instruction
+  const char* const Pb = reinterpret_cast<const char*>(a.PT) + c4 * 16;
+  char* const Ab = reinterpret_cast<char*>(a.acc) + c4 * 16;
+  const unsigned p_pitch = (unsigned)a.ldpt * 4u, a_pitch = (unsigned)a.Hp * 4u;
+  bool lane_on[VPL];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) lane_on[k] = c4 + k * LPE < nvec;
+
   auto flush = [&]() {
-    // all LPE lanes of the sub-group call this together with the same (cur, cnt)
-    if (cur < 0) return;
-    const int l = cur_loc;
-    if (l < 0 || l >= loc_limit) { bad = 1; cur = -1; cnt = 0; return; }
-    float* dst = a.acc + (size_t)l * a.Hp;
+    const int l = DIRECT ? cur : cur_loc;
+    if (!DIRECT && ((unsigned)l >= (unsigned)loc_limit)) { bad = 1; return; }
+    char* dst = Ab + (unsigned long long)(unsigned)l * a_pitch;
 #pragma unroll
     for (int k = 0; k < VPL; ++k)
-      if (c4 + k * LPE < nvec) red_add_v4(dst + 4 * (c4 + k * LPE), sum[k]);
-    if (c4 == 0) {
-      atomicAdd(&a.pend[cur], -cnt);   // result unused: a reduction; completion is read after the kernel
-      msgs += (unsigned)cnt;
-      if (l >= a.pool_slots) hub_msgs += (unsigned)cnt;
-    }
-    cur = -1; cnt = 0;
+      if (lane_on[k]) red_add_v4(reinterpret_cast<float*>(dst + k * LPE * 16), sum[k]);
+    if (c4 == 0) atomicAdd(&a.pend[cur], -cnt);   // result unused: a reduction; completion is read after the kernel
+    msgs += (unsigned)cnt;                          // counted by every lane; only lane c4 == 0 of each sub-group reports
+    groups += 1;
+    if (!DIRECT && l >= pool) hub_msgs += (unsigned)cnt;
   };
-  auto take = [&](int dj, int lj, const float4 (&row)[VPL]) {
-    if (dj != cur) {
-      flush();
-      cur = dj; cnt = 1; cur_loc = lj;
+  auto take = [&](int d, const float4 (&row)[VPL]) {
+    if (d != cur) {
+      if (cur >= 0) flush();
+      cur = d; cnt = 1;
+      if (!DIRECT) cur_loc = a.loc[d];
 #pragma unroll
       for (int k = 0; k < VPL; ++k) sum[k] = row[k];
     } else {
@@ -250,65 +263,50 @@ __global__ void __launch_bounds__(256) scatter_grouped_kernel(ChunkArgs a, const
       for (int k = 0; k < VPL; ++k) { sum[k].x += row[k].x; sum[k].y += row[k].y; sum[k].z += row[k].z; sum[k].w += row[k].w; }
     }
   };
-  auto fetch = [&](int sj, float4 (&row)[VPL]) {
-    const float4* p = reinterpret_cast<const float4*>(a.PT + (size_t)(sj - a.src_begin) * a.ldpt);
+  auto fetch = [&](int src_rel, float4 (&row)[VPL]) {
+    const char* p = Pb + (unsigned long long)(unsigned)src_rel * p_pitch;
 #pragma unroll
     for (int k = 0; k < VPL; ++k)
-      if (c4 + k * LPE < nvec) row[k] = p[c4 + k * LPE];
+      if (lane_on[k]) row[k] = *reinterpret_cast<const float4*>(p + k * LPE * 16);
   };
 
-  // A warp span is SPAN_TILES * 32 consecutive edges of the sorted list; sub-group g walks its own contiguous
-  // stretch of SPAN_TILES * LPE edges, LPE edges per round (loaded by its LPE lanes, one edge each).
-  // The rounds of all spans of this warp form one sequence that is software-pipelined: (destination, source)
-  // of round i+2 and the slots of round i+1 are requested while round i is processed.
-  constexpr int STRETCH = SPAN_TILES * LPE;
-  const long long my_spans = warp0 < spans ? (spans - warp0 + warps - 1) / warps : 0;
-  const long long rounds = my_spans * SPAN_TILES;
-  auto edge_of = [&](long long i) -> long long {   // this lane's edge in round i of the warp's sequence
-    const long long span = warp0 + (i / SPAN_TILES) * warps;
-    return e0 + span * (SPAN_TILES * 32) + (long long)sub * STRETCH + (i % SPAN_TILES) * LPE + c4;
-  };
-  auto load_ds = [&](long long i, int& d, int& sx) {
-    d = -1; sx = 0;
-    if (i < rounds) {
-      const long long e = edge_of(i);
-      if (e < e1 && (gmask == nullptr || ((gmask[e >> 5] >> (e & 31)) & 1u))) { d = g_dst[e]; sx = g_src[e]; }
-    }
-  };
-  int d0, s0, l0, d1, s1, d2, s2;
-  load_ds(0, d0, s0);
-  load_ds(1, d1, s1);
-  l0 = d0 >= 0 ? a.loc[d0] : -1;
+  for (long long span = warp0; span < spans; span += warps) {
+    long long x = e0 + span * SPAN_EDGES + (long long)sub * STRETCH;
+    const long long x_end = (x + STRETCH < e1) ? x + STRETCH : e1;
+    const int2* ge = g_edge + x;
+    int left = x_end > x ? (int)(x_end - x) : 0;
 #pragma unroll 1
-  for (long long i = 0; i < rounds; ++i) {
-    const int l1 = d1 >= 0 ? a.loc[d1] : -1;   // slots of the next round
-    load_ds(i + 2, d2, s2);                     // edges of the round after that
-    if (__any_sync(FULL, d0 >= 0)) {
-#pragma unroll 1
-      for (int j = 0; j < LPE; j += 4) {
-        // four edges per step: all rows are requested before any is used
-        int dd[4], ss[4], ll[4];
+    for (; left >= 4; left -= 4, ge += 4, x += 4) {   // fast path: four edges per step, all rows requested together
+      int2 ed[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          dd[q] = __shfl_sync(FULL, d0, sub * LPE + j + q);
-          ss[q] = __shfl_sync(FULL, s0, sub * LPE + j + q);
-          ll[q] = __shfl_sync(FULL, l0, sub * LPE + j + q);
-        }
-        float4 row[4][VPL];
+      for (int q = 0; q < 4; ++q) ed[q] = ge[q];
+      if (SAMPLED) {
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          if (dd[q] >= 0) fetch(ss[q], row[q]);
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          if (dd[q] >= 0) take(dd[q], ll[q], row[q]);
+          if (!((gmask[(x + q) >> 5] >> ((x + q) & 31)) & 1u)) ed[q].x = -1;
       }
+      float4 row[4][VPL];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (!SAMPLED || ed[q].x >= 0) fetch(ed[q].y, row[q]);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (!SAMPLED || ed[q].x >= 0) take(ed[q].x, row[q]);
     }
-    if ((i % SPAN_TILES) == SPAN_TILES - 1) flush();   // a group that continues in another warp's span is flushed by both
-    d0 = d1; s0 = s1; l0 = l1; d1 = d2; s1 = s2;
+#pragma unroll 1
+    for (; left > 0; --left, ++ge, ++x) {             // ragged end of the chunk's list
+      int2 ed = ge[0];
+      if (SAMPLED && !((gmask[x >> 5] >> (x & 31)) & 1u)) continue;
+      float4 row[VPL];
+      fetch(ed.y, row);
+      take(ed.x, row);
+    }
+    if (cur >= 0) flush();   // a group that continues in another stretch is flushed by both
+    cur = -1;
   }
-  flush();
+  if (c4 != 0) { msgs = 0; hub_msgs = 0; groups = 0; }
 
-  // self messages (one per chunk vertex), as in the CSR-order kernel
+  // self messages (one per chunk vertex)
   for (long long t = warp0; t < self_tiles; t += warps) {
     const long long u = a.src_begin + t * 32 + lane;
     int v = u < a.src_end ? (int)u : -1;
@@ -335,9 +333,9 @@ __global__ void __launch_bounds__(256) scatter_grouped_kernel(ChunkArgs a, const
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) {
-            float4 x = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
+            float4 xx = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
             float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];
-            red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(x.x + b.x * sc, x.y + b.y * sc, x.z + b.z * sc, x.w + b.w * sc));
+            red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(xx.x + b.x * sc, xx.y + b.y * sc, xx.z + b.z * sc, xx.w + b.w * sc));
           }
       }
     }
@@ -346,25 +344,44 @@ __global__ void __launch_bounds__(256) scatter_grouped_kernel(ChunkArgs a, const
   for (int o = 16; o; o >>= 1) {
     msgs += __shfl_xor_sync(FULL, msgs, o);
     hub_msgs += __shfl_xor_sync(FULL, hub_msgs, o);
+    groups += __shfl_xor_sync(FULL, groups, o);
     bad |= __shfl_xor_sync(FULL, bad, o);
   }
   if (lane == 0) {
-    if (msgs) atomicAdd((unsigned long long*)&ctl->total_messages, msgs);
-    if (hub_msgs) atomicAdd((unsigned long long*)&ctl->hub_messages, hub_msgs);
+    if (groups) atomicAdd((unsigned long long*)&ctl->scatter_groups, (unsigned long long)groups);
+    if (msgs) atomicAdd((unsigned long long*)&ctl->total_messages, (unsigned long long)msgs);
+    if (hub_msgs) atomicAdd((unsigned long long*)&ctl->hub_messages, (unsigned long long)hub_msgs);
     if (bad) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
   }
 }
 
-void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
-  const int blocks = c->sm_count * 8;
-  const int Hp = a.Hp;
+template <int LPE, int VPL, bool SAMPLED, bool DIRECT>
+static void launch_sg(taurus_ctx* c, const ChunkArgs& a, const uint32_t* gm, cudaStream_t st) {
+  static int blocks_per_sm = 0;
+  if (blocks_per_sm == 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, scatter_grouped_kernel<LPE, VPL, SAMPLED, DIRECT>, 256, 0) != cudaSuccess ||
+        blocks_per_sm < 1)
+      blocks_per_sm = 1;
+  }
+  scatter_grouped_kernel<LPE, VPL, SAMPLED, DIRECT><<<c->sm_count * blocks_per_sm, 256, 0, st>>>(a, c->d_gedge, gm);
+}
+
+template <int LPE, int VPL>
+static void launch_sg2(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   const uint32_t* gm = c->d_mask_cur ? c->d_gmask : nullptr;
-  if (Hp <= 16) scatter_grouped_kernel<4, 1><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
-  else if (Hp <= 32) scatter_grouped_kernel<8, 1><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
-  else if (Hp <= 64) scatter_grouped_kernel<16, 1><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
-  else if (Hp <= 128) scatter_grouped_kernel<32, 1><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
-  else if (Hp <= 256) scatter_grouped_kernel<32, 2><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
-  else if (Hp <= 512) scatter_grouped_kernel<32, 4><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
-  else scatter_grouped_kernel<32, 8><<<blocks, 256, 0, st>>>(a, c->d_gdst, c->d_gsrc, gm);
+  const bool direct = a.direct && c->hub_count == 0;
+  if (gm) { if (direct) launch_sg<LPE, VPL, true, true>(c, a, gm, st); else launch_sg<LPE, VPL, true, false>(c, a, gm, st); }
+  else    { if (direct) launch_sg<LPE, VPL, false, true>(c, a, gm, st); else launch_sg<LPE, VPL, false, false>(c, a, gm, st); }
+}
+
+void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  const int Hp = a.Hp;
+  if (Hp <= 16) launch_sg2<4, 1>(c, a, st);
+  else if (Hp <= 32) launch_sg2<8, 1>(c, a, st);
+  else if (Hp <= 64) launch_sg2<16, 1>(c, a, st);
+  else if (Hp <= 128) launch_sg2<32, 1>(c, a, st);
+  else if (Hp <= 256) launch_sg2<32, 2>(c, a, st);
+  else if (Hp <= 512) launch_sg2<32, 4>(c, a, st);
+  else launch_sg2<32, 8>(c, a, st);
   c->launches += 1;
 }

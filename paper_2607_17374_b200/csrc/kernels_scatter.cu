@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
     bad |= __shfl_xor_sync(FULL, bad, o);
   }
   if (lane == 0) {
-    if (msgs) atomicAdd((unsigned long long*)&ctl->total_messages, msgs);
+    if (msgs) { atomicAdd((unsigned long long*)&ctl->total_messages, msgs); atomicAdd((unsigned long long*)&ctl->scatter_groups, msgs); }
     if (hub_msgs) atomicAdd((unsigned long long*)&ctl->hub_messages, hub_msgs);
     if (bad) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
   }

@@ -71,7 +71,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X); cudaFree(c->d_PT);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
-  cudaFree(c->d_gdst); cudaFree(c->d_gsrc); cudaFree(c->d_geid); cudaFree(c->d_gmask);
+  cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
   cudaFree(c->d_ctl); cudaFree(c->d_chunk_log);
   if (c->h_ctl) cudaFreeHost(c->h_ctl);
   if (c->order_event) cudaEventDestroy(c->order_event);
@@ -451,7 +451,7 @@ static int fill_stats(taurus_ctx* c, taurus_stats* s) {
   s->evictions = h->evictions; s->reloads = h->reloads; s->peak_occupancy = h->peak_occupancy;
   s->hub_messages = h->hub_messages; s->total_messages = h->total_messages; s->hub_vertices = c->hub_count;
   s->completed = h->completed; s->sum_hs = h->sum_hs; s->sum_ns = h->sum_ns; s->sum_ev = h->sum_ev; s->sum_gs = h->sum_gs;
-  s->free_slots = h->free_top; s->chunks = h->chunks;
+  s->free_slots = h->free_top; s->chunks = h->chunks; s->scatter_groups = h->scatter_groups;
   return TAURUS_OK;
 }
 

@@ -40,6 +40,7 @@ struct DevCtl {
   // layer totals
   long long evictions, reloads, peak_occupancy, hub_messages, total_messages, completed;
   long long sum_hs, sum_ns, sum_ev, sum_gs, chunks;
+  long long scatter_groups; // accumulator-row reductions issued by the scatter (self messages not counted)
   long long bad_index;      // first out-of-range index seen by a checked kernel (debug aid)
 };
 
@@ -132,7 +133,7 @@ struct taurus_ctx {
   uint32_t* d_csc_eid = nullptr;
   uint32_t* d_mask = nullptr;
   int32_t* d_gdst = nullptr;      // grouped order (per grid chunk, edges sorted by destination): destinations
-  int32_t* d_gsrc = nullptr;      //   sources
+  int2* d_gedge = nullptr;        //   (destination, source - chunk start) pairs
   uint32_t* d_geid = nullptr;     //   CSR edge indices (kept only when some layer is sampled)
   uint32_t* d_gmask = nullptr;    // current layer's edge mask in grouped order
   uint32_t* d_mask_cur = nullptr; // d_mask when the current layer is sampled, else NULL (every edge propagated)
