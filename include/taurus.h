@@ -176,6 +176,19 @@ int taurus_drain_completed(taurus_ctx* ctx, int64_t* out_ids, float* out_rows, i
 int taurus_drain_dense(taurus_ctx* ctx, float* dense_rows, int64_t ld, int64_t* out_ids, int64_t capacity_rows,
                        int64_t* out_count);
 
+/*
+ * Dense-output mode for the current layer (Sect. 3.6 double-buffers graduation so that collecting and
+ * off-loading overlap; Sect. 3.7 keeps outputs in vertex order for the next layer).  Call after
+ * taurus_layer_begin and before the first push.  Every finalised row is then written to
+ * dense_rows[id * ld ...] (ld in floats, >= dims[layer+1]; device memory or pinned host memory) by the
+ * library itself: the graduation buffer is split in two halves, the rows of chunk k leave one half on an
+ * internal stream while chunk k+1 computes into the other, and the caller never drains (taurus_drain_*
+ * report zero rows).  A chunk whose completion bound exceeds drain_rows / 2 is refused with
+ * TAURUS_ERR_DRAIN_FULL (create the context with a larger drain_rows).  taurus_layer_end waits until
+ * every row has arrived.  The mode ends with the layer.
+ */
+int taurus_layer_set_dense_output(taurus_ctx* ctx, float* dense_rows, int64_t ld);
+
 /* Ends the layer: blocking; checks that every vertex completed and every slot is free (else
  * TAURUS_ERR_ORDER), and fills *stats (may be NULL). */
 int taurus_layer_end(taurus_ctx* ctx, taurus_stats* stats);

@@ -75,7 +75,7 @@ EXPORTS = [
     "taurus_layer_end", "taurus_get_stats", "taurus_get_chunk_log", "taurus_get_vertex_array",
     "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count",
     "taurus_set_timing", "taurus_get_phase_ms", "taurus_destroy", "taurus_strerror", "taurus_last_cuda_error",
-    "taurus_completion_counts_noalloc",
+    "taurus_completion_counts_noalloc", "taurus_layer_set_dense_output",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -97,6 +97,7 @@ def load_library():
     lib.taurus_drain_completed.argtypes = [vp, vp, vp, i64, ctypes.POINTER(i64)]
     lib.taurus_drain_dense.argtypes = [vp, vp, i64, vp, i64, ctypes.POINTER(i64)]
     lib.taurus_layer_end.argtypes = [vp, ctypes.POINTER(Stats)]
+    lib.taurus_layer_set_dense_output.argtypes = [vp, vp, i64]
     lib.taurus_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
     lib.taurus_get_chunk_log.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
     lib.taurus_get_vertex_array.argtypes = [vp, i32, vp]
@@ -202,6 +203,9 @@ class Context:
         self._check(self._lib.taurus_drain_dense(self._h, _ptr(dense_rows), ld, _ptr(out_ids), capacity_rows, ctypes.byref(n)),
                     "taurus_drain_dense")
         return int(n.value)
+
+    def layer_set_dense_output(self, dense_rows, ld: int):
+        self._check(self._lib.taurus_layer_set_dense_output(self._h, _ptr(dense_rows), ld), "taurus_layer_set_dense_output")
 
     def layer_end(self) -> dict:
         s = Stats()

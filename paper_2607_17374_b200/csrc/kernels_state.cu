@@ -372,7 +372,7 @@ __global__ void compact_done_kernel(ChunkArgs a) {
       int leader = __ffs(m) - 1, idx = 0;
       if (lane_id() == leader) idx = atomicAdd(&ctl->done_count, __popc(m));
       idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (done) { if (idx < a.drain_rows) a.done_list[idx] = v; else bad = 1; }
+      if (done) { if (idx < a.grad_cap) a.done_list[idx] = v; else bad = 1; }
     }
     // the slots of the completed non-hub vertices go back on the free stack (finalise still reads the rows:
     // nothing allocates before the next chunk)
@@ -396,11 +396,12 @@ __global__ void finalise_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
   const int n = ctl->done_count;
-  const long long base = ctl->grad_count;
+  const long long base = a.dense_half >= 0 ? a.grad_off : ctl->grad_count;
+  const long long limit = a.dense_half >= 0 ? a.grad_off + a.grad_cap : a.drain_rows;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    if (base + i >= a.drain_rows) {
+    if (base + i >= limit) {
       if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
       continue;
     }
@@ -443,7 +444,7 @@ __global__ void commit_kernel(ChunkArgs a) {
   ctl->evictions += ctl->deficit;
   ctl->reloads += ctl->reloaded;
   ctl->completed += ctl->done_count;
-  ctl->grad_count += ctl->done_count;
+  if (a.dense_half >= 0) ctl->out_count[a.dense_half] = ctl->done_count; else ctl->grad_count += ctl->done_count;
   ctl->chunks = c + 1;
   ctl->hs = ctl->ns = ctl->ev = ctl->gs = 0;
   ctl->need_count = 0; ctl->done_count = 0; ctl->touched_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;
@@ -502,6 +503,35 @@ __global__ void reload_histogram_kernel(long long V, const int32_t* reload, long
   __syncthreads();
   if (threadIdx.x < 17 && sh[threadIdx.x]) atomicAdd((unsigned long long*)&hist18[threadIdx.x], (unsigned long long)sh[threadIdx.x]);
   if (threadIdx.x == 0 && shmax) atomicMax(&hist18[17], (long long)shmax);
+}
+
+// Dense-output mode: the rows of one half of the graduation buffer go to dense[id * ld ...]; the row count is
+// read from the control block, so the launch needs no host round trip.
+__global__ void place_half_kernel(const DevCtl* ctl, int half, const long long* ids, const float* rows, int Hp, int d_out,
+                                  float* dense, long long ld) {
+  const long long count = ctl->out_count[half];
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const bool vec_ok = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(dense) & 15) == 0);
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < count; i += warps) {
+    long long id = ids[i];
+    const float* src = rows + (size_t)i * Hp;
+    float* dst = dense + (size_t)id * ld;
+    if (vec_ok) {
+      int full = d_out >> 2;
+      for (int k = lane_id(); k < full; k += 32)
+        reinterpret_cast<float4*>(dst)[k] = reinterpret_cast<const float4*>(src)[k];
+      for (int k = (full << 2) + lane_id(); k < d_out; k += 32) dst[k] = src[k];
+    } else {
+      for (int k = lane_id(); k < d_out; k += 32) dst[k] = src[k];
+    }
+  }
+}
+
+void launch_place_half(taurus_ctx* c, int half, int d_out, int Hp, cudaStream_t st) {
+  const long long off = (long long)half * (c->drain_rows / 2);
+  place_half_kernel<<<c->sm_count * 4, 256, 0, st>>>(c->d_ctl, half, c->d_grad_ids + off, c->d_grad_rows + (size_t)off * Hp, Hp, d_out,
+                                                     c->dense_out, c->dense_ld);
+  c->launches += 1;
 }
 
 void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st) {

@@ -69,12 +69,20 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
   cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
-  cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X); cudaFree(c->d_PT);
+  cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
   cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
   cudaFree(c->d_ctl); cudaFree(c->d_chunk_log);
   if (c->h_ctl) cudaFreeHost(c->h_ctl);
   if (c->order_event) cudaEventDestroy(c->order_event);
+  for (int i = 0; i < 2; ++i) {
+    if (c->x_ready[i]) cudaEventDestroy(c->x_ready[i]);
+    if (c->x_free[i]) cudaEventDestroy(c->x_free[i]);
+    if (c->fin_done[i]) cudaEventDestroy(c->fin_done[i]);
+    if (c->out_done[i]) cudaEventDestroy(c->out_done[i]);
+  }
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->out_stream) cudaStreamDestroy(c->out_stream);
   for (auto& e : c->phase_ev) if (e) cudaEventDestroy(e);
   cudaGetLastError();
   cudaSetDevice(prev);
@@ -181,7 +189,16 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   // graduation buffer, chunk buffers
   ALLOC(c->d_grad_ids, c->drain_rows); ALLOC(c->d_grad_rows, (size_t)c->drain_rows * c->Hmax); ALLOC(c->d_done_list, c->drain_rows);
-  ALLOC(c->d_X, (size_t)c->chunk_sources * c->Kmax);
+  ALLOC(c->d_X[0], (size_t)c->chunk_sources * c->Kmax);
+  ALLOC(c->d_X[1], (size_t)c->chunk_sources * c->Kmax);
+  CU(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  CU(cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    CU(cudaEventCreateWithFlags(&c->x_ready[i], cudaEventDisableTiming));
+    CU(cudaEventCreateWithFlags(&c->x_free[i], cudaEventDisableTiming));
+    CU(cudaEventCreateWithFlags(&c->fin_done[i], cudaEventDisableTiming));
+    CU(cudaEventCreateWithFlags(&c->out_done[i], cudaEventDisableTiming));
+  }
   ALLOC(c->d_PT, (size_t)c->chunk_sources * 2 * c->Hmax);
   // sampling
   if (any_sampled) {
@@ -239,6 +256,7 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
 // Reads the device control block (after synchronising `st`) and returns its sticky error.
 static int read_ctl(taurus_ctx* c, cudaStream_t st) {
   CU(cudaStreamSynchronize(st));
+  CU(cudaStreamSynchronize(c->out_stream));
   CU(cudaMemcpy(c->h_ctl, c->d_ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost));
   return c->h_ctl->error;
 }
@@ -248,7 +266,12 @@ extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_strea
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(cudaSetDevice(c->device));
   if (c->last_stream != st) CU(cudaStreamSynchronize(c->last_stream));
+  CU(cudaStreamSynchronize(c->copy_stream));
+  CU(cudaStreamSynchronize(c->out_stream));
   c->layer = layer;
+  c->dense_out = nullptr; c->dense_ld = 0;
+  c->half_used[0] = c->half_used[1] = false;
+  c->x_used[0] = c->x_used[1] = false;
   memset(c->h_ctl, 0, sizeof(DevCtl));
   c->next_src = 0; c->chunk_seq = 0; c->ub_since_drain = 0; c->last_stream = st;
   launch_layer_reset(c, layer, st);
@@ -308,6 +331,9 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.epoch = (int32_t)(c->chunk_seq + 1);
   a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.checked = (c->flags & TAURUS_FLAG_CHECKED) ? 1 : 0;
   a.direct = c->pool_slots >= c->V ? 1 : 0;
+  a.dense_half = c->dense_out ? (int)(c->chunk_seq & 1) : -1;
+  a.grad_cap = c->dense_out ? c->drain_rows / 2 : c->drain_rows;
+  a.grad_off = c->dense_out ? (long long)a.dense_half * (c->drain_rows / 2) : 0;
   return a;
 }
 
@@ -319,7 +345,7 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   if ((reinterpret_cast<uintptr_t>(features) & 3) != 0) return TAURUS_ERR_INVALID_ARG;
   if (c->h_ctl->error) return c->h_ctl->error;
   const long long bound = completion_bound(c, src_begin, src_end);
-  if (c->ub_since_drain + bound > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
+  if (c->dense_out ? bound > c->drain_rows / 2 : c->ub_since_drain + bound > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(cudaSetDevice(c->device));
   if (st != c->last_stream) {   // keep chunk order across streams
@@ -339,12 +365,19 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   }
   const bool timing = pev != nullptr;
   if (timing) cudaEventRecord(pev[0], st);
-  // S1: features to the device
+  // S1: features to the device.  Host chunks are copied on the library's copy stream into one of two staging
+  // buffers, so that the copy of chunk k+1 overlaps the kernels of chunk k.
   const float* X = features;
   int ldx = K;
+  int xbuf = -1;
   if (pointer_kind(features) != PK_DEVICE) {
-    CU(cudaMemcpyAsync(c->d_X, features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, st));
-    X = c->d_X;
+    xbuf = (int)(c->host_pushes & 1);
+    c->host_pushes += 1;
+    if (c->x_used[xbuf]) CU(cudaStreamWaitEvent(c->copy_stream, c->x_free[xbuf], 0));
+    CU(cudaMemcpyAsync(c->d_X[xbuf], features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+    CU(cudaEventRecord(c->x_ready[xbuf], c->copy_stream));
+    CU(cudaStreamWaitEvent(st, c->x_ready[xbuf], 0));
+    X = c->d_X[xbuf];
   }
   if (timing) cudaEventRecord(pev[1], st);
   ChunkArgs a = make_args(c, src_begin, src_end);
@@ -355,6 +388,7 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   } else {
     launch_project_simt(c, l, X, ldx, src_begin, n, st);
   }
+  if (xbuf >= 0) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }
   if (timing) cudaEventRecord(pev[2], st);
   // S3, S4
   const bool grouped = c->d_gdst != nullptr && src_begin % c->chunk_sources == 0 &&
@@ -366,12 +400,21 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
   if (timing) cudaEventRecord(pev[4], st);
   // S7
+  if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
   launch_finalise(c, a, st);
+  if (a.dense_half >= 0) {   // hand this chunk's rows to the output stream
+    const int h = a.dense_half, d_out = c->dims[l + 1];
+    CU(cudaEventRecord(c->fin_done[h], st));
+    CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
+    launch_place_half(c, h, d_out, a.Hp, c->out_stream);
+    CU(cudaEventRecord(c->out_done[h], c->out_stream));
+    c->half_used[h] = true;
+  }
   if (timing) cudaEventRecord(pev[5], st);
   CU(cudaGetLastError());
   c->next_src = src_end;
   c->chunk_seq += 1;
-  c->ub_since_drain += bound;
+  if (!c->dense_out) c->ub_since_drain += bound;
   return TAURUS_OK;
 }
 
@@ -432,6 +475,20 @@ extern "C" int taurus_drain_dense(taurus_ctx* c, float* dense_rows, int64_t ld, 
     CU(cudaGetLastError());
   }
   return drain_reset(c);
+}
+
+extern "C" int taurus_layer_set_dense_output(taurus_ctx* c, float* dense_rows, int64_t ld) {
+  if (!c || !dense_rows) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0 || c->chunk_seq != 0) return TAURUS_ERR_ORDER;
+  if (ld < c->dims[c->layer + 1]) return TAURUS_ERR_INVALID_ARG;
+  float* dev = dense_rows;
+  int kind = pointer_kind(dense_rows);
+  if (kind == PK_HOST_PAGEABLE) return TAURUS_ERR_INVALID_ARG;
+  if (kind == PK_HOST_PINNED && !cuda_ok(cudaHostGetDevicePointer((void**)&dev, dense_rows, 0), "cudaHostGetDevicePointer"))
+    return TAURUS_ERR_INVALID_ARG;
+  c->dense_out = dev;
+  c->dense_ld = ld;
+  return TAURUS_OK;
 }
 
 static int fill_stats(taurus_ctx* c, taurus_stats* s) {

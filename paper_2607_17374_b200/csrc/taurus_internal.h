@@ -31,6 +31,7 @@ struct DevCtl {
   long long free_top;       // entries on the free-slot stack
   long long host_free_top;  // entries on the free-host-row stack
   long long grad_count;     // rows waiting in the graduation buffer
+  long long out_count[2];   // dense-output mode: rows finalise left in each half of the graduation buffer
   long long alloc_base;       // this chunk: need-list entry i takes free_stack[alloc_base - 1 - i]
   long long evict_push_base;  // this chunk: victim i's slot goes to free_stack[evict_push_base + i]
   long long host_pop_base;    // this chunk: victim i's row goes to host row host_free[host_pop_base - 1 - i]
@@ -84,6 +85,9 @@ struct ChunkArgs {
   int32_t epoch;            // chunk sequence number + 1 within the layer
   int32_t Hp;               // padded accumulator width (multiple of 4)
   int32_t mode, act, fanout, checked;
+  long long grad_off;       // dense-output mode: first row of this chunk's half of the graduation buffer
+  long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
+  int32_t dense_half;       // -1: graduation buffer drained by the caller; 0 / 1: half used by this chunk
   int32_t direct;           // pool_slots >= V: vertex v owns slot v, no free stack, no eviction
 };
 
@@ -127,7 +131,17 @@ struct taurus_ctx {
   long long* d_grad_ids = nullptr;
   float* d_grad_rows = nullptr;
   int32_t* d_done_list = nullptr;
-  float* d_X = nullptr;          // staged feature chunk [chunk_sources x Kmax]
+  float* d_X[2] = {nullptr, nullptr};   // staged feature chunks [chunk_sources x Kmax], double-buffered
+  cudaStream_t copy_stream = nullptr;   // host -> device feature copies run here, ahead of the compute stream
+  cudaEvent_t x_ready[2] = {nullptr, nullptr}, x_free[2] = {nullptr, nullptr};
+  bool x_used[2] = {false, false};
+  long long host_pushes = 0;
+  // dense-output mode (taurus_layer_set_dense_output)
+  float* dense_out = nullptr;           // device-visible address of the caller's matrix, NULL = mode off
+  long long dense_ld = 0;
+  cudaStream_t out_stream = nullptr;    // rows leave the graduation buffer here while the next chunk computes
+  cudaEvent_t fin_done[2] = {nullptr, nullptr}, out_done[2] = {nullptr, nullptr};
+  bool half_used[2] = {false, false};
   float* d_PT = nullptr;         // projected chunk [chunk_sources x 2 Hmax]
   long long* d_csc_ptr = nullptr;
   uint32_t* d_csc_eid = nullptr;
@@ -167,6 +181,7 @@ void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);   // plan, select, evict, alloc/reload
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // finalise + commit
 void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st);
+void launch_place_half(taurus_ctx* c, int half, int d_out, int Hp, cudaStream_t st);   // dense-output mode
 void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st);
 void launch_completion_ranks(taurus_ctx* c, cudaStream_t st);                // fills d_rank_hist
 long long max_window_edges(taurus_ctx* c);                                  // most edges of any chunk_sources consecutive sources

@@ -8,7 +8,7 @@ import taurus_gen as tg
 
 
 def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_features=False, drain_rows=None,
-                host_evict_rows=None, chunk_plan=None, gemm_mode=None):
+                host_evict_rows=None, chunk_plan=None, gemm_mode=None, dense_output=False):
     """Runs every layer of workload w on the GPU.  Returns per-layer outputs (float32 [V, d_out]), the ids each
     chunk completed, stats and chunk logs.  Layer l+1 streams layer l's drained output."""
     import torch
@@ -21,7 +21,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
         0 if w.pool_slots >= V - w.hub_count else V - w.hub_count)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
-                     drain_rows or V, w.gemm_mode if gemm_mode is None else gemm_mode, flags)
+                     drain_rows or (2 * V if dense_output else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags)
     res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
     if host_features:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
@@ -30,7 +30,10 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
     stream = torch.cuda.current_stream()
     for l in range(L):
         d_out = w.dims[l + 1]
-        dense = torch.zeros((V, d_out), dtype=torch.float32, device=dev)
+        if dense_output and host_features:
+            dense = torch.zeros((V, d_out), dtype=torch.float32).pin_memory()
+        else:
+            dense = torch.zeros((V, d_out), dtype=torch.float32, device=dev)
         ids_buf = torch.empty(V, dtype=torch.int64, device=dev)
         ctx.layer_begin(l, stream)
         if w.fanout[l] > 0:
@@ -39,24 +42,31 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
             res["masks"].append(None)
         per_chunk = []
         plan = chunk_plan or [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
-        for (s, e) in plan:
-            rc = ctx.push_chunk(s, e, feat[s:e], stream, raise_on_drain_full=False)
-            if rc != 0:   # graduation buffer could overflow: drain, then push again
-                n = ctx.drain_dense(dense, d_out, V, ids_buf)
-                per_chunk.append(("drain", ids_buf[:n].cpu().numpy().copy()))
+        if dense_output:      # the library places every finalised row itself; nothing to drain
+            ctx.layer_set_dense_output(dense, d_out)
+            for (s, e) in plan:
                 ctx.push_chunk(s, e, feat[s:e], stream)
-            if drain_each_chunk:
-                n = ctx.drain_dense(dense, d_out, V, ids_buf)
-                per_chunk.append(ids_buf[:n].cpu().numpy().copy())
-        n = ctx.drain_dense(dense, d_out, V, ids_buf)
-        if n or not drain_each_chunk:
-            per_chunk.append(("tail", ids_buf[:n].cpu().numpy().copy()))
+            assert ctx.drain_dense(dense, d_out, V, ids_buf) == 0
+            per_chunk = None
+        else:
+            for (s, e) in plan:
+                rc = ctx.push_chunk(s, e, feat[s:e], stream, raise_on_drain_full=False)
+                if rc != 0:   # graduation buffer could overflow: drain, then push again
+                    n = ctx.drain_dense(dense, d_out, V, ids_buf)
+                    per_chunk.append(("drain", ids_buf[:n].cpu().numpy().copy()))
+                    ctx.push_chunk(s, e, feat[s:e], stream)
+                if drain_each_chunk:
+                    n = ctx.drain_dense(dense, d_out, V, ids_buf)
+                    per_chunk.append(ids_buf[:n].cpu().numpy().copy())
+            n = ctx.drain_dense(dense, d_out, V, ids_buf)
+            if n or not drain_each_chunk:
+                per_chunk.append(("tail", ids_buf[:n].cpu().numpy().copy()))
         res["stats"].append(ctx.layer_end())
         res["chunk_log"].append(ctx.get_chunk_log())
         res["reload_count"].append(ctx.get_vertex_array("reload_count"))
         res["completed"].append(per_chunk)
         res["outs"].append(dense.cpu().numpy())
-        feat = dense.cpu().pin_memory() if host_features else dense
+        feat = dense if (dense_output or not host_features) else dense.cpu().pin_memory()
     return res
 
 

@@ -45,6 +45,18 @@ def _full_check(w, g=None, bias_scale=0.3, tol=FP32_TOL, **kw):
     return lib, orc
 
 
+@pytest.mark.parametrize("host", [False, True])
+def test_dense_output_mode_overlapped_copies(host):
+    """The library places finalised rows itself (double-buffered graduation halves on an internal stream) and
+    stages host-pinned feature chunks on its copy stream; results and accounting are unchanged."""
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 60_000, chunk=1024)
+    w = replace(w, dims=(128, 256, 64), fanout=(0, 0), pool_slots=16_000, hub_count=60)
+    _full_check(w, dense_output=True, host_features=host)
+    w = tg.scaled(tg.WORKLOADS["mid"], 30_011, chunk=4096)
+    _full_check(w, dense_output=True, host_features=host)
+
+
 def test_eviction_and_hub_store_small_pool():
     """Scaled 'large' shape: pool well below the peak active set, hubs pinned; accounting bit-exact."""
     from dataclasses import replace
