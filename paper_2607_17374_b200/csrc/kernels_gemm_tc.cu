@@ -2,16 +2,17 @@
 // epilogue, for one pushed chunk (Sect. 3.6 puts the layer transform on the GPU; here it runs before the
 // aggregation, which is legal by linearity, SAGEConv paragraph of Sect. 3.9).
 //
-// One CTA per 128-row tile of X.  Roles (10 warps):
+// Persistent kernel: one CTA per SM walks (128-row tile of X, block of up to 256 output columns) units.  Roles (10 warps):
 //   warp 0        TMA producer: cp.async.bulk.tensor loads of the raw fp32 X tile and the W operand tiles
 //   warp 1        MMA issuer: tcgen05.mma, accumulators in TMEM (two buffers of up to 256 columns)
 //   warps 2..5    converter: turns the raw fp32 X tile in shared memory into tensor-core operands
 //                   fp32 mode : hi = x with the low 13 mantissa bits cleared (in place), lo = x - hi (exact);
 //                               acc += lo.Whi + hi.Wlo + hi.Whi   (three kind::tf32 MMAs, small terms first)
 //                   bf16 mode : bf16(x), one kind::f16 MMA
-//   warps 6..9    epilogue: tcgen05.ld of the accumulator, per-row scaling / bias, fp32 stores
-// The output columns are processed in blocks of up to 256; the epilogue of block j overlaps the main loop of
-// block j+1 through the second TMEM buffer.
+//   warps 6..9    epilogue: tcgen05.ld of the accumulator, per-row scaling / bias, 32 x 32 tiles staged in shared
+//                 memory and written with TMA stores (full 128-byte lines)
+// The output columns of a tile are processed in blocks of up to 256; (tile, block) units alternate between two
+// TMEM accumulator buffers, so the epilogue of one unit overlaps the main loop of the next, also across tiles.
 //
 // Every wait on an mbarrier is bounded: after WAIT_LIMIT polls the kernel raises a CTA-wide abort flag,
 // records TAURUS_ERR_INTERNAL in the control block, waits (bounded) for its TMA copies in flight, frees its
@@ -32,6 +33,8 @@ constexpr int TILE_A_BYTES = BM * 128;           // 128 rows x 128 B
 constexpr int TILE_B_BYTES = BN_MAX * 128;       // 256 rows x 128 B
 constexpr unsigned WAIT_LIMIT = 1u << 24;
 constexpr int NUM_THREADS = 320;
+constexpr int OUT_TILE_BYTES = 32 * 128;        // epilogue staging tile: 32 rows x 32 fp32, 128B-swizzled
+constexpr int OUT_STAGING_BYTES = 4 * 2 * OUT_TILE_BYTES;   // 4 epilogue warps x 2 tiles
 
 struct __align__(8) Barriers {
   unsigned long long full[STAGES], conv[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
@@ -118,16 +121,17 @@ struct GemmArgs {
 template <bool BF16>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_b0,
-                  const __grid_constant__ CUtensorMap map_b1, GemmArgs g) {
+                  const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_out, GemmArgs g) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int STAGE_BYTES = BF16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32;
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + STAGES * STAGE_BYTES);
+  unsigned char* out_staging = smem + STAGES * STAGE_BYTES;
+  Barriers* bars = reinterpret_cast<Barriers*>(out_staging + OUT_STAGING_BYTES);
   volatile int* abort_flag = &bars->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row0 = blockIdx.x * BM;
+  const int n_tiles = (g.n + BM - 1) / BM;
   const int n_blocks = (g.Np + BN_MAX - 1) / BN_MAX;
-  const int tmem_cols = g.Np <= 32 ? 32 : g.Np <= 64 ? 64 : g.Np <= 128 ? 128 : g.Np <= 256 ? 256 : 512;
+  const int tmem_cols = 512;   // two accumulator buffers of 256 columns; one CTA per SM
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->conv[s], 128); mbar_init(&bars->empty[s], 1); }
@@ -150,7 +154,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       int it = 0;
-      for (int nb = 0; nb < n_blocks && !*abort_flag; ++nb) {
+      for (int w = blockIdx.x; w < n_tiles * n_blocks && !*abort_flag; w += gridDim.x) {
+        const int tile = w / n_blocks, nb = w % n_blocks;
+        const int row0 = tile * BM;
         const int col0 = nb * BN_MAX;
         for (int ks = 0; ks < g.k_stages; ++ks, ++it) {
           const int s = it % STAGES;
@@ -174,11 +180,12 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      int it = 0;
-      for (int nb = 0; nb < n_blocks && !*abort_flag; ++nb) {
+      int it = 0, unit = 0;
+      for (int w = blockIdx.x; w < n_tiles * n_blocks && !*abort_flag; w += gridDim.x, ++unit) {
+        const int nb = w % n_blocks;
         const int bw = (g.Np - nb * BN_MAX) < BN_MAX ? (g.Np - nb * BN_MAX) : BN_MAX;
-        const int buf = nb & 1;
-        if (nb >= 2 && !mbar_wait(&bars->acc_empty[buf], ((nb >> 1) & 1) ^ 1, abort_flag)) break;
+        const int buf = unit & 1;
+        if (unit >= 2 && !mbar_wait(&bars->acc_empty[buf], ((unit >> 1) & 1) ^ 1, abort_flag)) break;
         tc_fence_after();
         const unsigned tmem_d = tmem_base + (unsigned)(buf * BN_MAX);
         const unsigned idesc = (1u << 4) | ((BF16 ? 1u : 2u) << 7) | ((BF16 ? 1u : 2u) << 10) |
@@ -214,7 +221,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     // ---------------------------------------------------------------- converter (128 threads)
     const int t = threadIdx.x - 64;
     int it = 0;
-    for (int nb = 0; nb < n_blocks && !*abort_flag; ++nb) {
+    for (int w = blockIdx.x; w < n_tiles * n_blocks && !*abort_flag; w += gridDim.x) {
       bool ok = true;
       for (int ks = 0; ks < g.k_stages; ++ks, ++it) {
         const int s = it % STAGES;
@@ -262,7 +269,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   } else {
     // ---------------------------------------------------------------- epilogue (warps 6..9, TMEM lanes 32 * (warp % 4))
     const int q = warp & 3;
-    const int r = row0 + q * 32 + lane;
+    int unit = 0, out_it = 0;
+    for (int w = blockIdx.x; w < n_tiles * n_blocks && !*abort_flag; w += gridDim.x, ++unit) {
+    const int tile = w / n_blocks, nb = w % n_blocks;
+    const int r = tile * BM + q * 32 + lane;
     float c_out = 1.f, self_mul = 1.f;
     if (r < g.n) {
       const long long u = g.src_begin + r;
@@ -274,10 +284,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         self_mul = (float)(m > 1 ? m : 1);
       }
     }
-    for (int nb = 0; nb < n_blocks && !*abort_flag; ++nb) {
+    {
       const int bw = (g.Np - nb * BN_MAX) < BN_MAX ? (g.Np - nb * BN_MAX) : BN_MAX;
-      const int buf = nb & 1;
-      if (!mbar_wait(&bars->acc_full[buf], (nb >> 1) & 1, abort_flag)) break;
+      const int buf = unit & 1;
+      if (!mbar_wait(&bars->acc_full[buf], (unit >> 1) & 1, abort_flag)) break;
       tc_fence_after();
       for (int c0 = 0; c0 < bw; c0 += 32) {
         unsigned v[32];
@@ -291,27 +301,41 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
               "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
             : "r"(taddr) : "memory");
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (r < g.n) {
-          const int cbase = nb * BN_MAX + c0;
-          float* out = g.PT + (size_t)r * g.N + cbase;
+        const int cbase = nb * BN_MAX + c0;
+        if (cbase >= g.N) continue;           // padding columns of the last block
+        // this warp's staging tile: 32 rows (lane = row) x 32 columns, 16-byte chunk c of row r at chunk c ^ (r & 7)
+        unsigned char* tile_smem = out_staging + (q * 2 + (out_it & 1)) * OUT_TILE_BYTES;
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store that last used this tile has read it
+        __syncwarp();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            if (cbase + j >= g.N) break;      // N is a multiple of 4: whole float4 in or out
-            float4 o;
-            float* po = &o.x;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int c = cbase + j + e;
-              float x = __uint_as_float(v[j + e]);
-              po[e] = (c < g.Hp) ? x * c_out : (x + g.bias[c - g.Hp]) * self_mul;
-            }
-            *reinterpret_cast<float4*>(out + j) = o;
+        for (int j = 0; j < 32; j += 4) {
+          float4 o;
+          float* po = &o.x;
+          const int c = cbase + j;
+          if (c >= g.Hp && c < g.N) {         // T columns: (x W_self + b) * max(|M(u)|, 1)
+            const float4 b = *reinterpret_cast<const float4*>(g.bias + (c - g.Hp));
+            po[0] = (__uint_as_float(v[j]) + b.x) * self_mul; po[1] = (__uint_as_float(v[j + 1]) + b.y) * self_mul;
+            po[2] = (__uint_as_float(v[j + 2]) + b.z) * self_mul; po[3] = (__uint_as_float(v[j + 3]) + b.w) * self_mul;
+          } else {                            // P columns: c_out(u) * (x W_neigh)
+            po[0] = __uint_as_float(v[j]) * c_out; po[1] = __uint_as_float(v[j + 1]) * c_out;
+            po[2] = __uint_as_float(v[j + 2]) * c_out; po[3] = __uint_as_float(v[j + 3]) * c_out;
           }
+          *reinterpret_cast<float4*>(tile_smem + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) = o;
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {                      // rows beyond n and columns beyond N are clipped by the tensor map
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                       ::"l"(&map_out), "r"(cbase), "r"(tile * BM + q * 32), "r"(smem_u32(tile_smem)) : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        ++out_it;
       }
       tc_fence_before();
       mbar_arrive(&bars->acc_empty[buf]);
     }
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all stores of this warp are complete
   }
 
   // ---------------------------------------------------------------- teardown
@@ -353,7 +377,8 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D row-major tensor [rows x cols] of `elem` bytes, box [box_rows x box_cols], 128-byte swizzle, zero fill.
+// 2-D row-major tensor [rows x cols] of `elem` bytes, box [box_rows x box_cols], 128-byte swizzle, zero fill
+// on loads, clipping on stores.
 bool make_map(CUtensorMap* m, const void* base, CUtensorMapDataType dt, int elem, long long rows, long long cols,
               long long ld_elems, int box_rows, int box_cols) {
   EncodeTiledFn fn = encode_fn();
@@ -438,20 +463,24 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   const int N = c->mode == TAURUS_SAGE_MEAN ? 2 * Hp : Hp;
   CUtensorMap map_x;
   if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, 32)) return TAURUS_ERR_CUDA;
+  CUtensorMap map_out;
+  if (!make_map(&map_out, c->d_PT, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, N, N, 32, 32)) return TAURUS_ERR_CUDA;
   GemmArgs g;
   g.PT = c->d_PT; g.n = n; g.N = N; g.Np = w->Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
   g.b_box_bytes = (w->Np < BN_MAX ? w->Np : BN_MAX) * 128;
   g.Hp = Hp; g.mode = c->mode; g.fanout = c->fanout[layer]; g.bias = c->d_bias[layer];
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = src_begin; g.ctl = c->d_ctl;
-  const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + (int)sizeof(Barriers) + 1024;
-  const int grid = (n + BM - 1) / BM;
+  const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
+  const int n_tiles = (n + BM - 1) / BM;
+  const int n_units = n_tiles * ((w->Np + BN_MAX - 1) / BN_MAX);
+  const int grid = n_units < c->sm_count ? n_units : c->sm_count;
   static bool attr_set[2] = {false, false};
   if (bf16) {
     if (!attr_set[1]) { cudaFuncSetAttribute(project_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); attr_set[1] = true; }
-    project_tc_kernel<true><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, g);
+    project_tc_kernel<true><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, map_out, g);
   } else {
     if (!attr_set[0]) { cudaFuncSetAttribute(project_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); attr_set[0] = true; }
-    project_tc_kernel<false><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, g);
+    project_tc_kernel<false><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, map_out, g);
   }
   c->launches += 1;
   return TAURUS_OK;
