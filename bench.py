@@ -29,8 +29,8 @@ import taurus_gen as tg  # noqa: E402
 
 
 # DRAM bytes (read + write) per accumulator-row reduction of scatter_grouped_kernel<32,2>, from the ncu capture
-# summarised in profiles/scatter_grouped_kernel_mid_1200k.md (2.70 GB per launch / 1.486 M groups).
-SCATTER_TRAFFIC_PER_GROUP_BYTES = 1817.0
+# summarised in profiles/scatter_grouped_kernel_mid_1200k.md (2.67 GB per launch / 0.98 M groups).
+SCATTER_TRAFFIC_PER_GROUP_BYTES = 2720.0
 
 
 def parse_args():
