@@ -149,6 +149,24 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------------------------- ranks
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time: every rank runs an independent replica, the job is as slow as its slowest rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank_step: float, steps: int, world: int, ms_max: float) -> float:
+    """Units all ranks processed / the slowest rank's time, in 1e9 units per second (weak scaling: replicas only)."""
+    return world * units_per_rank_step * steps / (ms_max * 1e-3) / 1e9
+
+
 # ----------------------------------------------------------------------------------------------- our arm
 
 def run_ours(args):
@@ -235,11 +253,8 @@ def run_ours(args):
     sampler.stop_flag.set()
     sampler.join()
     phases = ctx.get_phase_ms()   # [pushes, 5]
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max = float(t.item())
-    value = world * msgs_per_step * args.steps / (ms_max * 1e-3) / 1e9
+    ms_max = max_over_ranks(ms, world, dev)
+    value = whole_job_value(msgs_per_step, args.steps, world, ms_max)
 
     # ---- roofline of the dominant kernel (the scatter), from the events recorded inside the timed region
     n_push = len(chunks) * L * args.steps
@@ -293,11 +308,8 @@ def run_ours(args):
         e1.record(stream)
         barrier()
         wall = (time.time() - t0) * 1e3
-        t = torch.tensor([max(e0.elapsed_time(e1), wall)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-        e2e = dict(value=world * msgs_per_step * args.steps / (e2e_ms * 1e-3) / 1e9, unit="GTEPS",
+        e2e_ms = max_over_ranks(max(e0.elapsed_time(e1), wall), world, dev)
+        e2e = dict(value=whole_job_value(msgs_per_step, args.steps, world, e2e_ms), unit="GTEPS",
                    ms_per_step=e2e_ms / args.steps,
                    h2d_bytes_per_step=int(4 * V * w.dims[0]), d2h_bytes_per_step=int(4 * V * w.dims[-1]),
                    note="layer-0 features host -> device per chunk, last layer's rows device -> host; intermediate layers in HBM")
