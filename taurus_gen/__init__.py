@@ -56,6 +56,8 @@ def _lib():
         lib.tg_in_degrees.argtypes = [ctypes.c_int64, ctypes.c_int64, vp, vp]
         lib.tg_features.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int32, ctypes.c_int64, vp]
+        lib.tg_features_rows.argtypes = [ctypes.c_uint64, ctypes.c_uint64, vp, ctypes.c_int64, ctypes.c_int32,
+                                         ctypes.c_int64, vp]
         lib.tg_weights.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int32,
                                    ctypes.c_int32, vp]
         lib.tg_zipf_top_mass.restype = ctypes.c_double
@@ -205,6 +207,14 @@ def features(seed: int, layer_tag: int, v_begin: int, v_end: int, F: int, out: O
         out = np.zeros((n, ld), dtype=np.float32) if ld != F else np.empty((n, F), dtype=np.float32)
     assert out.dtype == np.float32 and out.flags.c_contiguous and out.size >= n * ld
     _lib().tg_features(seed, layer_tag, v_begin, v_end, F, ld, out.ctypes.data)
+    return out
+
+
+def features_rows(seed: int, layer_tag: int, ids: np.ndarray, F: int) -> np.ndarray:
+    """Feature rows of the listed vertices, [len(ids), F] fp32 (same values as features())."""
+    ids = np.ascontiguousarray(ids, dtype=np.int64)
+    out = np.empty((ids.size, F), dtype=np.float32)
+    _lib().tg_features_rows(seed, layer_tag, ids.ctypes.data, ids.size, F, F, out.ctypes.data)
     return out
 
 

@@ -207,6 +207,13 @@ int tg_features(uint64_t seed, uint64_t layer_tag, int64_t v_begin, int64_t v_en
   return 0;
 }
 
+/* The same rows for an arbitrary list of vertex ids (row i of out = features of ids[i]). */
+int tg_features_rows(uint64_t seed, uint64_t layer_tag, const int64_t* ids, int64_t n, int32_t F, int64_t ld, float* out) {
+#pragma omp parallel for schedule(static)
+  for (int64_t i = 0; i < n; ++i) tg_features(seed, layer_tag, ids[i], ids[i] + 1, F, ld, out + i * ld);
+  return 0;
+}
+
 /* Xavier-uniform rows x cols matrix, U(-a, a), a = sqrt(6 / (rows + cols)), row-major fp32 */
 int tg_weights(uint64_t seed, uint64_t layer, uint64_t which, int32_t rows, int32_t cols, float* out) {
   double a = sqrt(6.0 / ((double)rows + (double)cols));
