@@ -231,3 +231,20 @@ def test_gcn_bf16_mode():
     w = tg.scaled(tg.WORKLOADS["stress"], 30_000, chunk=2048)
     w = replace(w, dims=(512, 256, 256), pool_slots=30_000)
     _full_check(w, tol=BF16_TOL)
+
+
+def test_csr_order_kernels_under_eviction_sampling_and_hubs():
+    """TAURUS_FLAG_NO_GROUPING: every chunk takes the CSR-order classify / scatter kernels (the path of chunks that
+    are not cells of the chunk grid); same results, same accounting."""
+    import paper_2607_17374_b200 as tb
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["sampled"], 50_000, chunk=2048)
+    w = replace(w, dims=(128, 256, 256, 47), pool_slots=28_000, hub_count=50)
+    g = tg.make_graph(w)
+    lib, orc = _full_check(w, g, flags=tb.FLAG_NO_GROUPING)
+    for l in range(w.L):
+        want = np.packbits(orc["msets"][l].prop, bitorder="little")
+        assert (lib["masks"][l].view(np.uint8)[:want.size] == want).all()
+        assert lib["stats"][l]["scatter_groups"] == lib["stats"][l]["total_messages"]   # one reduction per message
+    w = replace(tg.scaled(tg.WORKLOADS["stress"], 40_000, chunk=1024), dims=(96, 128, 32), gemm_mode=tg.GEMM_FP32, pool_slots=20_000)
+    _full_check(w, flags=tb.FLAG_NO_GROUPING)
