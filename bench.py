@@ -64,33 +64,61 @@ def peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples the SM clock and the throttle reasons while the timed region runs: through NVML every 10 ms
+    when the bindings are importable (read-only queries), else through nvidia-smi every 200 ms."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    # NVML clocks-event reason bits
+    BITS = {"sw_power_cap": 0x4, "hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
 
     def __init__(self, index: int):
         super().__init__(daemon=True)
-        self.index, self.stop_flag, self.samples = index, threading.Event(), []
+        self.index, self.stop_flag = index, threading.Event()
+        self.mhz, self.reasons, self.max_mhz, self.source = [], set(), None, None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible and all(x.strip().isdigit() for x in visible.split(",")):
+                phys = int(visible.split(",")[index])
+            self.nvml, self.handle = pynvml, pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+            self.source = "nvml"
+        except Exception:
+            self.nvml = None
+            self.source = "nvidia-smi"
 
     def run(self):
         while not self.stop_flag.is_set():
             try:
-                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
-                f = [x.strip() for x in out.strip().split(",")]
-                if len(f) >= 6:
-                    self.samples.append(f)
+                if self.nvml is not None:
+                    self.mhz.append(float(self.nvml.nvmlDeviceGetClockInfo(self.handle, self.nvml.NVML_CLOCK_SM)))
+                    bits = int(self.nvml.nvmlDeviceGetCurrentClocksEventReasons(self.handle)) \
+                        if hasattr(self.nvml, "nvmlDeviceGetCurrentClocksEventReasons") \
+                        else int(self.nvml.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                    for name, bit in self.BITS.items():
+                        if bits & bit:
+                            self.reasons.add(name)
+                else:
+                    out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                    f = [x.strip() for x in out.strip().split(",")]
+                    if len(f) >= 6:
+                        self.mhz.append(float(f[0])); self.max_mhz = float(f[1])
+                        for i, name in enumerate(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]):
+                            if f[2 + i].lower().startswith("active"):
+                                self.reasons.add(name)
             except Exception:
                 pass
-            self.stop_flag.wait(0.2)
+            self.stop_flag.wait(0.01 if self.nvml is not None else 0.2)
 
     def summary(self):
-        if not self.samples:
-            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
-        mhz = sorted(float(s[0]) for s in self.samples)
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
-        return dict(sm_mhz=mhz[len(mhz) // 2], sm_max_mhz=float(self.samples[0][1]), reasons=reasons, samples=len(mhz))
+        if not self.mhz:
+            return dict(sm_mhz=None, sm_max_mhz=self.max_mhz, reasons=[], samples=0, source=self.source)
+        mhz = sorted(self.mhz)
+        return dict(sm_mhz=mhz[len(mhz) // 2], sm_max_mhz=self.max_mhz, reasons=sorted(self.reasons), samples=len(mhz),
+                    source=self.source)
 
 
 # ----------------------------------------------------------------------------------------------- reference arm / CPU baseline

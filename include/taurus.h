@@ -34,7 +34,7 @@
  * the exceptions stated at taurus_push_chunk.  The library owns all state
  * behind taurus_ctx.  A context is bound to the device current at
  * taurus_graph_init and is not thread-safe.  Errors found on the device
- * (pool too small, host store full, index out of bounds in a checked build)
+ * (pool too small, host store full, a slot / vertex index or pending count out of range)
  * are sticky: the chunk that hit one is not applied and every later call
  * on the context returns the code.
  */
@@ -102,7 +102,6 @@ typedef struct {
 } taurus_run;
 
 enum {
-  TAURUS_FLAG_CHECKED = 1,      /* bounds-check every slot / vertex index on the device (slower; sets ERR_INTERNAL) */
   TAURUS_FLAG_SIMT_GEMM = 2,    /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */
   TAURUS_FLAG_NO_GROUPING = 4   /* do not build the destination-grouped edge order: every chunk takes the CSR-order kernels */
 };

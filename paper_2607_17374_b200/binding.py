@@ -10,7 +10,7 @@ import numpy as np
 
 SAGE_MEAN, GCN_SYM = 0, 1
 GEMM_FP32, GEMM_BF16 = 0, 1
-FLAG_CHECKED, FLAG_SIMT_GEMM, FLAG_NO_GROUPING = 1, 2, 4
+FLAG_SIMT_GEMM, FLAG_NO_GROUPING = 2, 4
 CHUNK_LOG_COLUMNS = ["hs", "ns", "ev", "gs", "need", "evicted", "reloaded", "completed", "occupancy"]
 ERROR_CODES = {
     "OK": 0, "INVALID_ARG": -1, "ORDER": -2, "POOL_TOO_SMALL": -3, "HOST_STORE_FULL": -4, "DRAIN_FULL": -5,

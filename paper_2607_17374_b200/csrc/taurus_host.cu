@@ -329,7 +329,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.V = c->V; a.pool_slots = c->pool_slots; a.hub_count = c->hub_count; a.host_rows = c->host_rows; a.drain_rows = c->drain_rows;
   a.src_begin = s; a.src_end = e;
   a.epoch = (int32_t)(c->chunk_seq + 1);
-  a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.checked = (c->flags & TAURUS_FLAG_CHECKED) ? 1 : 0;
+  a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l];
   a.direct = c->pool_slots >= c->V ? 1 : 0;
   a.dense_half = c->dense_out ? (int)(c->chunk_seq & 1) : -1;
   a.grad_cap = c->dense_out ? c->drain_rows / 2 : c->drain_rows;

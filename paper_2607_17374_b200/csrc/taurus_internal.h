@@ -42,7 +42,6 @@ struct DevCtl {
   long long evictions, reloads, peak_occupancy, hub_messages, total_messages, completed;
   long long sum_hs, sum_ns, sum_ev, sum_gs, chunks;
   long long scatter_groups; // accumulator-row reductions issued by the scatter (self messages not counted)
-  long long bad_index;      // first out-of-range index seen by a checked kernel (debug aid)
 };
 
 // Everything the per-chunk kernels need, passed by value.
@@ -84,7 +83,7 @@ struct ChunkArgs {
   long long src_begin, src_end;
   int32_t epoch;            // chunk sequence number + 1 within the layer
   int32_t Hp;               // padded accumulator width (multiple of 4)
-  int32_t mode, act, fanout, checked;
+  int32_t mode, act, fanout;
   long long grad_off;       // dense-output mode: first row of this chunk's half of the graduation buffer
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
   int32_t dense_half;       // -1: graduation buffer drained by the caller; 0 / 1: half used by this chunk

@@ -248,3 +248,53 @@ def test_csr_order_kernels_under_eviction_sampling_and_hubs():
         assert lib["stats"][l]["scatter_groups"] == lib["stats"][l]["total_messages"]   # one reduction per message
     w = replace(tg.scaled(tg.WORKLOADS["stress"], 40_000, chunk=1024), dims=(96, 128, 32), gemm_mode=tg.GEMM_FP32, pool_slots=20_000)
     _full_check(w, flags=tb.FLAG_NO_GROUPING)
+
+
+def test_device_detected_capacity_errors_are_sticky():
+    """Too few eligible victims and an exhausted pinned host store are found on the device, reported by the next
+    blocking call and by every call after it; the context stays usable for destroy."""
+    import paper_2607_17374_b200 as tb
+    import torch
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 60_000, chunk=1024)
+    w = replace(w, dims=(128, 64), fanout=(0,), hub_count=60)
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    x = torch.from_numpy(tg.features(1, 0, 0, g.V, 128)).cuda()
+    ids = torch.empty(g.V, dtype=torch.int64, device="cuda"); rows = torch.empty((g.V, 64), device="cuda")
+
+    def run(pool, host_rows):
+        ctx = tb.Context(g.V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
+                         model.act, 1024, pool, 60, None, 1, host_rows, g.V, 0, 0)
+        ctx.layer_begin(0)
+        code = 0
+        try:
+            for s in range(0, g.V, 1024):
+                ctx.push_chunk(s, min(s + 1024, g.V), x[s:s + 1024])
+                ctx.drain_completed(ids, rows, g.V)
+        except tb.TaurusError as e:
+            code = e.code
+            with pytest.raises(tb.TaurusError) as again:      # sticky
+                ctx.get_stats()
+            assert again.value.code == code
+        ctx.destroy()
+        return code
+
+    assert run(16_000, g.V) == 0                                           # the reference point: this pool works
+    assert run(12_000, g.V) == tb.ERROR_CODES["POOL_TOO_SMALL"]           # need fits, but too few untouched victims
+    assert run(16_000, 2_000) == tb.ERROR_CODES["HOST_STORE_FULL"]        # more rows evicted at once than host rows
+
+
+def test_vertex_arrays_after_a_layer():
+    import paper_2607_17374_b200 as tb
+    w = tg.WORKLOADS["tiny"]
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
+    lib = run_library(w, g, model, x0)
+    ctx = lib["ctx"]
+    assert (ctx.get_vertex_array("state") == 4).all()          # every vertex COMPLETED
+    assert (ctx.get_vertex_array("pending") == 0).all()
+    assert (ctx.get_vertex_array("hub") == 0).all()
+    st = ctx.get_stats()
+    assert st["completed"] == g.V and st["free_slots"] == w.pool_slots and st["chunks"] == 10
