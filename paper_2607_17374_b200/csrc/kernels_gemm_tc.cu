@@ -474,14 +474,14 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   const int n_tiles = (n + BM - 1) / BM;
   const int n_units = n_tiles * ((w->Np + BN_MAX - 1) / BN_MAX);
   const int grid = n_units < c->sm_count ? n_units : c->sm_count;
-  static bool attr_set[2] = {false, false};
-  if (bf16) {
-    if (!attr_set[1]) { cudaFuncSetAttribute(project_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); attr_set[1] = true; }
-    project_tc_kernel<true><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, map_out, g);
-  } else {
-    if (!attr_set[0]) { cudaFuncSetAttribute(project_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); attr_set[0] = true; }
-    project_tc_kernel<false><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, map_out, g);
+  if (!c->tc_smem_set) {   // once per context (the attribute belongs to the context's device)
+    cudaError_t e = bf16 ? cudaFuncSetAttribute(project_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                         : cudaFuncSetAttribute(project_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) { cudaGetLastError(); return TAURUS_ERR_CUDA; }
+    c->tc_smem_set = true;
   }
+  if (bf16) project_tc_kernel<true><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, map_out, g);
+  else project_tc_kernel<false><<<grid, NUM_THREADS, smem, st>>>(map_x, w->map_hi, w->map_lo, map_out, g);
   c->launches += 1;
   return TAURUS_OK;
 }

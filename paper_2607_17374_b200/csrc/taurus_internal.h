@@ -107,6 +107,7 @@ struct taurus_ctx {
   // weights per layer: Wcat is [Kp x Ncat] row-major fp32 (P columns then T columns), bias [Hp]
   float* d_Wcat[TAURUS_MAX_LAYERS] = {nullptr};
   float* d_bias[TAURUS_MAX_LAYERS] = {nullptr};
+  bool tc_smem_set = false;                        // dynamic shared memory limit of the projection kernel raised
   void* tc_image[TAURUS_MAX_LAYERS] = {nullptr};   // tensor-core operand images of Wcat (owned by kernels_gemm_tc.cu)
   // state
   int32_t* d_pend = nullptr;
