@@ -99,7 +99,17 @@ typedef struct {
   int64_t drain_rows;       /* capacity (rows) of the graduation buffer; must hold the completions of any one
                                pushed range as bounded by taurus_completion_bound (64-source granularity)  */
   int32_t flags;            /* TAURUS_FLAG_*                                                               */
+  int32_t evict_policy;     /* TAURUS_EVICT_*: which IN_BUFFER vertices leave first when the pool is full     */
 } taurus_run;
+
+/* Eviction policies: the paper's (Sect. 3.5.3) and the alternatives of its ablation (Sect. 4.5).  Victims are
+ * always the `deficit` smallest (score, vertex id) among IN_BUFFER vertices the chunk does not touch. */
+enum {
+  TAURUS_EVICT_FEWEST_PENDING = 0,  /* score = pending messages: closest to completion first          */
+  TAURUS_EVICT_FIFO = 1,            /* score = chunk in which the vertex (last) entered the pool       */
+  TAURUS_EVICT_LRU = 2,             /* score = chunk that last touched the vertex                      */
+  TAURUS_EVICT_RANDOM = 3           /* score = 31-bit hash of (seed, vertex, chunk index)              */
+};
 
 enum {
   TAURUS_FLAG_SIMT_GEMM = 2,    /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */

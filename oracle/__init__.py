@@ -34,6 +34,9 @@ _handle = None
 SAGE_MEAN = 0
 GCN_SYM = 1
 
+# eviction policies: the paper's (Sect. 3.5.3) and the alternatives of its ablation (Sect. 4.5)
+EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
+
 # vertex states, Sect. 3.4
 NOT_STARTED, IN_BUFFER, EVICTED, ON_GPU, COMPLETED = 0, 1, 2, 3, 4
 
@@ -62,7 +65,9 @@ def _lib():
         lib.to_sample_positions.argtypes = [u64, i32, i64, i64, i32, vp]
         lib.to_message_sets.argtypes = [i64, vp, vp, vp, i32, u64, i32, vp, vp, vp, vp]
         lib.to_aggregate.argtypes = [i64, vp, vp, vp, vp, vp, i32, vp]
-        lib.to_simulate.argtypes = [i64, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp, vp]
+        lib.to_simulate.argtypes = [i64, vp, vp, vp, vp, vp, i64, i64, i32, u64, vp, vp, vp, vp, vp]
+        lib.to_evict_hash.restype = ctypes.c_uint32
+        lib.to_evict_hash.argtypes = [u64, u64, u64]
         _handle = lib
     return _handle
 
@@ -243,7 +248,7 @@ class SimResult:
 
 
 def simulate(V: int, row_ptr: np.ndarray, col: np.ndarray, ms: MessageSets, is_hub: np.ndarray,
-             chunk_sources: int, pool_slots: int) -> SimResult:
+             chunk_sources: int, pool_slots: int, policy: int = EVICT_FEWEST_PENDING, seed: int = 0) -> SimResult:
     """Chunk-granular state machine (Sect. 3.4-3.6).  rc: 0 ok, -2/-3 pool too small."""
     n_chunks = (V + chunk_sources - 1) // chunk_sources
     stats = np.zeros(len(STAT_KEYS), np.int64)
@@ -253,7 +258,7 @@ def simulate(V: int, row_ptr: np.ndarray, col: np.ndarray, ms: MessageSets, is_h
     evlog = np.empty(V, np.int32)
     m = np.ascontiguousarray(ms.m, dtype=np.int32)
     hub = np.ascontiguousarray(is_hub, dtype=np.uint8)
-    rc = _lib().to_simulate(V, _p(row_ptr), _p(col), _p(ms.prop), _p(m), _p(hub), chunk_sources, pool_slots,
+    rc = _lib().to_simulate(V, _p(row_ptr), _p(col), _p(ms.prop), _p(m), _p(hub), chunk_sources, pool_slots, policy, seed,
                             _p(stats), _p(cc), _p(rcount), _p(per), _p(evlog))
     if rc == -1:
         raise MemoryError

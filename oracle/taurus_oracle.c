@@ -154,8 +154,12 @@ int to_aggregate(int64_t n_dst, const int64_t* dst, const int64_t* msg_ptr, cons
  *      together with the non-hub vertices of [s, e) themselves.
  *   2. record the split of T by state, and the hub vertices touched.
  *   3. need = #{v in T : NOT_STARTED or EVICTED};  need > pool_slots -> error.
- *   4. deficit = need - free; if > 0 evict the `deficit` smallest (pend, id)
- *      among IN_BUFFER vertices outside T (too few -> error).
+ *   4. deficit = need - free; if > 0 evict the `deficit` smallest (score, id)
+ *      among IN_BUFFER vertices outside T (too few -> error).  The score is the
+ *      pending count (the paper's policy, Sect. 3.5.3) or, for the ablation of
+ *      Sect. 4.5: the chunk in which the vertex entered the pool (FIFO), the
+ *      chunk that last touched it (LRU), or a hash of (seed, vertex, chunk)
+ *      (random).
  *   5. EVICTED in T -> IN_BUFFER (a reload); NOT_STARTED in T -> IN_BUFFER.
  *   6. deliver: pend[v] -= messages from [s, e) into v, and -1 for v in [s, e).
  *   7. vertices whose pend reached 0 complete; non-hub ones free their slot.
@@ -168,7 +172,18 @@ enum {
 /* per-chunk record columns */
 enum { CK_HS = 0, CK_NS, CK_EV, CK_GS, CK_NEED, CK_EVICTED, CK_RELOADED, CK_COMPLETED, CK_OCC, CK_COUNT };
 
-typedef struct { int32_t pend; int32_t id; } to_key;
+enum { EV_FEWEST_PENDING = 0, EV_FIFO = 1, EV_LRU = 2, EV_RANDOM = 3 };
+
+/* 31-bit score of the random policy */
+uint32_t to_evict_hash(uint64_t seed, uint64_t vertex, uint64_t chunk) {
+  uint64_t h = 0x452821E638D01377ull;
+  h = to_absorb(h, seed);
+  h = to_absorb(h, vertex);
+  h = to_absorb(h, chunk);
+  return (uint32_t)(h >> 33);
+}
+
+typedef struct { int32_t pend; int32_t id; } to_key;   /* pend holds the policy's score */
 static int cmp_key(const void* a, const void* b) {
   const to_key* x = (const to_key*)a; const to_key* y = (const to_key*)b;
   if (x->pend != y->pend) return (x->pend > y->pend) - (x->pend < y->pend);
@@ -184,7 +199,7 @@ static int to_allowed(int a, int b) {
 /* returns 0, -1 (out of memory), -2 (pool too small: need > pool), -3 (pool too small: too few victims) */
 int to_simulate(int64_t V, const int64_t* row_ptr, const int32_t* col, const uint8_t* prop /*NULL = all*/,
                 const int32_t* m /*[V] = |M(v)|*/, const uint8_t* is_hub /*[V]*/,
-                int64_t chunk_sources, int64_t pool_slots,
+                int64_t chunk_sources, int64_t pool_slots, int32_t policy, uint64_t seed,
                 int64_t* stats /*[SK_COUNT]*/, int32_t* complete_chunk /*[V]*/, int32_t* reload_count /*[V]*/,
                 int64_t* per_chunk /*[n_chunks, CK_COUNT]*/, int32_t* evict_chunk_log /*[V] last chunk evicted, -1*/) {
   int64_t n_chunks = (V + chunk_sources - 1) / chunk_sources;
@@ -194,7 +209,9 @@ int to_simulate(int64_t V, const int64_t* row_ptr, const int32_t* col, const uin
   int32_t* T = (int32_t*)malloc(sizeof(int32_t) * (size_t)V);
   int32_t* hubT = (int32_t*)malloc(sizeof(int32_t) * (size_t)V);
   to_key* cand = (to_key*)malloc(sizeof(to_key) * (size_t)V);
-  if (!state || !pend || !stamp || !T || !hubT || !cand) return -1;
+  int32_t* entered = (int32_t*)calloc((size_t)V, sizeof(int32_t));   /* chunk of the latest NS/EV -> IB */
+  int32_t* touched_at = (int32_t*)calloc((size_t)V, sizeof(int32_t)); /* chunk of the latest touch */
+  if (!state || !pend || !stamp || !T || !hubT || !cand || !entered || !touched_at) return -1;
   memset(stats, 0, sizeof(int64_t) * SK_COUNT);
   int64_t free_slots = pool_slots, occupied = 0;
   int rc = 0;
@@ -234,7 +251,13 @@ int to_simulate(int64_t V, const int64_t* row_ptr, const int32_t* col, const uin
     if (deficit > 0) {
       int64_t nc = 0;
       for (int64_t v = 0; v < V; ++v)
-        if (state[v] == ST_IB && stamp[v] != c) { cand[nc].pend = pend[v]; cand[nc].id = (int32_t)v; nc++; }
+        if (state[v] == ST_IB && stamp[v] != c) {
+          int32_t score = pend[v];
+          if (policy == EV_FIFO) score = entered[v];
+          else if (policy == EV_LRU) score = touched_at[v];
+          else if (policy == EV_RANDOM) score = (int32_t)to_evict_hash(seed, (uint64_t)v, (uint64_t)c);
+          cand[nc].pend = score; cand[nc].id = (int32_t)v; nc++;
+        }
       if (nc < deficit) { rc = -3; break; }
       qsort(cand, (size_t)nc, sizeof(to_key), cmp_key);
       for (int64_t i = 0; i < deficit; ++i) {
@@ -249,6 +272,8 @@ int to_simulate(int64_t V, const int64_t* row_ptr, const int32_t* col, const uin
     /* step 5 */
     for (int64_t i = 0; i < nT; ++i) {
       int32_t v = T[i];
+      touched_at[v] = (int32_t)c;
+      if (state[v] != ST_IB) entered[v] = (int32_t)c;
       if (state[v] == ST_EV) {
         TRANSITION(v, ST_IB); stats[SK_RELOADS] += 1; rec[CK_RELOADED] += 1; reload_count[v] += 1;
         if (reload_count[v] > stats[SK_MAX_RELOAD]) stats[SK_MAX_RELOAD] = reload_count[v];
@@ -286,6 +311,6 @@ int to_simulate(int64_t V, const int64_t* row_ptr, const int32_t* col, const uin
   }
 #undef TRANSITION
   stats[SK_FREE_END] = free_slots;
-  free(state); free(pend); free(stamp); free(T); free(hubT); free(cand);
+  free(state); free(pend); free(stamp); free(T); free(hubT); free(cand); free(entered); free(touched_at);
   return rc;
 }

@@ -11,6 +11,7 @@ import numpy as np
 SAGE_MEAN, GCN_SYM = 0, 1
 GEMM_FP32, GEMM_BF16 = 0, 1
 FLAG_SIMT_GEMM, FLAG_NO_GROUPING = 2, 4
+EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
 CHUNK_LOG_COLUMNS = ["hs", "ns", "ev", "gs", "need", "evicted", "reloaded", "completed", "occupancy"]
 ERROR_CODES = {
     "OK": 0, "INVALID_ARG": -1, "ORDER": -2, "POOL_TOO_SMALL": -3, "HOST_STORE_FULL": -4, "DRAIN_FULL": -5,
@@ -51,7 +52,8 @@ class _Model(ctypes.Structure):
 class _Run(ctypes.Structure):
     _fields_ = [("chunk_sources", ctypes.c_int64), ("pool_slots", ctypes.c_int64), ("hub_count", ctypes.c_int64),
                 ("fanout", ctypes.POINTER(ctypes.c_int32)), ("seed", ctypes.c_uint64),
-                ("host_evict_rows", ctypes.c_int64), ("drain_rows", ctypes.c_int64), ("flags", ctypes.c_int32)]
+                ("host_evict_rows", ctypes.c_int64), ("drain_rows", ctypes.c_int64), ("flags", ctypes.c_int32),
+                ("evict_policy", ctypes.c_int32)]
 
 
 class Stats(ctypes.Structure):
@@ -155,7 +157,7 @@ class Context:
     def __init__(self, V: int, E: int, row_ptr, col_idx, in_degree, mode: int, dims: Sequence[int], W_neigh, W_self,
                  bias, act: Sequence[int], chunk_sources: int, pool_slots: int, hub_count: int = 0,
                  fanout: Optional[Sequence[int]] = None, seed: int = 1, host_evict_rows: int = 0, drain_rows: int = 0,
-                 gemm_mode: int = GEMM_FP32, flags: int = 0):
+                 gemm_mode: int = GEMM_FP32, flags: int = 0, evict_policy: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         L = len(dims) - 1
@@ -169,7 +171,7 @@ class Context:
         c_b = (ctypes.c_void_p * L)(*[_ptr(b) for b in bias]) if bias is not None else None
         m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode)
         c_f = (ctypes.c_int32 * L)(*[int(f) for f in fanout]) if fanout is not None else None
-        r = _Run(chunk_sources, pool_slots, hub_count, c_f, seed, host_evict_rows, drain_rows or chunk_sources, flags)
+        r = _Run(chunk_sources, pool_slots, hub_count, c_f, seed, host_evict_rows, drain_rows or chunk_sources, flags, evict_policy)
         rc = self._lib.taurus_graph_init(ctypes.byref(self._h), ctypes.byref(g), ctypes.byref(m), ctypes.byref(r))
         del keep
         if rc != 0:

@@ -174,6 +174,21 @@ __global__ void plan_kernel(ChunkArgs a) {
 // Victims are the `deficit` smallest keys (pending << 31 | id) among IN_BUFFER vertices the chunk does not
 // touch.  Keys are unique, so an MSB-first radix select over 6 digits of 11 bits finds the exact
 // threshold key; every key <= threshold is a victim.
+// 31-bit score of the random policy: a hash of (seed, vertex, chunk index); constants are part of its definition.
+static __device__ __forceinline__ unsigned long long ev_mix(unsigned long long x) {
+  x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+  x ^= x >> 27; x *= 0x94D049BB133111EBull;
+  x ^= x >> 31;
+  return x;
+}
+static __device__ __forceinline__ unsigned evict_hash(unsigned long long seed, unsigned long long vertex, unsigned long long chunk) {
+  unsigned long long h = 0x452821E638D01377ull;
+  h = ev_mix(h ^ (0x9E3779B97F4A7C15ull * (seed + 1ull)));
+  h = ev_mix(h ^ (0x9E3779B97F4A7C15ull * (vertex + 1ull)));
+  h = ev_mix(h ^ (0x9E3779B97F4A7C15ull * (chunk + 1ull)));
+  return (unsigned)(h >> 33);
+}
+
 static __device__ __forceinline__ int sel_shift(int pass) { return TAURUS_SEL_BITS * (TAURUS_SEL_PASSES - 1 - pass); }
 
 __global__ void select_keys_kernel(ChunkArgs a) {   // pass 0: gather keys, histogram of the top digit
@@ -186,7 +201,17 @@ __global__ void select_keys_kernel(ChunkArgs a) {   // pass 0: gather keys, hist
   for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < a.pool_slots; s += stride) {
     int v = a.owner[s];
     unsigned long long key = ~0ull;
-    if (v >= 0 && a.touch[v] != a.epoch) key = ((unsigned long long)(unsigned)a.pend[v] << 31) | (unsigned long long)v;
+    if (v >= 0) {
+      const int t = a.touch[v];
+      if (t != a.epoch) {
+        unsigned score;
+        if (a.evict_policy == TAURUS_EVICT_FIFO) score = (unsigned)a.slot_epoch[s];
+        else if (a.evict_policy == TAURUS_EVICT_LRU) score = (unsigned)t;
+        else if (a.evict_policy == TAURUS_EVICT_RANDOM) score = evict_hash(a.seed, (unsigned long long)v, (unsigned long long)(a.epoch - 1));
+        else score = (unsigned)a.pend[v];
+        key = ((unsigned long long)score << 31) | (unsigned long long)v;
+      }
+    }
     a.keys[s] = key;
     if (key != ~0ull) atomicAdd(&sh[(unsigned)(key >> sel_shift(0)) & (TAURUS_SEL_BINS - 1)], 1u);
   }
@@ -320,7 +345,7 @@ __global__ void alloc_kernel(ChunkArgs a) {
       for (int k = lane_id(); k < vec; k += 32) dst[k] = z;
     }
     if (lane_id() == 0) {
-      if (!a.direct) { a.loc[v] = slot; a.owner[slot] = v; }
+      if (!a.direct) { a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch; }
       a.state[v] = TAURUS_IN_BUFFER;
     }
   }

@@ -67,7 +67,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   free_tc_weights(c);
   cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
-  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
+  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
@@ -97,7 +97,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   c->V = g->V; c->E = g->E; c->L = m->L; c->mode = m->mode; c->gemm_mode = m->gemm_mode; c->flags = r->flags;
   c->seed = r->seed;
   c->chunk_sources = r->chunk_sources; c->pool_slots = r->pool_slots; c->hub_count = r->hub_count;
-  c->host_rows = r->host_evict_rows; c->drain_rows = r->drain_rows;
+  c->host_rows = r->host_evict_rows; c->drain_rows = r->drain_rows; c->evict_policy = r->evict_policy;
   bool any_sampled = false;
   for (int l = 0; l <= m->L; ++l) c->dims[l] = m->dims[l];
   for (int l = 0; l < m->L; ++l) {
@@ -180,7 +180,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     ALLOC(c->d_touched_list, c->touched_capacity);
   }
   ALLOC(c->d_owner, c->pool_slots); ALLOC(c->d_free_stack, c->pool_slots); ALLOC(c->d_need_list, c->pool_slots);
-  if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); }
+  if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); ALLOC(c->d_slot_epoch, c->pool_slots); }
   ALLOC(c->d_host_free, c->host_rows);
   if (c->host_rows > 0) {
     cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->host_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
@@ -243,6 +243,7 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
   if (r->chunk_sources < 1 || r->chunk_sources > (1 << 24) || r->pool_slots < 1 || r->pool_slots >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
   if (r->hub_count < 0 || r->hub_count > g->V || r->host_evict_rows < 0 || r->host_evict_rows >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
   if (r->drain_rows < 1 || r->drain_rows >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
+  if (r->evict_policy < TAURUS_EVICT_FEWEST_PENDING || r->evict_policy > TAURUS_EVICT_RANDOM) return TAURUS_ERR_INVALID_ARG;
   if (r->pool_slots + r->hub_count >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
   taurus_ctx* c = new (std::nothrow) taurus_ctx();
   if (!c) return TAURUS_ERR_NOMEM;
@@ -318,7 +319,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   const int l = c->layer;
   a.row_ptr = c->d_row_ptr; a.col = c->d_col; a.din = c->d_din; a.mask = c->d_mask_cur;
   a.pend = c->d_pend; a.state = c->d_state; a.loc = c->d_loc; a.touch = c->d_touch; a.reload_count = c->d_reload;
-  a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list;
+  a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list; a.slot_epoch = c->d_slot_epoch;
   a.touched_list = c->d_touched_list; a.touched_capacity = c->touched_capacity;
   a.victims = c->d_victims; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
@@ -329,7 +330,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.V = c->V; a.pool_slots = c->pool_slots; a.hub_count = c->hub_count; a.host_rows = c->host_rows; a.drain_rows = c->drain_rows;
   a.src_begin = s; a.src_end = e;
   a.epoch = (int32_t)(c->chunk_seq + 1);
-  a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l];
+  a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.evict_policy = c->evict_policy; a.seed = c->seed;
   a.direct = c->pool_slots >= c->V ? 1 : 0;
   a.dense_half = c->dense_out ? (int)(c->chunk_seq & 1) : -1;
   a.grad_cap = c->dense_out ? c->drain_rows / 2 : c->drain_rows;

@@ -60,6 +60,7 @@ struct ChunkArgs {
   // pool
   float* acc;               // [(pool_slots + hub_count) x Hp]
   int32_t* owner;           // [pool_slots] vertex in the slot, -1 = free
+  int32_t* slot_epoch;      // [pool_slots] chunk epoch at which the slot's vertex entered the pool (FIFO policy)
   int32_t* free_stack;      // [pool_slots]
   int32_t* need_list;       // [pool_slots]
   int32_t* touched_list;    // [touched_capacity] every vertex the chunk touches, listed at its first touch
@@ -84,6 +85,8 @@ struct ChunkArgs {
   int32_t epoch;            // chunk sequence number + 1 within the layer
   int32_t Hp;               // padded accumulator width (multiple of 4)
   int32_t mode, act, fanout;
+  int32_t evict_policy;
+  unsigned long long seed;
   long long grad_off;       // dense-output mode: first row of this chunk's half of the graduation buffer
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
   int32_t dense_half;       // -1: graduation buffer drained by the caller; 0 / 1: half used by this chunk
@@ -119,6 +122,8 @@ struct taurus_ctx {
   int32_t* d_hub_ids = nullptr;
   float* d_acc = nullptr;
   int32_t* d_owner = nullptr;
+  int32_t* d_slot_epoch = nullptr;
+  int evict_policy = 0;
   int32_t* d_free_stack = nullptr;
   int32_t* d_need_list = nullptr;
   int32_t* d_touched_list = nullptr;

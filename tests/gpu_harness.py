@@ -8,7 +8,7 @@ import taurus_gen as tg
 
 
 def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_features=False, drain_rows=None,
-                host_evict_rows=None, chunk_plan=None, gemm_mode=None, dense_output=False):
+                host_evict_rows=None, chunk_plan=None, gemm_mode=None, dense_output=False, evict_policy=0):
     """Runs every layer of workload w on the GPU.  Returns per-layer outputs (float32 [V, d_out]), the ids each
     chunk completed, stats and chunk logs.  Layer l+1 streams layer l's drained output."""
     import torch
@@ -21,7 +21,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
         0 if w.pool_slots >= V - w.hub_count else V - w.hub_count)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
-                     drain_rows or (2 * V if dense_output else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags)
+                     drain_rows or (2 * V if dense_output else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy)
     res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
     if host_features:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
@@ -70,7 +70,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
     return res
 
 
-def run_oracle(w, g, model, x0):
+def run_oracle(w, g, model, x0, evict_policy=0):
     """Oracle outputs for every layer plus the integer simulation per layer."""
     inl = oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
     din, dout = np.diff(inl.ptr), np.diff(g.row_ptr)
@@ -81,7 +81,7 @@ def run_oracle(w, g, model, x0):
         ms = oracle.message_sets(inl, w.fanout[l], w.seed, l)
         h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l])
         out["outs"].append(h)
-        out["sims"].append(oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, w.pool_slots))
+        out["sims"].append(oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, w.pool_slots, evict_policy, w.seed))
         out["msets"].append(ms)
     return out
 

@@ -37,7 +37,7 @@ def _full_check(w, g=None, bias_scale=0.3, tol=FP32_TOL, **kw):
     model = tg.make_model(w, bias_scale=bias_scale)
     x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
     lib = run_library(w, g, model, x0, **kw)
-    orc = run_oracle(w, g, model, x0)
+    orc = run_oracle(w, g, model, x0, kw.get("evict_policy", 0))
     _compare_layers(lib, orc, tol)
     for l in range(w.L):
         assert orc["sims"][l].rc == 0
@@ -298,3 +298,14 @@ def test_vertex_arrays_after_a_layer():
     assert (ctx.get_vertex_array("hub") == 0).all()
     st = ctx.get_stats()
     assert st["completed"] == g.V and st["free_slots"] == w.pool_slots and st["chunks"] == 10
+
+
+@pytest.mark.parametrize("policy", [1, 2, 3])
+def test_eviction_policy_variants(policy):
+    """FIFO, LRU and random eviction (the ablation of Sect. 4.5): same outputs, accounting bit-exact against the
+    oracle's simulator run with the same policy."""
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 60_000, chunk=1024)
+    w = replace(w, dims=(128, 64), fanout=(0,), pool_slots=20_000, hub_count=60)
+    lib, orc = _full_check(w, evict_policy=policy)
+    assert lib["stats"][0]["evictions"] > 1000

@@ -9,9 +9,10 @@ import taurus_gen as tg
 from helpers import random_multigraph
 
 
-def second_simulator(V, row_ptr, col, prop, m, is_hub, chunk, pool):
+def second_simulator(V, row_ptr, col, prop, m, is_hub, chunk, pool, policy=0, seed=0):
     """Independent restatement with Python sets; victims by a full sort of (pending, id)."""
     pend = {v: int(m[v]) + 1 for v in range(V)}
+    entered, touched_at = {}, {}
     in_pool, evicted, done, started_hubs = set(), set(), set(), set()
     ev = rl = 0
     reload_count = {v: 0 for v in range(V)}
@@ -32,13 +33,19 @@ def second_simulator(V, row_ptr, col, prop, m, is_hub, chunk, pool):
         deficit = need - (pool - len(in_pool))
         n_ev = 0
         if deficit > 0:
-            order = sorted((pend[v], v) for v in in_pool - T)
+            score = {0: lambda v: pend[v], 1: lambda v: entered[v], 2: lambda v: touched_at[v],
+                     3: lambda v: int(oracle._lib().to_evict_hash(seed, v, c))}[policy]
+            order = sorted((score(v), v) for v in in_pool - T)
             if len(order) < deficit:
                 return None
             for _, v in order[:deficit]:
                 in_pool.remove(v); evicted.add(v); ev += 1; n_ev += 1
         for v in evs:
             evicted.remove(v); in_pool.add(v); rl += 1; reload_count[v] += 1
+        for v in T:
+            touched_at[v] = c
+            if v in evs or v in ns:
+                entered[v] = c
         in_pool |= ns
         started_hubs |= {v for v in touched if is_hub[v]}
         peak = max(peak, len(in_pool))
@@ -168,3 +175,41 @@ def test_hub_set_takes_largest_in_degree_ties_by_smaller_id():
     assert oracle.hub_set(din, 2).tolist() == [0, 1, 1, 0, 0, 0]
     assert oracle.hub_set(din, 4).tolist() == [1, 1, 1, 0, 1, 0]
     assert oracle.hub_set(din, 0).sum() == 0
+
+
+@pytest.mark.parametrize("policy", [oracle.EVICT_FEWEST_PENDING, oracle.EVICT_FIFO, oracle.EVICT_LRU, oracle.EVICT_RANDOM])
+def test_eviction_policies_match_the_second_simulator(policy):
+    """The ablation policies of Sect. 4.5 (FIFO, LRU, random) beside the paper's fewest-pending rule."""
+    V, E, chunk = 60, 110, 2
+    checked = 0
+    for seed in range(8):
+        row_ptr, col, inl, ms, hub = _setup(V, E, seed, 0, 2)
+        for pool in (10, 14):
+            a = oracle.simulate(V, row_ptr, col, ms, hub, chunk, pool, policy, 77)
+            b = second_simulator(V, row_ptr, col, ms.prop, ms.m, hub, chunk, pool, policy, 77)
+            if b is None:
+                assert a.rc in (-2, -3)
+                continue
+            checked += 1
+            assert a.rc == 0 and a.stats["evictions"] == b["evictions"] and a.stats["reloads"] == b["reloads"]
+            assert all(a.reload_count[v] == b["reload_count"][v] for v in range(V))
+            for c, rec in enumerate(b["per_chunk"]):
+                for k, val in rec.items():
+                    assert a.per_chunk[k][c] == val, (k, c)
+    assert checked >= 4
+
+
+def test_fewest_pending_reloads_less_than_fifo_and_random():
+    """The claim behind Sect. 3.5.3, on a banded synthetic graph with a pool at 80 % of the peak active set:
+    evicting the vertices closest to completion causes fewer reloads than FIFO or random choice.  (Against LRU the
+    outcome depends on the graph; the paper's own margin there is its smallest.)"""
+    w = tg.scaled(tg.WORKLOADS["large"], 20_000, chunk=256)
+    g = tg.make_graph(w)
+    inl = oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
+    ms = oracle.message_sets(inl, 0, 1, 0)
+    hub = oracle.hub_set(g.in_degree, w.hub_count)
+    peak = oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, g.V).stats["peak_occupancy"]
+    reloads = {p: oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, int(peak * 0.8), p, 5).stats["reloads"]
+               for p in (oracle.EVICT_FEWEST_PENDING, oracle.EVICT_FIFO, oracle.EVICT_LRU, oracle.EVICT_RANDOM)}
+    assert reloads[oracle.EVICT_FEWEST_PENDING] < reloads[oracle.EVICT_FIFO]
+    assert reloads[oracle.EVICT_FEWEST_PENDING] < reloads[oracle.EVICT_RANDOM]
