@@ -22,6 +22,7 @@
  *   SAGE-mean: c_out = 1, c_in = 1 / max(|M(v)|, 1), c_self = 1
  *   GCN-sym  : c_out(u) = (dout(u)+1)^-1/2, c_in(v) = (din(v)+1)^-1/2,
  *              c_self = c_out * c_in, W_self = W_neigh
+ *   GIN-sum  : c_out = 1, c_in = 1, c_self = 1 + gin_eps, W_self = W_neigh ("GCN/GIN-style aggregation", Sect. 3.9)
  * M(v) is the multiset of propagated in-edges of v (all of them, or the
  * sampled ones); every CSR entry is one message, duplicates and self-loops
  * included.
@@ -60,7 +61,7 @@ enum {
   TAURUS_ERR_UNSUPPORTED = -9      /* shape or size outside what the kernels were built for                     */
 };
 
-enum { TAURUS_SAGE_MEAN = 0, TAURUS_GCN_SYM = 1 };
+enum { TAURUS_SAGE_MEAN = 0, TAURUS_GCN_SYM = 1, TAURUS_GIN_SUM = 2 };
 enum { TAURUS_GEMM_FP32 = 0, TAURUS_GEMM_BF16 = 1 };
 /* vertex states of Sect. 3.4 */
 enum { TAURUS_NOT_STARTED = 0, TAURUS_IN_BUFFER = 1, TAURUS_EVICTED = 2, TAURUS_ON_GPU = 3, TAURUS_COMPLETED = 4 };
@@ -77,14 +78,15 @@ typedef struct {
 
 /* Layer weights.  Copied at init.  dims[l] -> dims[l+1]; matrices are row-major dims[l] x dims[l+1] fp32. */
 typedef struct {
-  int32_t mode;                /* TAURUS_SAGE_MEAN or TAURUS_GCN_SYM                          */
+  int32_t mode;                /* TAURUS_SAGE_MEAN, TAURUS_GCN_SYM or TAURUS_GIN_SUM          */
   int32_t L;                   /* number of layers, 1..16                                     */
   const int32_t* dims;         /* [L+1], each in 1..1024 (host pointer)                       */
   const float* const* W_neigh; /* [L] (host array of pointers)                                */
-  const float* const* W_self;  /* [L]; ignored for GCN (the self term uses W_neigh)           */
+  const float* const* W_self;  /* [L]; used by SAGE only (GCN and GIN apply W_neigh to the self term) */
   const float* const* bias;    /* [L] each dims[l+1]; an entry may be NULL for zero bias      */
   const int32_t* act;          /* [L] 0 = identity, 1 = ReLU (host pointer)                   */
   int32_t gemm_mode;           /* TAURUS_GEMM_FP32: fp32-accurate projection; TAURUS_GEMM_BF16: bf16 operands, fp32 accumulate */
+  float gin_eps;               /* TAURUS_GIN_SUM only: the self message is weighted 1 + gin_eps */
 } taurus_model;
 
 typedef struct {

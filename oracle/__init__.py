@@ -33,6 +33,7 @@ _handle = None
 
 SAGE_MEAN = 0
 GCN_SYM = 1
+GIN_SUM = 2
 
 # eviction policies: the paper's (Sect. 3.5.3) and the alternatives of its ablation (Sect. 4.5)
 EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
@@ -144,7 +145,7 @@ def message_sets(inl: InLists, fanout: int, seed: int, layer: int) -> MessageSet
 
 # ----------------------------------------------------------------------------- one layer, pull-based, fp64
 
-def coefficients(mode: int, m: np.ndarray, din: np.ndarray, dout: np.ndarray):
+def coefficients(mode: int, m: np.ndarray, din: np.ndarray, dout: np.ndarray, gin_eps: float = 0.0):
     """(c_out[V], c_in[V], c_self[V]) in fp64.
 
     SAGE-mean (Sect. 3.4 normalised message, SAGEConv paragraph of Sect. 3.9):
@@ -152,10 +153,14 @@ def coefficients(mode: int, m: np.ndarray, din: np.ndarray, dout: np.ndarray):
     GCN symmetric norm with the implicit self message every vertex aggregates (Sect. 3.8):
         c_out(u) = (dout(u) + 1)^-1/2, c_in(v) = (din(v) + 1)^-1/2, c_self = c_out * c_in,
         with the full-graph degrees also under sampling.
+    GIN (sum aggregator; "GCN/GIN-style aggregation", Sect. 3.9; one of the models of Sect. 4.1):
+        c_out = 1, c_in = 1, c_self = 1 + eps, with one shared weight.
     """
     V = m.size
     if mode == SAGE_MEAN:
         return np.ones(V), 1.0 / np.maximum(m.astype(np.float64), 1.0), np.ones(V)
+    if mode == GIN_SUM:
+        return np.ones(V), np.ones(V), np.full(V, 1.0 + gin_eps)
     c_out = (dout.astype(np.float64) + 1.0) ** -0.5
     c_in = (din.astype(np.float64) + 1.0) ** -0.5
     return c_out, c_in, c_out * c_in
@@ -173,23 +178,23 @@ def aggregate(ms: MessageSets, dst: np.ndarray, c_out: Optional[np.ndarray], h: 
 
 def layer_forward(ms: MessageSets, mode: int, din: np.ndarray, dout: np.ndarray, h: np.ndarray,
                   W_neigh: np.ndarray, W_self: np.ndarray, bias: np.ndarray, act: int,
-                  dst: Optional[np.ndarray] = None) -> np.ndarray:
+                  dst: Optional[np.ndarray] = None, gin_eps: float = 0.0) -> np.ndarray:
     """out_v = act(c_in(v) * (agg_v @ W_neigh) + c_self(v) * (h_v @ W_self) + b) for v in dst (default: all), Eq. 1-2."""
     V = ms.m.size
     if dst is None:
         dst = np.arange(V, dtype=np.int64)
-    c_out, c_in, c_self = coefficients(mode, ms.m, din, dout)
+    c_out, c_in, c_self = coefficients(mode, ms.m, din, dout, gin_eps)
     h = np.asarray(h, dtype=np.float64)
-    agg = aggregate(ms, dst, None if mode == SAGE_MEAN else c_out, h)
+    agg = aggregate(ms, dst, c_out if mode == GCN_SYM else None, h)
     Wn = np.asarray(W_neigh, dtype=np.float64)
-    Ws = Wn if mode == GCN_SYM else np.asarray(W_self, dtype=np.float64)
+    Ws = np.asarray(W_self, dtype=np.float64) if mode == SAGE_MEAN else Wn
     z = c_in[dst, None] * (agg @ Wn) + c_self[dst, None] * (h[dst] @ Ws) + np.asarray(bias, dtype=np.float64)[None, :]
     return np.maximum(z, 0.0) if act else z
 
 
 def forward(V: int, row_ptr: np.ndarray, col: np.ndarray, x: np.ndarray, mode: int, W_neigh: Sequence[np.ndarray],
             W_self: Sequence[np.ndarray], bias: Sequence[np.ndarray], act: Sequence[int],
-            fanout: Sequence[int], seed: int, inl: Optional[InLists] = None) -> List[np.ndarray]:
+            fanout: Sequence[int], seed: int, inl: Optional[InLists] = None, gin_eps: float = 0.0) -> List[np.ndarray]:
     """All layers; layer l+1 consumes this oracle's own fp64 output of layer l.  Returns every layer's output."""
     inl = inl or build_in_lists(V, row_ptr, col)
     din = np.diff(inl.ptr)
@@ -198,7 +203,7 @@ def forward(V: int, row_ptr: np.ndarray, col: np.ndarray, x: np.ndarray, mode: i
     outs = []
     for l in range(len(W_neigh)):
         ms = message_sets(inl, fanout[l], seed, l)
-        h = layer_forward(ms, mode, din, dout, h, W_neigh[l], W_self[l], bias[l], act[l])
+        h = layer_forward(ms, mode, din, dout, h, W_neigh[l], W_self[l], bias[l], act[l], gin_eps=gin_eps)
         outs.append(h)
     return outs
 

@@ -8,7 +8,7 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-SAGE_MEAN, GCN_SYM = 0, 1
+SAGE_MEAN, GCN_SYM, GIN_SUM = 0, 1, 2
 GEMM_FP32, GEMM_BF16 = 0, 1
 FLAG_SIMT_GEMM, FLAG_NO_GROUPING = 2, 4
 EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
@@ -46,7 +46,7 @@ class _Model(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("L", ctypes.c_int32), ("dims", ctypes.POINTER(ctypes.c_int32)),
                 ("W_neigh", ctypes.POINTER(ctypes.c_void_p)), ("W_self", ctypes.POINTER(ctypes.c_void_p)),
                 ("bias", ctypes.POINTER(ctypes.c_void_p)), ("act", ctypes.POINTER(ctypes.c_int32)),
-                ("gemm_mode", ctypes.c_int32)]
+                ("gemm_mode", ctypes.c_int32), ("gin_eps", ctypes.c_float)]
 
 
 class _Run(ctypes.Structure):
@@ -157,7 +157,7 @@ class Context:
     def __init__(self, V: int, E: int, row_ptr, col_idx, in_degree, mode: int, dims: Sequence[int], W_neigh, W_self,
                  bias, act: Sequence[int], chunk_sources: int, pool_slots: int, hub_count: int = 0,
                  fanout: Optional[Sequence[int]] = None, seed: int = 1, host_evict_rows: int = 0, drain_rows: int = 0,
-                 gemm_mode: int = GEMM_FP32, flags: int = 0, evict_policy: int = 0):
+                 gemm_mode: int = GEMM_FP32, flags: int = 0, evict_policy: int = 0, gin_eps: float = 0.0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         L = len(dims) - 1
@@ -169,7 +169,7 @@ class Context:
         c_wn = (ctypes.c_void_p * L)(*[_ptr(w) for w in W_neigh])
         c_ws = (ctypes.c_void_p * L)(*[_ptr(w) for w in W_self]) if W_self is not None else None
         c_b = (ctypes.c_void_p * L)(*[_ptr(b) for b in bias]) if bias is not None else None
-        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode)
+        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode, gin_eps)
         c_f = (ctypes.c_int32 * L)(*[int(f) for f in fanout]) if fanout is not None else None
         r = _Run(chunk_sources, pool_slots, hub_count, c_f, seed, host_evict_rows, drain_rows or chunk_sources, flags, evict_policy)
         rc = self._lib.taurus_graph_init(ctypes.byref(self._h), ctypes.byref(g), ctypes.byref(m), ctypes.byref(r))

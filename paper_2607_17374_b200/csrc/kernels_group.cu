@@ -329,13 +329,15 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) red_add_v4(dst + 4 * (c4 + k * LPE), reinterpret_cast<const float4*>(p)[c4 + k * LPE]);
       } else {
-        const float sc = (float)sqrt((double)a.din[vj] + 1.0);
+        // one shared weight: GCN  P_v + b * sqrt(din(v) + 1);  GIN  (1 + eps) * P_v + b
+        const float ps = a.mode == TAURUS_GIN_SUM ? a.gin_self : 1.0f;
+        const float sc = a.mode == TAURUS_GIN_SUM ? 1.0f : (float)sqrt((double)a.din[vj] + 1.0);
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) {
             float4 xx = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
             float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];
-            red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(xx.x + b.x * sc, xx.y + b.y * sc, xx.z + b.z * sc, xx.w + b.w * sc));
+            red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(xx.x * ps + b.x * sc, xx.y * ps + b.y * sc, xx.z * ps + b.z * sc, xx.w * ps + b.w * sc));
           }
       }
     }

@@ -127,14 +127,16 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
 #pragma unroll
               for (int k = 0; k < VPL; ++k)
                 if (c4 + k * LPE < nvec) row[k] = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
-            } else {       // GCN: the self message is P_v + b / c_in(v)
-              const float s = (float)sqrt((double)a.din[sj] + 1.0);
+            } else {       // one shared weight: the self message is built from the vertex's own P row
+              // GCN: P_v (already scaled by c_out(v)) + b * sqrt(din(v) + 1);  GIN: (1 + eps) * P_v + b
+              const float ps = a.mode == TAURUS_GIN_SUM ? a.gin_self : 1.0f;
+              const float s = a.mode == TAURUS_GIN_SUM ? 1.0f : (float)sqrt((double)a.din[sj] + 1.0);
 #pragma unroll
               for (int k = 0; k < VPL; ++k)
                 if (c4 + k * LPE < nvec) {
                   float4 x = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
                   float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];
-                  row[k] = make_float4(x.x + b.x * s, x.y + b.y * s, x.z + b.z * s, x.w + b.w * s);
+                  row[k] = make_float4(x.x * ps + b.x * s, x.y * ps + b.y * s, x.z * ps + b.z * s, x.w * ps + b.w * s);
                 }
             }
           } else {

@@ -436,8 +436,10 @@ __global__ void finalise_kernel(ChunkArgs a) {
     if (a.mode == TAURUS_SAGE_MEAN) {
       int m = messages_of(a.din[v], a.fanout);
       scale = 1.0f / (float)(m > 1 ? m : 1);
-    } else {
+    } else if (a.mode == TAURUS_GCN_SYM) {
       scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+    } else {
+      scale = 1.0f;   // GIN: plain sum
     }
     const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
     float4* dst = reinterpret_cast<float4*>(a.grad_rows + (size_t)(base + i) * a.Hp);

@@ -96,6 +96,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   c->sm_count = prop.multiProcessorCount;
   c->V = g->V; c->E = g->E; c->L = m->L; c->mode = m->mode; c->gemm_mode = m->gemm_mode; c->flags = r->flags;
   c->seed = r->seed;
+  c->gin_eps = m->gin_eps;
   c->chunk_sources = r->chunk_sources; c->pool_slots = r->pool_slots; c->hub_count = r->hub_count;
   c->host_rows = r->host_evict_rows; c->drain_rows = r->drain_rows; c->evict_policy = r->evict_policy;
   bool any_sampled = false;
@@ -231,7 +232,7 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
   if (!g || !m || !r || !g->row_ptr || !g->in_degree || (g->E > 0 && !g->col_idx)) return TAURUS_ERR_INVALID_ARG;
   if (g->V < 1 || g->V >= (1ll << 31) || g->E < 0 || g->E >= (1ll << 32)) return TAURUS_ERR_INVALID_ARG;
   if (m->L < 1 || m->L > TAURUS_MAX_LAYERS || !m->dims || !m->W_neigh) return TAURUS_ERR_INVALID_ARG;
-  if (m->mode != TAURUS_SAGE_MEAN && m->mode != TAURUS_GCN_SYM) return TAURUS_ERR_INVALID_ARG;
+  if (m->mode != TAURUS_SAGE_MEAN && m->mode != TAURUS_GCN_SYM && m->mode != TAURUS_GIN_SUM) return TAURUS_ERR_INVALID_ARG;
   if (m->gemm_mode != TAURUS_GEMM_FP32 && m->gemm_mode != TAURUS_GEMM_BF16) return TAURUS_ERR_INVALID_ARG;
   if (m->mode == TAURUS_SAGE_MEAN && !m->W_self) return TAURUS_ERR_INVALID_ARG;
   for (int l = 0; l <= m->L; ++l)
@@ -331,6 +332,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.src_begin = s; a.src_end = e;
   a.epoch = (int32_t)(c->chunk_seq + 1);
   a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.evict_policy = c->evict_policy; a.seed = c->seed;
+  a.gin_self = 1.0f + c->gin_eps;
   a.direct = c->pool_slots >= c->V ? 1 : 0;
   a.dense_half = c->dense_out ? (int)(c->chunk_seq & 1) : -1;
   a.grad_cap = c->dense_out ? c->drain_rows / 2 : c->drain_rows;

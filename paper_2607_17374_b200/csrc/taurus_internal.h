@@ -86,6 +86,7 @@ struct ChunkArgs {
   int32_t Hp;               // padded accumulator width (multiple of 4)
   int32_t mode, act, fanout;
   int32_t evict_policy;
+  float gin_self;           // GIN: 1 + eps, the weight of the self message
   unsigned long long seed;
   long long grad_off;       // dense-output mode: first row of this chunk's half of the graduation buffer
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
@@ -124,6 +125,7 @@ struct taurus_ctx {
   int32_t* d_owner = nullptr;
   int32_t* d_slot_epoch = nullptr;
   int evict_policy = 0;
+  float gin_eps = 0.f;
   int32_t* d_free_stack = nullptr;
   int32_t* d_need_list = nullptr;
   int32_t* d_touched_list = nullptr;

@@ -74,6 +74,7 @@ def hash64(seed: int, tag: int, i: int, j: int) -> int:
 
 SAGE_MEAN = 0
 GCN_SYM = 1
+GIN_SUM = 2
 GEMM_FP32 = 0
 GEMM_BF16 = 1
 
@@ -91,13 +92,14 @@ class Workload:
     top_in: int                 # target for the largest in-degree (mode 1)
     symmetric: bool
     dims: Tuple[int, ...]       # F, hidden..., out
-    mode: int                   # SAGE_MEAN or GCN_SYM
+    mode: int                   # SAGE_MEAN, GCN_SYM or GIN_SUM
     chunk: int                  # sources per pushed chunk
     pool_slots: int             # accumulator slot pool capacity
     hub_count: int              # vertices pinned in the GPU-resident store
     fanout: Tuple[int, ...]     # per layer, 0 = exact
     gemm_mode: int = GEMM_FP32
     seed: int = 1
+    gin_eps: float = 0.0        # GIN_SUM only: the self weight is 1 + gin_eps
 
     @property
     def L(self) -> int:
@@ -240,7 +242,7 @@ def make_model(w: Workload, bias_scale: float = 0.0) -> Model:
     Wn, Ws, b = [], [], []
     for l in range(w.L):
         Wn.append(weights(w.seed, l, 0, w.dims[l], w.dims[l + 1]))
-        Ws.append(Wn[-1] if w.mode == GCN_SYM else weights(w.seed, l, 1, w.dims[l], w.dims[l + 1]))
+        Ws.append(weights(w.seed, l, 1, w.dims[l], w.dims[l + 1]) if w.mode == SAGE_MEAN else Wn[-1])
         if bias_scale > 0:
             b.append((weights(w.seed, l, 2, 1, w.dims[l + 1])[0] * bias_scale).astype(np.float32))
         else:

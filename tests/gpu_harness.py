@@ -21,7 +21,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
         0 if w.pool_slots >= V - w.hub_count else V - w.hub_count)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
-                     drain_rows or (2 * V if dense_output else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy)
+                     drain_rows or (2 * V if dense_output else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy, w.gin_eps)
     res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
     if host_features:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
@@ -79,7 +79,8 @@ def run_oracle(w, g, model, x0, evict_policy=0):
     out = dict(outs=[], sims=[], msets=[], hub=hub)
     for l in range(w.L):
         ms = oracle.message_sets(inl, w.fanout[l], w.seed, l)
-        h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l])
+        h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l],
+                                 gin_eps=w.gin_eps)
         out["outs"].append(h)
         out["sims"].append(oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, w.pool_slots, evict_policy, w.seed))
         out["msets"].append(ms)

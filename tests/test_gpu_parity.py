@@ -309,3 +309,12 @@ def test_eviction_policy_variants(policy):
     w = replace(w, dims=(128, 64), fanout=(0,), pool_slots=20_000, hub_count=60)
     lib, orc = _full_check(w, evict_policy=policy)
     assert lib["stats"][0]["evictions"] > 1000
+
+
+def test_gin_sum_mode():
+    """Sum aggregator with a (1 + eps) self weight and one shared matrix, under eviction, with hubs."""
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 40_000, chunk=1024)
+    w = replace(w, mode=tg.GIN_SUM, gin_eps=0.25, dims=(96, 128, 32), fanout=(0, 0), pool_slots=20_000, hub_count=40)
+    _full_check(w)
+    _full_check(replace(w, fanout=(6, 3)), flags=4)      # sampled, CSR-order kernels

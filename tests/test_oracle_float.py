@@ -49,6 +49,22 @@ def test_gcn_sym_equals_dense_products(V, E, seed):
     np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-12)
 
 
+@pytest.mark.parametrize("V,E,seed", [(9, 30, 13), (128, 700, 14)])
+def test_gin_sum_equals_dense_products(V, E, seed):
+    """act((A + (1 + eps) I) H W + b): sum aggregator, one shared weight ("GCN/GIN-style aggregation", Sect. 3.9)."""
+    rng = np.random.default_rng(seed)
+    row_ptr, col = random_multigraph(V, E, seed)
+    A = dense_adjacency(V, row_ptr, col)
+    H = rng.standard_normal((V, 4))
+    Wn, _, b = _weights(rng, 4, 6)
+    eps = 0.25
+    ref = np.maximum((A + (1 + eps) * np.eye(V)) @ H @ Wn + b, 0)
+    inl = oracle.build_in_lists(V, row_ptr, col)
+    ms = oracle.message_sets(inl, 0, 1, 0)
+    got = oracle.layer_forward(ms, oracle.GIN_SUM, np.diff(inl.ptr), np.diff(row_ptr), H, Wn, None, b, 1, gin_eps=eps)
+    np.testing.assert_allclose(got, ref, rtol=1e-12, atol=1e-12)
+
+
 def test_directed_ring_is_a_shifted_copy():
     V = 11
     row_ptr, col = csr_from_edges(V, [(u, (u + 1) % V) for u in range(V)])
