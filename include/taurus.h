@@ -265,6 +265,24 @@ int taurus_completion_counts_noalloc(int64_t V, int64_t E, const int64_t* row_pt
                                      const uint32_t* edge_mask, int32_t* out_counts, int32_t* out_bad_index,
                                      void* cuda_stream);
 
+/*
+ * Topology-aware reordering, Alg. 1 of Sect. 3.8 (pre-processing; needs no context).  Starting from the
+ * positions r(v) = initial_rank[v] (identity when NULL) it repeats `iterations` times
+ *     mu(v) = (r(v) + sum_{u -> v} r(u)) / d(v)                                     d(v) = in-degree + 1
+ *     r(w)  = (mu(w)/d(w) + sum_{w -> v} mu(v)/d(v)) / (1/d(w) + sum_{w -> v} 1/d(v))
+ * (every vertex also aggregates its own self message, so d >= 1 and each vertex belongs to its own
+ * neighbourhoods) and returns pi = ArgSort(r), ties by vertex id, as out_rank[v] = new processing rank of v.
+ * The real-valued positions are carried from one iteration to the next as Alg. 1 states them.
+ * out_positions ([V] doubles, may be NULL) receives the final r.  out_J and out_span ([iterations + 1], HOST
+ * memory, may be NULL) receive, for the initial order and after every iteration, the dispersion J and the
+ * total span C(pi) = sum_v (max - min) of the ranks of v's in-neighbours and v, both evaluated on the ordering
+ * itself (positions = ranks, centres = their optimum).  row_ptr, col_idx, initial_rank, out_rank and
+ * out_positions may be host or device memory.  Blocking; all arithmetic in fp64.
+ */
+int taurus_reorder(int64_t V, int64_t E, const int64_t* row_ptr, const int32_t* col_idx, const int32_t* initial_rank,
+                   int32_t iterations, int32_t* out_rank, double* out_positions, double* out_J, int64_t* out_span,
+                   void* cuda_stream);
+
 /* Kernels launched by this context since init (for launch accounting in benchmarks). */
 int64_t taurus_launch_count(const taurus_ctx* ctx);
 

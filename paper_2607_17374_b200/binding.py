@@ -77,7 +77,7 @@ EXPORTS = [
     "taurus_layer_end", "taurus_get_stats", "taurus_get_chunk_log", "taurus_get_vertex_array",
     "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count",
     "taurus_set_timing", "taurus_get_phase_ms", "taurus_destroy", "taurus_strerror", "taurus_last_cuda_error",
-    "taurus_completion_counts_noalloc", "taurus_layer_set_dense_output",
+    "taurus_completion_counts_noalloc", "taurus_layer_set_dense_output", "taurus_reorder",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -107,6 +107,7 @@ def load_library():
     lib.taurus_get_edge_mask.argtypes = [vp, vp]
     lib.taurus_completion_bound.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
     lib.taurus_completion_counts_noalloc.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
+    lib.taurus_reorder.argtypes = [i64, i64, vp, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -149,6 +150,20 @@ def completion_counts_noalloc(V: int, E: int, row_ptr, col_idx, edge_mask, out_c
     address owned by the caller; returns the C return code (0 = enqueued)."""
     return int(load_library().taurus_completion_counts_noalloc(V, E, _ptr(row_ptr), _ptr(col_idx), _ptr(edge_mask),
                                                                _ptr(out_counts), _ptr(out_bad_index), _stream(stream)))
+
+
+def reorder(V: int, E: int, row_ptr, col_idx, initial_rank=None, iterations: int = 5, stream=None):
+    """taurus_reorder (Alg. 1).  Returns (rank int32 [V], positions float64 [V], J float64 [iterations + 1],
+    span int64 [iterations + 1]) as numpy arrays."""
+    rank = np.empty(V, np.int32)
+    pos = np.empty(V, np.float64)
+    J = np.zeros(iterations + 1, np.float64)
+    span = np.zeros(iterations + 1, np.int64)
+    rc = load_library().taurus_reorder(V, E, _ptr(row_ptr), _ptr(col_idx), _ptr(initial_rank), iterations, rank.ctypes.data,
+                                       pos.ctypes.data, J.ctypes.data, span.ctypes.data, _stream(stream))
+    if rc != 0:
+        raise TaurusError(rc, "taurus_reorder")
+    return rank, pos, J, span
 
 
 class Context:
