@@ -58,7 +58,9 @@ enum {
   TAURUS_ERR_CUDA = -6,            /* a CUDA runtime call failed (see taurus_last_cuda_error)                   */
   TAURUS_ERR_INTERNAL = -7,        /* a device-side consistency check failed                                    */
   TAURUS_ERR_NOMEM = -8,           /* host or device allocation failed                                          */
-  TAURUS_ERR_UNSUPPORTED = -9      /* shape or size outside what the kernels were built for                     */
+  TAURUS_ERR_UNSUPPORTED = -9,     /* shape or size outside what the kernels were built for                     */
+  TAURUS_ERR_RUN_STORE_FULL = -10, /* a flush would exceed store_rows of the run store                          */
+  TAURUS_ERR_RUNS_INCOMPLETE = -11 /* a chunk read found fewer (or more) rows than vertices in its id range      */
 };
 
 enum { TAURUS_SAGE_MEAN = 0, TAURUS_GCN_SYM = 1, TAURUS_GIN_SUM = 2 };
@@ -282,6 +284,77 @@ int taurus_completion_counts_noalloc(int64_t V, int64_t E, const int64_t* row_pt
 int taurus_reorder(int64_t V, int64_t E, const int64_t* row_ptr, const int32_t* col_idx, const int32_t* initial_rank,
                    int32_t iterations, int32_t* out_rank, double* out_positions, double* out_J, int64_t* out_span,
                    void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------------------------
+ * Output side of a layer: sorted runs (embedding writer, Sect. 3.7) and merge-on-read (graph reader, Sect. 3.3).
+ *
+ * Finished rows leave the graduation buffer in completion order, not vertex order.  A taurus_runs object
+ * cuts the id space [0, V) into `partitions` fixed ranges of ceil(V / partitions) ids and keeps one
+ * partition buffer of `partition_rows` rows per range in device memory.  An appended row goes to the buffer
+ * of its range, in arrival order; a buffer that reaches partition_rows rows is sorted by vertex id on the
+ * GPU and written sequentially to the run store as one sorted run (ids I_f, rows X_f); runs are never
+ * merged.  taurus_runs_read_chunk rebuilds the matrix of a chunk [s, e) in vertex order: for every run that
+ * overlaps it, two binary searches (first id >= s, first id >= e) delimit a contiguous slice, the slice is
+ * copied to the device in one transfer, and the slices are merged by vertex id.  The run store stands for the
+ * paper's run files on SSD: pinned host memory (TAURUS_RUNS_HOST) or device memory (TAURUS_RUNS_DEVICE); the
+ * ids of all runs are always kept in pinned host memory, where the searches run.
+ *
+ * Run k of a range holds that range's arrivals k * partition_rows .. (k + 1) * partition_rows - 1 (arrival
+ * order = order of the rows within each append, appends in call order), so the set of runs is a function of
+ * the arrival sequence alone.  One object is used from one host thread at a time; calls on it are ordered on
+ * the streams given (the library inserts the dependencies between streams itself).
+ */
+typedef struct taurus_runs taurus_runs;
+enum { TAURUS_RUNS_HOST = 0, TAURUS_RUNS_DEVICE = 1 };
+typedef struct {
+  int64_t V;                /* vertex ids are in [0, V), V < 2^31                                              */
+  int32_t width;            /* floats per row, 1..1024                                                          */
+  int32_t store_kind;       /* TAURUS_RUNS_HOST | TAURUS_RUNS_DEVICE                                            */
+  int64_t partitions;       /* number of id ranges, 1..1024                                                     */
+  int64_t partition_rows;   /* rows a partition buffer holds before it is sorted and flushed                   */
+  int64_t store_rows;       /* capacity of the run store in rows (V holds one layer's output)                  */
+  int64_t max_append_rows;  /* most rows one taurus_runs_append call (or one chunk of a layer) may bring        */
+  int64_t max_chunk_rows;   /* most ids one taurus_runs_read_chunk call may span                                */
+} taurus_runs_config;
+
+/* Allocates the partition buffers, the run store and the scratch (all sizes fixed here).  TAURUS_ERR_NOMEM /
+ * TAURUS_ERR_INVALID_ARG on failure, *out untouched. */
+int taurus_runs_create(taurus_runs** out, const taurus_runs_config* config);
+/* Appends `count` rows: ids[i] is the vertex of rows[i * ld .. i * ld + width).  ids and rows are device
+ * memory or pinned host memory and must stay valid until the stream has passed this call.  Flushes every
+ * partition buffer that fills on the way.  Blocks the host once for the per-range counts.  An id outside
+ * [0, V) gives TAURUS_ERR_INVALID_ARG and appends nothing; a flush that does not fit the store gives
+ * TAURUS_ERR_RUN_STORE_FULL before anything is changed. */
+int taurus_runs_append(taurus_runs* runs, const int64_t* ids, const float* rows, int64_t ld, int64_t count, void* cuda_stream);
+/* End of the layer: every non-empty partition buffer is sorted and written as a (short) run. */
+int taurus_runs_flush(taurus_runs* runs, void* cuda_stream);
+/* Merge-on-read.  Writes rows of vertices [src_begin, src_end) in vertex order to out_rows (device memory,
+ * row v - src_begin at out_rows + (v - src_begin) * ld), asynchronously on the stream.  Every vertex of the
+ * range must be present in exactly one run: otherwise TAURUS_ERR_RUNS_INCOMPLETE (rows still held in a
+ * partition buffer do not count: flush first) and out_rows is untouched. */
+int taurus_runs_read_chunk(taurus_runs* runs, int64_t src_begin, int64_t src_end, float* out_rows, int64_t ld, void* cuda_stream);
+/* Counters (any pointer may be NULL): runs written, rows in the store, rows still in partition buffers. */
+int taurus_runs_info(taurus_runs* runs, int64_t* out_runs, int64_t* out_stored_rows, int64_t* out_buffered_rows);
+/* Directory in writing order: out[4 r + 0..3] = range, rows, first id, last id of run r (HOST memory).
+ * Blocking. */
+int taurus_runs_directory(taurus_runs* runs, int64_t* out, int64_t capacity_runs, int64_t* out_runs);
+/* Copies run `run` to HOST memory: out_ids [rows] and out_rows [rows x width] (either may be NULL).  Blocking. */
+int taurus_runs_get_run(taurus_runs* runs, int64_t run, int64_t* out_ids, float* out_rows);
+/* Forgets every run and every buffered row (the object is reused for the next layer's output).  Blocking. */
+int taurus_runs_reset(taurus_runs* runs);
+void taurus_runs_destroy(taurus_runs* runs);
+
+/* Run-output mode for the layer just begun (call after taurus_layer_begin, before the first push; exclusive
+ * with taurus_layer_set_dense_output).  Each chunk's finished rows are appended to `runs` (width must be
+ * dims[layer + 1]) on the library's output stream while the next chunk computes; the graduation buffer is
+ * split in halves as in dense-output mode (same drain_rows rule), runs->max_append_rows must be at least
+ * drain_rows / 2, and taurus_drain_* are not needed.  taurus_layer_end appends the last chunk's rows, flushes
+ * all partition buffers and waits, so that the runs can be read afterwards.  Which rows share a run depends
+ * on the order in which vertices of one chunk complete, which is not fixed; the rows themselves are. */
+int taurus_layer_set_run_output(taurus_ctx* ctx, taurus_runs* runs);
+/* taurus_push_chunk with the chunk's features read from `runs` (merge-on-read into the library's staging
+ * buffer on its copy stream, overlapping the previous chunk's kernels).  runs' width must be dims[layer]. */
+int taurus_push_chunk_from_runs(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, taurus_runs* runs, void* cuda_stream);
 
 /* Kernels launched by this context since init (for launch accounting in benchmarks). */
 int64_t taurus_launch_count(const taurus_ctx* ctx);

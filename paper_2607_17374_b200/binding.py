@@ -15,8 +15,9 @@ EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
 CHUNK_LOG_COLUMNS = ["hs", "ns", "ev", "gs", "need", "evicted", "reloaded", "completed", "occupancy"]
 ERROR_CODES = {
     "OK": 0, "INVALID_ARG": -1, "ORDER": -2, "POOL_TOO_SMALL": -3, "HOST_STORE_FULL": -4, "DRAIN_FULL": -5,
-    "CUDA": -6, "INTERNAL": -7, "NOMEM": -8, "UNSUPPORTED": -9,
+    "CUDA": -6, "INTERNAL": -7, "NOMEM": -8, "UNSUPPORTED": -9, "RUN_STORE_FULL": -10, "RUNS_INCOMPLETE": -11,
 }
+RUNS_HOST, RUNS_DEVICE = 0, 1
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _lib = None
@@ -72,12 +73,21 @@ class Stats(ctypes.Structure):
         return d
 
 
+class _RunsConfig(ctypes.Structure):
+    _fields_ = [("V", ctypes.c_int64), ("width", ctypes.c_int32), ("store_kind", ctypes.c_int32),
+                ("partitions", ctypes.c_int64), ("partition_rows", ctypes.c_int64), ("store_rows", ctypes.c_int64),
+                ("max_append_rows", ctypes.c_int64), ("max_chunk_rows", ctypes.c_int64)]
+
+
 EXPORTS = [
     "taurus_graph_init", "taurus_layer_begin", "taurus_push_chunk", "taurus_drain_completed", "taurus_drain_dense",
     "taurus_layer_end", "taurus_get_stats", "taurus_get_chunk_log", "taurus_get_vertex_array",
     "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count",
     "taurus_set_timing", "taurus_get_phase_ms", "taurus_destroy", "taurus_strerror", "taurus_last_cuda_error",
     "taurus_completion_counts_noalloc", "taurus_layer_set_dense_output", "taurus_reorder",
+    "taurus_runs_create", "taurus_runs_append", "taurus_runs_flush", "taurus_runs_read_chunk", "taurus_runs_info",
+    "taurus_runs_directory", "taurus_runs_get_run", "taurus_runs_reset", "taurus_runs_destroy",
+    "taurus_layer_set_run_output", "taurus_push_chunk_from_runs",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -108,6 +118,18 @@ def load_library():
     lib.taurus_completion_bound.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
     lib.taurus_completion_counts_noalloc.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
     lib.taurus_reorder.argtypes = [i64, i64, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.taurus_runs_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_RunsConfig)]
+    lib.taurus_runs_append.argtypes = [vp, vp, vp, i64, i64, vp]
+    lib.taurus_runs_flush.argtypes = [vp, vp]
+    lib.taurus_runs_read_chunk.argtypes = [vp, i64, i64, vp, i64, vp]
+    lib.taurus_runs_info.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.taurus_runs_directory.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
+    lib.taurus_runs_get_run.argtypes = [vp, i64, vp, vp]
+    lib.taurus_runs_reset.argtypes = [vp]
+    lib.taurus_runs_destroy.argtypes = [vp]
+    lib.taurus_runs_destroy.restype = None
+    lib.taurus_layer_set_run_output.argtypes = [vp, vp]
+    lib.taurus_push_chunk_from_runs.argtypes = [vp, i64, i64, vp, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -164,6 +186,69 @@ def reorder(V: int, E: int, row_ptr, col_idx, initial_rank=None, iterations: int
     if rc != 0:
         raise TaurusError(rc, "taurus_reorder")
     return rank, pos, J, span
+
+
+class Runs:
+    """One taurus_runs: sorted runs of (vertex id, row) records and the merge-on-read chunk reader."""
+
+    def __init__(self, V: int, width: int, partitions: int, partition_rows: int, store_rows: int = 0,
+                 max_append_rows: int = 0, max_chunk_rows: int = 0, store_kind: int = RUNS_HOST):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        self.V, self.width = V, width
+        cfg = _RunsConfig(V, width, store_kind, partitions, partition_rows, store_rows or V, max_append_rows or V,
+                          max_chunk_rows or V)
+        rc = self._lib.taurus_runs_create(ctypes.byref(self._h), ctypes.byref(cfg))
+        if rc != 0:
+            self._h = ctypes.c_void_p()
+            raise TaurusError(rc, "taurus_runs_create", self._lib.taurus_last_cuda_error().decode())
+
+    def _check(self, rc: int, where: str):
+        if rc != 0:
+            raise TaurusError(rc, where, self._lib.taurus_last_cuda_error().decode() if rc == ERROR_CODES["CUDA"] else "")
+
+    def append(self, ids, rows, ld: int, count: int, stream=None):
+        self._check(self._lib.taurus_runs_append(self._h, _ptr(ids), _ptr(rows), ld, count, _stream(stream)), "taurus_runs_append")
+
+    def flush(self, stream=None):
+        self._check(self._lib.taurus_runs_flush(self._h, _stream(stream)), "taurus_runs_flush")
+
+    def read_chunk(self, src_begin: int, src_end: int, out_rows, ld: int, stream=None):
+        self._check(self._lib.taurus_runs_read_chunk(self._h, src_begin, src_end, _ptr(out_rows), ld, _stream(stream)),
+                    "taurus_runs_read_chunk")
+
+    def info(self) -> dict:
+        a, b, c = ctypes.c_int64(0), ctypes.c_int64(0), ctypes.c_int64(0)
+        self._check(self._lib.taurus_runs_info(self._h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)), "taurus_runs_info")
+        return {"runs": int(a.value), "stored_rows": int(b.value), "buffered_rows": int(c.value)}
+
+    def directory(self) -> np.ndarray:
+        """int64 [runs, 4]: id range, rows, first id, last id of every run in writing order."""
+        n_runs = self.info()["runs"]
+        out = np.zeros((max(n_runs, 1), 4), np.int64)
+        n = ctypes.c_int64(0)
+        self._check(self._lib.taurus_runs_directory(self._h, out.ctypes.data, n_runs, ctypes.byref(n)), "taurus_runs_directory")
+        return out[:n.value].copy()
+
+    def get_run(self, run: int, rows_in_run: int):
+        ids = np.empty(rows_in_run, np.int64)
+        rows = np.empty((rows_in_run, self.width), np.float32)
+        self._check(self._lib.taurus_runs_get_run(self._h, run, ids.ctypes.data, rows.ctypes.data), "taurus_runs_get_run")
+        return ids, rows
+
+    def reset(self):
+        self._check(self._lib.taurus_runs_reset(self._h), "taurus_runs_reset")
+
+    def destroy(self):
+        if self._h:
+            self._lib.taurus_runs_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 class Context:
@@ -223,6 +308,13 @@ class Context:
 
     def layer_set_dense_output(self, dense_rows, ld: int):
         self._check(self._lib.taurus_layer_set_dense_output(self._h, _ptr(dense_rows), ld), "taurus_layer_set_dense_output")
+
+    def layer_set_run_output(self, runs: "Runs"):
+        self._check(self._lib.taurus_layer_set_run_output(self._h, runs._h), "taurus_layer_set_run_output")
+
+    def push_chunk_from_runs(self, src_begin: int, src_end: int, runs: "Runs", stream=None):
+        self._check(self._lib.taurus_push_chunk_from_runs(self._h, src_begin, src_end, runs._h, _stream(stream)),
+                    "taurus_push_chunk_from_runs")
 
     def layer_end(self) -> dict:
         s = Stats()

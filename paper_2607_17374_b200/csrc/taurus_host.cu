@@ -18,6 +18,7 @@ static bool cuda_ok(cudaError_t e, const char* what) {
   cudaGetLastError();
   return false;
 }
+void taurus_note_cuda_error(cudaError_t e, const char* what) { cuda_ok(e, what); }
 #define CU(call) do { if (!cuda_ok((call), #call)) return TAURUS_ERR_CUDA; } while (0)
 
 template <class T>
@@ -52,6 +53,8 @@ extern "C" const char* taurus_strerror(int code) {
     case TAURUS_ERR_INTERNAL: return "device-side consistency check failed";
     case TAURUS_ERR_NOMEM: return "out of memory";
     case TAURUS_ERR_UNSUPPORTED: return "unsupported shape or size";
+    case TAURUS_ERR_RUN_STORE_FULL: return "run store is full";
+    case TAURUS_ERR_RUNS_INCOMPLETE: return "the runs do not hold every vertex of the chunk exactly once";
     default: return "unknown error";
   }
 }
@@ -272,6 +275,7 @@ extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_strea
   CU(cudaStreamSynchronize(c->out_stream));
   c->layer = layer;
   c->dense_out = nullptr; c->dense_ld = 0;
+  c->run_out = nullptr; c->run_pending_half = -1;
   c->half_used[0] = c->half_used[1] = false;
   c->x_used[0] = c->x_used[1] = false;
   memset(c->h_ctl, 0, sizeof(DevCtl));
@@ -334,21 +338,40 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.evict_policy = c->evict_policy; a.seed = c->seed;
   a.gin_self = 1.0f + c->gin_eps;
   a.direct = c->pool_slots >= c->V ? 1 : 0;
-  a.dense_half = c->dense_out ? (int)(c->chunk_seq & 1) : -1;
-  a.grad_cap = c->dense_out ? c->drain_rows / 2 : c->drain_rows;
-  a.grad_off = c->dense_out ? (long long)a.dense_half * (c->drain_rows / 2) : 0;
+  const bool halves = c->dense_out || c->run_out;   // the graduation buffer alternates between two halves
+  a.dense_half = halves ? (int)(c->chunk_seq & 1) : -1;
+  a.grad_cap = halves ? c->drain_rows / 2 : c->drain_rows;
+  a.grad_off = halves ? (long long)a.dense_half * (c->drain_rows / 2) : 0;
   return a;
 }
 
-extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream) {
-  if (!c || !features) return TAURUS_ERR_INVALID_ARG;
+// Run-output mode: phase 2 of the append that is still open (rows of half run_pending_half), on the output stream.
+static int finish_run_append(taurus_ctx* c) {
+  if (!c->run_out || c->run_pending_half < 0) return TAURUS_OK;
+  const int h = c->run_pending_half;
+  c->run_pending_half = -1;
+  int rc = runs_phase2(c->run_out, c->out_stream);
+  if (rc) return rc;
+  CU(cudaEventRecord(c->out_done[h], c->out_stream));
+  c->half_used[h] = true;
+  return TAURUS_OK;
+}
+
+// One chunk through S1..S7.  The features come from `features` (host or device memory) or, when `src_runs` is
+// given, from the sorted runs of the previous layer by merge-on-read.
+static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, taurus_runs* src_runs, void* cuda_stream) {
+  if (!c || (!features && !src_runs)) return TAURUS_ERR_INVALID_ARG;
   if (c->layer < 0) return TAURUS_ERR_ORDER;
   if (src_begin != c->next_src) return TAURUS_ERR_ORDER;
   if (src_end <= src_begin || src_end > c->V || src_end - src_begin > c->chunk_sources) return TAURUS_ERR_INVALID_ARG;
-  if ((reinterpret_cast<uintptr_t>(features) & 3) != 0) return TAURUS_ERR_INVALID_ARG;
+  if (features && (reinterpret_cast<uintptr_t>(features) & 3) != 0) return TAURUS_ERR_INVALID_ARG;
+  if (src_runs && (runs_width(src_runs) != c->dims[c->layer] || runs_vertices(src_runs) != c->V ||
+                   runs_max_chunk(src_runs) < src_end - src_begin || src_runs == c->run_out))
+    return TAURUS_ERR_INVALID_ARG;
   if (c->h_ctl->error) return c->h_ctl->error;
   const long long bound = completion_bound(c, src_begin, src_end);
-  if (c->dense_out ? bound > c->drain_rows / 2 : c->ub_since_drain + bound > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
+  const bool halves = c->dense_out || c->run_out;
+  if (halves ? bound > c->drain_rows / 2 : c->ub_since_drain + bound > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(cudaSetDevice(c->device));
   if (st != c->last_stream) {   // keep chunk order across streams
@@ -373,11 +396,16 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   const float* X = features;
   int ldx = K;
   int xbuf = -1;
-  if (pointer_kind(features) != PK_DEVICE) {
+  if (src_runs || pointer_kind(features) != PK_DEVICE) {
     xbuf = (int)(c->host_pushes & 1);
-    c->host_pushes += 1;
     if (c->x_used[xbuf]) CU(cudaStreamWaitEvent(c->copy_stream, c->x_free[xbuf], 0));
-    CU(cudaMemcpyAsync(c->d_X[xbuf], features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+    if (src_runs) {   // merge-on-read; fails before anything is enqueued when the runs do not cover the chunk
+      int rc = runs_read_into(src_runs, src_begin, src_end, c->d_X[xbuf], K, c->copy_stream);
+      if (rc) return rc;
+    } else {
+      CU(cudaMemcpyAsync(c->d_X[xbuf], features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+    }
+    c->host_pushes += 1;
     CU(cudaEventRecord(c->x_ready[xbuf], c->copy_stream));
     CU(cudaStreamWaitEvent(st, c->x_ready[xbuf], 0));
     X = c->d_X[xbuf];
@@ -405,19 +433,56 @@ extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_e
   // S7
   if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
   launch_finalise(c, a, st);
-  if (a.dense_half >= 0) {   // hand this chunk's rows to the output stream
+  int run_rc = TAURUS_OK;
+  if (a.dense_half >= 0 && c->dense_out) {   // hand this chunk's rows to the output stream
     const int h = a.dense_half, d_out = c->dims[l + 1];
     CU(cudaEventRecord(c->fin_done[h], st));
     CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
     launch_place_half(c, h, d_out, a.Hp, c->out_stream);
     CU(cudaEventRecord(c->out_done[h], c->out_stream));
     c->half_used[h] = true;
+  } else if (a.dense_half >= 0) {
+    // Run-output mode.  The previous chunk's rows are already grouped by id range and its per-range counts are
+    // on their way to the host: now that this chunk's kernels are queued behind it, wait for them (the device
+    // stays busy), move those rows into the partition buffers and flush the full ones; then group this chunk's
+    // rows once its finalise has run.
+    const int h = a.dense_half;
+    CU(cudaEventRecord(c->fin_done[h], st));
+    run_rc = finish_run_append(c);
+    if (!run_rc) {
+      CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
+      const long long off = a.grad_off;
+      run_rc = runs_phase1(c->run_out, c->d_grad_ids + off, c->d_grad_rows + (size_t)off * a.Hp, a.Hp, std::min(bound, a.grad_cap),
+                           &c->d_ctl->out_count[h], 0, c->out_stream);
+      if (!run_rc) c->run_pending_half = h;
+    }
   }
   if (timing) cudaEventRecord(pev[5], st);
   CU(cudaGetLastError());
   c->next_src = src_end;
   c->chunk_seq += 1;
-  if (!c->dense_out) c->ub_since_drain += bound;
+  if (!halves) c->ub_since_drain += bound;
+  return run_rc;
+}
+
+extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream) {
+  if (!features) return TAURUS_ERR_INVALID_ARG;
+  return push_core(c, src_begin, src_end, features, nullptr, cuda_stream);
+}
+
+extern "C" int taurus_push_chunk_from_runs(taurus_ctx* c, int64_t src_begin, int64_t src_end, taurus_runs* runs, void* cuda_stream) {
+  if (!runs) return TAURUS_ERR_INVALID_ARG;
+  return push_core(c, src_begin, src_end, nullptr, runs, cuda_stream);
+}
+
+extern "C" int taurus_layer_set_run_output(taurus_ctx* c, taurus_runs* runs) {
+  if (!c || !runs) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0 || c->chunk_seq != 0 || c->dense_out) return TAURUS_ERR_ORDER;
+  if (runs_width(runs) != c->dims[c->layer + 1] || runs_vertices(runs) != c->V || runs_max_append(runs) < c->drain_rows / 2 ||
+      runs_pending(runs))
+    return TAURUS_ERR_INVALID_ARG;
+  c->run_out = runs;
+  c->run_pending_half = -1;
   return TAURUS_OK;
 }
 
@@ -528,6 +593,11 @@ extern "C" int taurus_layer_end(taurus_ctx* c, taurus_stats* stats) {
   if (!c) return TAURUS_ERR_INVALID_ARG;
   if (c->layer < 0) return TAURUS_ERR_ORDER;
   CU(cudaSetDevice(c->device));
+  if (c->run_out) {   // last chunk's rows, then every partition buffer leaves as a run
+    int rc = finish_run_append(c);
+    if (!rc) rc = runs_flush_all(c->run_out, c->out_stream);
+    if (rc) return rc;
+  }
   int err = read_ctl(c, c->last_stream);
   if (err) return err;
   if (stats) { int rc = fill_stats(c, stats); if (rc) return rc; }

@@ -146,6 +146,8 @@ struct taurus_ctx {
   // dense-output mode (taurus_layer_set_dense_output)
   float* dense_out = nullptr;           // device-visible address of the caller's matrix, NULL = mode off
   long long dense_ld = 0;
+  struct taurus_runs* run_out = nullptr;  // run-output mode (taurus_layer_set_run_output), NULL = mode off
+  int run_pending_half = -1;            // half whose rows are grouped but not yet moved to the partition buffers
   cudaStream_t out_stream = nullptr;    // rows leave the graduation buffer here while the next chunk computes
   cudaEvent_t fin_done[2] = {nullptr, nullptr}, out_done[2] = {nullptr, nullptr};
   bool half_used[2] = {false, false};
@@ -193,6 +195,21 @@ void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st
 void launch_completion_ranks(taurus_ctx* c, cudaStream_t st);                // fills d_rank_hist
 long long max_window_edges(taurus_ctx* c);                                  // most edges of any chunk_sources consecutive sources
 int check_in_degrees(taurus_ctx* c, cudaStream_t st);                        // 0 ok, 1 mismatch
+// ---- run_store.cu (sorted runs and merge-on-read)
+struct taurus_runs;
+int runs_width(const taurus_runs* r);
+long long runs_max_append(const taurus_runs* r);
+long long runs_max_chunk(const taurus_runs* r);
+long long runs_vertices(const taurus_runs* r);
+bool runs_pending(const taurus_runs* r);
+long long runs_launches(const taurus_runs* r);
+int runs_phase1(taurus_runs* r, const long long* ids, const float* rows, long long ld, long long n_bound, const long long* d_count,
+                long long count_host, cudaStream_t st);
+int runs_phase2(taurus_runs* r, cudaStream_t st);
+int runs_flush_all(taurus_runs* r, cudaStream_t st);
+int runs_read_into(taurus_runs* r, long long s, long long e, float* out, long long ld, cudaStream_t st);
+// ---- taurus_host.cu
+void taurus_note_cuda_error(cudaError_t e, const char* what);   // keeps the text for taurus_last_cuda_error
 // ---- kernels_scatter.cu
 void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_gemm_simt.cu

@@ -8,7 +8,7 @@ import taurus_gen as tg
 
 
 def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_features=False, drain_rows=None,
-                host_evict_rows=None, chunk_plan=None, gemm_mode=None, dense_output=False, evict_policy=0):
+                host_evict_rows=None, chunk_plan=None, gemm_mode=None, dense_output=False, evict_policy=0, run_output=None):
     """Runs every layer of workload w on the GPU.  Returns per-layer outputs (float32 [V, d_out]), the ids each
     chunk completed, stats and chunk logs.  Layer l+1 streams layer l's drained output."""
     import torch
@@ -21,13 +21,15 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
         0 if w.pool_slots >= V - w.hub_count else V - w.hub_count)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
-                     drain_rows or (2 * V if dense_output else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy, w.gin_eps)
+                     drain_rows or (2 * V if (dense_output or run_output) else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy, w.gin_eps)
     res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
     if host_features:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
     else:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).to(dev)
     stream = torch.cuda.current_stream()
+    prev_runs = None
+    res["runs"] = []
     for l in range(L):
         d_out = w.dims[l + 1]
         if dense_output and host_features:
@@ -42,7 +44,17 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
             res["masks"].append(None)
         per_chunk = []
         plan = chunk_plan or [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
-        if dense_output:      # the library places every finalised row itself; nothing to drain
+        if run_output:        # rows leave as sorted runs; layers after the first read their input back from runs
+            P, R, kind = run_output
+            runs = tb.Runs(V, d_out, P, R, store_rows=V, max_append_rows=V, max_chunk_rows=w.chunk, store_kind=kind)
+            ctx.layer_set_run_output(runs)
+            for (s, e) in plan:
+                if prev_runs is None:
+                    ctx.push_chunk(s, e, feat[s:e], stream)
+                else:
+                    ctx.push_chunk_from_runs(s, e, prev_runs, stream)
+            per_chunk = None
+        elif dense_output:    # the library places every finalised row itself; nothing to drain
             ctx.layer_set_dense_output(dense, d_out)
             for (s, e) in plan:
                 ctx.push_chunk(s, e, feat[s:e], stream)
@@ -62,6 +74,14 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
             if n or not drain_each_chunk:
                 per_chunk.append(("tail", ids_buf[:n].cpu().numpy().copy()))
         res["stats"].append(ctx.layer_end())
+        if run_output:
+            for (s, e) in [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]:
+                runs.read_chunk(s, e, dense[s:e], d_out, stream)
+            torch.cuda.synchronize()
+            if prev_runs is not None:
+                prev_runs.destroy()
+            prev_runs = runs
+            res["runs"].append(runs)
         res["chunk_log"].append(ctx.get_chunk_log())
         res["reload_count"].append(ctx.get_vertex_array("reload_count"))
         res["completed"].append(per_chunk)
