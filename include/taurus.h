@@ -63,7 +63,7 @@ enum {
   TAURUS_ERR_RUNS_INCOMPLETE = -11 /* a chunk read found fewer (or more) rows than vertices in its id range      */
 };
 
-enum { TAURUS_SAGE_MEAN = 0, TAURUS_GCN_SYM = 1, TAURUS_GIN_SUM = 2 };
+enum { TAURUS_SAGE_MEAN = 0, TAURUS_GCN_SYM = 1, TAURUS_GIN_SUM = 2, TAURUS_GAT = 3 };
 enum { TAURUS_GEMM_FP32 = 0, TAURUS_GEMM_BF16 = 1 };
 /* vertex states of Sect. 3.4 */
 enum { TAURUS_NOT_STARTED = 0, TAURUS_IN_BUFFER = 1, TAURUS_EVICTED = 2, TAURUS_ON_GPU = 3, TAURUS_COMPLETED = 4 };
@@ -80,7 +80,7 @@ typedef struct {
 
 /* Layer weights.  Copied at init.  dims[l] -> dims[l+1]; matrices are row-major dims[l] x dims[l+1] fp32. */
 typedef struct {
-  int32_t mode;                /* TAURUS_SAGE_MEAN, TAURUS_GCN_SYM or TAURUS_GIN_SUM          */
+  int32_t mode;                /* TAURUS_SAGE_MEAN, TAURUS_GCN_SYM, TAURUS_GIN_SUM or TAURUS_GAT */
   int32_t L;                   /* number of layers, 1..16                                     */
   const int32_t* dims;         /* [L+1], each in 1..1024 (host pointer)                       */
   const float* const* W_neigh; /* [L] (host array of pointers)                                */
@@ -89,6 +89,9 @@ typedef struct {
   const int32_t* act;          /* [L] 0 = identity, 1 = ReLU (host pointer)                   */
   int32_t gemm_mode;           /* TAURUS_GEMM_FP32: fp32-accurate projection; TAURUS_GEMM_BF16: bf16 operands, fp32 accumulate */
   float gin_eps;               /* TAURUS_GIN_SUM only: the self message is weighted 1 + gin_eps */
+  const float* const* att_src; /* TAURUS_GAT only: [L] each dims[l+1], the half of the attention vector applied to the source */
+  const float* const* att_dst; /* TAURUS_GAT only: [L] each dims[l+1], the half applied to the destination      */
+  float leaky_slope;           /* TAURUS_GAT only: negative slope of the LeakyReLU on the scores, in [0, 1]     */
 } taurus_model;
 
 typedef struct {
@@ -171,6 +174,29 @@ int taurus_layer_begin(taurus_ctx* ctx, int32_t layer, void* cuda_stream);
  * fit the graduation buffer: drain and push the same chunk again.
  */
 int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream);
+
+/*
+ * GATConv in three sequential passes (GATConv paragraph of Sect. 3.9); contexts created with TAURUS_GAT, one
+ * attention head (several heads are several contexts), fp32 projection only.  With h' = h W,
+ *     e_uv = LeakyReLU(att_src . h'_u + att_dst . h'_v),  alpha_uv = softmax over u in N(v) of e_uv,
+ *     out_v = act(sum_{u in N(v)} alpha_uv h'_u + b),
+ * where N(v) is the propagated in-multiset of v (all in-edges, or the layer's sampled ones) plus v itself:
+ * every vertex aggregates its own self message.  After taurus_layer_begin:
+ *   pass 1  taurus_gat_project_chunk for every chunk in ascending, contiguous order: writes the transformed rows
+ *           h' of sources [src_begin, src_end) to hprime_out (DEVICE memory, row i at hprime_out + i * ld,
+ *           ld >= dims[layer+1] floats) and keeps the two scalars att_src . h'_u and att_dst . h'_u of every
+ *           vertex.  `features` as in taurus_push_chunk.  Asynchronous on the stream.
+ *   pass 2  taurus_gat_attention, once all vertices are projected: a topology-only sweep over the CSR that
+ *           computes, per destination, the maximum score and the softmax normaliser (no per-edge state is
+ *           stored; the coefficients are recomputed from four per-vertex scalars where they are used).
+ *   pass 3  taurus_push_chunk / taurus_push_chunk_from_runs for every chunk with the transformed rows as
+ *           `features` ([n] x dims[layer+1], rows contiguous): the broadcast of Sect. 3.1 with each message
+ *           weighted by its attention coefficient; draining and taurus_layer_end as for the other modes.
+ * Calls out of this order return TAURUS_ERR_ORDER.
+ */
+int taurus_gat_project_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const float* features, float* hprime_out,
+                             int64_t ld, void* cuda_stream);
+int taurus_gat_attention(taurus_ctx* ctx, void* cuda_stream);
 
 /*
  * Copies out the vertices finalised since the last drain (Sect. 3.6): out_ids[i] and the dims[layer+1]

@@ -8,7 +8,7 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-SAGE_MEAN, GCN_SYM, GIN_SUM = 0, 1, 2
+SAGE_MEAN, GCN_SYM, GIN_SUM, GAT = 0, 1, 2, 3
 GEMM_FP32, GEMM_BF16 = 0, 1
 FLAG_SIMT_GEMM, FLAG_NO_GROUPING = 2, 4
 EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
@@ -47,7 +47,9 @@ class _Model(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("L", ctypes.c_int32), ("dims", ctypes.POINTER(ctypes.c_int32)),
                 ("W_neigh", ctypes.POINTER(ctypes.c_void_p)), ("W_self", ctypes.POINTER(ctypes.c_void_p)),
                 ("bias", ctypes.POINTER(ctypes.c_void_p)), ("act", ctypes.POINTER(ctypes.c_int32)),
-                ("gemm_mode", ctypes.c_int32), ("gin_eps", ctypes.c_float)]
+                ("gemm_mode", ctypes.c_int32), ("gin_eps", ctypes.c_float),
+                ("att_src", ctypes.POINTER(ctypes.c_void_p)), ("att_dst", ctypes.POINTER(ctypes.c_void_p)),
+                ("leaky_slope", ctypes.c_float)]
 
 
 class _Run(ctypes.Structure):
@@ -87,7 +89,7 @@ EXPORTS = [
     "taurus_completion_counts_noalloc", "taurus_layer_set_dense_output", "taurus_reorder",
     "taurus_runs_create", "taurus_runs_append", "taurus_runs_flush", "taurus_runs_read_chunk", "taurus_runs_info",
     "taurus_runs_directory", "taurus_runs_get_run", "taurus_runs_reset", "taurus_runs_destroy",
-    "taurus_layer_set_run_output", "taurus_push_chunk_from_runs",
+    "taurus_layer_set_run_output", "taurus_push_chunk_from_runs", "taurus_gat_project_chunk", "taurus_gat_attention",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -130,6 +132,8 @@ def load_library():
     lib.taurus_runs_destroy.restype = None
     lib.taurus_layer_set_run_output.argtypes = [vp, vp]
     lib.taurus_push_chunk_from_runs.argtypes = [vp, i64, i64, vp, vp]
+    lib.taurus_gat_project_chunk.argtypes = [vp, i64, i64, vp, vp, i64, vp]
+    lib.taurus_gat_attention.argtypes = [vp, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -257,7 +261,8 @@ class Context:
     def __init__(self, V: int, E: int, row_ptr, col_idx, in_degree, mode: int, dims: Sequence[int], W_neigh, W_self,
                  bias, act: Sequence[int], chunk_sources: int, pool_slots: int, hub_count: int = 0,
                  fanout: Optional[Sequence[int]] = None, seed: int = 1, host_evict_rows: int = 0, drain_rows: int = 0,
-                 gemm_mode: int = GEMM_FP32, flags: int = 0, evict_policy: int = 0, gin_eps: float = 0.0):
+                 gemm_mode: int = GEMM_FP32, flags: int = 0, evict_policy: int = 0, gin_eps: float = 0.0,
+                 att_src=None, att_dst=None, leaky_slope: float = 0.2):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         L = len(dims) - 1
@@ -269,7 +274,10 @@ class Context:
         c_wn = (ctypes.c_void_p * L)(*[_ptr(w) for w in W_neigh])
         c_ws = (ctypes.c_void_p * L)(*[_ptr(w) for w in W_self]) if W_self is not None else None
         c_b = (ctypes.c_void_p * L)(*[_ptr(b) for b in bias]) if bias is not None else None
-        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode, gin_eps)
+        c_as = (ctypes.c_void_p * L)(*[_ptr(a) for a in att_src]) if att_src is not None else None
+        c_ad = (ctypes.c_void_p * L)(*[_ptr(a) for a in att_dst]) if att_dst is not None else None
+        keep += [att_src, att_dst]
+        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode, gin_eps, c_as, c_ad, leaky_slope)
         c_f = (ctypes.c_int32 * L)(*[int(f) for f in fanout]) if fanout is not None else None
         r = _Run(chunk_sources, pool_slots, hub_count, c_f, seed, host_evict_rows, drain_rows or chunk_sources, flags, evict_policy)
         rc = self._lib.taurus_graph_init(ctypes.byref(self._h), ctypes.byref(g), ctypes.byref(m), ctypes.byref(r))
@@ -293,6 +301,13 @@ class Context:
             return rc
         self._check(rc, "taurus_push_chunk")
         return rc
+
+    def gat_project_chunk(self, src_begin: int, src_end: int, features, hprime_out, ld: int, stream=None):
+        self._check(self._lib.taurus_gat_project_chunk(self._h, src_begin, src_end, _ptr(features), _ptr(hprime_out), ld,
+                                                       _stream(stream)), "taurus_gat_project_chunk")
+
+    def gat_attention(self, stream=None):
+        self._check(self._lib.taurus_gat_attention(self._h, _stream(stream)), "taurus_gat_attention")
 
     def drain_completed(self, out_ids, out_rows, capacity_rows: int) -> int:
         n = ctypes.c_int64(0)

@@ -1,0 +1,104 @@
+// GATConv passes 1 and 2 (GATConv paragraph of Sect. 3.9).
+//
+// Pass 1 is the projection kernel with two extra weight columns, W att_src and W att_dst, so that the scalars
+// s_u = att_src . h'_u and t_u = att_dst . h'_u fall out of the same GEMM; gat_split_kernel files the rows
+// h' and the scalars away.  Pass 2 is topology-only: because LeakyReLU is non-decreasing, the maximum score
+// of destination v is LeakyReLU(max_u s_u + t_v), so one sweep over the CSR takes a running maximum of s_u per
+// destination and a second sweep sums exp(e_uv - max) into the normaliser; both use scalar atomics on
+// V-sized arrays and read no feature row.  Nothing per edge is stored: pass 3 recomputes
+// exp(LeakyReLU(s_u + t_v) - max_v) where it adds the message and divides by the normaliser at finalise.
+#include "taurus_internal.h"
+
+namespace {
+
+__device__ __forceinline__ int gl() { return threadIdx.x & 31; }
+__device__ __forceinline__ float lrelu(float x, float slope) { return x > 0.f ? x : slope * x; }
+
+// Order-preserving atomic maximum for finite floats of either sign.
+__device__ __forceinline__ void atomic_max_float(float* addr, float v) {
+  v += 0.f;   // -0 -> +0, whose bit pattern orders correctly among the non-negative values
+  if (v >= 0.f) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(v));
+  else atomicMin(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
+}
+
+__global__ void gat_split_kernel(const float* __restrict__ PT, int ldpt, int n, int Hp, int d_out, long long src_begin,
+                                 float* __restrict__ hprime, long long ld, float* __restrict__ att_s, float* __restrict__ att_t,
+                                 float* __restrict__ att_max) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    const float* src = PT + (size_t)r * ldpt;
+    float* dst = hprime + (size_t)r * ld;
+    for (int k = gl(); k < d_out; k += 32) dst[k] = src[k];
+    if (gl() == 0) {
+      const float s = src[Hp], t = src[Hp + 1];
+      att_s[src_begin + r] = s;
+      att_t[src_begin + r] = t;
+      att_max[src_begin + r] = s;   // the self message takes part in the maximum
+    }
+  }
+}
+
+// max over propagated in-edges (u -> v) of s_u, one warp per source row
+__global__ void gat_edge_max_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                                    const uint32_t* __restrict__ mask, const float* __restrict__ att_s, float* __restrict__ att_max) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    const float s = att_s[u];
+    for (long long e = row_ptr[u] + gl(); e < row_ptr[u + 1]; e += 32)
+      if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) atomic_max_float(&att_max[col[e]], s);
+  }
+}
+
+// tm[v] = (t_v, LeakyReLU(max_u s_u + t_v));  z[v] starts with the self term
+__global__ void gat_tm_kernel(long long V, const float* __restrict__ att_s, const float* __restrict__ att_t,
+                              const float* __restrict__ att_max, float slope, float2* __restrict__ tm, float* __restrict__ z) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
+    const float t = att_t[v];
+    const float m = lrelu(att_max[v] + t, slope);
+    tm[v] = make_float2(t, m);
+    z[v] = __expf(lrelu(att_s[v] + t, slope) - m);
+  }
+}
+
+__global__ void gat_edge_sum_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                                    const uint32_t* __restrict__ mask, const float* __restrict__ att_s,
+                                    const float2* __restrict__ tm, float slope, float* __restrict__ z) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    const float s = att_s[u];
+    for (long long e = row_ptr[u] + gl(); e < row_ptr[u + 1]; e += 32)
+      if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) {
+        const int v = col[e];
+        const float2 x = tm[v];
+        atomicAdd(&z[v], __expf(lrelu(s + x.x, slope) - x.y));
+      }
+  }
+}
+
+__global__ void gat_repack_kernel(const float* __restrict__ X, int n, int d_out, int Hp, float* __restrict__ PT) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps)
+    for (int k = gl(); k < Hp; k += 32) PT[(size_t)r * Hp + k] = k < d_out ? X[(size_t)r * d_out + k] : 0.f;
+}
+
+}  // namespace
+
+void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st) {
+  gat_split_kernel<<<c->sm_count * 8, 256, 0, st>>>(c->d_PT, Hp + 4, n, Hp, d_out, src_begin, hprime_out, ld, c->d_att_s, c->d_att_t,
+                                                    c->d_att_max);
+  c->launches += 1;
+}
+
+void launch_gat_attention(taurus_ctx* c, cudaStream_t st) {
+  const int grid = c->sm_count * 8;
+  gat_edge_max_kernel<<<grid, 256, 0, st>>>(c->V, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_max);
+  gat_tm_kernel<<<grid, 256, 0, st>>>(c->V, c->d_att_s, c->d_att_t, c->d_att_max, c->leaky, c->d_att_tm, c->d_att_z);
+  gat_edge_sum_kernel<<<grid, 256, 0, st>>>(c->V, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_tm, c->leaky, c->d_att_z);
+  c->launches += 3;
+}
+
+void launch_gat_repack(taurus_ctx* c, const float* X, int n, int d_out, int Hp, cudaStream_t st) {
+  gat_repack_kernel<<<c->sm_count * 8, 256, 0, st>>>(X, n, d_out, Hp, c->d_PT);
+  c->launches += 1;
+}

@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restri
     float c_out = 1.f, self_mul = 1.f;
     if (mode == TAURUS_GCN_SYM) {
       c_out = (float)(1.0 / sqrt((double)(row_ptr[u + 1] - row_ptr[u]) + 1.0));
-    } else {
+    } else if (mode == TAURUS_SAGE_MEAN) {
       int d = din[u];
       int m = (fanout > 0 && d > fanout) ? fanout : d;
       self_mul = (float)(m > 1 ? m : 1);
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restri
       if (cidx >= N) continue;
       float x = acc[i][j];
       if (cidx < Hp) x *= c_out;
-      else x = (x + bias[cidx - Hp]) * self_mul;
+      else if (mode != TAURUS_GAT) x = (x + bias[cidx - Hp]) * self_mul;   // GAT: the attention scalars as they are
       PT[(size_t)r * N + cidx] = x;
     }
   }
@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restri
 
 void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st) {
   const int Hp = taurus_round_up(c->dims[layer + 1], 4);
-  const int N = c->mode == TAURUS_SAGE_MEAN ? 2 * Hp : Hp;
+  const int N = taurus_proj_width(c->mode, Hp);
   dim3 grid((N + BN - 1) / BN, (n + BM - 1) / BM);
   project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, c->dims[layer], c->d_Wcat[layer], N, c->d_PT, n, Hp, c->mode,
                                             c->d_bias[layer], c->d_row_ptr, c->d_din, c->fanout[layer], src_begin);

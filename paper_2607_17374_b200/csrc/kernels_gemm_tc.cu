@@ -278,7 +278,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       const long long u = g.src_begin + r;
       if (g.mode == TAURUS_GCN_SYM) {
         c_out = (float)(1.0 / sqrt((double)(g.row_ptr[u + 1] - g.row_ptr[u]) + 1.0));
-      } else {
+      } else if (g.mode == TAURUS_SAGE_MEAN) {
         const int d = g.din[u];
         const int m = (g.fanout > 0 && d > g.fanout) ? g.fanout : d;
         self_mul = (float)(m > 1 ? m : 1);
@@ -312,8 +312,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           float4 o;
           float* po = &o.x;
           const int c = cbase + j;
-          if (c >= g.Hp && c < g.N) {         // T columns: (x W_self + b) * max(|M(u)|, 1)
-            const float4 b = *reinterpret_cast<const float4*>(g.bias + (c - g.Hp));
+          if (c >= g.Hp && c < g.N) {         // T columns: (x W_self + b) * max(|M(u)|, 1); GAT: the two attention scalars as they are
+            const float4 b = g.mode == TAURUS_GAT ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(g.bias + (c - g.Hp));
             po[0] = (__uint_as_float(v[j]) + b.x) * self_mul; po[1] = (__uint_as_float(v[j + 1]) + b.y) * self_mul;
             po[2] = (__uint_as_float(v[j + 2]) + b.z) * self_mul; po[3] = (__uint_as_float(v[j + 3]) + b.w) * self_mul;
           } else {                            // P columns: c_out(u) * (x W_neigh)
@@ -460,7 +460,7 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
   WImage* w = static_cast<WImage*>(c->tc_image[layer]);
   const int K = c->dims[layer], Hp = taurus_round_up(c->dims[layer + 1], 4);
-  const int N = c->mode == TAURUS_SAGE_MEAN ? 2 * Hp : Hp;
+  const int N = taurus_proj_width(c->mode, Hp);
   CUtensorMap map_x;
   if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, 32)) return TAURUS_ERR_CUDA;
   CUtensorMap map_out;

@@ -204,7 +204,9 @@ void launch_classify_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st)
 // instructions per edge: an earlier version with lane-parallel edge loads and shuffles was issue-bound.
 #define SPAN_EDGES 128   // edges per warp span (all sub-groups together)
 
-template <int LPE, int VPL, bool SAMPLED, bool DIRECT>
+// With GAT every message is weighted by exp(LeakyReLU(s_u + t_v) - max_v), recomputed from per-vertex scalars
+// (the 1 / normaliser factor is applied at finalise).
+template <int LPE, int VPL, bool SAMPLED, bool DIRECT, bool GAT>
 __global__ void __launch_bounds__(256, (VPL <= 2 ? 3 : 1))
 scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
@@ -229,6 +231,8 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
   int bad = 0;
 
   int cur = -1, cnt = 0, cur_loc = -1;
+  float2 cur_tm = make_float2(0.f, 0.f);
+  const float* const att_s_chunk = GAT ? a.att_s + a.src_begin : nullptr;
   float4 sum[VPL];
   // byte addressing with 32-bit x 32-bit -> 64-bit products keeps the address arithmetic to one instruction
   const char* const Pb = reinterpret_cast<const char*>(a.PT) + c4 * 16;
@@ -250,15 +254,28 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
     groups += 1;
     if (!DIRECT && l >= pool) hub_msgs += (unsigned)cnt;
   };
-  auto take = [&](int d, const float4 (&row)[VPL]) {
-    if (d != cur) {
+  auto take = [&](int d, int src_rel, const float4 (&row)[VPL]) {
+    const bool fresh = d != cur;
+    if (fresh) {
       if (cur >= 0) flush();
-      cur = d; cnt = 1;
+      cur = d; cnt = 0;
       if (!DIRECT) cur_loc = a.loc[d];
+      if (GAT) cur_tm = a.att_tm[d];
+    }
+    cnt++;
+    if (GAT) {
+      const float e = att_s_chunk[src_rel] + cur_tm.x;
+      const float w = __expf((e > 0.f ? e : a.leaky * e) - cur_tm.y);
+#pragma unroll
+      for (int k = 0; k < VPL; ++k) {
+        if (fresh) sum[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        sum[k].x = fmaf(w, row[k].x, sum[k].x); sum[k].y = fmaf(w, row[k].y, sum[k].y);
+        sum[k].z = fmaf(w, row[k].z, sum[k].z); sum[k].w = fmaf(w, row[k].w, sum[k].w);
+      }
+    } else if (fresh) {
 #pragma unroll
       for (int k = 0; k < VPL; ++k) sum[k] = row[k];
     } else {
-      cnt++;
 #pragma unroll
       for (int k = 0; k < VPL; ++k) { sum[k].x += row[k].x; sum[k].y += row[k].y; sum[k].z += row[k].z; sum[k].w += row[k].w; }
     }
@@ -291,7 +308,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
         if (!SAMPLED || ed[q].x >= 0) fetch(ed[q].y, row[q]);
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        if (!SAMPLED || ed[q].x >= 0) take(ed[q].x, row[q]);
+        if (!SAMPLED || ed[q].x >= 0) take(ed[q].x, ed[q].y, row[q]);
     }
 #pragma unroll 1
     for (; left > 0; --left, ++ge, ++x) {             // ragged end of the chunk's list
@@ -299,7 +316,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
       if (SAMPLED && !((gmask[x >> 5] >> (x & 31)) & 1u)) continue;
       float4 row[VPL];
       fetch(ed.y, row);
-      take(ed.x, row);
+      take(ed.x, ed.y, row);
     }
     if (cur >= 0) flush();   // a group that continues in another stretch is flushed by both
     cur = -1;
@@ -329,9 +346,17 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) red_add_v4(dst + 4 * (c4 + k * LPE), reinterpret_cast<const float4*>(p)[c4 + k * LPE]);
       } else {
-        // one shared weight: GCN  P_v + b * sqrt(din(v) + 1);  GIN  (1 + eps) * P_v + b
-        const float ps = a.mode == TAURUS_GIN_SUM ? a.gin_self : 1.0f;
-        const float sc = a.mode == TAURUS_GIN_SUM ? 1.0f : (float)sqrt((double)a.din[vj] + 1.0);
+        // one shared weight: GCN  P_v + b * sqrt(din(v) + 1);  GIN  (1 + eps) * P_v + b;
+        // GAT  exp(e_vv - max_v) * h'_v + b * normaliser(v)
+        float ps = 1.0f, sc = 1.0f;
+        if (a.mode == TAURUS_GIN_SUM) ps = a.gin_self;
+        else if (a.mode == TAURUS_GCN_SYM) sc = (float)sqrt((double)a.din[vj] + 1.0);
+        else {
+          const float2 tm = a.att_tm[vj];
+          const float e = a.att_s[vj] + tm.x;
+          ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
+          sc = a.att_z[vj];
+        }
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) {
@@ -357,23 +382,27 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
   }
 }
 
-template <int LPE, int VPL, bool SAMPLED, bool DIRECT>
+template <int LPE, int VPL, bool SAMPLED, bool DIRECT, bool GAT>
 static void launch_sg(taurus_ctx* c, const ChunkArgs& a, const uint32_t* gm, cudaStream_t st) {
   static int blocks_per_sm = 0;
   if (blocks_per_sm == 0) {
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, scatter_grouped_kernel<LPE, VPL, SAMPLED, DIRECT>, 256, 0) != cudaSuccess ||
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, scatter_grouped_kernel<LPE, VPL, SAMPLED, DIRECT, GAT>, 256, 0) != cudaSuccess ||
         blocks_per_sm < 1)
       blocks_per_sm = 1;
   }
-  scatter_grouped_kernel<LPE, VPL, SAMPLED, DIRECT><<<c->sm_count * blocks_per_sm, 256, 0, st>>>(a, c->d_gedge, gm);
+  scatter_grouped_kernel<LPE, VPL, SAMPLED, DIRECT, GAT><<<c->sm_count * blocks_per_sm, 256, 0, st>>>(a, c->d_gedge, gm);
 }
 
 template <int LPE, int VPL>
 static void launch_sg2(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   const uint32_t* gm = c->d_mask_cur ? c->d_gmask : nullptr;
   const bool direct = a.direct && c->hub_count == 0;
-  if (gm) { if (direct) launch_sg<LPE, VPL, true, true>(c, a, gm, st); else launch_sg<LPE, VPL, true, false>(c, a, gm, st); }
-  else    { if (direct) launch_sg<LPE, VPL, false, true>(c, a, gm, st); else launch_sg<LPE, VPL, false, false>(c, a, gm, st); }
+  if (a.mode == TAURUS_GAT) {   // the weighted variants exist for the general (slot-mapped) addressing only
+    if (gm) launch_sg<LPE, VPL, true, false, true>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, true>(c, a, gm, st);
+    return;
+  }
+  if (gm) { if (direct) launch_sg<LPE, VPL, true, true, false>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, false>(c, a, gm, st); }
+  else    { if (direct) launch_sg<LPE, VPL, false, true, false>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, false>(c, a, gm, st); }
 }
 
 void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {

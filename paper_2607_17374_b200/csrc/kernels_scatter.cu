@@ -97,6 +97,13 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
         const long long u = a.src_begin + t * 32 + lane;
         if (u < a.src_end) { v = (int)u; src = u; }
       }
+      // GAT: weight of this lane's message, exp(LeakyReLU(s_u + t_v) - max_v)
+      float wgt = 1.f;
+      if (a.mode == TAURUS_GAT && v >= 0 && !self_run) {
+        const float2 tm = a.att_tm[v];
+        const float e = a.att_s[src] + tm.x;
+        wgt = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
+      }
       // pending count and slot of this lane's destination
       int l = -1;
       if (v >= 0) {
@@ -117,6 +124,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
         const int j = step + sub;
         const int lj = __shfl_sync(FULL, l, j);
         const long long sj = __shfl_sync(FULL, src, j);
+        const float wj = __shfl_sync(FULL, wgt, j);
         if (lj < 0) continue;
         if (sj != held) {
           held = sj;
@@ -128,9 +136,17 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
               for (int k = 0; k < VPL; ++k)
                 if (c4 + k * LPE < nvec) row[k] = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
             } else {       // one shared weight: the self message is built from the vertex's own P row
-              // GCN: P_v (already scaled by c_out(v)) + b * sqrt(din(v) + 1);  GIN: (1 + eps) * P_v + b
-              const float ps = a.mode == TAURUS_GIN_SUM ? a.gin_self : 1.0f;
-              const float s = a.mode == TAURUS_GIN_SUM ? 1.0f : (float)sqrt((double)a.din[sj] + 1.0);
+              // GCN: P_v (already scaled by c_out(v)) + b * sqrt(din(v) + 1);  GIN: (1 + eps) * P_v + b;
+              // GAT: exp(e_vv - max_v) * h'_v + b * normaliser(v)
+              float ps = 1.0f, s = 1.0f;
+              if (a.mode == TAURUS_GIN_SUM) ps = a.gin_self;
+              else if (a.mode == TAURUS_GCN_SYM) s = (float)sqrt((double)a.din[sj] + 1.0);
+              else {
+                const float2 tm = a.att_tm[sj];
+                const float e = a.att_s[sj] + tm.x;
+                ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
+                s = a.att_z[sj];
+              }
 #pragma unroll
               for (int k = 0; k < VPL; ++k)
                 if (c4 + k * LPE < nvec) {
@@ -146,9 +162,16 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
           }
         }
         float* dst = a.acc + (size_t)lj * a.Hp;
+        if (a.mode == TAURUS_GAT && !self_run) {
 #pragma unroll
-        for (int k = 0; k < VPL; ++k)
-          if (c4 + k * LPE < nvec) red_add_v4(dst + 4 * (c4 + k * LPE), row[k]);
+          for (int k = 0; k < VPL; ++k)
+            if (c4 + k * LPE < nvec)
+              red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(row[k].x * wj, row[k].y * wj, row[k].z * wj, row[k].w * wj));
+        } else {
+#pragma unroll
+          for (int k = 0; k < VPL; ++k)
+            if (c4 + k * LPE < nvec) red_add_v4(dst + 4 * (c4 + k * LPE), row[k]);
+        }
       }
     }
   }

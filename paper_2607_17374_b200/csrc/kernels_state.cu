@@ -438,6 +438,8 @@ __global__ void finalise_kernel(ChunkArgs a) {
       scale = 1.0f / (float)(m > 1 ? m : 1);
     } else if (a.mode == TAURUS_GCN_SYM) {
       scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+    } else if (a.mode == TAURUS_GAT) {
+      scale = 1.0f / a.att_z[v];   // softmax normaliser
     } else {
       scale = 1.0f;   // GIN: plain sum
     }

@@ -73,6 +73,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
+  cudaFree(c->d_att_s); cudaFree(c->d_att_t); cudaFree(c->d_att_max); cudaFree(c->d_att_tm); cudaFree(c->d_att_z);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
   cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
   cudaFree(c->d_ctl); cudaFree(c->d_chunk_log);
@@ -100,6 +101,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   c->V = g->V; c->E = g->E; c->L = m->L; c->mode = m->mode; c->gemm_mode = m->gemm_mode; c->flags = r->flags;
   c->seed = r->seed;
   c->gin_eps = m->gin_eps;
+  c->leaky = m->leaky_slope;
   c->chunk_sources = r->chunk_sources; c->pool_slots = r->pool_slots; c->hub_count = r->hub_count;
   c->host_rows = r->host_evict_rows; c->drain_rows = r->drain_rows; c->evict_policy = r->evict_policy;
   bool any_sampled = false;
@@ -110,6 +112,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     any_sampled |= c->fanout[l] > 0;
     c->Hmax = std::max(c->Hmax, taurus_round_up(c->dims[l + 1], 4));
     c->Kmax = std::max(c->Kmax, taurus_round_up(c->dims[l], 4));
+    if (c->mode == TAURUS_GAT) c->Kmax = std::max(c->Kmax, taurus_round_up(c->dims[l + 1], 4));   // pass 3 streams h' rows
   }
   const long long V = c->V, E = c->E;
 
@@ -148,7 +151,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   // weights: Wcat = [W_neigh | W_self] with both halves padded to Hp columns
   for (int l = 0; l < c->L; ++l) {
     const int K = c->dims[l], d_out = c->dims[l + 1], Hp = taurus_round_up(d_out, 4);
-    const int N = c->mode == TAURUS_SAGE_MEAN ? 2 * Hp : Hp;
+    const int N = taurus_proj_width(c->mode, Hp);
     std::vector<float> wn((size_t)K * d_out), ws, b((size_t)Hp, 0.f), cat((size_t)K * N, 0.f);
     CU(cudaMemcpy(wn.data(), m->W_neigh[l], wn.size() * sizeof(float), cudaMemcpyDefault));
     if (c->mode == TAURUS_SAGE_MEAN) {
@@ -161,6 +164,17 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
         cat[(size_t)k * N + j] = wn[(size_t)k * d_out + j];
         if (c->mode == TAURUS_SAGE_MEAN) cat[(size_t)k * N + Hp + j] = ws[(size_t)k * d_out + j];
       }
+    if (c->mode == TAURUS_GAT) {   // two more columns, W att_src and W att_dst: the attention scalars come out of the same GEMM
+      std::vector<float> as((size_t)d_out), ad((size_t)d_out);
+      CU(cudaMemcpy(as.data(), m->att_src[l], as.size() * sizeof(float), cudaMemcpyDefault));
+      CU(cudaMemcpy(ad.data(), m->att_dst[l], ad.size() * sizeof(float), cudaMemcpyDefault));
+      for (int k = 0; k < K; ++k) {
+        double ss = 0.0, sd = 0.0;
+        for (int j = 0; j < d_out; ++j) { ss += (double)wn[(size_t)k * d_out + j] * as[(size_t)j]; sd += (double)wn[(size_t)k * d_out + j] * ad[(size_t)j]; }
+        cat[(size_t)k * N + Hp] = (float)ss;
+        cat[(size_t)k * N + Hp + 1] = (float)sd;
+      }
+    }
     ALLOC(c->d_Wcat[l], cat.size()); ALLOC(c->d_bias[l], b.size());
     CU(cudaMemcpy(c->d_Wcat[l], cat.data(), cat.size() * sizeof(float), cudaMemcpyHostToDevice));
     CU(cudaMemcpy(c->d_bias[l], b.data(), b.size() * sizeof(float), cudaMemcpyHostToDevice));
@@ -204,6 +218,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     CU(cudaEventCreateWithFlags(&c->out_done[i], cudaEventDisableTiming));
   }
   ALLOC(c->d_PT, (size_t)c->chunk_sources * 2 * c->Hmax);
+  if (c->mode == TAURUS_GAT) { ALLOC(c->d_att_s, V); ALLOC(c->d_att_t, V); ALLOC(c->d_att_max, V); ALLOC(c->d_att_tm, V); ALLOC(c->d_att_z, V); }
   // sampling
   if (any_sampled) {
     int rc = build_in_edge_order(c);
@@ -235,7 +250,13 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
   if (!g || !m || !r || !g->row_ptr || !g->in_degree || (g->E > 0 && !g->col_idx)) return TAURUS_ERR_INVALID_ARG;
   if (g->V < 1 || g->V >= (1ll << 31) || g->E < 0 || g->E >= (1ll << 32)) return TAURUS_ERR_INVALID_ARG;
   if (m->L < 1 || m->L > TAURUS_MAX_LAYERS || !m->dims || !m->W_neigh) return TAURUS_ERR_INVALID_ARG;
-  if (m->mode != TAURUS_SAGE_MEAN && m->mode != TAURUS_GCN_SYM && m->mode != TAURUS_GIN_SUM) return TAURUS_ERR_INVALID_ARG;
+  if (m->mode != TAURUS_SAGE_MEAN && m->mode != TAURUS_GCN_SYM && m->mode != TAURUS_GIN_SUM && m->mode != TAURUS_GAT) return TAURUS_ERR_INVALID_ARG;
+  if (m->mode == TAURUS_GAT) {
+    if (!m->att_src || !m->att_dst || !(m->leaky_slope >= 0.f && m->leaky_slope <= 1.f)) return TAURUS_ERR_INVALID_ARG;
+    if (m->gemm_mode != TAURUS_GEMM_FP32) return TAURUS_ERR_UNSUPPORTED;   // the scores need the fp32-accurate projection
+    for (int l = 0; l < m->L; ++l)
+      if (!m->att_src[l] || !m->att_dst[l]) return TAURUS_ERR_INVALID_ARG;
+  }
   if (m->gemm_mode != TAURUS_GEMM_FP32 && m->gemm_mode != TAURUS_GEMM_BF16) return TAURUS_ERR_INVALID_ARG;
   if (m->mode == TAURUS_SAGE_MEAN && !m->W_self) return TAURUS_ERR_INVALID_ARG;
   for (int l = 0; l <= m->L; ++l)
@@ -276,6 +297,7 @@ extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_strea
   c->layer = layer;
   c->dense_out = nullptr; c->dense_ld = 0;
   c->run_out = nullptr; c->run_pending_half = -1;
+  c->gat_next_src = 0; c->gat_ready = false;
   c->half_used[0] = c->half_used[1] = false;
   c->x_used[0] = c->x_used[1] = false;
   memset(c->h_ctl, 0, sizeof(DevCtl));
@@ -329,7 +351,8 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.victims = c->d_victims; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
   a.Hp = taurus_round_up(c->dims[l + 1], 4);
-  a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;
+  a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;   // GAT pass 3 scatters h' rows repacked to pitch Hp
+  a.att_s = c->d_att_s; a.att_tm = c->d_att_tm; a.att_z = c->d_att_z; a.leaky = c->leaky;
   a.bias = c->d_bias[l];
   a.ctl = c->d_ctl; a.chunk_log = c->d_chunk_log; a.log_capacity = c->log_capacity;
   a.V = c->V; a.pool_slots = c->pool_slots; a.hub_count = c->hub_count; a.host_rows = c->host_rows; a.drain_rows = c->drain_rows;
@@ -357,6 +380,30 @@ static int finish_run_append(taurus_ctx* c) {
   return TAURUS_OK;
 }
 
+// S1: features of sources [s, e) ([n x K], rows contiguous) to the device.  Host chunks are copied on the library's
+// copy stream into one of two staging buffers, so that the copy of chunk k+1 overlaps the kernels of chunk k; a
+// chunk read from sorted runs is merged into the same buffers; a device pointer is used in place (*xbuf = -1).
+static int stage_chunk(taurus_ctx* c, const float* features, taurus_runs* src_runs, long long s, long long e, int K, cudaStream_t st,
+                       const float** X, int* xbuf) {
+  *X = features;
+  *xbuf = -1;
+  if (!src_runs && pointer_kind(features) == PK_DEVICE) return TAURUS_OK;
+  const int b = (int)(c->host_pushes & 1);
+  if (c->x_used[b]) CU(cudaStreamWaitEvent(c->copy_stream, c->x_free[b], 0));
+  if (src_runs) {   // merge-on-read; fails before anything is enqueued when the runs do not cover the chunk
+    int rc = runs_read_into(src_runs, s, e, c->d_X[b], K, c->copy_stream);
+    if (rc) return rc;
+  } else {
+    CU(cudaMemcpyAsync(c->d_X[b], features, (size_t)(e - s) * K * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
+  }
+  c->host_pushes += 1;
+  CU(cudaEventRecord(c->x_ready[b], c->copy_stream));
+  CU(cudaStreamWaitEvent(st, c->x_ready[b], 0));
+  *X = c->d_X[b];
+  *xbuf = b;
+  return TAURUS_OK;
+}
+
 // One chunk through S1..S7.  The features come from `features` (host or device memory) or, when `src_runs` is
 // given, from the sorted runs of the previous layer by merge-on-read.
 static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, taurus_runs* src_runs, void* cuda_stream) {
@@ -365,7 +412,9 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   if (src_begin != c->next_src) return TAURUS_ERR_ORDER;
   if (src_end <= src_begin || src_end > c->V || src_end - src_begin > c->chunk_sources) return TAURUS_ERR_INVALID_ARG;
   if (features && (reinterpret_cast<uintptr_t>(features) & 3) != 0) return TAURUS_ERR_INVALID_ARG;
-  if (src_runs && (runs_width(src_runs) != c->dims[c->layer] || runs_vertices(src_runs) != c->V ||
+  const bool gat = c->mode == TAURUS_GAT;   // pass 3: the features are the transformed rows h'
+  if (gat && !c->gat_ready) return TAURUS_ERR_ORDER;
+  if (src_runs && (runs_width(src_runs) != c->dims[c->layer + (gat ? 1 : 0)] || runs_vertices(src_runs) != c->V ||
                    runs_max_chunk(src_runs) < src_end - src_begin || src_runs == c->run_out))
     return TAURUS_ERR_INVALID_ARG;
   if (c->h_ctl->error) return c->h_ctl->error;
@@ -380,7 +429,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
     c->last_stream = st;
   }
   const int l = c->layer;
-  const int K = c->dims[l];
+  const int K = gat ? c->dims[l + 1] : c->dims[l];
   const int n = (int)(src_end - src_begin);
   cudaEvent_t* pev = nullptr;
   if (c->timing && c->timed_pushes < TAURUS_MAX_TIMED_PUSHES) {
@@ -391,35 +440,25 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   }
   const bool timing = pev != nullptr;
   if (timing) cudaEventRecord(pev[0], st);
-  // S1: features to the device.  Host chunks are copied on the library's copy stream into one of two staging
-  // buffers, so that the copy of chunk k+1 overlaps the kernels of chunk k.
-  const float* X = features;
+  // S1: features to the device
+  const float* X = nullptr;
   int ldx = K;
   int xbuf = -1;
-  if (src_runs || pointer_kind(features) != PK_DEVICE) {
-    xbuf = (int)(c->host_pushes & 1);
-    if (c->x_used[xbuf]) CU(cudaStreamWaitEvent(c->copy_stream, c->x_free[xbuf], 0));
-    if (src_runs) {   // merge-on-read; fails before anything is enqueued when the runs do not cover the chunk
-      int rc = runs_read_into(src_runs, src_begin, src_end, c->d_X[xbuf], K, c->copy_stream);
-      if (rc) return rc;
-    } else {
-      CU(cudaMemcpyAsync(c->d_X[xbuf], features, (size_t)n * K * sizeof(float), cudaMemcpyHostToDevice, c->copy_stream));
-    }
-    c->host_pushes += 1;
-    CU(cudaEventRecord(c->x_ready[xbuf], c->copy_stream));
-    CU(cudaStreamWaitEvent(st, c->x_ready[xbuf], 0));
-    X = c->d_X[xbuf];
-  }
+  { int rc = stage_chunk(c, features, src_runs, src_begin, src_end, K, st, &X, &xbuf); if (rc) return rc; }
   if (timing) cudaEventRecord(pev[1], st);
   ChunkArgs a = make_args(c, src_begin, src_end);
-  // S2: projection
-  if (project_tc_usable(c, l, X, ldx)) {
+  // S2: projection (GAT: already done in pass 1; rows narrower than their padded width are repacked)
+  bool x_in_use = false;
+  if (gat) {
+    if (K == a.Hp && (reinterpret_cast<uintptr_t>(X) & 15) == 0) { a.PT = X; x_in_use = true; }
+    else launch_gat_repack(c, X, n, K, a.Hp, st);
+  } else if (project_tc_usable(c, l, X, ldx)) {
     int rc = launch_project_tc(c, l, X, ldx, src_begin, n, st);
     if (rc) return rc;
   } else {
     launch_project_simt(c, l, X, ldx, src_begin, n, st);
   }
-  if (xbuf >= 0) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }
+  if (xbuf >= 0 && !x_in_use) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }
   if (timing) cudaEventRecord(pev[2], st);
   // S3, S4
   const bool grouped = c->d_gdst != nullptr && src_begin % c->chunk_sources == 0 &&
@@ -429,6 +468,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   if (timing) cudaEventRecord(pev[3], st);
   // S5, S5', S6
   if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
+  if (xbuf >= 0 && x_in_use) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }   // the scatter read the staged rows in place
   if (timing) cudaEventRecord(pev[4], st);
   // S7
   if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
@@ -463,6 +503,55 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   c->chunk_seq += 1;
   if (!halves) c->ub_since_drain += bound;
   return run_rc;
+}
+
+extern "C" int taurus_gat_project_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, float* hprime_out,
+                                        int64_t ld, void* cuda_stream) {
+  if (!c || !features || !hprime_out) return TAURUS_ERR_INVALID_ARG;
+  if (c->mode != TAURUS_GAT) return TAURUS_ERR_UNSUPPORTED;
+  if (c->layer < 0 || c->gat_ready || c->chunk_seq != 0 || src_begin != c->gat_next_src) return TAURUS_ERR_ORDER;
+  if (src_end <= src_begin || src_end > c->V || src_end - src_begin > c->chunk_sources) return TAURUS_ERR_INVALID_ARG;
+  const int l = c->layer, K = c->dims[l], d_out = c->dims[l + 1], Hp = taurus_round_up(d_out, 4);
+  if (ld < d_out || (reinterpret_cast<uintptr_t>(features) & 3) != 0 || pointer_kind(hprime_out) != PK_DEVICE) return TAURUS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CU(cudaSetDevice(c->device));
+  if (st != c->last_stream) {
+    CU(cudaEventRecord(c->order_event, c->last_stream));
+    CU(cudaStreamWaitEvent(st, c->order_event, 0));
+    c->last_stream = st;
+  }
+  const int n = (int)(src_end - src_begin);
+  const float* X = nullptr;
+  int xbuf = -1;
+  { int rc = stage_chunk(c, features, nullptr, src_begin, src_end, K, st, &X, &xbuf); if (rc) return rc; }
+  if (project_tc_usable(c, l, X, K)) {
+    int rc = launch_project_tc(c, l, X, K, src_begin, n, st);
+    if (rc) return rc;
+  } else {
+    launch_project_simt(c, l, X, K, src_begin, n, st);
+  }
+  if (xbuf >= 0) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }
+  launch_gat_split(c, n, Hp, d_out, src_begin, hprime_out, ld, st);
+  CU(cudaGetLastError());
+  c->gat_next_src = src_end;
+  return TAURUS_OK;
+}
+
+extern "C" int taurus_gat_attention(taurus_ctx* c, void* cuda_stream) {
+  if (!c) return TAURUS_ERR_INVALID_ARG;
+  if (c->mode != TAURUS_GAT) return TAURUS_ERR_UNSUPPORTED;
+  if (c->layer < 0 || c->gat_ready || c->gat_next_src != c->V) return TAURUS_ERR_ORDER;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CU(cudaSetDevice(c->device));
+  if (st != c->last_stream) {
+    CU(cudaEventRecord(c->order_event, c->last_stream));
+    CU(cudaStreamWaitEvent(st, c->order_event, 0));
+    c->last_stream = st;
+  }
+  launch_gat_attention(c, st);
+  CU(cudaGetLastError());
+  c->gat_ready = true;
+  return TAURUS_OK;
 }
 
 extern "C" int taurus_push_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream) {

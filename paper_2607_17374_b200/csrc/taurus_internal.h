@@ -87,6 +87,11 @@ struct ChunkArgs {
   int32_t mode, act, fanout;
   int32_t evict_policy;
   float gin_self;           // GIN: 1 + eps, the weight of the self message
+  // GAT: per-vertex scalars from which every attention coefficient is recomputed
+  const float* att_s;       // [V] att_src . h'_u
+  const float2* att_tm;     // [V] (att_dst . h'_v, maximum score of v's neighbourhood)
+  const float* att_z;       // [V] softmax normaliser
+  float leaky;              // LeakyReLU slope
   unsigned long long seed;
   long long grad_off;       // dense-output mode: first row of this chunk's half of the graduation buffer
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
@@ -126,6 +131,15 @@ struct taurus_ctx {
   int32_t* d_slot_epoch = nullptr;
   int evict_policy = 0;
   float gin_eps = 0.f;
+  // GAT mode
+  float leaky = 0.2f;
+  float* d_att_s = nullptr;     // [V] att_src . h'
+  float* d_att_t = nullptr;     // [V] att_dst . h'
+  float* d_att_max = nullptr;   // [V] running maximum of att_src . h'_u over the neighbourhood
+  float2* d_att_tm = nullptr;   // [V] (t, maximum score)
+  float* d_att_z = nullptr;     // [V] normaliser
+  long long gat_next_src = 0;   // next source taurus_gat_project_chunk expects
+  bool gat_ready = false;       // taurus_gat_attention has run for this layer
   int32_t* d_free_stack = nullptr;
   int32_t* d_need_list = nullptr;
   int32_t* d_touched_list = nullptr;
@@ -183,6 +197,8 @@ struct taurus_ctx {
 };
 
 static inline int taurus_round_up(int x, int m) { return (x + m - 1) / m * m; }
+// Columns of the projection output: [P | T] for SAGE, [h' | att_src.h' att_dst.h' 0 0] for GAT, P otherwise.
+static inline int taurus_proj_width(int mode, int Hp) { return mode == TAURUS_SAGE_MEAN ? 2 * Hp : mode == TAURUS_GAT ? Hp + 4 : Hp; }
 
 // ---- kernels_state.cu
 void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st);
@@ -210,6 +226,10 @@ int runs_flush_all(taurus_runs* r, cudaStream_t st);
 int runs_read_into(taurus_runs* r, long long s, long long e, float* out, long long ld, cudaStream_t st);
 // ---- taurus_host.cu
 void taurus_note_cuda_error(cudaError_t e, const char* what);   // keeps the text for taurus_last_cuda_error
+// ---- kernels_gat.cu
+void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st);
+void launch_gat_attention(taurus_ctx* c, cudaStream_t st);
+void launch_gat_repack(taurus_ctx* c, const float* X, int n, int d_out, int Hp, cudaStream_t st);   // X [n x d_out] -> d_PT [n x Hp]
 // ---- kernels_scatter.cu
 void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_gemm_simt.cu

@@ -75,6 +75,7 @@ def hash64(seed: int, tag: int, i: int, j: int) -> int:
 SAGE_MEAN = 0
 GCN_SYM = 1
 GIN_SUM = 2
+GAT = 3
 GEMM_FP32 = 0
 GEMM_BF16 = 1
 
@@ -92,7 +93,7 @@ class Workload:
     top_in: int                 # target for the largest in-degree (mode 1)
     symmetric: bool
     dims: Tuple[int, ...]       # F, hidden..., out
-    mode: int                   # SAGE_MEAN, GCN_SYM or GIN_SUM
+    mode: int                   # SAGE_MEAN, GCN_SYM, GIN_SUM or GAT
     chunk: int                  # sources per pushed chunk
     pool_slots: int             # accumulator slot pool capacity
     hub_count: int              # vertices pinned in the GPU-resident store
@@ -100,6 +101,7 @@ class Workload:
     gemm_mode: int = GEMM_FP32
     seed: int = 1
     gin_eps: float = 0.0        # GIN_SUM only: the self weight is 1 + gin_eps
+    leaky_slope: float = 0.2    # GAT only: negative slope of the LeakyReLU on the attention scores
 
     @property
     def L(self) -> int:
@@ -235,6 +237,8 @@ class Model:
     W_self: list
     bias: list
     act: Tuple[int, ...]
+    att_src: Optional[list] = None   # GAT only: per layer, dims[l+1] floats
+    att_dst: Optional[list] = None
 
 
 def make_model(w: Workload, bias_scale: float = 0.0) -> Model:
@@ -247,4 +251,8 @@ def make_model(w: Workload, bias_scale: float = 0.0) -> Model:
             b.append((weights(w.seed, l, 2, 1, w.dims[l + 1])[0] * bias_scale).astype(np.float32))
         else:
             b.append(np.zeros(w.dims[l + 1], dtype=np.float32))
-    return Model(w.mode, w.dims, Wn, Ws, b, w.act)
+    att_s = att_d = None
+    if w.mode == GAT:      # attention vectors drawn like weight columns (which = 3 and 4)
+        att_s = [weights(w.seed, l, 3, w.dims[l + 1], 1)[:, 0].copy() for l in range(w.L)]
+        att_d = [weights(w.seed, l, 4, w.dims[l + 1], 1)[:, 0].copy() for l in range(w.L)]
+    return Model(w.mode, w.dims, Wn, Ws, b, w.act, att_s, att_d)

@@ -21,7 +21,8 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
         0 if w.pool_slots >= V - w.hub_count else V - w.hub_count)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
-                     drain_rows or (2 * V if (dense_output or run_output) else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy, w.gin_eps)
+                     drain_rows or (2 * V if (dense_output or run_output) else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy, w.gin_eps,
+                     model.att_src, model.att_dst, w.leaky_slope)
     res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
     if host_features:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
@@ -44,6 +45,12 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
             res["masks"].append(None)
         per_chunk = []
         plan = chunk_plan or [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
+        if w.mode == tg.GAT:  # passes 1 and 2; pass 3 below streams the transformed rows instead of the features
+            hprime = torch.empty((V, d_out), dtype=torch.float32, device=dev)
+            for (s, e) in plan:
+                ctx.gat_project_chunk(s, e, feat[s:e], hprime[s:e], d_out, stream)
+            ctx.gat_attention(stream)
+            layer_in, feat = feat, (hprime.cpu().pin_memory() if host_features else hprime)
         if run_output:        # rows leave as sorted runs; layers after the first read their input back from runs
             P, R, kind = run_output
             runs = tb.Runs(V, d_out, P, R, store_rows=V, max_append_rows=V, max_chunk_rows=w.chunk, store_kind=kind)
@@ -99,8 +106,13 @@ def run_oracle(w, g, model, x0, evict_policy=0):
     out = dict(outs=[], sims=[], msets=[], hub=hub)
     for l in range(w.L):
         ms = oracle.message_sets(inl, w.fanout[l], w.seed, l)
-        h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l],
-                                 gin_eps=w.gin_eps)
+        if w.mode == tg.GAT:
+            from oracle import gat
+            h = gat.gat_layer_forward(ms, h, model.W_neigh[l], model.att_src[l], model.att_dst[l], model.bias[l], model.act[l],
+                                      w.leaky_slope)
+        else:
+            h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l],
+                                     gin_eps=w.gin_eps)
         out["outs"].append(h)
         out["sims"].append(oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, w.pool_slots, evict_policy, w.seed))
         out["msets"].append(ms)
