@@ -220,11 +220,12 @@ int taurus_drain_dense(taurus_ctx* ctx, float* dense_rows, int64_t ld, int64_t* 
  * off-loading overlap; Sect. 3.7 keeps outputs in vertex order for the next layer).  Call after
  * taurus_layer_begin and before the first push.  Every finalised row is then written to
  * dense_rows[id * ld ...] (ld in floats, >= dims[layer+1]; device memory or pinned host memory) by the
- * library itself: the graduation buffer is split in two halves, the rows of chunk k leave one half on an
- * internal stream while chunk k+1 computes into the other, and the caller never drains (taurus_drain_*
- * report zero rows).  A chunk whose completion bound exceeds drain_rows / 2 is refused with
- * TAURUS_ERR_DRAIN_FULL (create the context with a larger drain_rows).  taurus_layer_end waits until
- * every row has arrived.  The mode ends with the layer.
+ * library itself and the caller never drains (taurus_drain_* report zero rows).  Device memory: the
+ * finalise kernel writes each row straight to its place; a chunk whose completion bound exceeds drain_rows
+ * is refused with TAURUS_ERR_DRAIN_FULL.  Pinned host memory: the graduation buffer is split in two halves,
+ * the rows of chunk k leave one half on an internal stream while chunk k+1 computes into the other, and the
+ * refusal threshold is drain_rows / 2 (create the context with a larger drain_rows).  taurus_layer_end waits
+ * until every row has arrived.  The mode ends with the layer.
  */
 int taurus_layer_set_dense_output(taurus_ctx* ctx, float* dense_rows, int64_t ld);
 

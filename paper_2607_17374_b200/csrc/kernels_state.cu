@@ -426,7 +426,7 @@ __global__ void finalise_kernel(ChunkArgs a) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    if (base + i >= limit) {
+    if (!a.dense_direct && base + i >= limit) {
       if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
       continue;
     }
@@ -444,6 +444,26 @@ __global__ void finalise_kernel(ChunkArgs a) {
       scale = 1.0f;   // GIN: plain sum
     }
     const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
+    if (a.dense_direct) {   // the caller's vertex-ordered matrix is device memory: no detour through the graduation buffer
+      float* drow = a.dense_direct + (size_t)v * a.dense_ld;
+      const bool vec_ok = (a.dense_ld & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dense_direct) & 15) == 0;
+      for (int k = lane_id(); k < vec; k += 32) {
+        float4 x = src[k];
+        x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
+        if (a.act) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
+        const int c0 = k << 2;
+        if (vec_ok && c0 + 3 < a.d_out) {
+          reinterpret_cast<float4*>(drow)[k] = x;
+        } else {
+          if (c0 < a.d_out) drow[c0] = x.x;
+          if (c0 + 1 < a.d_out) drow[c0 + 1] = x.y;
+          if (c0 + 2 < a.d_out) drow[c0 + 2] = x.z;
+          if (c0 + 3 < a.d_out) drow[c0 + 3] = x.w;
+        }
+      }
+      if (lane_id() == 0) a.state[v] = TAURUS_COMPLETED;
+      continue;
+    }
     float4* dst = reinterpret_cast<float4*>(a.grad_rows + (size_t)(base + i) * a.Hp);
     for (int k = lane_id(); k < vec; k += 32) {
       float4 x = src[k];
@@ -473,7 +493,9 @@ __global__ void commit_kernel(ChunkArgs a) {
   ctl->evictions += ctl->deficit;
   ctl->reloads += ctl->reloaded;
   ctl->completed += ctl->done_count;
-  if (a.dense_half >= 0) ctl->out_count[a.dense_half] = ctl->done_count; else ctl->grad_count += ctl->done_count;
+  if (a.dense_direct) { /* rows already sit in the caller's matrix */ }
+  else if (a.dense_half >= 0) ctl->out_count[a.dense_half] = ctl->done_count;
+  else ctl->grad_count += ctl->done_count;
   ctl->chunks = c + 1;
   ctl->hs = ctl->ns = ctl->ev = ctl->gs = 0;
   ctl->need_count = 0; ctl->done_count = 0; ctl->touched_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;

@@ -361,7 +361,11 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.evict_policy = c->evict_policy; a.seed = c->seed;
   a.gin_self = 1.0f + c->gin_eps;
   a.direct = c->pool_slots >= c->V ? 1 : 0;
-  const bool halves = c->dense_out || c->run_out;   // the graduation buffer alternates between two halves
+  const bool direct_dense = c->dense_out && c->dense_is_device;
+  const bool halves = (c->dense_out && !direct_dense) || c->run_out;   // the graduation buffer alternates between two halves
+  a.dense_direct = direct_dense ? c->dense_out : nullptr;
+  a.dense_ld = c->dense_ld;
+  a.d_out = c->dims[l + 1];
   a.dense_half = halves ? (int)(c->chunk_seq & 1) : -1;
   a.grad_cap = halves ? c->drain_rows / 2 : c->drain_rows;
   a.grad_off = halves ? (long long)a.dense_half * (c->drain_rows / 2) : 0;
@@ -419,8 +423,9 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
     return TAURUS_ERR_INVALID_ARG;
   if (c->h_ctl->error) return c->h_ctl->error;
   const long long bound = completion_bound(c, src_begin, src_end);
-  const bool halves = c->dense_out || c->run_out;
-  if (halves ? bound > c->drain_rows / 2 : c->ub_since_drain + bound > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
+  const bool direct_dense = c->dense_out && c->dense_is_device;   // rows are finalised straight into the caller's matrix
+  const bool halves = (c->dense_out && !direct_dense) || c->run_out;
+  if (halves ? bound > c->drain_rows / 2 : (direct_dense ? bound : c->ub_since_drain + bound) > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(cudaSetDevice(c->device));
   if (st != c->last_stream) {   // keep chunk order across streams
@@ -474,7 +479,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
   launch_finalise(c, a, st);
   int run_rc = TAURUS_OK;
-  if (a.dense_half >= 0 && c->dense_out) {   // hand this chunk's rows to the output stream
+  if (a.dense_half >= 0 && c->dense_out) {   // hand this chunk's rows to the output stream (matrix in pinned host memory)
     const int h = a.dense_half, d_out = c->dims[l + 1];
     CU(cudaEventRecord(c->fin_done[h], st));
     CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
@@ -501,7 +506,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   CU(cudaGetLastError());
   c->next_src = src_end;
   c->chunk_seq += 1;
-  if (!halves) c->ub_since_drain += bound;
+  if (!halves && !direct_dense) c->ub_since_drain += bound;
   return run_rc;
 }
 
@@ -645,6 +650,7 @@ extern "C" int taurus_layer_set_dense_output(taurus_ctx* c, float* dense_rows, i
     return TAURUS_ERR_INVALID_ARG;
   c->dense_out = dev;
   c->dense_ld = ld;
+  c->dense_is_device = kind == PK_DEVICE;
   return TAURUS_OK;
 }
 

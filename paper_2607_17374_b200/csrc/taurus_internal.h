@@ -97,6 +97,9 @@ struct ChunkArgs {
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
   int32_t dense_half;       // -1: graduation buffer drained by the caller; 0 / 1: half used by this chunk
   int32_t direct;           // pool_slots >= V: vertex v owns slot v, no free stack, no eviction
+  float* dense_direct;      // dense-output mode with the matrix in device memory: finalise writes row v at dense_direct + v * dense_ld
+  long long dense_ld;
+  int32_t d_out;            // unpadded output width
 };
 
 struct taurus_ctx {
@@ -160,6 +163,7 @@ struct taurus_ctx {
   // dense-output mode (taurus_layer_set_dense_output)
   float* dense_out = nullptr;           // device-visible address of the caller's matrix, NULL = mode off
   long long dense_ld = 0;
+  bool dense_is_device = false;         // the matrix is device memory: rows are finalised straight into it (no graduation halves)
   struct taurus_runs* run_out = nullptr;  // run-output mode (taurus_layer_set_run_output), NULL = mode off
   int run_pending_half = -1;            // half whose rows are grouped but not yet moved to the partition buffers
   cudaStream_t out_stream = nullptr;    // rows leave the graduation buffer here while the next chunk computes
