@@ -207,7 +207,7 @@ void launch_classify_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st)
 // With GAT every message is weighted by exp(LeakyReLU(s_u + t_v) - max_v), recomputed from per-vertex scalars
 // (the 1 / normaliser factor is applied at finalise).
 template <int LPE, int VPL, bool SAMPLED, bool DIRECT, bool GAT>
-__global__ void __launch_bounds__(256, (VPL <= 2 ? 3 : 1))
+__global__ void __launch_bounds__(256, (VPL <= 2 ? 3 : VPL == 3 ? 2 : 1))
 scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
@@ -409,6 +409,7 @@ void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) 
   const int Hp = a.Hp;
   if (Hp <= 16) launch_sg2<4, 1>(c, a, st);
   else if (Hp <= 32) launch_sg2<8, 1>(c, a, st);
+  else if (Hp <= 48) launch_sg2<4, 3>(c, a, st);     // 12 float4: four lanes x three, no idle lanes
   else if (Hp <= 64) launch_sg2<16, 1>(c, a, st);
   else if (Hp <= 128) launch_sg2<32, 1>(c, a, st);
   else if (Hp <= 256) launch_sg2<32, 2>(c, a, st);
