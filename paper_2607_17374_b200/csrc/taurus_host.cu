@@ -198,7 +198,8 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     ALLOC(c->d_touched_list, c->touched_capacity);
   }
   ALLOC(c->d_owner, c->pool_slots); ALLOC(c->d_free_stack, c->pool_slots); ALLOC(c->d_need_list, c->pool_slots);
-  if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); ALLOC(c->d_slot_epoch, c->pool_slots); }
+  ALLOC(c->d_slot_epoch, c->pool_slots);   // written at every slot hand-out, also when no eviction can happen
+  if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); }
   ALLOC(c->d_host_free, c->host_rows);
   if (c->host_rows > 0) {
     cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->host_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
