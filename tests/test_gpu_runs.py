@@ -238,3 +238,53 @@ def test_run_output_argument_checks():
     st = ctx.layer_end()
     assert st["completed"] == g.V and out.info()["stored_rows"] == g.V
     ctx.destroy()
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_writer_reader_configurations(seed):
+    """Random V / ranges / buffer sizes / widths / append sizes (more ranges than vertices, one-row buffers, wide
+    rows, partial layers) against the oracle's writer and reader."""
+    import torch
+    import paper_2607_17374_b200 as tb
+    dev = torch.device("cuda:0")
+    rng = np.random.default_rng(500 + seed)
+    V = int(rng.choice([1, 2, 17, 300, 1000, 4097, 20000]))
+    P = int(rng.choice([1, 2, 3, 16, 100, 1024]))
+    R = int(rng.choice([1, 2, 7, 64, 1000, 50000]))
+    if V // max(1, min(P, V)) > 400 * R:          # keep the number of runs (each a few launches) bounded
+        R = max(R, V // (400 * P) + 1)
+    width = int(rng.choice([1, 3, 4, 12, 64, 257, 1024])) if V <= 4097 else int(rng.choice([1, 4, 12, 64]))
+    ld = width + int(rng.choice([0, 0, 1, 4]))
+    kind = tb.RUNS_HOST if rng.integers(0, 2) else tb.RUNS_DEVICE
+    present = rng.permutation(V)[:max(1, int(V * rng.choice([1.0, 1.0, 0.6])))].astype(np.int64)   # sometimes a partial layer
+    runs = tb.Runs(V, width, P, R, store_kind=kind)
+    w = rs.RunWriter(V, P, R, width)
+    at = 0
+    while at < present.size:
+        n = int(min(present.size - at, rng.choice([1, 3, 50, 1000, V])))
+        ids = present[at:at + n]
+        rows = np.full((n, ld), -3.0, np.float32)
+        rows[:, :width] = rows_for(ids, width)
+        w.append(ids, rows[:, :width])
+        runs.append(torch.from_numpy(ids).to(dev), torch.from_numpy(rows).to(dev), ld, n)
+        at += n
+    runs.flush(); w.flush()
+    assert runs.info() == {"runs": len(w.runs), "stored_rows": int(present.size), "buffered_rows": 0}
+    compare_with_oracle(runs, w, width)
+    have = np.zeros(V, bool)
+    have[present] = True
+    chunk = int(rng.choice([1, 5, 64, 1000, V]))
+    chunk = max(chunk, V // 200 + 1)
+    for s in range(0, V, chunk):
+        e = min(V, s + chunk)
+        out = torch.full((e - s, width), -1.0, device=dev)
+        if have[s:e].all():
+            runs.read_chunk(s, e, out, width)
+            ref_ids, ref_rows = rs.read_chunk(w.runs, s, e, width)
+            assert ref_ids.tolist() == list(range(s, e)) and np.array_equal(out.cpu().numpy(), ref_rows)
+        else:
+            with pytest.raises(tb.TaurusError) as ei:
+                runs.read_chunk(s, e, out, width)
+            assert ei.value.code == tb.ERROR_CODES["RUNS_INCOMPLETE"]
+            assert (out == -1.0).all()
+    runs.destroy()
