@@ -415,8 +415,10 @@ __global__ void compact_done_kernel(ChunkArgs a) {
   if (__any_sync(FULL, bad) && lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
 }
 
-// One warp per completed vertex (listed by compact_done_kernel):
-// out = act(c_in(v) * acc) into the graduation buffer (Sect. 3.6); the slot is released.
+// Completed vertices (listed by compact_done_kernel) in batches of 32 per warp: each lane first fetches the
+// vertex, its slot and its normalisation of one row of the batch (one dependent chain for 32 rows), then the
+// warp walks the batch row by row: out = act(c_in(v) * acc) into the graduation buffer, or straight into the
+// caller's vertex-ordered matrix (Sect. 3.6); the slot is released by compact_done_kernel.
 __global__ void finalise_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
@@ -425,55 +427,65 @@ __global__ void finalise_kernel(ChunkArgs a) {
   const long long limit = a.dense_half >= 0 ? a.grad_off + a.grad_cap : a.drain_rows;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
-  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    if (!a.dense_direct && base + i >= limit) {
-      if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
-      continue;
+  const bool vec_ok = a.dense_direct && (a.dense_ld & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dense_direct) & 15) == 0;
+  // rows per warp batch: as many as keep every warp busy, at most one per lane
+  int per = (int)((n + warps - 1) / warps);
+  per = per < 1 ? 1 : per > 32 ? 32 : per;
+  for (long long i0 = (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * per; i0 < n; i0 += warps * per) {
+    const long long mine = i0 + lane_id();
+    int v = -1, l = 0;
+    float scale = 1.0f;
+    if (lane_id() < per && mine < n) {
+      if (!a.dense_direct && base + mine >= limit) {
+        atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+      } else {
+        v = a.done_list[mine];
+        l = a.loc[v];
+        if (a.mode == TAURUS_SAGE_MEAN) {
+          int m = messages_of(a.din[v], a.fanout);
+          scale = 1.0f / (float)(m > 1 ? m : 1);
+        } else if (a.mode == TAURUS_GCN_SYM) {
+          scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+        } else if (a.mode == TAURUS_GAT) {
+          scale = 1.0f / a.att_z[v];   // softmax normaliser
+        }                              // GIN: plain sum
+        a.state[v] = TAURUS_COMPLETED;
+        if (!a.dense_direct) a.grad_ids[base + mine] = v;
+      }
     }
-    int v = a.done_list[i];
-    int l = a.loc[v];
-    float scale;
-    if (a.mode == TAURUS_SAGE_MEAN) {
-      int m = messages_of(a.din[v], a.fanout);
-      scale = 1.0f / (float)(m > 1 ? m : 1);
-    } else if (a.mode == TAURUS_GCN_SYM) {
-      scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
-    } else if (a.mode == TAURUS_GAT) {
-      scale = 1.0f / a.att_z[v];   // softmax normaliser
-    } else {
-      scale = 1.0f;   // GIN: plain sum
-    }
-    const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
-    if (a.dense_direct) {   // the caller's vertex-ordered matrix is device memory: no detour through the graduation buffer
-      float* drow = a.dense_direct + (size_t)v * a.dense_ld;
-      const bool vec_ok = (a.dense_ld & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dense_direct) & 15) == 0;
-      for (int k = lane_id(); k < vec; k += 32) {
-        float4 x = src[k];
-        x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
-        if (a.act) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
-        const int c0 = k << 2;
-        if (vec_ok && c0 + 3 < a.d_out) {
-          reinterpret_cast<float4*>(drow)[k] = x;
-        } else {
-          if (c0 < a.d_out) drow[c0] = x.x;
-          if (c0 + 1 < a.d_out) drow[c0 + 1] = x.y;
-          if (c0 + 2 < a.d_out) drow[c0 + 2] = x.z;
-          if (c0 + 3 < a.d_out) drow[c0 + 3] = x.w;
+    const int rows = n - i0 < per ? (int)(n - i0) : per;
+    for (int j = 0; j < rows; ++j) {
+      const int vj = __shfl_sync(FULL, v, j);
+      if (vj < 0) continue;
+      const int lj = __shfl_sync(FULL, l, j);
+      const float sj = __shfl_sync(FULL, scale, j);
+      const float4* __restrict__ src = reinterpret_cast<const float4*>(a.acc + (size_t)lj * a.Hp);
+      float* __restrict__ drow = a.dense_direct ? a.dense_direct + (size_t)vj * a.dense_ld : a.grad_rows + (size_t)(base + i0 + j) * a.Hp;
+      for (int k0 = 0; k0 < vec; k0 += 128) {   // up to four float4 per lane in flight before the first store
+        float4 x[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int k = k0 + q * 32 + lane_id();
+          if (k < vec) x[q] = src[k];
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int k = k0 + q * 32 + lane_id();
+          if (k >= vec) continue;
+          float4 y = x[q];
+          y.x *= sj; y.y *= sj; y.z *= sj; y.w *= sj;
+          if (a.act) { y.x = fmaxf(y.x, 0.f); y.y = fmaxf(y.y, 0.f); y.z = fmaxf(y.z, 0.f); y.w = fmaxf(y.w, 0.f); }
+          const int c0 = k << 2;
+          if (!a.dense_direct || (vec_ok && c0 + 3 < a.d_out)) {
+            reinterpret_cast<float4*>(drow)[k] = y;
+          } else {   // ragged last columns, or a matrix whose rows are not 16-byte aligned
+            if (c0 < a.d_out) drow[c0] = y.x;
+            if (c0 + 1 < a.d_out) drow[c0 + 1] = y.y;
+            if (c0 + 2 < a.d_out) drow[c0 + 2] = y.z;
+            if (c0 + 3 < a.d_out) drow[c0 + 3] = y.w;
+          }
         }
       }
-      if (lane_id() == 0) a.state[v] = TAURUS_COMPLETED;
-      continue;
-    }
-    float4* dst = reinterpret_cast<float4*>(a.grad_rows + (size_t)(base + i) * a.Hp);
-    for (int k = lane_id(); k < vec; k += 32) {
-      float4 x = src[k];
-      x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
-      if (a.act) { x.x = fmaxf(x.x, 0.f); x.y = fmaxf(x.y, 0.f); x.z = fmaxf(x.z, 0.f); x.w = fmaxf(x.w, 0.f); }
-      dst[k] = x;
-    }
-    if (lane_id() == 0) {
-      a.grad_ids[base + i] = v;
-      a.state[v] = TAURUS_COMPLETED;
     }
   }
 }
