@@ -45,6 +45,11 @@ def parse_args():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--simt-gemm", action="store_true", help="use the plain FFMA projection kernel")
     p.add_argument("--no-grouping", action="store_true", help="CSR-order scatter for every chunk")
+    p.add_argument("--model", default="", choices=["", "sage", "gcn", "gin", "gat"],
+                   help="aggregation of every layer (default: the workload's); gat runs its three passes per layer")
+    p.add_argument("--output", default="dense", choices=["dense", "runs-device", "runs-host"],
+                   help="where a layer's rows go: a dense matrix in HBM (default), or sorted runs (in HBM / pinned host "
+                        "memory) that the next layer reads back by merge-on-read")
     return p.parse_args()
 
 
@@ -52,6 +57,10 @@ def workload_of(args):
     w = tg.WORKLOADS[args.workload]
     if args.vertices:
         w = tg.scaled(w, args.vertices)
+    if args.model:
+        from dataclasses import replace
+        w = replace(w, mode={"sage": tg.SAGE_MEAN, "gcn": tg.GCN_SYM, "gin": tg.GIN_SUM, "gat": tg.GAT}[args.model],
+                    gemm_mode=tg.GEMM_FP32 if args.model == "gat" else w.gemm_mode)
     return w
 
 
@@ -226,7 +235,18 @@ def run_ours(args):
     host_evict = 0 if w.pool_slots >= V - w.hub_count else V - w.hub_count
     flags = (tb.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (tb.FLAG_NO_GROUPING if args.no_grouping else 0)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
-                     model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags)
+                     model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags,
+                     0, w.gin_eps, model.att_src, model.att_dst, w.leaky_slope)
+    gat = w.mode == tg.GAT
+    use_runs = args.output != "dense"
+    if gat and use_runs:
+        raise SystemExit("--model gat reads its features through pointers: use --output dense")
+    hprime = torch.zeros((V, max(w.dims[1:])), dtype=torch.float32, device=dev) if gat else None
+    runs = None
+    if use_runs:   # one run store per layer output: 16 id ranges, buffers of 32 768 rows
+        kind = tb.RUNS_DEVICE if args.output == "runs-device" else tb.RUNS_HOST
+        runs = [tb.Runs(V, w.dims[l + 1], 16, 32768, store_rows=V, max_append_rows=max(V, w.chunk), max_chunk_rows=w.chunk,
+                        store_kind=kind) for l in range(L)]
     x_host = torch.empty((V, w.dims[0]), dtype=torch.float32).pin_memory()
     tg.features(w.seed, 0, 0, V, w.dims[0], out=x_host.numpy())
     x_dev = x_host.to(dev)
@@ -246,14 +266,33 @@ def run_ours(args):
             d_out = w.dims[l + 1]
             out = final_out if l == L - 1 else dense_dev[l % 2][:V * d_out].view(V, d_out)
             ctx.layer_begin(l, stream)
-            ctx.layer_set_dense_output(out, d_out)   # finalised rows are placed by the library while the next chunk runs
-            for (s, e) in chunks:
-                ctx.push_chunk(s, e, feat[s:e], stream)
+            src = feat
+            if gat:    # passes 1 and 2: transformed rows and attention scalars, then the topology-only sweep
+                hp = hprime.view(-1)[:V * d_out].view(V, d_out)
+                for (s, e) in chunks:
+                    ctx.gat_project_chunk(s, e, feat[s:e], hp[s:e], d_out, stream)
+                ctx.gat_attention(stream)
+                src = hp
+            if use_runs:
+                runs[l].reset()
+                ctx.layer_set_run_output(runs[l])
+                for (s, e) in chunks:
+                    if l == 0:
+                        ctx.push_chunk(s, e, src[s:e], stream)
+                    else:
+                        ctx.push_chunk_from_runs(s, e, runs[l - 1], stream)
+            else:
+                ctx.layer_set_dense_output(out, d_out)   # finalised rows go straight to their place in the matrix
+                for (s, e) in chunks:
+                    ctx.push_chunk(s, e, src[s:e], stream)
             st = ctx.layer_end()
             if collect_stats:
                 edges_per_layer.append(st["total_messages"])
                 groups_per_layer.append(st["scatter_groups"])
             feat = out
+        if use_runs:   # the result is read back from the last layer's runs in vertex order
+            for (s, e) in chunks:
+                runs[L - 1].read_chunk(s, e, final_out[s:e], w.dims[-1], stream)
         return feat
 
     # warm-up (also collects the per-layer message counts)
@@ -349,7 +388,7 @@ def run_ours(args):
         del out_host
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not gat:
         v, info, _ = oracle_sample(w, g, 12.0)
         cpu = dict(value=v / 1e9, unit="GTEPS", **info)
 
@@ -359,12 +398,15 @@ def run_ours(args):
                     vs_baseline=None, dtype="f32", data="synthetic",
                     config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=w.chunk, chunks_per_layer=len(chunks),
                                 pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
-                                mode="sage_mean" if w.mode == 0 else "gcn_sym", messages_per_step=msgs_per_step,
+                                mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], output=args.output,
+                                messages_per_step=msgs_per_step,
                                 l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
                                 parallelism="replicas only" if world > 1 else "1 gpu",
                                 layer_ms=[float(ph[:, l].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
                     clocks=sampler.summary(), roofline=roofline, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
         print(json.dumps(line))
+    for r in runs or []:
+        r.destroy()
     ctx.destroy()
     if world > 1:
         dist.destroy_process_group()
