@@ -6,9 +6,9 @@
 // counts go to pinned host memory.  Phase 2 (host plans, device moves): with the counts known the host cuts
 // each range's rows into what still fits its partition buffer, what fills the next buffer load, and so on;
 // each pass moves one such piece per range (one launch for all ranges) and then sorts and flushes the
-// buffers that are full: radix sort of the buffered ids with the buffer positions as payload, then one gather
-// that writes ids and rows of the run sequentially into the run store (directly over PCIe when the store is
-// pinned host memory).  Because the grouping sort is stable, run k of a range holds that range's arrivals
+// buffers that are full: their ids are collected, radix-sorted together with the buffer positions as payload
+// (the ranges are contiguous in id, so one sort leaves them range after range), and one gather writes ids and
+// rows of the runs sequentially into the run store (directly over PCIe when the store is pinned host memory).  Because the grouping sort is stable, run k of a range holds that range's arrivals
 // k R .. (k + 1) R - 1 whatever the other ranges did.
 //
 // Reader.  The ids of all runs live in pinned host memory; for a chunk [s, e) the host bisects each
@@ -83,12 +83,19 @@ __global__ void rs_move_kernel(const MoveSeg* __restrict__ segs, const int32_t* 
   }
 }
 
-__global__ void rs_iota_kernel(long long n, int32_t* out) {
+// Buffers that leave together: ids of piece q go to fkeys[dst ..], their partition-buffer row numbers to fvals[dst ..].
+__global__ void rs_collect_kernel(const MoveSeg* __restrict__ segs, const int32_t* __restrict__ pids, int32_t* __restrict__ fkeys,
+                                  int32_t* __restrict__ fvals) {
+  const MoveSeg sg = segs[blockIdx.y];
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) out[i] = (int32_t)i;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < sg.n; i += stride) {
+    fkeys[sg.dst + i] = pids[sg.src + i];
+    fvals[sg.dst + i] = (int32_t)(sg.src + i);
+  }
 }
 
-// Writes one sorted run: ids and rows in id order, sequentially, into the store.
+// Writes sorted runs: ids and rows in id order, sequentially, into the store (the id ranges are contiguous, so
+// buffers sorted together come out range after range).
 __global__ void rs_gather_kernel(long long n, const int32_t* __restrict__ sid, const int32_t* __restrict__ sidx,
                                  const float* __restrict__ prows, int width, int32_t* __restrict__ run_ids,
                                  float* __restrict__ run_rows) {
@@ -105,6 +112,16 @@ __global__ void rs_place_kernel(long long n, const int32_t* __restrict__ sid, co
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps)
     copy_row(out + (size_t)(sid[i] - s) * ld, srows + (size_t)i * width, width);
+}
+
+// The same for a store in device memory: slice q of the chunk (rows src .. src + n of the store, their ids staged
+// at dst ..) is read in place, without a staging copy of the rows.
+__global__ void rs_place_slices_kernel(const MoveSeg* __restrict__ segs, const int32_t* __restrict__ sid, const float* __restrict__ store,
+                                       int width, long long s, float* __restrict__ out, long long ld) {
+  const MoveSeg sg = segs[blockIdx.y];
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < sg.n; i += warps)
+    copy_row(out + (size_t)(sid[sg.dst + i] - s) * ld, store + (size_t)(sg.src + i) * width, width);
 }
 
 int bits_for(long long values) {   // bits needed to tell `values` different keys apart
@@ -140,7 +157,8 @@ struct taurus_runs {
   bool seg_used[SEG_RING] = {false};
   long long seg_seq = 0;
   // flush scratch
-  int32_t *d_iota = nullptr, *d_sid = nullptr, *d_sidx = nullptr;
+  int32_t *d_fkeys = nullptr, *d_fvals = nullptr, *d_sid = nullptr, *d_sidx = nullptr;   // [flush_cap]
+  long long flush_cap = 0;       // most rows sorted in one go
   void* d_tmp = nullptr;
   size_t tmp_bytes = 0;
   // read staging
@@ -186,7 +204,7 @@ extern "C" void taurus_runs_destroy(taurus_runs* r) {
   if (r->kind == TAURUS_RUNS_HOST) cudaFreeHost(r->store_host); else cudaFree(r->store_dev);
   cudaFreeHost(r->h_ids); cudaFreeHost(r->h_cnt); cudaFreeHost(r->h_segs);
   cudaFree(r->d_key); cudaFree(r->d_key_s); cudaFree(r->d_idx); cudaFree(r->d_idx_s); cudaFree(r->d_cnt); cudaFree(r->d_segs);
-  cudaFree(r->d_iota); cudaFree(r->d_sid); cudaFree(r->d_sidx); cudaFree(r->d_tmp);
+  cudaFree(r->d_fkeys); cudaFree(r->d_fvals); cudaFree(r->d_sid); cudaFree(r->d_sidx); cudaFree(r->d_tmp);
   cudaFree(r->d_stage_rows); cudaFree(r->d_stage_ids);
   for (int i = 0; i < SEG_RING; ++i) if (r->seg_done[i]) cudaEventDestroy(r->seg_done[i]);
   if (r->cnt_ready) cudaEventDestroy(r->cnt_ready);
@@ -202,6 +220,7 @@ extern "C" int taurus_runs_create(taurus_runs** out, const taurus_runs_config* c
   if (cfg->V < 1 || cfg->V >= (1ll << 31) || cfg->width < 1 || cfg->width > TAURUS_MAX_DIM || cfg->partitions < 1 ||
       cfg->partitions > 1024 || cfg->partition_rows < 1 || cfg->partition_rows >= (1ll << 31) || cfg->store_rows < 1 ||
       cfg->max_append_rows < 1 || cfg->max_append_rows >= (1ll << 31) || cfg->max_chunk_rows < 1 ||
+      cfg->partitions * cfg->partition_rows >= (1ll << 31) ||
       (cfg->store_kind != TAURUS_RUNS_HOST && cfg->store_kind != TAURUS_RUNS_DEVICE))
     return TAURUS_ERR_INVALID_ARG;
   taurus_runs* r = new (std::nothrow) taurus_runs();
@@ -231,10 +250,11 @@ extern "C" int taurus_runs_create(taurus_runs** out, const taurus_runs_config* c
   RPINNED(r->h_cnt, (size_t)r->P + 2);
   RALLOC(r->d_segs, (size_t)SEG_RING * r->P);
   RPINNED(r->h_segs, (size_t)SEG_RING * r->P);
-  RALLOC(r->d_iota, r->R); RALLOC(r->d_sid, r->R); RALLOC(r->d_sidx, r->R);
+  r->flush_cap = std::max<long long>(r->R, std::min<long long>(r->P * r->R, 1ll << 26));
+  RALLOC(r->d_fkeys, r->flush_cap); RALLOC(r->d_fvals, r->flush_cap); RALLOC(r->d_sid, r->flush_cap); RALLOC(r->d_sidx, r->flush_cap);
   size_t t1 = 0, t2 = 0;
   cub::DeviceRadixSort::SortPairs(nullptr, t1, r->d_key, r->d_key_s, r->d_idx, r->d_idx_s, (int)r->max_append, 0, r->part_bits);
-  cub::DeviceRadixSort::SortPairs(nullptr, t2, r->d_pids, r->d_sid, r->d_iota, r->d_sidx, (int)r->R, 0, r->id_bits);
+  cub::DeviceRadixSort::SortPairs(nullptr, t2, r->d_fkeys, r->d_sid, r->d_fvals, r->d_sidx, (int)r->flush_cap, 0, r->id_bits);
   r->tmp_bytes = std::max(t1, t2);
   { char* t = nullptr; RALLOC(t, r->tmp_bytes); r->d_tmp = t; }
   RALLOC(r->d_stage_rows, (size_t)r->max_chunk * w);
@@ -244,7 +264,6 @@ extern "C" int taurus_runs_create(taurus_runs** out, const taurus_runs_config* c
   if (cudaEventCreateWithFlags(&r->cnt_ready, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&r->write_done, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&r->stage_free, cudaEventDisableTiming) != cudaSuccess) { taurus_runs_destroy(r); return TAURUS_ERR_CUDA; }
-  rs_iota_kernel<<<256, 256>>>(r->R, r->d_iota);
   if (cudaDeviceSynchronize() != cudaSuccess) { taurus_note_cuda_error(cudaGetLastError(), "taurus_runs_create"); taurus_runs_destroy(r); return TAURUS_ERR_CUDA; }
   *out = r;
   return TAURUS_OK;
@@ -279,23 +298,72 @@ int runs_phase1(taurus_runs* r, const long long* ids, const float* rows, long lo
   return TAURUS_OK;
 }
 
-// Sort partition buffer p (n rows) by id and write it to the store as one run.
-static int flush_partition(taurus_runs* r, long long p, cudaStream_t st) {
-  const long long n = r->fill[(size_t)p];
-  if (n == 0) return TAURUS_OK;
-  if (r->store_top + n > r->store_rows) return TAURUS_ERR_RUN_STORE_FULL;
-  size_t tb = r->tmp_bytes;
-  RCU(cub::DeviceRadixSort::SortPairs(r->d_tmp, tb, r->d_pids + p * r->R, r->d_sid, r->d_iota, r->d_sidx, (int)n, 0, r->id_bits, st));
-  const long long off = r->store_top;
-  const int grid = (int)std::min<long long>((n * 32 + 255) / 256, (long long)r->sm_count * 8);
-  rs_gather_kernel<<<grid, 256, 0, st>>>(n, r->d_sid, r->d_sidx, r->d_prows + (size_t)p * r->R * r->width, r->width, r->d_ids + off,
-                                         r->store_dev + (size_t)off * r->width);
-  r->launches += 3;
-  r->by_part[(size_t)p].push_back((int)r->dir.size());
-  r->dir.push_back(RunRec{p, off, n});
-  r->store_top += n;
-  r->fill[(size_t)p] = 0;
-  r->dirty = true;
+// One slot of the piece-table ring, filled by the caller through *hs and uploaded by push_segs.
+static int next_seg_slot(taurus_runs* r, MoveSeg** hs, MoveSeg** ds, int* slot) {
+  *slot = (int)(r->seg_seq % SEG_RING);
+  r->seg_seq += 1;
+  if (r->seg_used[*slot]) RCU(cudaEventSynchronize(r->seg_done[*slot]));
+  *hs = r->h_segs + (size_t)*slot * r->P;
+  *ds = r->d_segs + (size_t)*slot * r->P;
+  return TAURUS_OK;
+}
+static int push_segs(taurus_runs* r, int slot, int nseg, cudaStream_t st) {
+  RCU(cudaMemcpyAsync(r->d_segs + (size_t)slot * r->P, r->h_segs + (size_t)slot * r->P, (size_t)nseg * sizeof(MoveSeg),
+                      cudaMemcpyHostToDevice, st));
+  return TAURUS_OK;
+}
+// Called after the kernel that reads the table has been launched: the slot (host and device copy) may be
+// reused once that kernel has run, on whichever stream the next user works.
+static int release_seg_slot(taurus_runs* r, int slot, cudaStream_t st) {
+  RCU(cudaEventRecord(r->seg_done[slot], st));
+  r->seg_used[slot] = true;
+  return TAURUS_OK;
+}
+
+// Sorts the listed partition buffers (ascending range numbers) by id and writes each to the store as one run.
+// Buffers are sorted together, as many per radix sort as the scratch holds: the ranges are contiguous in id,
+// so one sort by id leaves them range after range, each in id order.
+static int flush_many(taurus_runs* r, const std::vector<long long>& parts, cudaStream_t st) {
+  long long total = 0;
+  for (long long p : parts) total += r->fill[(size_t)p];
+  if (r->store_top + total > r->store_rows) return TAURUS_ERR_RUN_STORE_FULL;
+  size_t at = 0;
+  while (at < parts.size()) {
+    MoveSeg *hs, *ds;
+    int slot;
+    { int rc = next_seg_slot(r, &hs, &ds, &slot); if (rc) return rc; }
+    int nseg = 0;
+    long long m = 0, most = 0;
+    const size_t first = at;
+    while (at < parts.size()) {
+      const long long p = parts[at], n = r->fill[(size_t)p];
+      if (n == 0) { ++at; continue; }
+      if (m + n > r->flush_cap) break;   // n <= R <= flush_cap, so every batch takes at least one buffer
+      hs[nseg++] = MoveSeg{p * r->R, n, m};
+      m += n; most = std::max(most, n);
+      ++at;
+    }
+    if (m == 0) continue;
+    { int rc = push_segs(r, slot, nseg, st); if (rc) return rc; }
+    const int gx = (int)std::max<long long>(1, std::min<long long>((most + 255) / 256, std::max<long long>(1, (long long)r->sm_count * 8 / nseg)));
+    rs_collect_kernel<<<dim3(gx, nseg), 256, 0, st>>>(ds, r->d_pids, r->d_fkeys, r->d_fvals);
+    { int rc = release_seg_slot(r, slot, st); if (rc) return rc; }
+    size_t tb = r->tmp_bytes;
+    RCU(cub::DeviceRadixSort::SortPairs(r->d_tmp, tb, r->d_fkeys, r->d_sid, r->d_fvals, r->d_sidx, (int)m, 0, r->id_bits, st));
+    const long long off = r->store_top;
+    const int grid = (int)std::min<long long>((m * 32 + 255) / 256, (long long)r->sm_count * 8);
+    rs_gather_kernel<<<grid, 256, 0, st>>>(m, r->d_sid, r->d_sidx, r->d_prows, r->width, r->d_ids + off, r->store_dev + (size_t)off * r->width);
+    r->launches += 4;
+    for (size_t q = first; q < at; ++q) {
+      const long long p = parts[q], n = r->fill[(size_t)p];
+      if (n == 0) continue;
+      r->by_part[(size_t)p].push_back((int)r->dir.size());
+      r->dir.push_back(RunRec{p, r->store_top, n});
+      r->store_top += n;
+      r->fill[(size_t)p] = 0;
+    }
+    r->dirty = true;
+  }
   return TAURUS_OK;
 }
 
@@ -313,11 +381,11 @@ int runs_phase2(taurus_runs* r, cudaStream_t st) {
   std::vector<long long> src((size_t)r->P), left((size_t)r->P);
   long long acc = 0, remaining = 0;
   for (long long p = 0; p < r->P; ++p) { src[(size_t)p] = acc; left[(size_t)p] = cnt[p]; acc += cnt[p]; remaining += cnt[p]; }
+  std::vector<long long> full;
   while (remaining > 0) {
-    const int slot = (int)(r->seg_seq % SEG_RING);
-    r->seg_seq += 1;
-    if (r->seg_used[slot]) RCU(cudaEventSynchronize(r->seg_done[slot]));
-    MoveSeg* hs = r->h_segs + (size_t)slot * r->P;
+    MoveSeg *hs, *ds;
+    int slot;
+    { int rc = next_seg_slot(r, &hs, &ds, &slot); if (rc) return rc; }
     int nseg = 0;
     long long most = 0;
     for (long long p = 0; p < r->P; ++p) {
@@ -327,15 +395,15 @@ int runs_phase2(taurus_runs* r, cudaStream_t st) {
       r->fill[(size_t)p] += take; src[(size_t)p] += take; left[(size_t)p] -= take; remaining -= take;
       most = std::max(most, take);
     }
-    MoveSeg* ds = r->d_segs + (size_t)slot * r->P;
-    RCU(cudaMemcpyAsync(ds, hs, (size_t)nseg * sizeof(MoveSeg), cudaMemcpyHostToDevice, st));
-    RCU(cudaEventRecord(r->seg_done[slot], st));
-    r->seg_used[slot] = true;
+    { int rc = push_segs(r, slot, nseg, st); if (rc) return rc; }
     const int gx = (int)std::max<long long>(1, std::min<long long>((most * 32 + 255) / 256, std::max<long long>(1, (long long)r->sm_count * 8 / nseg)));
     rs_move_kernel<<<dim3(gx, nseg), 256, 0, st>>>(ds, r->d_idx_s, r->p_ids, r->p_rows, r->p_ld, r->width, r->d_pids, r->d_prows);
+    { int rc = release_seg_slot(r, slot, st); if (rc) return rc; }
     r->launches += 1;
+    full.clear();
     for (long long p = 0; p < r->P; ++p)
-      if (r->fill[(size_t)p] == r->R) { int rc = flush_partition(r, p, st); if (rc) return rc; }
+      if (r->fill[(size_t)p] == r->R) full.push_back(p);
+    if (!full.empty()) { int rc = flush_many(r, full, st); if (rc) return rc; }
   }
   RCU(cudaGetLastError());
   RCU(cudaEventRecord(r->write_done, st));
@@ -348,7 +416,10 @@ int runs_flush_all(taurus_runs* r, cudaStream_t st) {
   long long total = 0;
   for (long long p = 0; p < r->P; ++p) total += r->fill[(size_t)p];
   if (r->store_top + total > r->store_rows) return TAURUS_ERR_RUN_STORE_FULL;
-  for (long long p = 0; p < r->P; ++p) { int rc = flush_partition(r, p, st); if (rc) return rc; }
+  std::vector<long long> parts;
+  for (long long p = 0; p < r->P; ++p)
+    if (r->fill[(size_t)p] > 0) parts.push_back(p);
+  if (!parts.empty()) { int rc = flush_many(r, parts, st); if (rc) return rc; }
   RCU(cudaGetLastError());
   RCU(cudaEventRecord(r->write_done, st));
   r->dirty = true;
@@ -383,14 +454,31 @@ int runs_read_into(taurus_runs* r, long long s, long long e, float* out, long lo
   if (r->stage_used) RCU(cudaStreamWaitEvent(st, r->stage_free, 0));
   long long at = 0;
   const size_t w = (size_t)r->width;
-  for (const Slice& sl : slices) {
-    const float* src = r->kind == TAURUS_RUNS_HOST ? r->store_host + (size_t)sl.off * w : r->store_dev + (size_t)sl.off * w;
-    RCU(cudaMemcpyAsync(r->d_stage_rows + (size_t)at * w, src, (size_t)sl.n * w * sizeof(float), cudaMemcpyDefault, st));
-    RCU(cudaMemcpyAsync(r->d_stage_ids + at, r->h_ids + sl.off, (size_t)sl.n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-    at += sl.n;
+  if (r->kind == TAURUS_RUNS_DEVICE && (long long)slices.size() <= r->P) {   // rows are read from the store in place
+    MoveSeg *hs, *ds;
+    int slot;
+    { int rc2 = next_seg_slot(r, &hs, &ds, &slot); if (rc2) return rc2; }
+    int nseg = 0;
+    long long most = 0;
+    for (const Slice& sl : slices) {
+      RCU(cudaMemcpyAsync(r->d_stage_ids + at, r->h_ids + sl.off, (size_t)sl.n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+      hs[nseg++] = MoveSeg{sl.off, sl.n, at};
+      at += sl.n; most = std::max(most, sl.n);
+    }
+    { int rc2 = push_segs(r, slot, nseg, st); if (rc2) return rc2; }
+    const int gx = (int)std::max<long long>(1, std::min<long long>((most * 32 + 255) / 256, std::max<long long>(1, (long long)r->sm_count * 8 / nseg)));
+    rs_place_slices_kernel<<<dim3(gx, nseg), 256, 0, st>>>(ds, r->d_stage_ids, r->store_dev, r->width, s, out, ld);
+    { int rc2 = release_seg_slot(r, slot, st); if (rc2) return rc2; }
+  } else {
+    for (const Slice& sl : slices) {
+      const float* src = r->kind == TAURUS_RUNS_HOST ? r->store_host + (size_t)sl.off * w : r->store_dev + (size_t)sl.off * w;
+      RCU(cudaMemcpyAsync(r->d_stage_rows + (size_t)at * w, src, (size_t)sl.n * w * sizeof(float), cudaMemcpyDefault, st));
+      RCU(cudaMemcpyAsync(r->d_stage_ids + at, r->h_ids + sl.off, (size_t)sl.n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+      at += sl.n;
+    }
+    const int grid = (int)std::min<long long>((total * 32 + 255) / 256, (long long)r->sm_count * 8);
+    rs_place_kernel<<<grid, 256, 0, st>>>(total, r->d_stage_ids, r->d_stage_rows, r->width, s, out, ld);
   }
-  const int grid = (int)std::min<long long>((total * 32 + 255) / 256, (long long)r->sm_count * 8);
-  rs_place_kernel<<<grid, 256, 0, st>>>(total, r->d_stage_ids, r->d_stage_rows, r->width, s, out, ld);
   r->launches += 1;
   RCU(cudaGetLastError());
   RCU(cudaEventRecord(r->stage_free, st));
