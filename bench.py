@@ -327,7 +327,7 @@ def run_ours(args):
     n_push = len(chunks) * L * args.steps
     ph = phases[:n_push].reshape(args.steps, L, len(chunks), 5)
     scatter_ms = ph[..., 3]
-    # Algorithmic bytes of the scatter ("Kernels"): per accumulator-row reduction a read-modify-write of
+    # Algorithmic bytes of the scatter: per accumulator-row reduction a read-modify-write of
     # the row (2 * 4 Hp) plus slot and pending-count words (8); per propagated edge its (destination, source)
     # words (8); per source its projected row read once (4 Hp) and its self message (row read 4 Hp + RMW 2 * 4 Hp + 8).
     # In CSR order a "group" is one edge.  The per-edge cold-miss model (12 + 2 * 4 Hp per edge) is kept beside it.
