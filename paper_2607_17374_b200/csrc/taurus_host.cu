@@ -642,7 +642,7 @@ extern "C" int taurus_drain_dense(taurus_ctx* c, float* dense_rows, int64_t ld, 
 
 extern "C" int taurus_layer_set_dense_output(taurus_ctx* c, float* dense_rows, int64_t ld) {
   if (!c || !dense_rows) return TAURUS_ERR_INVALID_ARG;
-  if (c->layer < 0 || c->chunk_seq != 0) return TAURUS_ERR_ORDER;
+  if (c->layer < 0 || c->chunk_seq != 0 || c->run_out) return TAURUS_ERR_ORDER;
   if (ld < c->dims[c->layer + 1]) return TAURUS_ERR_INVALID_ARG;
   float* dev = dense_rows;
   int kind = pointer_kind(dense_rows);
