@@ -8,7 +8,9 @@ At these sizes the full oracle is out of reach, so the checks are
     evaluation of exactly those destinations, their in-lists taken from the CSR by a scan;
   * per-chunk completion counts against the closed form floor(max(v, max in-neighbour) / chunk) (exact layers);
   * conservation laws of the state machine (completed == V, evictions == reloads, free == pool at layer end);
-  * for sampled layers: the kept edge lists of the sampled destinations, bit-exact.
+  * for sampled layers: the kept edge lists of the sampled destinations, bit-exact; the library's whole edge mask
+    (one bit per CSR edge, all E of them) against the oracle's propagated-edge flags from its own full in-lists and
+    its own sampler; and the per-chunk completion counts against the closed form over the sampled message sets.
 Each layer is run on its own generated input rows of the right width (the paper's convention of dummy inputs of
 matching dimensions for layers whose real input cannot be materialised, Sect. 4.2)."""
 import os
@@ -97,6 +99,10 @@ def test_full_config(name):
     completed_closed_form = np.bincount(last // chunk, minlength=n_chunks)
     del last, src_of_edge
     print("subset in-lists: %d destinations, %d in-edges, %.0f s" % (dsts.size, src.size, time.time() - t0), flush=True)
+    full_inl = None
+    if any(f > 0 for f in w.fanout):     # the oracle's own in-lists of the whole graph, for the full-mask comparison
+        full_inl = oracle.build_in_lists(V, g.row_ptr, g.col_idx)
+        print("full in-lists built, %.0f s" % (time.time() - t0), flush=True)
 
     drain_rows = int(completed_closed_form.max() * 1.05) + chunk
     host_rows = int(os.environ.get("TAURUS_FULL_HOST_ROWS", min(V - w.hub_count, 56_000_000)))
@@ -116,6 +122,17 @@ def test_full_config(name):
         got_ids, got_rows, counts = [], [], []
         t1 = time.time()
         ctx.layer_begin(l, stream)
+        sampled_counts = None
+        if w.fanout[l] > 0:                  # every bit of the edge mask, and the completion chunks of the sampled sets
+            ms_full = oracle.message_sets(full_inl, w.fanout[l], w.seed, l)
+            want_words = np.packbits(ms_full.prop, bitorder="little")
+            want_words = np.concatenate([want_words, np.zeros((-want_words.size) % 4, np.uint8)]).view(np.uint32)
+            got_words = ctx.get_edge_mask()
+            assert got_words.size == want_words.size and np.array_equal(got_words, want_words)
+            sampled_counts = np.bincount(oracle.complete_chunk_closed_form(ms_full, chunk), minlength=n_chunks)
+            print("%s layer %d: edge mask identical on all %d edges (%d propagated), %.0f s" %
+                  (name, l, g.E, int(ms_full.m.sum()), time.time() - t0), flush=True)
+            del ms_full, want_words, got_words
         for c, s in enumerate(range(0, V, chunk)):
             e = min(s + chunk, V)
             x = xbuf[c & 1]
@@ -144,6 +161,7 @@ def test_full_config(name):
             assert (np.asarray(counts) == completed_closed_form).all()
         else:
             assert st["total_messages"] == int(np.minimum(g.in_degree.astype(np.int64), w.fanout[l]).sum())
+            assert (np.asarray(counts) == sampled_counts).all()
             for i in list(range(0, dsts.size, 97)) + list(np.argsort(-np.diff(ptr))[:16]):   # kept edge lists, bit-exact
                 eids, srcs, n = ctx.get_sampled_edges(l, int(dsts[i]), capacity=128)
                 assert n == keep_ptr[i + 1] - keep_ptr[i] and (eids == keep_eid[keep_ptr[i]:keep_ptr[i + 1]]).all()
