@@ -158,9 +158,9 @@ __global__ void plan_kernel(ChunkArgs a) {
   ctl->sel_prefix = 0ull;
   ctl->sel_k = deficit;
   ctl->victim_count = 0;
-  // Stack positions are handed out by list index, not by per-item atomics: victim i frees into
-  // free_stack[F + i] and takes host row host_free[H - 1 - i]; need-list entry i takes
-  // free_stack[F + deficit - 1 - i].  The counters are brought to their end-of-chunk values here.
+  // Stack positions are handed out by list index, not by per-item atomics: victim i takes host row
+  // host_free[H - 1 - i]; need-list entry i < deficit takes over the slot of victim deficit - 1 - i, entry
+  // i >= deficit pops free_stack[F + deficit - 1 - i].  The counters are brought to their end-of-chunk values here.
   const long long F = ctl->free_top, H = ctl->host_free_top;
   ctl->evict_push_base = F;
   ctl->host_pop_base = H;
@@ -272,79 +272,85 @@ __global__ void evict_list_kernel(ChunkArgs a) {
       int leader = __ffs(m) - 1, idx = 0;
       if (lane_id() == leader) idx = atomicAdd(&ctl->victim_count, __popc(m));
       idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (hit && idx < a.pool_slots) a.victims[idx] = (int32_t)s;
+      // victim idx takes the host row host_free[H - 1 - idx]; read here, before this chunk's reloads push rows back
+      if (hit && idx < a.victim_capacity) a.victims[idx] = make_int2((int)s, a.host_free[ctl->host_pop_base - 1 - idx]);
     }
   }
 }
 
-// One warp per victim: accumulator row -> pinned host row, IN_BUFFER -> EVICTED, slot back on the free stack.
-__global__ void evict_copy_kernel(ChunkArgs a) {
+// One warp per vertex that needs a slot.  Need-list entry i < deficit takes over the slot of victim
+// deficit - 1 - i: the warp reads the victim's accumulator row and, if its own vertex was EVICTED, the vertex's
+// host row, then writes the victim's row to its pinned host row (IN_BUFFER -> EVICTED) and the reloaded row (or
+// zeros for a NOT_STARTED vertex) into the slot, so that evictions (device -> host) and reloads (host -> device)
+// use both directions of the link at the same time.  Entries i >= deficit pop the free stack.  Either way
+// the vertex is IN_BUFFER afterwards.
+__global__ void alloc_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->deficit == 0) return;
-  const int n = ctl->deficit;
-  if (ctl->victim_count != n) {   // the select must have produced exactly `deficit` victims
+  if (ctl->error) return;
+  const int n = ctl->need_count;
+  const int deficit = ctl->deficit;
+  if (deficit > 0 && ctl->victim_count != deficit) {   // the select must have produced exactly `deficit` victims
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
     return;
   }
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
-  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    int slot = a.victims[i];
-    int v = a.owner[slot];
-    const int hrow = a.host_free[ctl->host_pop_base - 1 - i];
-    const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)slot * a.Hp);
-    float4* dst = reinterpret_cast<float4*>(a.host_store + (size_t)hrow * a.Hp);
-    for (int k = lane_id(); k < vec; k += 32) dst[k] = src[k];
-    if (lane_id() == 0) {
-      a.loc[v] = -2 - hrow;
-      a.state[v] = TAURUS_EVICTED;
-      a.owner[slot] = -1;
-      a.free_stack[ctl->evict_push_base + i] = slot;
-    }
-  }
-}
-
-// One warp per vertex that needs a slot: pop a slot; EVICTED -> copy the host row back (a reload),
-// NOT_STARTED -> zero the row; either way the vertex is IN_BUFFER afterwards.
-__global__ void alloc_kernel(ChunkArgs a) {
-  DevCtl* ctl = a.ctl;
-  if (ctl->error) return;
-  const int n = ctl->need_count;
-  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const int vec = a.Hp >> 2;
   int reloaded = 0;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
     int v = a.need_list[i];
-    int slot = -1, st = 0, l = 0;
+    int slot = -1, st = 0, l = 0, out_hrow = -1, victim = -1;
     if (lane_id() == 0) {
       if (a.direct) slot = v;
-      else { long long f = ctl->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
+      else if (i < deficit) {
+        const int2 vic = a.victims[deficit - 1 - i];
+        slot = vic.x; out_hrow = vic.y; victim = a.owner[slot];
+      } else { long long f = ctl->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
       st = a.state[v];
       l = a.loc[v];
     }
     slot = __shfl_sync(FULL, slot, 0);
     st = __shfl_sync(FULL, st, 0);
     l = __shfl_sync(FULL, l, 0);
+    out_hrow = __shfl_sync(FULL, out_hrow, 0);
     if (slot < 0) {
       if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
       continue;
     }
-    float4* dst = reinterpret_cast<float4*>(a.acc + (size_t)slot * a.Hp);
-    if (st == TAURUS_EVICTED) {
-      int hrow = -2 - l;
-      const float4* src = reinterpret_cast<const float4*>(a.host_store + (size_t)hrow * a.Hp);
-      for (int k = lane_id(); k < vec; k += 32) dst[k] = src[k];
-      if (lane_id() == 0) {
+    float4* __restrict__ row = reinterpret_cast<float4*>(a.acc + (size_t)slot * a.Hp);
+    float4* __restrict__ host_out = out_hrow >= 0 ? reinterpret_cast<float4*>(a.host_store + (size_t)out_hrow * a.Hp) : nullptr;
+    const int in_hrow = st == TAURUS_EVICTED ? -2 - l : -1;
+    const float4* __restrict__ host_in = in_hrow >= 0 ? reinterpret_cast<const float4*>(a.host_store + (size_t)in_hrow * a.Hp) : nullptr;
+    for (int k0 = 0; k0 < vec; k0 += 128) {   // four float4 per lane and direction in flight
+      float4 keep[4], in[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = k0 + q * 32 + lane_id();
+        in[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (k < vec) {
+          if (host_out) keep[q] = row[k];
+          if (host_in) in[q] = host_in[k];
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = k0 + q * 32 + lane_id();
+        if (k < vec) {
+          if (host_out) host_out[k] = keep[q];
+          row[k] = in[q];
+        }
+      }
+    }
+    if (lane_id() == 0) {
+      if (out_hrow >= 0) {
+        a.loc[victim] = -2 - out_hrow;
+        a.state[victim] = TAURUS_EVICTED;
+      }
+      if (in_hrow >= 0) {
         long long h = atomicAdd((unsigned long long*)&ctl->host_free_top, 1ull);
-        a.host_free[h] = hrow;
+        a.host_free[h] = in_hrow;
         a.reload_count[v] += 1;
         reloaded++;
       }
-    } else {
-      const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int k = lane_id(); k < vec; k += 32) dst[k] = z;
-    }
-    if (lane_id() == 0) {
       if (!a.direct) { a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch; }
       a.state[v] = TAURUS_IN_BUFFER;
     }
@@ -364,8 +370,7 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
       select_resolve_kernel<<<1, 1024, 0, st>>>(a, p);
     }
     evict_list_kernel<<<blocks, 256, 0, st>>>(a);
-    evict_copy_kernel<<<blocks, 256, 0, st>>>(a);
-    c->launches += 2 * TAURUS_SEL_PASSES + 2;
+    c->launches += 2 * TAURUS_SEL_PASSES + 1;
   }
   alloc_kernel<<<blocks, 256, 0, st>>>(a);
   c->launches += 1;

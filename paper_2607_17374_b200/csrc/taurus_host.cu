@@ -199,7 +199,10 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   ALLOC(c->d_owner, c->pool_slots); ALLOC(c->d_free_stack, c->pool_slots); ALLOC(c->d_need_list, c->pool_slots);
   ALLOC(c->d_slot_epoch, c->pool_slots);   // written at every slot hand-out, also when no eviction can happen
-  if (c->pool_slots < V - c->hub_count) { ALLOC(c->d_victims, c->pool_slots); ALLOC(c->d_keys, c->pool_slots); }
+  if (c->pool_slots < V - c->hub_count) {   // a chunk evicts at most what it needs, and it needs at most what it touches
+    c->victim_capacity = std::min<long long>(c->pool_slots, c->touched_capacity);
+    ALLOC(c->d_victims, c->victim_capacity); ALLOC(c->d_keys, c->pool_slots);
+  }
   ALLOC(c->d_host_free, c->host_rows);
   if (c->host_rows > 0) {
     cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->host_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
@@ -349,7 +352,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.pend = c->d_pend; a.state = c->d_state; a.loc = c->d_loc; a.touch = c->d_touch; a.reload_count = c->d_reload;
   a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list; a.slot_epoch = c->d_slot_epoch;
   a.touched_list = c->d_touched_list; a.touched_capacity = c->touched_capacity;
-  a.victims = c->d_victims; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
+  a.victims = c->d_victims; a.victim_capacity = c->victim_capacity; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
   a.Hp = taurus_round_up(c->dims[l + 1], 4);
   a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;   // GAT pass 3 scatters h' rows repacked to pitch Hp

@@ -33,7 +33,7 @@ struct DevCtl {
   long long grad_count;     // rows waiting in the graduation buffer
   long long out_count[2];   // dense-output mode: rows finalise left in each half of the graduation buffer
   long long alloc_base;       // this chunk: need-list entry i takes free_stack[alloc_base - 1 - i]
-  long long evict_push_base;  // this chunk: victim i's slot goes to free_stack[evict_push_base + i]
+  long long evict_push_base;  // this chunk: free-stack height before the chunk (victims' slots go straight to the vertices that need them)
   long long host_pop_base;    // this chunk: victim i's row goes to host row host_free[host_pop_base - 1 - i]
   unsigned long long sel_prefix;  // radix select: digits fixed so far (high bits)
   long long sel_k;                // radix select: rank still to resolve inside the prefix bucket
@@ -65,7 +65,8 @@ struct ChunkArgs {
   int32_t* need_list;       // [pool_slots]
   int32_t* touched_list;    // [touched_capacity] every vertex the chunk touches, listed at its first touch
   long long touched_capacity;
-  int32_t* victims;         // [pool_slots]
+  int2* victims;            // [victim_capacity] (slot, pinned host row) of this chunk's victims
+  long long victim_capacity;
   unsigned long long* keys; // [pool_slots]
   float* host_store;        // device alias of the pinned host rows [host_evict_rows x Hp]
   int32_t* host_free;       // [host_evict_rows]
@@ -147,7 +148,8 @@ struct taurus_ctx {
   int32_t* d_need_list = nullptr;
   int32_t* d_touched_list = nullptr;
   long long touched_capacity = 0;
-  int32_t* d_victims = nullptr;
+  int2* d_victims = nullptr;
+  long long victim_capacity = 0;
   unsigned long long* d_keys = nullptr;
   float* h_store = nullptr;      // pinned, mapped
   float* d_store_alias = nullptr;

@@ -122,6 +122,7 @@ def test_full_config(name):
         got_ids, got_rows, counts = [], [], []
         t1 = time.time()
         ctx.layer_begin(l, stream)
+        ctx.set_timing(True)
         sampled_counts = None
         if w.fanout[l] > 0:                  # every bit of the edge mask, and the completion chunks of the sampled sets
             ms_full = oracle.message_sets(full_inl, w.fanout[l], w.seed, l)
@@ -146,6 +147,11 @@ def test_full_config(name):
                     got_ids.append(ids_buf[:n][hit].cpu().numpy()); got_rows.append(rows_buf[:n][hit].cpu().numpy())
         st = ctx.layer_end()
         dt = time.time() - t1
+        ph = ctx.get_phase_ms().sum(axis=0)
+        ctx.set_timing(False)
+        print("%s layer %d: device time %.0f ms (copy-in %.0f, projection %.0f, classify + make-room %.0f, scatter %.0f, finalise %.0f) "
+              "= %.2f G messages/s on the device" % (name, l, ph.sum(), ph[0], ph[1], ph[2], ph[3], ph[4],
+                                                    st["total_messages"] / max(ph.sum(), 1e-9) / 1e6), flush=True)
         print("%s layer %d: %.1f s, %.3f G messages/s incl. host feature generation; evictions %d reloads %d peak occupancy %d "
               "max reloads of one vertex %d hub messages %.1f %%" %
               (name, l, dt, st["total_messages"] / dt / 1e9, st["evictions"], st["reloads"], st["peak_occupancy"],
