@@ -255,6 +255,15 @@ int taurus_get_sampled_edges(taurus_ctx* ctx, int32_t layer, int64_t dst, int64_
  * host output of ceil(E / 32) words; all ones in exact mode. */
 int taurus_get_edge_mask(taurus_ctx* ctx, uint32_t* out_words);
 
+/* Per-destination digest of the current layer's propagated in-edges, for checking sampled neighbour sets of all
+ * V vertices at once (Sect. 3.9 sampling paragraph): with h(u, e) = mix64(((u << 32) | e) + 0x9E3779B97F4A7C15)
+ * for a propagated edge number e (its CSR index) from source u, where mix64(x) is x ^= x >> 30;
+ * x *= 0xBF58476D1CE4E5B9; x ^= x >> 27; x *= 0x94D049BB133111EB; x ^= x >> 31 on 64-bit words,
+ * out_digest[2 v] = sum of h over the propagated in-edges of v (mod 2^64) and out_digest[2 v + 1] = their
+ * xor; both 0 for a vertex without propagated in-edges.  out_digest: [2 V] words, host or device memory.
+ * Blocking. */
+int taurus_get_sample_digest(taurus_ctx* ctx, uint64_t* out_digest);
+
 /* Upper bound on the vertices that sources [src_begin, src_end) complete in the current layer
  * (exact when both ends are multiples of 64 or the ends of the graph). */
 int taurus_completion_bound(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, int64_t* out_bound);

@@ -143,6 +143,25 @@ def message_sets(inl: InLists, fanout: int, seed: int, layer: int) -> MessageSet
     return MessageSets(ptr, src, eid, prop, m.astype(np.int32))
 
 
+def sample_digest(ms: MessageSets) -> np.ndarray:
+    """uint64 [V, 2]: per destination the sum (mod 2^64) and the xor of mix64(((u << 32) | e) + golden) over its
+    propagated in-edges (source u, CSR edge index e); (0, 0) for an empty set.  A commutative fingerprint of M(v)
+    (Sect. 3.9 sampling paragraph: the sampled set is a function of seed, layer and destination)."""
+    M64 = np.uint64(0xFFFFFFFFFFFFFFFF)
+    with np.errstate(over="ignore"):
+        x = ((ms.src.astype(np.uint64) << np.uint64(32)) | (ms.eid.astype(np.uint64) & np.uint64(0xFFFFFFFF))) + np.uint64(0x9E3779B97F4A7C15)
+        x ^= x >> np.uint64(30); x = (x * np.uint64(0xBF58476D1CE4E5B9)) & M64
+        x ^= x >> np.uint64(27); x = (x * np.uint64(0x94D049BB133111EB)) & M64
+        x ^= x >> np.uint64(31)
+        V = ms.m.size
+        out = np.zeros((V, 2), np.uint64)
+        nz = np.flatnonzero(ms.m > 0)
+        if nz.size:
+            out[nz, 0] = np.add.reduceat(x, ms.ptr[nz])
+            out[nz, 1] = np.bitwise_xor.reduceat(x, ms.ptr[nz])
+    return out
+
+
 # ----------------------------------------------------------------------------- one layer, pull-based, fp64
 
 def coefficients(mode: int, m: np.ndarray, din: np.ndarray, dout: np.ndarray, gin_eps: float = 0.0):

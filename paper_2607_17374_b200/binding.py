@@ -90,6 +90,7 @@ EXPORTS = [
     "taurus_runs_create", "taurus_runs_append", "taurus_runs_flush", "taurus_runs_read_chunk", "taurus_runs_info",
     "taurus_runs_directory", "taurus_runs_get_run", "taurus_runs_reset", "taurus_runs_destroy",
     "taurus_layer_set_run_output", "taurus_push_chunk_from_runs", "taurus_gat_project_chunk", "taurus_gat_attention",
+    "taurus_get_sample_digest",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -117,6 +118,7 @@ def load_library():
     lib.taurus_get_vertex_array.argtypes = [vp, i32, vp]
     lib.taurus_get_sampled_edges.argtypes = [vp, i32, i64, vp, vp, i32, ctypes.POINTER(i32)]
     lib.taurus_get_edge_mask.argtypes = [vp, vp]
+    lib.taurus_get_sample_digest.argtypes = [vp, vp]
     lib.taurus_completion_bound.argtypes = [vp, i64, i64, ctypes.POINTER(i64)]
     lib.taurus_completion_counts_noalloc.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp]
     lib.taurus_reorder.argtypes = [i64, i64, vp, vp, vp, i32, vp, vp, vp, vp, vp]
@@ -367,6 +369,12 @@ class Context:
         words = np.empty((self.E + 31) // 32, np.uint32)
         self._check(self._lib.taurus_get_edge_mask(self._h, words.ctypes.data), "taurus_get_edge_mask")
         return words
+
+    def get_sample_digest(self) -> np.ndarray:
+        """uint64 [V, 2]: (sum, xor) of the mixed (source, CSR edge index) pairs of every vertex's propagated in-edges."""
+        out = np.empty((self.V, 2), np.uint64)
+        self._check(self._lib.taurus_get_sample_digest(self._h, out.ctypes.data), "taurus_get_sample_digest")
+        return out
 
     def completion_bound(self, src_begin: int, src_end: int) -> int:
         n = ctypes.c_int64(0)

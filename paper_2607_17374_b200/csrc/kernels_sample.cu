@@ -184,3 +184,28 @@ int sampled_edges_of(taurus_ctx* c, int layer, long long dst, long long* out_eid
   cudaFree(d_e); cudaFree(d_s); cudaFree(d_n);
   return rc;
 }
+
+// Digest of every destination's propagated in-edges: commutative sum and xor of a 64-bit mix of (source, CSR
+// edge index), accumulated push-based with one warp per source row.
+__global__ void sample_digest_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                                     const uint32_t* __restrict__ mask, unsigned long long* __restrict__ digest) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    for (long long e = row_ptr[u] + lane; e < row_ptr[u + 1]; e += 32) {
+      if (mask && !((mask[e >> 5] >> (e & 31)) & 1u)) continue;
+      unsigned long long x = (((unsigned long long)u << 32) | (unsigned long long)(e & 0xffffffffll)) + 0x9E3779B97F4A7C15ull;
+      x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+      x ^= x >> 27; x *= 0x94D049BB133111EBull;
+      x ^= x >> 31;
+      const long long v = col[e];
+      atomicAdd(&digest[2 * v], x);
+      atomicXor(&digest[2 * v + 1], x);
+    }
+  }
+}
+
+void launch_sample_digest(taurus_ctx* c, unsigned long long* d_digest, cudaStream_t st) {
+  sample_digest_kernel<<<c->sm_count * 8, 256, 0, st>>>(c->V, c->d_row_ptr, c->d_col, c->d_mask_cur, d_digest);
+  c->launches += 1;
+}

@@ -753,6 +753,21 @@ extern "C" int taurus_get_edge_mask(taurus_ctx* c, uint32_t* out_words) {
   return TAURUS_OK;
 }
 
+extern "C" int taurus_get_sample_digest(taurus_ctx* c, uint64_t* out_digest) {
+  if (!c || !out_digest) return TAURUS_ERR_INVALID_ARG;
+  if (c->layer < 0) return TAURUS_ERR_ORDER;
+  CU(cudaSetDevice(c->device));
+  CU(cudaStreamSynchronize(c->last_stream));
+  unsigned long long* d = nullptr;
+  ALLOC(d, (size_t)2 * c->V);
+  cudaError_t e = cudaMemset(d, 0, (size_t)2 * c->V * sizeof(unsigned long long));
+  if (e == cudaSuccess) { launch_sample_digest(c, d, nullptr); e = cudaGetLastError(); }
+  if (e == cudaSuccess) e = cudaMemcpy(out_digest, d, (size_t)2 * c->V * sizeof(unsigned long long), cudaMemcpyDefault);
+  cudaFree(d);
+  CU(e);
+  return TAURUS_OK;
+}
+
 extern "C" int64_t taurus_launch_count(const taurus_ctx* c) { return c ? c->launches : 0; }
 
 extern "C" int taurus_set_timing(taurus_ctx* c, int32_t on) {

@@ -254,3 +254,4 @@ void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 int build_in_edge_order(taurus_ctx* c);                                      // csc_ptr, csc_eid
 void launch_sample_mask(taurus_ctx* c, int layer, cudaStream_t st);
 int sampled_edges_of(taurus_ctx* c, int layer, long long dst, long long* out_eids, int32_t* out_src, int cap, int* n);
+void launch_sample_digest(taurus_ctx* c, unsigned long long* d_digest, cudaStream_t st);   // d_digest [2V], zeroed by the caller

@@ -43,6 +43,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
             res["masks"].append(ctx.get_edge_mask())
         else:
             res["masks"].append(None)
+        res.setdefault("digests", []).append(ctx.get_sample_digest())
         per_chunk = []
         plan = chunk_plan or [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
         if w.mode == tg.GAT:  # passes 1 and 2; pass 3 below streams the transformed rows instead of the features

@@ -130,6 +130,7 @@ def test_full_config(name):
             want_words = np.concatenate([want_words, np.zeros((-want_words.size) % 4, np.uint8)]).view(np.uint32)
             got_words = ctx.get_edge_mask()
             assert got_words.size == want_words.size and np.array_equal(got_words, want_words)
+            assert np.array_equal(ctx.get_sample_digest(), oracle.sample_digest(ms_full))   # per-destination fingerprints, all V
             sampled_counts = np.bincount(oracle.complete_chunk_closed_form(ms_full, chunk), minlength=n_chunks)
             print("%s layer %d: edge mask identical on all %d edges (%d propagated), %.0f s" %
                   (name, l, g.E, int(ms_full.m.sum()), time.time() - t0), flush=True)

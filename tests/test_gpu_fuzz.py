@@ -78,6 +78,7 @@ def test_random_configuration(seed):
             scale = np.abs(orc["outs"][l]).max() + 1e-6
             assert np.abs(lib["outs"][l] - orc["outs"][l]).max() <= 1e-4 * scale, (l, row, elem_max)
         assert orc["sims"][l].rc == 0
+        assert np.array_equal(lib["digests"][l], oracle.sample_digest(orc["msets"][l]))   # the propagated in-edge sets, all V
         completed = lib["completed"][l]
         per_chunk = completed if (completed and kw.get("drain_each_chunk", True) and not kw.get("dense_output")) else None
         if per_chunk is not None and any(isinstance(c, tuple) for c in per_chunk):

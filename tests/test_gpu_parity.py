@@ -2,6 +2,7 @@
 import numpy as np
 import pytest
 
+import oracle
 import taurus_gen as tg
 from gpu_harness import check_accounting, row_error, run_library, run_oracle
 
@@ -77,6 +78,7 @@ def test_sampled_inference_masks_and_outputs():
         want = np.packbits(orc["msets"][l].prop, bitorder="little")
         got = lib["masks"][l].view(np.uint8)[:want.size]
         assert (got == want).all(), l
+        assert np.array_equal(lib["digests"][l], oracle.sample_digest(orc["msets"][l])), l   # per-destination fingerprints, all V
     # kept edge lists of single destinations, hubs included
     ctx = lib["ctx"]
     order = np.argsort(-g.in_degree)

@@ -77,3 +77,44 @@ def test_frozen_hash_values():
     assert len(rows) >= 16
     for seed, layer, dst, k, h in rows:
         assert oracle._lib().to_sample_hash(int(seed), int(layer), int(dst), int(k)) == int(h, 16)
+
+
+def test_sample_digest_against_python_integers_and_its_invariances():
+    """The digest is the plain definition (checked with Python's unbounded integers), does not depend on the order
+    of the entries, and changes when one kept edge is exchanged for another."""
+    rng = np.random.default_rng(12)
+    V, E = 60, 700
+    src = np.sort(rng.integers(0, V, E))
+    col = rng.integers(0, V, E).astype(np.int32)
+    row_ptr = np.zeros(V + 1, np.int64)
+    np.cumsum(np.bincount(src, minlength=V), out=row_ptr[1:])
+    inl = oracle.build_in_lists(V, row_ptr, col)
+    for fanout in (0, 4):
+        ms = oracle.message_sets(inl, fanout, 5, 1)
+        d = oracle.sample_digest(ms)
+
+        def mix(u, e):
+            m = (1 << 64) - 1
+            x = (((u << 32) | e) + 0x9E3779B97F4A7C15) & m
+            x ^= x >> 30; x = (x * 0xBF58476D1CE4E5B9) & m
+            x ^= x >> 27; x = (x * 0x94D049BB133111EB) & m
+            x ^= x >> 31
+            return x
+        for v in range(V):
+            hs = [mix(int(ms.src[k]), int(ms.eid[k])) for k in range(ms.ptr[v], ms.ptr[v + 1])]
+            s, x = 0, 0
+            for h in hs:
+                s = (s + h) & ((1 << 64) - 1)
+                x ^= h
+            assert (int(d[v, 0]), int(d[v, 1])) == (s, x)
+        # order of the entries inside a list does not matter
+        perm = np.concatenate([ms.ptr[v] + rng.permutation(ms.ptr[v + 1] - ms.ptr[v]) for v in range(V)]).astype(np.int64)
+        shuffled = oracle.MessageSets(ms.ptr, ms.src[perm], ms.eid[perm], ms.prop, ms.m)
+        assert np.array_equal(oracle.sample_digest(shuffled), d)
+    exact, sampled = oracle.message_sets(inl, 0, 5, 1), oracle.message_sets(inl, 4, 5, 1)
+    de, ds = oracle.sample_digest(exact), oracle.sample_digest(sampled)
+    big = np.diff(inl.ptr) > 4
+    assert big.any() and (de[big] != ds[big]).any(axis=1).all()       # a thinned list has another digest
+    assert np.array_equal(de[~big], ds[~big])                          # lists that were kept whole have the same
+    other = oracle.sample_digest(oracle.message_sets(inl, 4, 6, 1))   # another seed keeps other edges somewhere
+    assert not np.array_equal(other, ds)
