@@ -45,7 +45,21 @@ def random_config(seed):
         pool = int(pool * 1.3) + 1
     w = replace(w, pool_slots=pool)
     kw = dict(flags=int(rng.choice([0, 0, 2, 4, 6])), evict_policy=policy)
-    out_mode = int(rng.integers(0, 4))
+    out_mode = int(rng.integers(0, 6))
+    if out_mode == 4 and mode != tg.GAT:       # layers chained through sorted runs
+        import paper_2607_17374_b200 as tb
+        kw["run_output"] = (int(rng.choice([1, 3, 16])), int(rng.choice([1, 50, 4000])) if g.V < 1500 else int(rng.choice([50, 4000])),
+                            tb.RUNS_HOST if rng.integers(0, 2) else tb.RUNS_DEVICE)
+    elif out_mode == 5:                        # pushes that are not cells of the chunk grid (CSR-order kernels), small graduation buffer
+        cuts = sorted(set([0, g.V] + [int(x) for x in rng.integers(1, g.V, size=int(rng.integers(1, 12)))]))
+        plan = []
+        for a, b in zip(cuts[:-1], cuts[1:]):
+            while b - a > chunk:
+                plan.append((a, a + chunk)); a += chunk
+            plan.append((a, b))
+        kw["chunk_plan"] = plan
+        kw["drain_each_chunk"] = bool(rng.integers(0, 2))
+        w = replace(w, pool_slots=g.V)         # the simulator works on the chunk grid: no eviction, outputs and sets only
     if out_mode == 1:
         kw["dense_output"] = True
     elif out_mode == 2:
@@ -77,10 +91,14 @@ def test_random_configuration(seed):
             # several hundred terms meets a bound relative to that row: gate such layers on the layer's own scale
             scale = np.abs(orc["outs"][l]).max() + 1e-6
             assert np.abs(lib["outs"][l] - orc["outs"][l]).max() <= 1e-4 * scale, (l, row, elem_max)
-        assert orc["sims"][l].rc == 0
+        assert orc["sims"][l].rc == 0 or kw.get("chunk_plan")
         assert np.array_equal(lib["digests"][l], oracle.sample_digest(orc["msets"][l]))   # the propagated in-edge sets, all V
         completed = lib["completed"][l]
-        per_chunk = completed if (completed and kw.get("drain_each_chunk", True) and not kw.get("dense_output")) else None
+        per_chunk = completed if (completed and kw.get("drain_each_chunk", True) and not kw.get("dense_output")
+                                  and not kw.get("chunk_plan")) else None
         if per_chunk is not None and any(isinstance(c, tuple) for c in per_chunk):
             per_chunk = None
-        check_accounting(lib["stats"][l], lib["chunk_log"][l], lib["reload_count"][l], orc["sims"][l], per_chunk)
+        if kw.get("chunk_plan"):
+            assert lib["stats"][l]["completed"] == g.V and lib["stats"][l]["total_messages"] == int(orc["msets"][l].m.sum())
+        else:
+            check_accounting(lib["stats"][l], lib["chunk_log"][l], lib["reload_count"][l], orc["sims"][l], per_chunk)
