@@ -239,8 +239,6 @@ def run_ours(args):
                      0, w.gin_eps, model.att_src, model.att_dst, w.leaky_slope)
     gat = w.mode == tg.GAT
     use_runs = args.output != "dense"
-    if gat and use_runs:
-        raise SystemExit("--model gat reads its features through pointers: use --output dense")
     hprime = torch.zeros((V, max(w.dims[1:])), dtype=torch.float32, device=dev) if gat else None
     runs = None
     if use_runs:   # one run store per layer output: 16 id ranges, buffers of 32 768 rows
@@ -270,14 +268,17 @@ def run_ours(args):
             if gat:    # passes 1 and 2: transformed rows and attention scalars, then the topology-only sweep
                 hp = hprime.view(-1)[:V * d_out].view(V, d_out)
                 for (s, e) in chunks:
-                    ctx.gat_project_chunk(s, e, feat[s:e], hp[s:e], d_out, stream)
+                    if use_runs and l > 0:
+                        ctx.gat_project_chunk_from_runs(s, e, runs[l - 1], hp[s:e], d_out, stream)
+                    else:
+                        ctx.gat_project_chunk(s, e, feat[s:e], hp[s:e], d_out, stream)
                 ctx.gat_attention(stream)
                 src = hp
             if use_runs:
                 runs[l].reset()
                 ctx.layer_set_run_output(runs[l])
                 for (s, e) in chunks:
-                    if l == 0:
+                    if l == 0 or gat:      # gat: pass 3 streams the transformed rows of pass 1
                         ctx.push_chunk(s, e, src[s:e], stream)
                     else:
                         ctx.push_chunk_from_runs(s, e, runs[l - 1], stream)

@@ -69,6 +69,7 @@ enum { TAURUS_GEMM_FP32 = 0, TAURUS_GEMM_BF16 = 1 };
 enum { TAURUS_NOT_STARTED = 0, TAURUS_IN_BUFFER = 1, TAURUS_EVICTED = 2, TAURUS_ON_GPU = 3, TAURUS_COMPLETED = 4 };
 
 typedef struct taurus_ctx taurus_ctx;
+typedef struct taurus_runs taurus_runs;   /* sorted runs of (vertex id, row) records: the output side, declared below */
 
 /* CSR out-edge topology (Sect. 3.2).  Copied at init. */
 typedef struct {
@@ -197,6 +198,10 @@ int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const
 int taurus_gat_project_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const float* features, float* hprime_out,
                              int64_t ld, void* cuda_stream);
 int taurus_gat_attention(taurus_ctx* ctx, void* cuda_stream);
+/* Pass 1 with the chunk's features read from sorted runs (see taurus_runs below; width dims[layer]) by
+ * merge-on-read, as taurus_push_chunk_from_runs does for the other modes. */
+int taurus_gat_project_chunk_from_runs(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, taurus_runs* runs,
+                                       float* hprime_out, int64_t ld, void* cuda_stream);
 
 /*
  * Copies out the vertices finalised since the last drain (Sect. 3.6): out_ids[i] and the dims[layer+1]
@@ -340,7 +345,6 @@ int taurus_reorder(int64_t V, int64_t E, const int64_t* row_ptr, const int32_t* 
  * the arrival sequence alone.  One object is used from one host thread at a time; calls on it are ordered on
  * the streams given (the library inserts the dependencies between streams itself).
  */
-typedef struct taurus_runs taurus_runs;
 enum { TAURUS_RUNS_HOST = 0, TAURUS_RUNS_DEVICE = 1 };
 typedef struct {
   int64_t V;                /* vertex ids are in [0, V), V < 2^31                                              */

@@ -90,7 +90,7 @@ EXPORTS = [
     "taurus_runs_create", "taurus_runs_append", "taurus_runs_flush", "taurus_runs_read_chunk", "taurus_runs_info",
     "taurus_runs_directory", "taurus_runs_get_run", "taurus_runs_reset", "taurus_runs_destroy",
     "taurus_layer_set_run_output", "taurus_push_chunk_from_runs", "taurus_gat_project_chunk", "taurus_gat_attention",
-    "taurus_get_sample_digest",
+    "taurus_get_sample_digest", "taurus_gat_project_chunk_from_runs",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -136,6 +136,7 @@ def load_library():
     lib.taurus_push_chunk_from_runs.argtypes = [vp, i64, i64, vp, vp]
     lib.taurus_gat_project_chunk.argtypes = [vp, i64, i64, vp, vp, i64, vp]
     lib.taurus_gat_attention.argtypes = [vp, vp]
+    lib.taurus_gat_project_chunk_from_runs.argtypes = [vp, i64, i64, vp, vp, i64, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -307,6 +308,10 @@ class Context:
     def gat_project_chunk(self, src_begin: int, src_end: int, features, hprime_out, ld: int, stream=None):
         self._check(self._lib.taurus_gat_project_chunk(self._h, src_begin, src_end, _ptr(features), _ptr(hprime_out), ld,
                                                        _stream(stream)), "taurus_gat_project_chunk")
+
+    def gat_project_chunk_from_runs(self, src_begin: int, src_end: int, runs: "Runs", hprime_out, ld: int, stream=None):
+        self._check(self._lib.taurus_gat_project_chunk_from_runs(self._h, src_begin, src_end, runs._h, _ptr(hprime_out), ld,
+                                                                 _stream(stream)), "taurus_gat_project_chunk_from_runs")
 
     def gat_attention(self, stream=None):
         self._check(self._lib.taurus_gat_attention(self._h, _stream(stream)), "taurus_gat_attention")

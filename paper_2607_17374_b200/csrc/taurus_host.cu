@@ -514,14 +514,16 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   return run_rc;
 }
 
-extern "C" int taurus_gat_project_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, float* hprime_out,
-                                        int64_t ld, void* cuda_stream) {
-  if (!c || !features || !hprime_out) return TAURUS_ERR_INVALID_ARG;
+static int gat_project_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, taurus_runs* src_runs,
+                            float* hprime_out, int64_t ld, void* cuda_stream) {
+  if (!c || (!features && !src_runs) || !hprime_out) return TAURUS_ERR_INVALID_ARG;
   if (c->mode != TAURUS_GAT) return TAURUS_ERR_UNSUPPORTED;
   if (c->layer < 0 || c->gat_ready || c->chunk_seq != 0 || src_begin != c->gat_next_src) return TAURUS_ERR_ORDER;
   if (src_end <= src_begin || src_end > c->V || src_end - src_begin > c->chunk_sources) return TAURUS_ERR_INVALID_ARG;
   const int l = c->layer, K = c->dims[l], d_out = c->dims[l + 1], Hp = taurus_round_up(d_out, 4);
-  if (ld < d_out || (reinterpret_cast<uintptr_t>(features) & 3) != 0 || pointer_kind(hprime_out) != PK_DEVICE) return TAURUS_ERR_INVALID_ARG;
+  if (ld < d_out || (features && (reinterpret_cast<uintptr_t>(features) & 3) != 0) || pointer_kind(hprime_out) != PK_DEVICE) return TAURUS_ERR_INVALID_ARG;
+  if (src_runs && (runs_width(src_runs) != K || runs_vertices(src_runs) != c->V || runs_max_chunk(src_runs) < src_end - src_begin))
+    return TAURUS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(cudaSetDevice(c->device));
   if (st != c->last_stream) {
@@ -532,7 +534,7 @@ extern "C" int taurus_gat_project_chunk(taurus_ctx* c, int64_t src_begin, int64_
   const int n = (int)(src_end - src_begin);
   const float* X = nullptr;
   int xbuf = -1;
-  { int rc = stage_chunk(c, features, nullptr, src_begin, src_end, K, st, &X, &xbuf); if (rc) return rc; }
+  { int rc = stage_chunk(c, features, src_runs, src_begin, src_end, K, st, &X, &xbuf); if (rc) return rc; }
   if (project_tc_usable(c, l, X, K)) {
     int rc = launch_project_tc(c, l, X, K, src_begin, n, st);
     if (rc) return rc;
@@ -544,6 +546,18 @@ extern "C" int taurus_gat_project_chunk(taurus_ctx* c, int64_t src_begin, int64_
   CU(cudaGetLastError());
   c->gat_next_src = src_end;
   return TAURUS_OK;
+}
+
+extern "C" int taurus_gat_project_chunk(taurus_ctx* c, int64_t src_begin, int64_t src_end, const float* features, float* hprime_out,
+                                        int64_t ld, void* cuda_stream) {
+  if (!features) return TAURUS_ERR_INVALID_ARG;
+  return gat_project_core(c, src_begin, src_end, features, nullptr, hprime_out, ld, cuda_stream);
+}
+
+extern "C" int taurus_gat_project_chunk_from_runs(taurus_ctx* c, int64_t src_begin, int64_t src_end, taurus_runs* runs, float* hprime_out,
+                                                  int64_t ld, void* cuda_stream) {
+  if (!runs) return TAURUS_ERR_INVALID_ARG;
+  return gat_project_core(c, src_begin, src_end, nullptr, runs, hprime_out, ld, cuda_stream);
 }
 
 extern "C" int taurus_gat_attention(taurus_ctx* c, void* cuda_stream) {

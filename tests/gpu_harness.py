@@ -49,7 +49,10 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
         if w.mode == tg.GAT:  # passes 1 and 2; pass 3 below streams the transformed rows instead of the features
             hprime = torch.empty((V, d_out), dtype=torch.float32, device=dev)
             for (s, e) in plan:
-                ctx.gat_project_chunk(s, e, feat[s:e], hprime[s:e], d_out, stream)
+                if run_output and prev_runs is not None:
+                    ctx.gat_project_chunk_from_runs(s, e, prev_runs, hprime[s:e], d_out, stream)
+                else:
+                    ctx.gat_project_chunk(s, e, feat[s:e], hprime[s:e], d_out, stream)
             ctx.gat_attention(stream)
             layer_in, feat = feat, (hprime.cpu().pin_memory() if host_features else hprime)
         if run_output:        # rows leave as sorted runs; layers after the first read their input back from runs
@@ -57,7 +60,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
             runs = tb.Runs(V, d_out, P, R, store_rows=V, max_append_rows=V, max_chunk_rows=w.chunk, store_kind=kind)
             ctx.layer_set_run_output(runs)
             for (s, e) in plan:
-                if prev_runs is None:
+                if prev_runs is None or w.mode == tg.GAT:      # GAT: pass 3 streams the transformed rows of pass 1
                     ctx.push_chunk(s, e, feat[s:e], stream)
                 else:
                     ctx.push_chunk_from_runs(s, e, prev_runs, stream)

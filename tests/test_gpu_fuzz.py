@@ -46,7 +46,7 @@ def random_config(seed):
     w = replace(w, pool_slots=pool)
     kw = dict(flags=int(rng.choice([0, 0, 2, 4, 6])), evict_policy=policy)
     out_mode = int(rng.integers(0, 6))
-    if out_mode == 4 and mode != tg.GAT:       # layers chained through sorted runs
+    if out_mode == 4:                          # layers chained through sorted runs
         import paper_2607_17374_b200 as tb
         kw["run_output"] = (int(rng.choice([1, 3, 16])), int(rng.choice([1, 50, 4000])) if g.V < 1500 else int(rng.choice([50, 4000])),
                             tb.RUNS_HOST if rng.integers(0, 2) else tb.RUNS_DEVICE)
