@@ -254,30 +254,37 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
     groups += 1;
     if (!DIRECT && l >= pool) hub_msgs += (unsigned)cnt;
   };
+  auto weight = [&](int src_rel) {   // GAT: exp(LeakyReLU(s_u + t_v) - max_v) for the current destination
+    const float e = att_s_chunk[src_rel] + cur_tm.x;
+    return __expf((e > 0.f ? e : a.leaky * e) - cur_tm.y);
+  };
   auto take = [&](int d, int src_rel, const float4 (&row)[VPL]) {
-    const bool fresh = d != cur;
-    if (fresh) {
+    if (d != cur) {
       if (cur >= 0) flush();
-      cur = d; cnt = 0;
+      cur = d; cnt = 1;
       if (!DIRECT) cur_loc = a.loc[d];
-      if (GAT) cur_tm = a.att_tm[d];
-    }
-    cnt++;
-    if (GAT) {
-      const float e = att_s_chunk[src_rel] + cur_tm.x;
-      const float w = __expf((e > 0.f ? e : a.leaky * e) - cur_tm.y);
+      if (GAT) {
+        cur_tm = a.att_tm[d];
+        const float w = weight(src_rel);
 #pragma unroll
-      for (int k = 0; k < VPL; ++k) {
-        if (fresh) sum[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        sum[k].x = fmaf(w, row[k].x, sum[k].x); sum[k].y = fmaf(w, row[k].y, sum[k].y);
-        sum[k].z = fmaf(w, row[k].z, sum[k].z); sum[k].w = fmaf(w, row[k].w, sum[k].w);
+        for (int k = 0; k < VPL; ++k) sum[k] = make_float4(w * row[k].x, w * row[k].y, w * row[k].z, w * row[k].w);
+      } else {
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) sum[k] = row[k];
       }
-    } else if (fresh) {
-#pragma unroll
-      for (int k = 0; k < VPL; ++k) sum[k] = row[k];
     } else {
+      cnt++;
+      if (GAT) {
+        const float w = weight(src_rel);
 #pragma unroll
-      for (int k = 0; k < VPL; ++k) { sum[k].x += row[k].x; sum[k].y += row[k].y; sum[k].z += row[k].z; sum[k].w += row[k].w; }
+        for (int k = 0; k < VPL; ++k) {
+          sum[k].x = fmaf(w, row[k].x, sum[k].x); sum[k].y = fmaf(w, row[k].y, sum[k].y);
+          sum[k].z = fmaf(w, row[k].z, sum[k].z); sum[k].w = fmaf(w, row[k].w, sum[k].w);
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) { sum[k].x += row[k].x; sum[k].y += row[k].y; sum[k].z += row[k].z; sum[k].w += row[k].w; }
+      }
     }
   };
   auto fetch = [&](int src_rel, float4 (&row)[VPL]) {
