@@ -396,6 +396,21 @@ int taurus_layer_set_run_output(taurus_ctx* ctx, taurus_runs* runs);
  * buffer on its copy stream, overlapping the previous chunk's kernels).  runs' width must be dims[layer]. */
 int taurus_push_chunk_from_runs(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, taurus_runs* runs, void* cuda_stream);
 
+/*
+ * Applying an ordering (Sect. 3.8: topology relabelling and feature relabelling).  rank is a permutation of
+ * [0, V), e.g. out_rank of taurus_reorder: vertex v becomes vertex rank[v].
+ * taurus_relabel_csr: row rank[u] of the output holds the out-edges of u in their original order with every
+ * destination v renamed rank[v]; out_in_degree (may be NULL) receives the in-degrees of the relabelled graph.
+ * All pointers host or device memory; blocking; TAURUS_ERR_INVALID_ARG when rank is not a permutation or a
+ * destination lies outside [0, V) (outputs then undefined).
+ * taurus_permute_rows: out_rows[rank[v]] = in_rows[v] for a [V x width] matrix (ld_in, ld_out in floats);
+ * DEVICE memory only, in_rows != out_rows, asynchronous on the stream; rank is not checked here.
+ */
+int taurus_relabel_csr(int64_t V, int64_t E, const int64_t* row_ptr, const int32_t* col_idx, const int32_t* rank,
+                       int64_t* out_row_ptr, int32_t* out_col_idx, int32_t* out_in_degree, void* cuda_stream);
+int taurus_permute_rows(int64_t V, int32_t width, const float* in_rows, int64_t ld_in, const int32_t* rank, float* out_rows,
+                        int64_t ld_out, void* cuda_stream);
+
 /* Kernels launched by this context since init (for launch accounting in benchmarks). */
 int64_t taurus_launch_count(const taurus_ctx* ctx);
 

@@ -338,6 +338,22 @@ def total_span(V: int, row_ptr: np.ndarray, col: np.ndarray, rank: np.ndarray) -
     return int((hi - lo).sum())
 
 
+def relabel_csr(V: int, row_ptr: np.ndarray, col: np.ndarray, rank: np.ndarray):
+    """The graph with vertex v renamed rank[v] (Sect. 3.8, topology relabelling): row rank[u] = the out-edges of u in
+    their original order, destinations renamed.  Returns (row_ptr, col, in_degree)."""
+    rank = np.asarray(rank, dtype=np.int64)
+    old_of_new = np.empty(V, np.int64)
+    old_of_new[rank] = np.arange(V)
+    deg = np.diff(row_ptr)
+    new_ptr = np.zeros(V + 1, np.int64)
+    np.cumsum(deg[old_of_new], out=new_ptr[1:])
+    new_col = np.empty(int(row_ptr[V]), np.int32)
+    for nu in range(V):
+        u = old_of_new[nu]
+        new_col[new_ptr[nu]:new_ptr[nu + 1]] = rank[col[row_ptr[u]:row_ptr[u + 1]]]
+    return new_ptr, new_col, np.bincount(new_col, minlength=V).astype(np.int32)
+
+
 def ranks_of(r: np.ndarray) -> np.ndarray:
     """pi = ArgSort(r), ties by vertex id; returned as the rank of every vertex."""
     order = np.argsort(r, kind="stable")

@@ -90,7 +90,7 @@ EXPORTS = [
     "taurus_runs_create", "taurus_runs_append", "taurus_runs_flush", "taurus_runs_read_chunk", "taurus_runs_info",
     "taurus_runs_directory", "taurus_runs_get_run", "taurus_runs_reset", "taurus_runs_destroy",
     "taurus_layer_set_run_output", "taurus_push_chunk_from_runs", "taurus_gat_project_chunk", "taurus_gat_attention",
-    "taurus_get_sample_digest", "taurus_gat_project_chunk_from_runs",
+    "taurus_get_sample_digest", "taurus_gat_project_chunk_from_runs", "taurus_relabel_csr", "taurus_permute_rows",
 ]
 NOALLOC_MAX_VERTICES = 4 * 1024 * 1024
 
@@ -137,6 +137,8 @@ def load_library():
     lib.taurus_gat_project_chunk.argtypes = [vp, i64, i64, vp, vp, i64, vp]
     lib.taurus_gat_attention.argtypes = [vp, vp]
     lib.taurus_gat_project_chunk_from_runs.argtypes = [vp, i64, i64, vp, vp, i64, vp]
+    lib.taurus_relabel_csr.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp, vp]
+    lib.taurus_permute_rows.argtypes = [i64, i32, vp, i64, vp, vp, i64, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -193,6 +195,25 @@ def reorder(V: int, E: int, row_ptr, col_idx, initial_rank=None, iterations: int
     if rc != 0:
         raise TaurusError(rc, "taurus_reorder")
     return rank, pos, J, span
+
+
+def relabel_csr(V: int, E: int, row_ptr, col_idx, rank, stream=None):
+    """taurus_relabel_csr.  Returns (row_ptr int64 [V+1], col_idx int32 [E], in_degree int32 [V]) as numpy arrays."""
+    new_ptr = np.empty(V + 1, np.int64)
+    new_col = np.empty(max(E, 1), np.int32)
+    new_din = np.empty(V, np.int32)
+    rc = load_library().taurus_relabel_csr(V, E, _ptr(row_ptr), _ptr(col_idx), _ptr(rank), new_ptr.ctypes.data, new_col.ctypes.data,
+                                           new_din.ctypes.data, _stream(stream))
+    if rc != 0:
+        raise TaurusError(rc, "taurus_relabel_csr")
+    return new_ptr, new_col[:E], new_din
+
+
+def permute_rows(V: int, width: int, in_rows, ld_in: int, rank, out_rows, ld_out: int, stream=None):
+    """taurus_permute_rows: out_rows[rank[v]] = in_rows[v] (device tensors)."""
+    rc = load_library().taurus_permute_rows(V, width, _ptr(in_rows), ld_in, _ptr(rank), _ptr(out_rows), ld_out, _stream(stream))
+    if rc != 0:
+        raise TaurusError(rc, "taurus_permute_rows")
 
 
 class Runs:

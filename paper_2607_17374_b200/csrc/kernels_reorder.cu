@@ -224,3 +224,116 @@ extern "C" int taurus_reorder(int64_t V, int64_t E, const int64_t* row_ptr, cons
 #undef RO
   return TAURUS_OK;
 }
+
+// ------------------------------------------------------------------------------------------------ relabelling
+// Applying an ordering (Sect. 3.8: topology relabelling and feature relabelling): vertex v becomes rank[v].
+namespace {
+
+__global__ void rl_check_kernel(long long V, const int32_t* __restrict__ rank, int32_t* __restrict__ seen, int* bad) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
+    const int r = rank[v];
+    if (r < 0 || r >= V || atomicAdd(&seen[r], 1) != 0) *bad = 1;   // not a permutation of [0, V)
+  }
+}
+__global__ void rl_degree_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ rank,
+                                 long long* __restrict__ new_ptr) {
+  long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v <= V; v += stride) {
+    if (v < V) new_ptr[rank[v]] = row_ptr[v + 1] - row_ptr[v];
+    else new_ptr[V] = 0;
+  }
+}
+// row rank[u] of the output = the out-edges of u in their original order, destinations renamed
+__global__ void rl_edges_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                                const int32_t* __restrict__ rank, const long long* __restrict__ new_ptr, int32_t* __restrict__ new_col,
+                                int32_t* __restrict__ new_din, int* bad) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    const long long b = row_ptr[u], n = row_ptr[u + 1] - b, nb = new_ptr[rank[u]];
+    for (long long k = lane(); k < n; k += 32) {
+      const int v = col[b + k];
+      if (v < 0 || v >= V) { *bad = 1; continue; }
+      const int nv = rank[v];
+      new_col[nb + k] = nv;
+      if (new_din) atomicAdd(&new_din[nv], 1);
+    }
+  }
+}
+__global__ void rl_rows_kernel(long long V, int width, const float* __restrict__ in, long long ld_in, const int32_t* __restrict__ rank,
+                               float* __restrict__ out, long long ld_out) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long v = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; v < V; v += warps) {
+    const float* src = in + (size_t)v * ld_in;
+    float* dst = out + (size_t)rank[v] * ld_out;
+    for (int k = lane(); k < width; k += 32) dst[k] = src[k];
+  }
+}
+
+}  // namespace
+
+extern "C" int taurus_relabel_csr(int64_t V, int64_t E, const int64_t* row_ptr, const int32_t* col_idx, const int32_t* rank,
+                                  int64_t* out_row_ptr, int32_t* out_col_idx, int32_t* out_in_degree, void* cuda_stream) {
+  if (V < 1 || V >= (1ll << 31) || E < 0 || E >= (1ll << 32) || !row_ptr || (E > 0 && (!col_idx || !out_col_idx)) || !rank || !out_row_ptr)
+    return TAURUS_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int sms = 148, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = sms * 8;
+  Buffers B;
+  long long* d_row = B.get<long long>((size_t)V + 1);
+  int32_t* d_col = B.get<int32_t>((size_t)E);
+  int32_t* d_rank = B.get<int32_t>((size_t)V);
+  int32_t* d_seen = B.get<int32_t>((size_t)V);
+  long long* d_nptr = B.get<long long>((size_t)V + 1);
+  int32_t* d_ncol = B.get<int32_t>((size_t)E);
+  int32_t* d_ndin = out_in_degree ? B.get<int32_t>((size_t)V) : nullptr;
+  int* d_bad = B.get<int>(1);
+  size_t tb = 0;
+  cub::DeviceScan::ExclusiveSum(nullptr, tb, d_nptr, d_nptr, V + 1, st);
+  void* d_tmp = B.get<char>(tb);
+  if (!d_row || !d_col || !d_rank || !d_seen || !d_nptr || !d_ncol || (out_in_degree && !d_ndin) || !d_bad || !d_tmp) return TAURUS_ERR_NOMEM;
+#define RL(call) do { if ((call) != cudaSuccess) { cudaGetLastError(); return TAURUS_ERR_CUDA; } } while (0)
+  RL(cudaMemcpyAsync(d_row, row_ptr, (size_t)(V + 1) * sizeof(long long), cudaMemcpyDefault, st));
+  if (E > 0) RL(cudaMemcpyAsync(d_col, col_idx, (size_t)E * sizeof(int32_t), cudaMemcpyDefault, st));
+  RL(cudaMemcpyAsync(d_rank, rank, (size_t)V * sizeof(int32_t), cudaMemcpyDefault, st));
+  RL(cudaMemsetAsync(d_seen, 0, (size_t)V * sizeof(int32_t), st));
+  RL(cudaMemsetAsync(d_bad, 0, sizeof(int), st));
+  if (d_ndin) RL(cudaMemsetAsync(d_ndin, 0, (size_t)V * sizeof(int32_t), st));
+  rl_check_kernel<<<grid, 256, 0, st>>>(V, d_rank, d_seen, d_bad);
+  int bad = 0;
+  RL(cudaMemcpyAsync(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, st));
+  RL(cudaStreamSynchronize(st));
+  if (bad) return TAURUS_ERR_INVALID_ARG;      // before any index derived from rank is used as an address
+  rl_degree_kernel<<<grid, 256, 0, st>>>(V, d_row, d_rank, d_nptr);
+  RL(cub::DeviceScan::ExclusiveSum(d_tmp, tb, d_nptr, d_nptr, V + 1, st));
+  rl_edges_kernel<<<grid, 256, 0, st>>>(V, d_row, d_col, d_rank, d_nptr, d_ncol, d_ndin, d_bad);
+  RL(cudaMemcpyAsync(&bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, st));
+  RL(cudaMemcpyAsync(out_row_ptr, d_nptr, (size_t)(V + 1) * sizeof(long long), cudaMemcpyDefault, st));
+  if (E > 0) RL(cudaMemcpyAsync(out_col_idx, d_ncol, (size_t)E * sizeof(int32_t), cudaMemcpyDefault, st));
+  if (out_in_degree) RL(cudaMemcpyAsync(out_in_degree, d_ndin, (size_t)V * sizeof(int32_t), cudaMemcpyDefault, st));
+  RL(cudaStreamSynchronize(st));
+  RL(cudaGetLastError());
+  return bad ? TAURUS_ERR_INVALID_ARG : TAURUS_OK;
+#undef RL
+}
+
+extern "C" int taurus_permute_rows(int64_t V, int32_t width, const float* in_rows, int64_t ld_in, const int32_t* rank, float* out_rows,
+                                   int64_t ld_out, void* cuda_stream) {
+  if (V < 1 || V >= (1ll << 31) || width < 1 || !in_rows || !rank || !out_rows || ld_in < width || ld_out < width || in_rows == out_rows)
+    return TAURUS_ERR_INVALID_ARG;
+  cudaPointerAttributes a_in, a_out, a_rank;
+  if (cudaPointerGetAttributes(&a_in, in_rows) != cudaSuccess || cudaPointerGetAttributes(&a_out, out_rows) != cudaSuccess ||
+      cudaPointerGetAttributes(&a_rank, rank) != cudaSuccess || a_in.type != cudaMemoryTypeDevice || a_out.type != cudaMemoryTypeDevice ||
+      a_rank.type != cudaMemoryTypeDevice) {
+    cudaGetLastError();
+    return TAURUS_ERR_INVALID_ARG;             // device memory only: the matrices are too large to stage
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int sms = 148, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  rl_rows_kernel<<<sms * 8, 256, 0, st>>>(V, width, in_rows, ld_in, rank, out_rows, ld_out);
+  return cudaGetLastError() == cudaSuccess ? TAURUS_OK : TAURUS_ERR_CUDA;
+}

@@ -75,3 +75,39 @@ def test_five_iterations_reduce_the_span_of_a_scrambled_banded_graph():
     assert sorted(rank.tolist()) == list(range(g.V))
     assert hist[-1][1] < 0.85 * hist[0][1] and hist[-1][0] < hist[0][0]
     assert hist[1][1] < hist[0][1]
+
+
+def test_relabelling_is_an_isomorphism():
+    """Relabelled graph: same edges under the renaming, inverse relabelling restores the original, and a GNN layer
+    on the relabelled graph with permuted features gives the permuted outputs (message passing does not depend on
+    the names of the vertices)."""
+    rng = np.random.default_rng(21)
+    V, E = 300, 2500
+    src = np.sort(rng.integers(0, V, E))
+    col = rng.integers(0, V, E).astype(np.int32)
+    row_ptr = np.zeros(V + 1, np.int64)
+    np.cumsum(np.bincount(src, minlength=V), out=row_ptr[1:])
+    rank = rng.permutation(V).astype(np.int32)
+    p2, c2, d2 = oracle.relabel_csr(V, row_ptr, col, rank)
+    # the same multiset of edges under the renaming
+    old_edges = sorted(zip(rank[src].tolist(), rank[col].tolist()))
+    src2 = np.repeat(np.arange(V), np.diff(p2))
+    assert sorted(zip(src2.tolist(), c2.tolist())) == old_edges
+    assert np.array_equal(d2, np.bincount(rank[col], minlength=V))
+    # the inverse renaming restores the original arrays exactly (edge order inside a row is kept)
+    inv = np.empty(V, np.int32); inv[rank] = np.arange(V, dtype=np.int32)
+    p3, c3, _ = oracle.relabel_csr(V, p2, c2, inv)
+    assert np.array_equal(p3, row_ptr) and np.array_equal(c3, col)
+    ident = np.arange(V, dtype=np.int32)
+    p4, c4, _ = oracle.relabel_csr(V, row_ptr, col, ident)
+    assert np.array_equal(p4, row_ptr) and np.array_equal(c4, col)
+    # one exact SAGE layer: out'[rank[v]] == out[v]
+    h = rng.normal(size=(V, 6)); Wn = rng.normal(size=(6, 4)); Ws = rng.normal(size=(6, 4)); b = rng.normal(size=4)
+    def layer(rp, cc, x):
+        inl = oracle.build_in_lists(V, rp, cc)
+        ms = oracle.message_sets(inl, 0, 1, 0)
+        return oracle.layer_forward(ms, oracle.SAGE_MEAN, np.diff(inl.ptr), np.diff(rp), x, Wn, Ws, b, 1)
+    out = layer(row_ptr, col, h)
+    h2 = np.empty_like(h); h2[rank] = h
+    out2 = layer(p2, c2, h2)
+    assert np.allclose(out2[rank], out, rtol=1e-12, atol=1e-12)
