@@ -45,6 +45,8 @@ def random_config(seed):
         pool = int(pool * 1.3) + 1
     w = replace(w, pool_slots=pool)
     kw = dict(flags=int(rng.choice([0, 0, 2, 4, 6])), evict_policy=policy)
+    if mode != tg.GAT and L <= 2 and rng.integers(0, 8) == 0:
+        kw["gemm_mode"] = tg.GEMM_BF16          # bf16 operands, fp32 accumulate
     out_mode = int(rng.integers(0, 6))
     if out_mode == 4:                          # layers chained through sorted runs
         import paper_2607_17374_b200 as tb
@@ -84,13 +86,18 @@ def test_random_configuration(seed):
     orc = run_oracle(w, g, model, x0, kw["evict_policy"])
     for l in range(w.L):
         row, elem_max, _ = row_error(lib["outs"][l], orc["outs"][l])
-        if w.dims[l + 1] >= (32 if w.mode == tg.GAT else 16):   # attention adds the exponent's rounding to every term
-            assert row <= 1e-4, (l, row, elem_max)
+        # The row-wise bound presumes rows that are not dominated by cancellation: a layer fed by one or a few input
+        # columns produces rows that are all multiples of a few near-cancelling sums, a row of a few output columns can
+        # have every entry small, and attention adds the rounding of an exponent to every term.  Those layers are
+        # gated on the layer's own scale instead; outputs of well-conditioned layers on the row-wise bound.
+        bf16 = kw.get("gemm_mode") == tg.GEMM_BF16 and not (kw["flags"] & 2)
+        wide = min(w.dims[l], w.dims[l + 1]) >= (32 if bf16 else 16) and (w.mode != tg.GAT or w.dims[l + 1] >= 64)
+        tol = 2e-2 if bf16 else 1e-4
+        if wide:
+            assert row <= tol, (l, row, elem_max)
         else:
-            # a row of a few columns can have all its entries small through cancellation, and then no fp32 sum of
-            # several hundred terms meets a bound relative to that row: gate such layers on the layer's own scale
             scale = np.abs(orc["outs"][l]).max() + 1e-6
-            assert np.abs(lib["outs"][l] - orc["outs"][l]).max() <= 1e-4 * scale, (l, row, elem_max)
+            assert np.abs(lib["outs"][l] - orc["outs"][l]).max() <= tol * scale, (l, row, elem_max)
         assert orc["sims"][l].rc == 0 or kw.get("chunk_plan")
         assert np.array_equal(lib["digests"][l], oracle.sample_digest(orc["msets"][l]))   # the propagated in-edge sets, all V
         completed = lib["completed"][l]
