@@ -45,6 +45,8 @@ def parse_args():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--simt-gemm", action="store_true", help="use the plain FFMA projection kernel")
     p.add_argument("--no-grouping", action="store_true", help="CSR-order scatter for every chunk")
+    p.add_argument("--pool-fraction", type=float, default=0.0,
+                   help="accumulator pool as a fraction of V (0 = the workload's own pool); below the peak active set it forces eviction")
     p.add_argument("--model", default="", choices=["", "sage", "gcn", "gin", "gat"],
                    help="aggregation of every layer (default: the workload's); gat runs its three passes per layer")
     p.add_argument("--output", default="dense", choices=["dense", "runs-device", "runs-host"],
@@ -57,6 +59,9 @@ def workload_of(args):
     w = tg.WORKLOADS[args.workload]
     if args.vertices:
         w = tg.scaled(w, args.vertices)
+    if args.pool_fraction > 0:
+        from dataclasses import replace
+        w = replace(w, pool_slots=max(1, int(w.V * args.pool_fraction)))
     if args.model:
         from dataclasses import replace
         w = replace(w, mode={"sage": tg.SAGE_MEAN, "gcn": tg.GCN_SYM, "gin": tg.GIN_SUM, "gat": tg.GAT}[args.model],
