@@ -47,6 +47,8 @@ def parse_args():
     p.add_argument("--no-grouping", action="store_true", help="CSR-order scatter for every chunk")
     p.add_argument("--pool-fraction", type=float, default=0.0,
                    help="accumulator pool as a fraction of V (0 = the workload's own pool); below the peak active set it forces eviction")
+    p.add_argument("--evict-policy", default="fewest", choices=["fewest", "fifo", "lru", "random"],
+                   help="which IN_BUFFER rows leave first when the pool is full (the paper's policy and its ablation's alternatives)")
     p.add_argument("--model", default="", choices=["", "sage", "gcn", "gin", "gat"],
                    help="aggregation of every layer (default: the workload's); gat runs its three passes per layer")
     p.add_argument("--output", default="dense", choices=["dense", "runs-device", "runs-host"],
@@ -241,7 +243,8 @@ def run_ours(args):
     flags = (tb.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (tb.FLAG_NO_GROUPING if args.no_grouping else 0)
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags,
-                     0, w.gin_eps, model.att_src, model.att_dst, w.leaky_slope)
+                     {"fewest": 0, "fifo": 1, "lru": 2, "random": 3}[args.evict_policy], w.gin_eps, model.att_src, model.att_dst,
+                     w.leaky_slope)
     gat = w.mode == tg.GAT
     use_runs = args.output != "dense"
     hprime = torch.zeros((V, max(w.dims[1:])), dtype=torch.float32, device=dev) if gat else None
@@ -404,7 +407,7 @@ def run_ours(args):
                     vs_baseline=None, dtype="f32", data="synthetic",
                     config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=w.chunk, chunks_per_layer=len(chunks),
                                 pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
-                                mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], output=args.output,
+                                mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], output=args.output, evict_policy=args.evict_policy,
                                 messages_per_step=msgs_per_step,
                                 l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
                                 parallelism="replicas only" if world > 1 else "1 gpu",
