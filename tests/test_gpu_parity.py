@@ -320,3 +320,31 @@ def test_gin_sum_mode():
     w = replace(w, mode=tg.GIN_SUM, gin_eps=0.25, dims=(96, 128, 32), fanout=(0, 0), pool_slots=20_000, hub_count=40)
     _full_check(w)
     _full_check(replace(w, fanout=(6, 3)), flags=4)      # sampled, CSR-order kernels
+
+
+@pytest.mark.parametrize("mode", [tg.SAGE_MEAN, tg.GCN_SYM, tg.GAT])
+def test_smallest_and_edgeless_graphs(mode):
+    """Degenerate inputs: a graph without edges (every vertex completes on its self message alone), a single vertex
+    with and without a self-loop, a two-vertex multigraph, chunks of one source, a pool of one slot per vertex."""
+    from dataclasses import replace
+    cases = [
+        (5, []),                                        # no edges at all
+        (1, []),                                        # one vertex
+        (1, [(0, 0), (0, 0)]),                          # one vertex, a double self-loop
+        (2, [(0, 1), (0, 1), (1, 0), (1, 1)]),          # multi-edges and a self-loop
+        (40, [(u, (u + 1) % 40) for u in range(40)]),   # a ring, one source per chunk
+    ]
+    from helpers import csr_from_edges
+    for V, edges in cases:
+        row_ptr, col = csr_from_edges(V, edges)
+        g = tg.Graph(V, len(edges), row_ptr, col, np.bincount(col, minlength=V).astype(np.int32) if edges else np.zeros(V, np.int32))
+        for chunk in (1, 64):
+            w = replace(tg.WORKLOADS["tiny"], V=V, E=g.E, mode=mode, dims=(8, 12, 4), fanout=(0, 1), chunk=chunk, pool_slots=V, hub_count=0)
+            model = tg.make_model(w, bias_scale=0.3)
+            x0 = tg.features(w.seed, 0, 0, V, 8)
+            lib = run_library(w, g, model, x0)
+            orc = run_oracle(w, g, model, x0)
+            for l in range(w.L):
+                scale = np.abs(orc["outs"][l]).max() + 1e-6
+                assert np.abs(lib["outs"][l] - orc["outs"][l]).max() <= 1e-4 * scale, (V, edges, chunk, l)
+                check_accounting(lib["stats"][l], lib["chunk_log"][l], lib["reload_count"][l], orc["sims"][l], lib["completed"][l])
