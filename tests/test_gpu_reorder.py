@@ -120,3 +120,17 @@ def test_reordered_graph_runs_through_the_hot_path():
     assert row_error(outs[1][rank], ref1)[0] <= 1e-4          # the reordered run gives the same rows under the renaming
     print("evictions scrambled %d -> reordered %d" % tuple(evictions))
     assert evictions[1] < evictions[0]
+
+
+def test_reorder_and_relabel_on_edgeless_and_single_vertex_graphs():
+    import oracle
+    import paper_2607_17374_b200 as tb
+    for V in (1, 5):
+        row_ptr = np.zeros(V + 1, np.int64)
+        col = np.zeros(1, np.int32)[:0]
+        start = np.arange(V, dtype=np.int32)[::-1].copy()
+        rank, pos, J, span = tb.reorder(V, 0, row_ptr, col, start, 3)
+        want_rank, _, _ = oracle.reorder(V, row_ptr, col, start, 3)
+        assert np.array_equal(rank, want_rank) and (span == 0).all() and np.allclose(J, 0.0)
+        p, c, d = tb.relabel_csr(V, 0, row_ptr, col, rank)
+        assert np.array_equal(p, row_ptr) and c.size == 0 and (d == 0).all()
