@@ -348,3 +348,14 @@ def test_smallest_and_edgeless_graphs(mode):
                 scale = np.abs(orc["outs"][l]).max() + 1e-6
                 assert np.abs(lib["outs"][l] - orc["outs"][l]).max() <= 1e-4 * scale, (V, edges, chunk, l)
                 check_accounting(lib["stats"][l], lib["chunk_log"][l], lib["reload_count"][l], orc["sims"][l], lib["completed"][l])
+
+
+@pytest.mark.parametrize("mode", [tg.SAGE_MEAN, tg.GAT])
+def test_maximum_widths_and_fanout(mode):
+    """Rows of 1 024 floats in and out (the largest the library takes), a 512-wide last layer, fanout 64."""
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 6_000, chunk=512)
+    w = replace(w, mode=mode, dims=(1024, 1024, 512), fanout=(0, 64), pool_slots=5_000, hub_count=6)
+    for flags in (0, 4):
+        lib, _ = _full_check(w, flags=flags)
+    assert lib["stats"][0]["evictions"] > 0
