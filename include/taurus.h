@@ -121,7 +121,12 @@ enum {
 
 enum {
   TAURUS_FLAG_SIMT_GEMM = 2,    /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */
-  TAURUS_FLAG_NO_GROUPING = 4   /* do not build the destination-grouped edge order: every chunk takes the CSR-order kernels */
+  TAURUS_FLAG_NO_GROUPING = 4,  /* do not build the destination-grouped edge order: every chunk takes the CSR-order kernels */
+  TAURUS_FLAG_PROJECT_FIRST = 8 /* always project a chunk before scattering it.  Without this flag a SAGE / GCN / GIN layer whose
+                                   input rows are at most 3/4 as wide as its output rows aggregates the (scaled) input rows and
+                                   applies the weights to the finished rows instead (exact by linearity, Sect. 3.6 / 3.9): the
+                                   accumulators, the scatter traffic and every evicted row shrink by d_in / d_out.  SAGE layers
+                                   do so only when the per-vertex store of x_v W_self (V x d_out floats) stays below 16 GiB */
 };
 
 /* Integer accounting of one layer pass (Sect. 4.4-4.7 report these quantities). */

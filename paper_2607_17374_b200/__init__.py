@@ -6,5 +6,5 @@ library (python -m paper_2607_17374_b200.build) and a CUDA device.
 """
 from .binding import (  # noqa: F401
     Context, Runs, RUNS_HOST, RUNS_DEVICE, TaurusError, Stats, library_path, load_library, completion_counts_noalloc, NOALLOC_MAX_VERTICES, reorder, relabel_csr, permute_rows,
-    SAGE_MEAN, GCN_SYM, GIN_SUM, GAT, GEMM_FP32, GEMM_BF16, FLAG_SIMT_GEMM, FLAG_NO_GROUPING, EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM, CHUNK_LOG_COLUMNS, ERROR_CODES,
+    SAGE_MEAN, GCN_SYM, GIN_SUM, GAT, GEMM_FP32, GEMM_BF16, FLAG_SIMT_GEMM, FLAG_NO_GROUPING, FLAG_PROJECT_FIRST, EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM, CHUNK_LOG_COLUMNS, ERROR_CODES,
 )

@@ -10,7 +10,7 @@ import numpy as np
 
 SAGE_MEAN, GCN_SYM, GIN_SUM, GAT = 0, 1, 2, 3
 GEMM_FP32, GEMM_BF16 = 0, 1
-FLAG_SIMT_GEMM, FLAG_NO_GROUPING = 2, 4
+FLAG_SIMT_GEMM, FLAG_NO_GROUPING, FLAG_PROJECT_FIRST = 2, 4, 8
 EVICT_FEWEST_PENDING, EVICT_FIFO, EVICT_LRU, EVICT_RANDOM = 0, 1, 2, 3
 CHUNK_LOG_COLUMNS = ["hs", "ns", "ev", "gs", "need", "evicted", "reloaded", "completed", "occupancy"]
 ERROR_CODES = {

@@ -1,0 +1,154 @@
+// Aggregate-first layers.  When a layer's input rows are narrower than its output rows, the accumulators hold
+// sums of (scaled) INPUT rows and the weight matrix is applied to the finished rows, as the paper's graduation
+// processor does (Sect. 3.6; the split W = [W_agg  W_self] of the SAGEConv paragraph in Sect. 3.9 is what makes it
+// exact): by linearity
+//     c_in(v) * sum_u c_out(u) (h_u W)  =  (c_in(v) * sum_u c_out(u) h_u) W,
+// and the read-modify-write traffic of the scatter, the pool and every evicted row shrink by d_in / d_out.
+//   push     : S_u = c_out(u) h_u (padded to a multiple of 4 columns) is what the scatter pushes;
+//              GCN / GIN add the self message in input space (c_out(v) h_v, or (1 + eps) h_v: one shared matrix);
+//              SAGE keeps T_v = h_v W_self in a per-vertex store from v's own chunk until v completes.
+//   finalise : A_i = c_in(v_i) * acc(v_i) gathered for the completed vertices, O = A W_neigh on the tensor cores,
+//              out = act(O_i + T_v + b).
+#include "taurus_internal.h"
+
+namespace {
+
+__device__ __forceinline__ int al() { return threadIdx.x & 31; }
+__device__ __forceinline__ int af_messages(int din, int fanout) { return (fanout > 0 && din > fanout) ? fanout : din; }
+
+// S[r][k] = c_out(u) * X[r][k] for k < K, 0 for the padding columns; u = src_begin + r.
+__global__ void af_prep_kernel(const float* __restrict__ X, int ldx, int n, int K, int Kp, long long src_begin, int mode,
+                               const long long* __restrict__ row_ptr, float* __restrict__ S) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    float scale = 1.0f;
+    if (mode == TAURUS_GCN_SYM) {
+      const long long u = src_begin + r;
+      scale = (float)(1.0 / sqrt((double)(row_ptr[u + 1] - row_ptr[u]) + 1.0));
+    }
+    const float* src = X + (size_t)r * ldx;
+    float* dst = S + (size_t)r * Kp;
+    for (int k = al(); k < Kp; k += 32) dst[k] = k < K ? src[k] * scale : 0.f;
+  }
+}
+
+// A[i] = c_in(v_i) * acc(v_i) for the completed vertices, zero rows up to `rows` (the row count the host sized the
+// transform for).  The slot is released by compact_done_kernel; its row stays intact until the next chunk.
+__global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long rows) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const int n = ctl->done_count;
+  const int vec = a.Hp >> 2;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < rows; i += warps) {
+    float4* dst = reinterpret_cast<float4*>(A + (size_t)i * a.Hp);
+    if (i >= n) {
+      for (int k = al(); k < vec; k += 32) dst[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      continue;
+    }
+    const int v = a.done_list[i];
+    const int l = a.loc[v];
+    float scale = 1.0f;
+    if (a.mode == TAURUS_SAGE_MEAN) {
+      const int m = af_messages(a.din[v], a.fanout);
+      scale = 1.0f / (float)(m > 1 ? m : 1);
+    } else if (a.mode == TAURUS_GCN_SYM) {
+      scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+    }
+    const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
+    for (int k = al(); k < vec; k += 32) {
+      float4 x = src[k];
+      x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
+      dst[k] = x;
+    }
+  }
+}
+
+// out = act(O_i + T_v + b) into the graduation buffer or straight into the caller's vertex-ordered matrix.
+// O has pitch a.Hout; rows of the graduation buffer too.
+__global__ void af_finish_kernel(ChunkArgs a, const float* __restrict__ O, const float* __restrict__ T, long long rows) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const int n = ctl->done_count;
+  if (n > rows) {   // the host sized the transform for fewer rows than completed: its bound was wrong
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+    return;
+  }
+  const long long base = a.dense_half >= 0 ? a.grad_off : ctl->grad_count;
+  const long long limit = a.dense_half >= 0 ? a.grad_off + a.grad_cap : a.drain_rows;
+  const int vec = a.Hout >> 2;
+  const bool vec_ok = a.dense_direct && (a.dense_ld & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dense_direct) & 15) == 0;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    if (!a.dense_direct && base + i >= limit) {
+      if (al() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+      continue;
+    }
+    const int v = a.done_list[i];
+    const float4* __restrict__ o = reinterpret_cast<const float4*>(O + (size_t)i * a.Hout);
+    const float4* __restrict__ t = T ? reinterpret_cast<const float4*>(T + (size_t)v * a.Hout) : nullptr;
+    const float4* __restrict__ b = reinterpret_cast<const float4*>(a.bias);
+    float* __restrict__ drow = a.dense_direct ? a.dense_direct + (size_t)v * a.dense_ld : a.grad_rows + (size_t)(base + i) * a.Hout;
+    for (int k = al(); k < vec; k += 32) {
+      float4 y = o[k];
+      const float4 bb = b[k];
+      y.x += bb.x; y.y += bb.y; y.z += bb.z; y.w += bb.w;
+      if (t) { const float4 tt = t[k]; y.x += tt.x; y.y += tt.y; y.z += tt.z; y.w += tt.w; }
+      if (a.act) { y.x = fmaxf(y.x, 0.f); y.y = fmaxf(y.y, 0.f); y.z = fmaxf(y.z, 0.f); y.w = fmaxf(y.w, 0.f); }
+      const int c0 = k << 2;
+      if (!a.dense_direct || (vec_ok && c0 + 3 < a.d_out)) {
+        reinterpret_cast<float4*>(drow)[k] = y;
+      } else {
+        if (c0 < a.d_out) drow[c0] = y.x;
+        if (c0 + 1 < a.d_out) drow[c0 + 1] = y.y;
+        if (c0 + 2 < a.d_out) drow[c0 + 2] = y.z;
+        if (c0 + 3 < a.d_out) drow[c0 + 3] = y.w;
+      }
+    }
+    if (al() == 0) {
+      a.state[v] = TAURUS_COMPLETED;
+      if (!a.dense_direct) a.grad_ids[base + i] = v;
+    }
+  }
+}
+
+}  // namespace
+
+void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, cudaStream_t st) {
+  af_prep_kernel<<<c->sm_count * 8, 256, 0, st>>>(X, ldx, n, K, Kp, src_begin, c->mode, c->d_row_ptr, c->d_PT);
+  c->launches += 1;
+}
+
+// S6 + S7 of an aggregate-first layer: compact, gather, transform, finish, commit.  `rows` is the host's bound on the
+// vertices this chunk completes (the transform is sized for it; rows beyond the actual count are zero).
+int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long rows, cudaStream_t st) {
+  launch_compact_done(c, a, st);
+  if (rows > 0) {
+    const int grid = c->sm_count * 8;
+    float* O;
+    if (a.dense_direct) O = c->d_grad_rows;
+    else if (a.dense_half >= 0) O = c->d_grad_rows + (size_t)a.grad_off * a.Hout;
+    else {
+      if (!c->d_af_O) {   // the place in the graduation buffer is known only on the device: transform into a scratch matrix
+        if (cudaMalloc((void**)&c->d_af_O, (size_t)c->drain_rows * c->Hmax * sizeof(float)) != cudaSuccess) {
+          cudaGetLastError();
+          c->d_af_O = nullptr;
+          return TAURUS_ERR_NOMEM;
+        }
+      }
+      O = c->d_af_O;
+    }
+    af_gather_kernel<<<grid, 256, 0, st>>>(a, c->d_af_A, rows);
+    c->launches += 1;
+    if (gemm_plain_tc_usable(c, layer, c->d_af_A, a.Hp, O, a.Hout)) {
+      int rc = launch_gemm_plain_tc(c, layer, 0, a.Hout, c->d_af_A, a.Hp, a.Hp, (int)rows, O, a.Hout, st);
+      if (rc) return rc;
+    } else {
+      launch_gemm_plain_simt(c, layer, 0, a.Hout, c->d_af_A, a.Hp, c->dims[layer], (int)rows, O, a.Hout, st);
+    }
+    af_finish_kernel<<<grid, 256, 0, st>>>(a, O, c->mode == TAURUS_SAGE_MEAN ? c->d_af_T : nullptr, rows);
+    c->launches += 1;
+  }
+  launch_commit(c, a, st);
+  return TAURUS_OK;
+}

@@ -14,7 +14,7 @@
 #define BK 16
 
 __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restrict__ X, int ldx, int K, const float* __restrict__ W,
-                                                           int N, float* __restrict__ PT, int n, int Hp, int mode,
+                                                           int ldw, int N, float* __restrict__ PT, long long ldo, int n, int Hp, int mode,
                                                            const float* __restrict__ bias, const long long* __restrict__ row_ptr,
                                                            const int32_t* __restrict__ din, int fanout, long long src_begin) {
   __shared__ float sA[BK][BM + 1];
@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restri
     for (int i = threadIdx.x; i < BK * BN; i += 256) {
       int k = i / BN, cidx = i % BN;
       int gk = k0 + k, gc = col0 + cidx;
-      sB[k][cidx] = (gk < K && gc < N) ? W[(size_t)gk * N + gc] : 0.f;
+      sB[k][cidx] = (gk < K && gc < N) ? W[(size_t)gk * ldw + gc] : 0.f;
     }
     __syncthreads();
 #pragma unroll
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restri
       float x = acc[i][j];
       if (cidx < Hp) x *= c_out;
       else if (mode != TAURUS_GAT) x = (x + bias[cidx - Hp]) * self_mul;   // GAT: the attention scalars as they are
-      PT[(size_t)r * N + cidx] = x;
+      PT[(size_t)r * ldo + cidx] = x;
     }
   }
 }
@@ -77,7 +77,18 @@ void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long
   const int Hp = taurus_round_up(c->dims[layer + 1], 4);
   const int N = taurus_proj_width(c->mode, Hp);
   dim3 grid((N + BN - 1) / BN, (n + BM - 1) / BM);
-  project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, c->dims[layer], c->d_Wcat[layer], N, c->d_PT, n, Hp, c->mode,
+  project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, c->dims[layer], c->d_Wcat[layer], N, N, c->d_PT, N, n, Hp, c->mode,
                                             c->d_bias[layer], c->d_row_ptr, c->d_din, c->fanout[layer], src_begin);
+  c->launches += 1;
+}
+
+// out[n x N] (pitch ld_out) = X[n x K] (pitch ldx) . columns [col0, col0 + N) of the layer's weight matrix, no epilogue.
+void launch_gemm_plain_simt(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out,
+                            long long ld_out, cudaStream_t st) {
+  const int Hp = taurus_round_up(c->dims[layer + 1], 4);
+  const int ldw = taurus_proj_width(c->mode, Hp);
+  dim3 grid((N + BN - 1) / BN, (n + BM - 1) / BM);
+  project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, K, c->d_Wcat[layer] + col0, ldw, N, out, ld_out, n, N, TAURUS_GIN_SUM, c->d_bias[layer],
+                                            c->d_row_ptr, c->d_din, 0, 0);
   c->launches += 1;
 }

@@ -485,3 +485,56 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   c->launches += 1;
   return TAURUS_OK;
 }
+
+// Plain product on the tensor cores: out[n x N] (pitch ld_out floats) = X[n x K] (pitch ldx) . columns
+// [col0, col0 + N) of the layer's weight image, no epilogue scaling (used when a layer aggregates raw rows
+// first and transforms the finished rows afterwards).  col0 and N are multiples of 4.
+bool gemm_plain_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx, const float* out, long long ld_out) {
+  if (c->flags & TAURUS_FLAG_SIMT_GEMM) return false;
+  if (!c->tc_image[layer] || !encode_fn()) return false;
+  if ((ldx & 3) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0) return false;
+  if ((ld_out & 3) != 0 || (reinterpret_cast<uintptr_t>(out) & 15) != 0) return false;
+  return true;
+}
+
+int launch_gemm_plain_tc(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
+                         cudaStream_t st) {
+  if (n <= 0) return TAURUS_OK;
+  const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
+  WImage* w = static_cast<WImage*>(c->tc_image[layer]);
+  const int rows_left = w->Np - col0;                       // image rows (= output columns) from col0 on
+  const int Np = std::min(taurus_round_up(N, 16), rows_left);
+  const int bw = Np < BN_MAX ? Np : BN_MAX;
+  const int elem = bf16 ? 2 : 4;
+  CUtensorMap map_x, map_out, map_hi, map_lo;
+  if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, 32)) return TAURUS_ERR_CUDA;
+  if (!make_map(&map_out, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, N, ld_out, 32, 32)) return TAURUS_ERR_CUDA;
+  const char* hi = static_cast<const char*>(w->hi) + (size_t)col0 * w->Kp * elem;
+  if (!make_map(&map_hi, hi, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, elem, rows_left, w->Kp, w->Kp, bw,
+                bf16 ? 64 : 32))
+    return TAURUS_ERR_CUDA;
+  map_lo = map_hi;
+  if (!bf16) {
+    const char* lo = static_cast<const char*>(w->lo) + (size_t)col0 * w->Kp * elem;
+    if (!make_map(&map_lo, lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, rows_left, w->Kp, w->Kp, bw, 32)) return TAURUS_ERR_CUDA;
+  }
+  GemmArgs g;
+  g.PT = out; g.n = n; g.N = N; g.Np = Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
+  g.b_box_bytes = bw * 128;
+  g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = c->d_bias[layer];
+  g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = 0; g.ctl = c->d_ctl;
+  const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
+  const int n_tiles = (n + BM - 1) / BM;
+  const int n_units = n_tiles * ((Np + BN_MAX - 1) / BN_MAX);
+  const int grid = n_units < c->sm_count ? n_units : c->sm_count;
+  if (!c->tc_smem_set) {
+    cudaError_t e = bf16 ? cudaFuncSetAttribute(project_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                         : cudaFuncSetAttribute(project_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) { cudaGetLastError(); return TAURUS_ERR_CUDA; }
+    c->tc_smem_set = true;
+  }
+  if (bf16) project_tc_kernel<true><<<grid, NUM_THREADS, smem, st>>>(map_x, map_hi, map_lo, map_out, g);
+  else project_tc_kernel<false><<<grid, NUM_THREADS, smem, st>>>(map_x, map_hi, map_lo, map_out, g);
+  c->launches += 1;
+  return TAURUS_OK;
+}

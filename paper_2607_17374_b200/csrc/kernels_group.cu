@@ -344,7 +344,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
       const int j = step + sub;
       const int lj = __shfl_sync(FULL, l, j);
       const int vj = __shfl_sync(FULL, v, j);
-      if (lj < 0) continue;
+      if (lj < 0 || !a.self_rows) continue;   // aggregate-first SAGE: the self message is only counted here
       const float* p = a.PT + (size_t)(vj - a.src_begin) * a.ldpt;
       float* dst = a.acc + (size_t)lj * a.Hp;
       if (a.mode == TAURUS_SAGE_MEAN) {
@@ -364,6 +364,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
           ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
           sc = a.att_z[vj];
         }
+        if (!a.self_bias) sc = 0.f;             // aggregate-first: the bias is added after the transform
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) {

@@ -126,6 +126,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
         const long long sj = __shfl_sync(FULL, src, j);
         const float wj = __shfl_sync(FULL, wgt, j);
         if (lj < 0) continue;
+        if (self_run && !a.self_rows) continue;   // aggregate-first SAGE: the self message is only counted
         if (sj != held) {
           held = sj;
           const float* p = a.PT + (size_t)(sj - a.src_begin) * a.ldpt;
@@ -147,6 +148,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
                 ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
                 s = a.att_z[sj];
               }
+              if (!a.self_bias) s = 0.f;          // aggregate-first: the bias is added after the transform
 #pragma unroll
               for (int k = 0; k < VPL; ++k)
                 if (c4 + k * LPE < nvec) {

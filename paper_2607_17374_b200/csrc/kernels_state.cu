@@ -55,7 +55,8 @@ void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st) {
                                                 c->d_touch, c->d_reload, c->pool_slots >= c->V ? 1 : 0);
   reset_pool_kernel<<<blocks, 256, 0, st>>>(c->pool_slots, c->host_rows, c->hub_count, c->d_hub_ids, c->d_loc, c->d_owner,
                                             c->d_free_stack, c->d_host_free, c->d_ctl);
-  int Hp = taurus_round_up(c->dims[layer + 1], 4);
+  // accumulator rows are as wide as what the scatter pushes: input rows in aggregate-first layers, output rows otherwise
+  int Hp = taurus_round_up(c->agg_first[layer] ? c->dims[layer] : c->dims[layer + 1], 4);
   if (c->hub_count > 0)
     cudaMemsetAsync(c->d_acc + (size_t)c->pool_slots * Hp, 0, (size_t)c->hub_count * Hp * sizeof(float), st);
   c->launches += 2;
@@ -516,6 +517,15 @@ __global__ void commit_kernel(ChunkArgs a) {
   ctl->chunks = c + 1;
   ctl->hs = ctl->ns = ctl->ev = ctl->gs = 0;
   ctl->need_count = 0; ctl->done_count = 0; ctl->touched_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;
+}
+
+void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  compact_done_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
+  c->launches += 1;
+}
+void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  commit_kernel<<<1, 32, 0, st>>>(a);
+  c->launches += 1;
 }
 
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {

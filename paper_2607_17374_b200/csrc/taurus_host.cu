@@ -73,6 +73,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
+  cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_T);
   cudaFree(c->d_att_s); cudaFree(c->d_att_t); cudaFree(c->d_att_max); cudaFree(c->d_att_tm); cudaFree(c->d_att_z);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
   cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
@@ -223,6 +224,21 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   ALLOC(c->d_PT, (size_t)c->chunk_sources * 2 * c->Hmax);
   if (c->mode == TAURUS_GAT) { ALLOC(c->d_att_s, V); ALLOC(c->d_att_t, V); ALLOC(c->d_att_max, V); ALLOC(c->d_att_tm, V); ALLOC(c->d_att_z, V); }
+  // aggregate-first layers: input rows at most 3/4 as wide as output rows
+  {
+    int af_kmax = 0, af_hmax = 0;
+    for (int l = 0; l < c->L; ++l) {
+      const int Kp = taurus_round_up(c->dims[l], 4), Hp = taurus_round_up(c->dims[l + 1], 4);
+      bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && c->mode != TAURUS_GAT && 4 * Kp <= 3 * Hp;
+      if (af && c->mode == TAURUS_SAGE_MEAN && (size_t)V * Hp * sizeof(float) > ((size_t)16 << 30)) af = false;
+      c->agg_first[l] = af;
+      if (af) { af_kmax = std::max(af_kmax, Kp); af_hmax = std::max(af_hmax, Hp); }
+    }
+    if (af_kmax > 0) {
+      ALLOC(c->d_af_A, (size_t)c->drain_rows * af_kmax);
+      if (c->mode == TAURUS_SAGE_MEAN) ALLOC(c->d_af_T, (size_t)V * af_hmax);
+    }
+  }
   // sampling
   if (any_sampled) {
     int rc = build_in_edge_order(c);
@@ -370,6 +386,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.dense_direct = direct_dense ? c->dense_out : nullptr;
   a.dense_ld = c->dense_ld;
   a.d_out = c->dims[l + 1];
+  a.Hout = a.Hp; a.self_rows = 1; a.self_bias = 1;
   a.dense_half = halves ? (int)(c->chunk_seq & 1) : -1;
   a.grad_cap = halves ? c->drain_rows / 2 : c->drain_rows;
   a.grad_off = halves ? (long long)a.dense_half * (c->drain_rows / 2) : 0;
@@ -456,9 +473,27 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   { int rc = stage_chunk(c, features, src_runs, src_begin, src_end, K, st, &X, &xbuf); if (rc) return rc; }
   if (timing) cudaEventRecord(pev[1], st);
   ChunkArgs a = make_args(c, src_begin, src_end);
-  // S2: projection (GAT: already done in pass 1; rows narrower than their padded width are repacked)
+  // S2: projection (GAT: already done in pass 1; rows narrower than their padded width are repacked).
+  // Aggregate-first layers push the (scaled, padded) input rows instead and transform the finished rows in S7.
   bool x_in_use = false;
-  if (gat) {
+  const bool af = c->agg_first[l];
+  if (af) {
+    const int Kp = taurus_round_up(K, 4);
+    a.Hout = a.Hp; a.Hp = Kp; a.ldpt = Kp;
+    a.self_rows = c->mode == TAURUS_SAGE_MEAN ? 0 : 1;
+    a.self_bias = 0;
+    if (c->mode == TAURUS_SAGE_MEAN) {   // T_v = x_v W_self, kept per vertex until v completes
+      float* T = c->d_af_T + (size_t)src_begin * a.Hout;
+      if (gemm_plain_tc_usable(c, l, X, ldx, T, a.Hout)) {
+        int rc = launch_gemm_plain_tc(c, l, a.Hout, a.Hout, X, ldx, K, n, T, a.Hout, st);
+        if (rc) return rc;
+      } else {
+        launch_gemm_plain_simt(c, l, a.Hout, a.Hout, X, ldx, K, n, T, a.Hout, st);
+      }
+    }
+    if (c->mode != TAURUS_GCN_SYM && K == Kp && (reinterpret_cast<uintptr_t>(X) & 15) == 0) { a.PT = X; x_in_use = true; }
+    else launch_af_prep(c, X, ldx, n, K, Kp, src_begin, st);
+  } else if (gat) {
     if (K == a.Hp && (reinterpret_cast<uintptr_t>(X) & 15) == 0) { a.PT = X; x_in_use = true; }
     else launch_gat_repack(c, X, n, K, a.Hp, st);
   } else if (project_tc_usable(c, l, X, ldx)) {
@@ -481,13 +516,18 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   if (timing) cudaEventRecord(pev[4], st);
   // S7
   if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
-  launch_finalise(c, a, st);
+  if (af) {
+    int rc = launch_af_finalise(c, a, l, std::min<long long>(bound, a.grad_cap), st);
+    if (rc) return rc;
+  } else {
+    launch_finalise(c, a, st);
+  }
   int run_rc = TAURUS_OK;
   if (a.dense_half >= 0 && c->dense_out) {   // hand this chunk's rows to the output stream (matrix in pinned host memory)
     const int h = a.dense_half, d_out = c->dims[l + 1];
     CU(cudaEventRecord(c->fin_done[h], st));
     CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
-    launch_place_half(c, h, d_out, a.Hp, c->out_stream);
+    launch_place_half(c, h, d_out, a.Hout, c->out_stream);
     CU(cudaEventRecord(c->out_done[h], c->out_stream));
     c->half_used[h] = true;
   } else if (a.dense_half >= 0) {
@@ -501,7 +541,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
     if (!run_rc) {
       CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
       const long long off = a.grad_off;
-      run_rc = runs_phase1(c->run_out, c->d_grad_ids + off, c->d_grad_rows + (size_t)off * a.Hp, a.Hp, std::min(bound, a.grad_cap),
+      run_rc = runs_phase1(c->run_out, c->d_grad_ids + off, c->d_grad_rows + (size_t)off * a.Hout, a.Hout, std::min(bound, a.grad_cap),
                            &c->d_ctl->out_count[h], 0, c->out_stream);
       if (!run_rc) c->run_pending_half = h;
     }

@@ -101,6 +101,11 @@ struct ChunkArgs {
   float* dense_direct;      // dense-output mode with the matrix in device memory: finalise writes row v at dense_direct + v * dense_ld
   long long dense_ld;
   int32_t d_out;            // unpadded output width
+  // aggregate-first layers (input rows narrower than output rows): the accumulators hold sums of input rows, Hp is
+  // the padded INPUT width, and the transform runs on the finished rows
+  int32_t Hout;             // padded output width (= Hp for project-first layers)
+  int32_t self_rows;        // 1: the scatter adds a self row; 0: it only counts the self message (the self term is added after the transform)
+  int32_t self_bias;        // 1: the self row carries the bias (project-first); 0: the bias is added after the transform
 };
 
 struct taurus_ctx {
@@ -144,6 +149,11 @@ struct taurus_ctx {
   float* d_att_z = nullptr;     // [V] normaliser
   long long gat_next_src = 0;   // next source taurus_gat_project_chunk expects
   bool gat_ready = false;       // taurus_gat_attention has run for this layer
+  // aggregate-first layers
+  bool agg_first[TAURUS_MAX_LAYERS] = {false};
+  float* d_af_A = nullptr;      // [drain_rows x max padded input width of such layers] finished rows gathered for the transform
+  float* d_af_O = nullptr;      // [drain_rows x Hmax] transform output when its place in the graduation buffer is known only on the device
+  float* d_af_T = nullptr;      // [V x Hp] SAGE: x_v W_self of every vertex, kept from its chunk until it completes
   int32_t* d_free_stack = nullptr;
   int32_t* d_need_list = nullptr;
   int32_t* d_touched_list = nullptr;
@@ -210,7 +220,9 @@ static inline int taurus_proj_width(int mode, int Hp) { return mode == TAURUS_SA
 void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st);
 void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);   // plan, select, evict, alloc/reload
-void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // finalise + commit
+void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // compact + finalise + commit
+void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
+void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st);
 void launch_place_half(taurus_ctx* c, int half, int d_out, int Hp, cudaStream_t st);   // dense-output mode
 void launch_reload_histogram(taurus_ctx* c, long long* d_hist18, cudaStream_t st);
@@ -232,6 +244,9 @@ int runs_flush_all(taurus_runs* r, cudaStream_t st);
 int runs_read_into(taurus_runs* r, long long s, long long e, float* out, long long ld, cudaStream_t st);
 // ---- taurus_host.cu
 void taurus_note_cuda_error(cudaError_t e, const char* what);   // keeps the text for taurus_last_cuda_error
+// ---- kernels_aggfirst.cu
+void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, cudaStream_t st);   // -> d_PT [n x Kp]
+int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long bound, cudaStream_t st);
 // ---- kernels_gat.cu
 void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st);
 void launch_gat_attention(taurus_ctx* c, cudaStream_t st);
@@ -240,7 +255,12 @@ void launch_gat_repack(taurus_ctx* c, const float* X, int n, int d_out, int Hp, 
 void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_gemm_simt.cu
 void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
+void launch_gemm_plain_simt(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
+                            cudaStream_t st);
 // ---- kernels_gemm_tc.cu
+bool gemm_plain_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx, const float* out, long long ld_out);
+int launch_gemm_plain_tc(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
+                         cudaStream_t st);
 int prepare_tc_weights(taurus_ctx* c, int layer, const std::vector<float>& cat, int K, int N);
 void free_tc_weights(taurus_ctx* c);
 bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);

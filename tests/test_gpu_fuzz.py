@@ -44,7 +44,7 @@ def random_config(seed):
             break
         pool = int(pool * 1.3) + 1
     w = replace(w, pool_slots=pool)
-    kw = dict(flags=int(rng.choice([0, 0, 2, 4, 6])), evict_policy=policy)
+    kw = dict(flags=int(rng.choice([0, 0, 0, 2, 4, 6, 8, 10, 12])), evict_policy=policy)   # 8: always project first
     if mode != tg.GAT and L <= 2 and rng.integers(0, 8) == 0:
         kw["gemm_mode"] = tg.GEMM_BF16          # bf16 operands, fp32 accumulate
     out_mode = int(rng.integers(0, 6))
