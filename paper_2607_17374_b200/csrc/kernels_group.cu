@@ -419,6 +419,7 @@ void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) 
   else if (Hp <= 32) launch_sg2<8, 1>(c, a, st);
   else if (Hp <= 48) launch_sg2<4, 3>(c, a, st);     // 12 float4: four lanes x three, no idle lanes
   else if (Hp <= 64) launch_sg2<16, 1>(c, a, st);
+  else if (Hp <= 112) launch_sg2<16, 2>(c, a, st);   // up to 28 float4: sixteen lanes x two leave fewer lanes idle than thirty-two x one
   else if (Hp <= 128) launch_sg2<32, 1>(c, a, st);
   else if (Hp <= 256) launch_sg2<32, 2>(c, a, st);
   else if (Hp <= 512) launch_sg2<32, 4>(c, a, st);
