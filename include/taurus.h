@@ -126,7 +126,9 @@ enum {
                                    input rows are at most 3/4 as wide as its output rows aggregates the (scaled) input rows and
                                    applies the weights to the finished rows instead (exact by linearity, Sect. 3.6 / 3.9): the
                                    accumulators, the scatter traffic and every evicted row shrink by d_in / d_out.  SAGE layers
-                                   do so only when the per-vertex store of x_v W_self (V x d_out floats) stays below 16 GiB */
+                                   keep every vertex's input row on the device until the vertex completes (its self term goes
+                                   through W_self with the transform) and do so only while that store (V x d_in floats) stays
+                                   below 64 GiB */
 };
 
 /* Integer accounting of one layer pass (Sect. 4.4-4.7 report these quantities). */

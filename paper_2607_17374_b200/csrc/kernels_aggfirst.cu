@@ -6,9 +6,10 @@
 // and the read-modify-write traffic of the scatter, the pool and every evicted row shrink by d_in / d_out.
 //   push     : S_u = c_out(u) h_u (padded to a multiple of 4 columns) is what the scatter pushes;
 //              GCN / GIN add the self message in input space (c_out(v) h_v, or (1 + eps) h_v: one shared matrix);
-//              SAGE keeps T_v = h_v W_self in a per-vertex store from v's own chunk until v completes.
-//   finalise : A_i = c_in(v_i) * acc(v_i) gathered for the completed vertices, O = A W_neigh on the tensor cores,
-//              out = act(O_i + T_v + b).
+//              SAGE keeps every vertex's input row h_v in a per-vertex store from v's own chunk until v completes
+//              (the scatter pushes the chunk's rows from that store).
+//   finalise : A_i = c_in(v_i) * acc(v_i) gathered for the completed vertices (SAGE: [c_in * acc | h_v]),
+//              O = A W_neigh (SAGE: A [W_neigh ; W_self]) on the tensor cores, out = act(O_i + b).
 #include "taurus_internal.h"
 
 namespace {
@@ -32,18 +33,20 @@ __global__ void af_prep_kernel(const float* __restrict__ X, int ldx, int n, int 
   }
 }
 
-// A[i] = c_in(v_i) * acc(v_i) for the completed vertices, zero rows up to `rows` (the row count the host sized the
-// transform for).  The slot is released by compact_done_kernel; its row stays intact until the next chunk.
-__global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long rows) {
+// A[i] = c_in(v_i) * acc(v_i) for the completed vertices (followed by v_i's own input row when `self_store` is given:
+// SAGE), zero rows up to `rows` (the row count the host sized the transform for).  The slot is released by
+// compact_done_kernel; its row stays intact until the next chunk.
+__global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long rows, const float* __restrict__ self_store) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
   const int n = ctl->done_count;
   const int vec = a.Hp >> 2;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < rows; i += warps) {
-    float4* dst = reinterpret_cast<float4*>(A + (size_t)i * a.Hp);
+    const int pitch = self_store ? 2 * a.Hp : a.Hp;
+    float4* dst = reinterpret_cast<float4*>(A + (size_t)i * pitch);
     if (i >= n) {
-      for (int k = al(); k < vec; k += 32) dst[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int k = al(); k < (pitch >> 2); k += 32) dst[k] = make_float4(0.f, 0.f, 0.f, 0.f);
       continue;
     }
     const int v = a.done_list[i];
@@ -61,12 +64,16 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
       x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
       dst[k] = x;
     }
+    if (self_store) {
+      const float4* own = reinterpret_cast<const float4*>(self_store + (size_t)v * a.Hp);
+      for (int k = al(); k < vec; k += 32) dst[vec + k] = own[k];
+    }
   }
 }
 
-// out = act(O_i + T_v + b) into the graduation buffer or straight into the caller's vertex-ordered matrix.
+// out = act(O_i + b) into the graduation buffer or straight into the caller's vertex-ordered matrix.
 // O has pitch a.Hout; rows of the graduation buffer too.
-__global__ void af_finish_kernel(ChunkArgs a, const float* __restrict__ O, const float* __restrict__ T, long long rows) {
+__global__ void af_finish_kernel(ChunkArgs a, const float* __restrict__ O, long long rows) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
   const int n = ctl->done_count;
@@ -86,14 +93,12 @@ __global__ void af_finish_kernel(ChunkArgs a, const float* __restrict__ O, const
     }
     const int v = a.done_list[i];
     const float4* __restrict__ o = reinterpret_cast<const float4*>(O + (size_t)i * a.Hout);
-    const float4* __restrict__ t = T ? reinterpret_cast<const float4*>(T + (size_t)v * a.Hout) : nullptr;
     const float4* __restrict__ b = reinterpret_cast<const float4*>(a.bias);
     float* __restrict__ drow = a.dense_direct ? a.dense_direct + (size_t)v * a.dense_ld : a.grad_rows + (size_t)(base + i) * a.Hout;
     for (int k = al(); k < vec; k += 32) {
       float4 y = o[k];
       const float4 bb = b[k];
       y.x += bb.x; y.y += bb.y; y.z += bb.z; y.w += bb.w;
-      if (t) { const float4 tt = t[k]; y.x += tt.x; y.y += tt.y; y.z += tt.z; y.w += tt.w; }
       if (a.act) { y.x = fmaxf(y.x, 0.f); y.y = fmaxf(y.y, 0.f); y.z = fmaxf(y.z, 0.f); y.w = fmaxf(y.w, 0.f); }
       const int c0 = k << 2;
       if (!a.dense_direct || (vec_ok && c0 + 3 < a.d_out)) {
@@ -114,8 +119,8 @@ __global__ void af_finish_kernel(ChunkArgs a, const float* __restrict__ O, const
 
 }  // namespace
 
-void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, cudaStream_t st) {
-  af_prep_kernel<<<c->sm_count * 8, 256, 0, st>>>(X, ldx, n, K, Kp, src_begin, c->mode, c->d_row_ptr, c->d_PT);
+void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, float* out, cudaStream_t st) {
+  af_prep_kernel<<<c->sm_count * 8, 256, 0, st>>>(X, ldx, n, K, Kp, src_begin, c->mode, c->d_row_ptr, out);
   c->launches += 1;
 }
 
@@ -138,15 +143,20 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
       }
       O = c->d_af_O;
     }
-    af_gather_kernel<<<grid, 256, 0, st>>>(a, c->d_af_A, rows);
+    const bool sage = c->mode == TAURUS_SAGE_MEAN;
+    const int Ka = sage ? 2 * a.Hp : a.Hp;               // columns of the gathered matrix
+    af_gather_kernel<<<grid, 256, 0, st>>>(a, c->d_af_A, rows, sage ? c->d_af_X : nullptr);
     c->launches += 1;
-    if (gemm_plain_tc_usable(c, layer, c->d_af_A, a.Hp, O, a.Hout)) {
-      int rc = launch_gemm_plain_tc(c, layer, 0, a.Hout, c->d_af_A, a.Hp, a.Hp, (int)rows, O, a.Hout, st);
+    void* image = sage ? c->tc_image_af[layer] : c->tc_image[layer];
+    if (gemm_plain_tc_usable(c, image, c->d_af_A, Ka, O, a.Hout)) {
+      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);
       if (rc) return rc;
+    } else if (sage) {
+      launch_gemm_plain_simt(c, c->d_Waf[layer], a.Hout, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);
     } else {
-      launch_gemm_plain_simt(c, layer, 0, a.Hout, c->d_af_A, a.Hp, c->dims[layer], (int)rows, O, a.Hout, st);
+      launch_gemm_plain_simt(c, c->d_Wcat[layer], a.Hout, a.Hout, c->d_af_A, Ka, c->dims[layer], (int)rows, O, a.Hout, st);
     }
-    af_finish_kernel<<<grid, 256, 0, st>>>(a, O, c->mode == TAURUS_SAGE_MEAN ? c->d_af_T : nullptr, rows);
+    af_finish_kernel<<<grid, 256, 0, st>>>(a, O, rows);
     c->launches += 1;
   }
   launch_commit(c, a, st);

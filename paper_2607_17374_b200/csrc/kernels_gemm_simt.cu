@@ -82,13 +82,11 @@ void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long
   c->launches += 1;
 }
 
-// out[n x N] (pitch ld_out) = X[n x K] (pitch ldx) . columns [col0, col0 + N) of the layer's weight matrix, no epilogue.
-void launch_gemm_plain_simt(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out,
+// out[n x N] (pitch ld_out) = X[n x K] (pitch ldx) . W[:, 0..N) (row-major, pitch ldw), no epilogue.
+void launch_gemm_plain_simt(taurus_ctx* c, const float* W, int ldw, int N, const float* X, int ldx, int K, int n, float* out,
                             long long ld_out, cudaStream_t st) {
-  const int Hp = taurus_round_up(c->dims[layer + 1], 4);
-  const int ldw = taurus_proj_width(c->mode, Hp);
+  if (n <= 0) return;
   dim3 grid((N + BN - 1) / BN, (n + BM - 1) / BM);
-  project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, K, c->d_Wcat[layer] + col0, ldw, N, out, ld_out, n, N, TAURUS_GIN_SUM, c->d_bias[layer],
-                                            c->d_row_ptr, c->d_din, 0, 0);
+  project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, K, W, ldw, N, out, ld_out, n, N, TAURUS_GIN_SUM, nullptr, c->d_row_ptr, c->d_din, 0, 0);
   c->launches += 1;
 }

@@ -401,10 +401,10 @@ struct WImage {
 
 }  // namespace
 
-int prepare_tc_weights(taurus_ctx* c, int layer, const std::vector<float>& cat, int K, int N) {
+int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat, int K, int N) {
   const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
   WImage* w = new WImage();
-  c->tc_image[layer] = w;
+  *slot = w;
   w->Np = taurus_round_up(N, 16);
   w->Kp = taurus_round_up(K, bf16 ? 64 : 32);
   const size_t cnt = (size_t)w->Np * w->Kp;
@@ -439,12 +439,13 @@ int prepare_tc_weights(taurus_ctx* c, int layer, const std::vector<float>& cat, 
 }
 
 void free_tc_weights(taurus_ctx* c) {
-  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) {
-    WImage* w = static_cast<WImage*>(c->tc_image[l]);
+  for (int l = 0; l < 2 * TAURUS_MAX_LAYERS; ++l) {
+    void** slot = l < TAURUS_MAX_LAYERS ? &c->tc_image[l] : &c->tc_image_af[l - TAURUS_MAX_LAYERS];
+    WImage* w = static_cast<WImage*>(*slot);
     if (!w) continue;
     cudaFree(w->hi); cudaFree(w->lo);
     delete w;
-    c->tc_image[l] = nullptr;
+    *slot = nullptr;
   }
 }
 
@@ -489,19 +490,19 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
 // Plain product on the tensor cores: out[n x N] (pitch ld_out floats) = X[n x K] (pitch ldx) . columns
 // [col0, col0 + N) of the layer's weight image, no epilogue scaling (used when a layer aggregates raw rows
 // first and transforms the finished rows afterwards).  col0 and N are multiples of 4.
-bool gemm_plain_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx, const float* out, long long ld_out) {
+bool gemm_plain_tc_usable(const taurus_ctx* c, const void* image, const float* X, int ldx, const float* out, long long ld_out) {
   if (c->flags & TAURUS_FLAG_SIMT_GEMM) return false;
-  if (!c->tc_image[layer] || !encode_fn()) return false;
+  if (!image || !encode_fn()) return false;
   if ((ldx & 3) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0) return false;
   if ((ld_out & 3) != 0 || (reinterpret_cast<uintptr_t>(out) & 15) != 0) return false;
   return true;
 }
 
-int launch_gemm_plain_tc(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
+int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
                          cudaStream_t st) {
   if (n <= 0) return TAURUS_OK;
   const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
-  WImage* w = static_cast<WImage*>(c->tc_image[layer]);
+  WImage* w = static_cast<WImage*>(image);
   const int rows_left = w->Np - col0;                       // image rows (= output columns) from col0 on
   const int Np = std::min(taurus_round_up(N, 16), rows_left);
   const int bw = Np < BN_MAX ? Np : BN_MAX;
@@ -521,7 +522,7 @@ int launch_gemm_plain_tc(taurus_ctx* c, int layer, int col0, int N, const float*
   GemmArgs g;
   g.PT = out; g.n = n; g.N = N; g.Np = Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
   g.b_box_bytes = bw * 128;
-  g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = c->d_bias[layer];
+  g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = nullptr;
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = 0; g.ctl = c->d_ctl;
   const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
   const int n_tiles = (n + BM - 1) / BM;

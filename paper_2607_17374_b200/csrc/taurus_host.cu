@@ -73,7 +73,8 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
-  cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_T);
+  cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_X);
+  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) cudaFree(c->d_Waf[l]);
   cudaFree(c->d_att_s); cudaFree(c->d_att_t); cudaFree(c->d_att_max); cudaFree(c->d_att_tm); cudaFree(c->d_att_z);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
   cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
@@ -149,6 +150,17 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     CU(cudaMemcpy(c->d_hub, flag.data(), flag.size(), cudaMemcpyHostToDevice));
   }
 
+  // aggregate-first layers: input rows at most 3/4 as wide as output rows.  SAGE keeps every vertex's input row until
+  // the vertex completes (its self term goes through W_self with the transform): only while that store stays small.
+  int af_kmax = 0;
+  for (int l = 0; l < c->L; ++l) {
+    const int Kp = taurus_round_up(c->dims[l], 4), Hp = taurus_round_up(c->dims[l + 1], 4);
+    bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && c->mode != TAURUS_GAT && 4 * Kp <= 3 * Hp;
+    if (af && c->mode == TAURUS_SAGE_MEAN && (size_t)V * Kp * sizeof(float) > ((size_t)64 << 30)) af = false;
+    c->agg_first[l] = af;
+    if (af) af_kmax = std::max(af_kmax, Kp);
+  }
+
   // weights: Wcat = [W_neigh | W_self] with both halves padded to Hp columns
   for (int l = 0; l < c->L; ++l) {
     const int K = c->dims[l], d_out = c->dims[l + 1], Hp = taurus_round_up(d_out, 4);
@@ -180,9 +192,26 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     CU(cudaMemcpy(c->d_Wcat[l], cat.data(), cat.size() * sizeof(float), cudaMemcpyHostToDevice));
     CU(cudaMemcpy(c->d_bias[l], b.data(), b.size() * sizeof(float), cudaMemcpyHostToDevice));
     if (!(c->flags & TAURUS_FLAG_SIMT_GEMM)) {
-      int rc = prepare_tc_weights(c, l, cat, K, N);
+      int rc = prepare_tc_weights(c, &c->tc_image[l], cat, K, N);
       if (rc == TAURUS_ERR_NOMEM) return rc;
       if (rc != TAURUS_OK) { cudaGetLastError(); free_tc_weights(c); }   // no tensor-map support: the FFMA kernel is used
+    }
+    if (c->agg_first[l] && c->mode == TAURUS_SAGE_MEAN) {
+      // [W_neigh ; W_self] stacked along K (each padded to Kp rows): one product transforms [c_in * agg | h_v]
+      const int Kp = taurus_round_up(K, 4);
+      std::vector<float> st2((size_t)2 * Kp * Hp, 0.f);
+      for (int k = 0; k < K; ++k)
+        for (int j = 0; j < d_out; ++j) {
+          st2[(size_t)k * Hp + j] = wn[(size_t)k * d_out + j];
+          st2[(size_t)(Kp + k) * Hp + j] = ws[(size_t)k * d_out + j];
+        }
+      ALLOC(c->d_Waf[l], st2.size());
+      CU(cudaMemcpy(c->d_Waf[l], st2.data(), st2.size() * sizeof(float), cudaMemcpyHostToDevice));
+      if (!(c->flags & TAURUS_FLAG_SIMT_GEMM) && c->tc_image[l]) {
+        int rc = prepare_tc_weights(c, &c->tc_image_af[l], st2, 2 * Kp, Hp);
+        if (rc == TAURUS_ERR_NOMEM) return rc;
+        if (rc != TAURUS_OK) { cudaGetLastError(); free_tc_weights(c); }
+      }
     }
   }
 
@@ -224,20 +253,10 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   ALLOC(c->d_PT, (size_t)c->chunk_sources * 2 * c->Hmax);
   if (c->mode == TAURUS_GAT) { ALLOC(c->d_att_s, V); ALLOC(c->d_att_t, V); ALLOC(c->d_att_max, V); ALLOC(c->d_att_tm, V); ALLOC(c->d_att_z, V); }
-  // aggregate-first layers: input rows at most 3/4 as wide as output rows
-  {
-    int af_kmax = 0, af_hmax = 0;
-    for (int l = 0; l < c->L; ++l) {
-      const int Kp = taurus_round_up(c->dims[l], 4), Hp = taurus_round_up(c->dims[l + 1], 4);
-      bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && c->mode != TAURUS_GAT && 4 * Kp <= 3 * Hp;
-      if (af && c->mode == TAURUS_SAGE_MEAN && (size_t)V * Hp * sizeof(float) > ((size_t)16 << 30)) af = false;
-      c->agg_first[l] = af;
-      if (af) { af_kmax = std::max(af_kmax, Kp); af_hmax = std::max(af_hmax, Hp); }
-    }
-    if (af_kmax > 0) {
-      ALLOC(c->d_af_A, (size_t)c->drain_rows * af_kmax);
-      if (c->mode == TAURUS_SAGE_MEAN) ALLOC(c->d_af_T, (size_t)V * af_hmax);
-    }
+  if (af_kmax > 0) {
+    const bool sage = c->mode == TAURUS_SAGE_MEAN;
+    ALLOC(c->d_af_A, (size_t)c->drain_rows * af_kmax * (sage ? 2 : 1));
+    if (sage) ALLOC(c->d_af_X, (size_t)V * af_kmax);
   }
   // sampling
   if (any_sampled) {
@@ -482,17 +501,17 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
     a.Hout = a.Hp; a.Hp = Kp; a.ldpt = Kp;
     a.self_rows = c->mode == TAURUS_SAGE_MEAN ? 0 : 1;
     a.self_bias = 0;
-    if (c->mode == TAURUS_SAGE_MEAN) {   // T_v = x_v W_self, kept per vertex until v completes
-      float* T = c->d_af_T + (size_t)src_begin * a.Hout;
-      if (gemm_plain_tc_usable(c, l, X, ldx, T, a.Hout)) {
-        int rc = launch_gemm_plain_tc(c, l, a.Hout, a.Hout, X, ldx, K, n, T, a.Hout, st);
-        if (rc) return rc;
-      } else {
-        launch_gemm_plain_simt(c, l, a.Hout, a.Hout, X, ldx, K, n, T, a.Hout, st);
-      }
+    if (c->mode == TAURUS_SAGE_MEAN) {
+      // the chunk's (padded) input rows go to the per-vertex store: the scatter pushes them from there, and the
+      // transform of a finished vertex reads its own row back for the W_self term
+      float* rows = c->d_af_X + (size_t)src_begin * Kp;
+      launch_af_prep(c, X, ldx, n, K, Kp, src_begin, rows, st);
+      a.PT = rows;
+    } else if (c->mode != TAURUS_GCN_SYM && K == Kp && (reinterpret_cast<uintptr_t>(X) & 15) == 0) {
+      a.PT = X; x_in_use = true;
+    } else {
+      launch_af_prep(c, X, ldx, n, K, Kp, src_begin, c->d_PT, st);
     }
-    if (c->mode != TAURUS_GCN_SYM && K == Kp && (reinterpret_cast<uintptr_t>(X) & 15) == 0) { a.PT = X; x_in_use = true; }
-    else launch_af_prep(c, X, ldx, n, K, Kp, src_begin, st);
   } else if (gat) {
     if (K == a.Hp && (reinterpret_cast<uintptr_t>(X) & 15) == 0) { a.PT = X; x_in_use = true; }
     else launch_gat_repack(c, X, n, K, a.Hp, st);

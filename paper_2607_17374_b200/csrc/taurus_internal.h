@@ -127,6 +127,8 @@ struct taurus_ctx {
   float* d_bias[TAURUS_MAX_LAYERS] = {nullptr};
   bool tc_smem_set = false;                        // dynamic shared memory limit of the projection kernel raised
   void* tc_image[TAURUS_MAX_LAYERS] = {nullptr};   // tensor-core operand images of Wcat (owned by kernels_gemm_tc.cu)
+  void* tc_image_af[TAURUS_MAX_LAYERS] = {nullptr};   // SAGE aggregate-first layers: image of [W_neigh ; W_self] stacked along K
+  float* d_Waf[TAURUS_MAX_LAYERS] = {nullptr};       //   the same matrix row-major [2 Kp x Hp] for the FFMA kernel
   // state
   int32_t* d_pend = nullptr;
   uint8_t* d_state = nullptr;
@@ -153,7 +155,8 @@ struct taurus_ctx {
   bool agg_first[TAURUS_MAX_LAYERS] = {false};
   float* d_af_A = nullptr;      // [drain_rows x max padded input width of such layers] finished rows gathered for the transform
   float* d_af_O = nullptr;      // [drain_rows x Hmax] transform output when its place in the graduation buffer is known only on the device
-  float* d_af_T = nullptr;      // [V x Hp] SAGE: x_v W_self of every vertex, kept from its chunk until it completes
+  float* d_af_X = nullptr;      // [V x Kp] SAGE: the (padded) input row of every vertex, kept from its chunk until it completes;
+                                //   the scatter reads the chunk's rows from here and the transform multiplies them by W_self
   int32_t* d_free_stack = nullptr;
   int32_t* d_need_list = nullptr;
   int32_t* d_touched_list = nullptr;
@@ -245,7 +248,7 @@ int runs_read_into(taurus_runs* r, long long s, long long e, float* out, long lo
 // ---- taurus_host.cu
 void taurus_note_cuda_error(cudaError_t e, const char* what);   // keeps the text for taurus_last_cuda_error
 // ---- kernels_aggfirst.cu
-void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, cudaStream_t st);   // -> d_PT [n x Kp]
+void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, float* out, cudaStream_t st);   // out [n x Kp]
 int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long bound, cudaStream_t st);
 // ---- kernels_gat.cu
 void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st);
@@ -255,13 +258,13 @@ void launch_gat_repack(taurus_ctx* c, const float* X, int n, int d_out, int Hp, 
 void launch_scatter(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_gemm_simt.cu
 void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
-void launch_gemm_plain_simt(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
-                            cudaStream_t st);
+void launch_gemm_plain_simt(taurus_ctx* c, const float* W, int ldw, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
+                            cudaStream_t st);   // out = X . W[:, 0..N), W row-major with pitch ldw
 // ---- kernels_gemm_tc.cu
-bool gemm_plain_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx, const float* out, long long ld_out);
-int launch_gemm_plain_tc(taurus_ctx* c, int layer, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
+bool gemm_plain_tc_usable(const taurus_ctx* c, const void* image, const float* X, int ldx, const float* out, long long ld_out);
+int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
                          cudaStream_t st);
-int prepare_tc_weights(taurus_ctx* c, int layer, const std::vector<float>& cat, int K, int N);
+int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat, int K, int N);   // image of cat [K x N] into *slot
 void free_tc_weights(taurus_ctx* c);
 bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);
 int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
