@@ -8,8 +8,6 @@
 #include <new>
 #include <vector>
 
-#include <sys/mman.h>
-
 #include "taurus_internal.h"
 
 static thread_local char g_cuda_err[256] = "";
@@ -73,8 +71,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
   cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
-  if (c->h_store && c->h_store_registered) { cudaHostUnregister(c->h_store); free(c->h_store); }
-  else if (c->h_store) cudaFreeHost(c->h_store);
+  if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_X);
   for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) cudaFree(c->d_Waf[l]);
@@ -238,27 +235,8 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   ALLOC(c->d_host_free, c->host_rows);
   if (c->host_rows > 0) {
-    const size_t bytes = (size_t)c->host_rows * c->Hmax * sizeof(float);
-    // Large stores are backed by transparent huge pages where the system grants them: evicted rows are scattered over
-    // the whole region, and 2 MiB pages keep the address translation of the device's loads and stores cheap.
-    if (bytes >= ((size_t)1 << 30) && !getenv("TAURUS_NO_HUGEPAGES")) {
-      const size_t huge = (size_t)2 << 20, rounded = (bytes + huge - 1) / huge * huge;
-      void* p = nullptr;
-      if (posix_memalign(&p, huge, rounded) == 0 && p) {
-        madvise(p, rounded, MADV_HUGEPAGE);
-        if (cudaHostRegister(p, rounded, cudaHostRegisterMapped | cudaHostRegisterPortable) == cudaSuccess) {
-          c->h_store = static_cast<float*>(p);
-          c->h_store_registered = true;
-        } else {
-          cudaGetLastError();
-          free(p);
-        }
-      }
-    }
-    if (!c->h_store) {
-      cudaError_t e = cudaHostAlloc((void**)&c->h_store, bytes, cudaHostAllocMapped);
-      if (e != cudaSuccess) { cuda_ok(e, "cudaHostAlloc(evicted-row store)"); c->h_store = nullptr; return TAURUS_ERR_NOMEM; }
-    }
+    cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->host_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
+    if (e != cudaSuccess) { cuda_ok(e, "cudaHostAlloc(evicted-row store)"); c->h_store = nullptr; return TAURUS_ERR_NOMEM; }
     CU(cudaHostGetDevicePointer((void**)&c->d_store_alias, c->h_store, 0));
   }
   // graduation buffer, chunk buffers

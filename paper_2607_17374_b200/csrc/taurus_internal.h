@@ -165,7 +165,6 @@ struct taurus_ctx {
   long long victim_capacity = 0;
   unsigned long long* d_keys = nullptr;
   float* h_store = nullptr;      // pinned, mapped
-  bool h_store_registered = false;   // allocated with posix_memalign + cudaHostRegister (huge pages) instead of cudaHostAlloc
   float* d_store_alias = nullptr;
   int32_t* d_host_free = nullptr;
   long long* d_grad_ids = nullptr;
