@@ -245,9 +245,9 @@ def run_ours(args):
     flags = (tb.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (tb.FLAG_NO_GROUPING if args.no_grouping else 0) | \
         (tb.FLAG_PROJECT_FIRST if args.project_first else 0)
     pad4 = lambda x: (x + 3) // 4 * 4
-    # the library's rule: a SAGE / GCN / GIN layer whose input rows are at most 3/4 as wide as its output rows aggregates
-    # input rows and transforms the finished rows (SAGE: while its per-vertex store of input rows stays below 64 GiB)
-    agg_first = [(not args.project_first) and w.mode != tg.GAT and 4 * pad4(w.dims[l]) <= 3 * pad4(w.dims[l + 1]) and
+    # the library's rule: a layer whose input rows are at most 3/4 as wide as its output rows aggregates input rows and
+    # transforms the finished rows (SAGE: while its per-vertex store of input rows stays below 64 GiB)
+    agg_first = [(not args.project_first) and 4 * pad4(w.dims[l]) <= 3 * pad4(w.dims[l + 1]) and
                  (w.mode != tg.SAGE_MEAN or V * pad4(w.dims[l]) * 4 <= (64 << 30)) for l in range(L)]
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags,

@@ -122,7 +122,7 @@ enum {
 enum {
   TAURUS_FLAG_SIMT_GEMM = 2,    /* use the plain fp32 FFMA projection kernel instead of the tensor-core one         */
   TAURUS_FLAG_NO_GROUPING = 4,  /* do not build the destination-grouped edge order: every chunk takes the CSR-order kernels */
-  TAURUS_FLAG_PROJECT_FIRST = 8 /* always project a chunk before scattering it.  Without this flag a SAGE / GCN / GIN layer whose
+  TAURUS_FLAG_PROJECT_FIRST = 8 /* always project a chunk before scattering it.  Without this flag a layer whose
                                    input rows are at most 3/4 as wide as its output rows aggregates the (scaled) input rows and
                                    applies the weights to the finished rows instead (exact by linearity, Sect. 3.6 / 3.9): the
                                    accumulators, the scatter traffic and every evicted row shrink by d_in / d_out.  SAGE layers
@@ -190,14 +190,16 @@ int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const
  *     out_v = act(sum_{u in N(v)} alpha_uv h'_u + b),
  * where N(v) is the propagated in-multiset of v (all in-edges, or the layer's sampled ones) plus v itself:
  * every vertex aggregates its own self message.  After taurus_layer_begin:
- *   pass 1  taurus_gat_project_chunk for every chunk in ascending, contiguous order: writes the transformed rows
- *           h' of sources [src_begin, src_end) to hprime_out (DEVICE memory, row i at hprime_out + i * ld,
- *           ld >= dims[layer+1] floats) and keeps the two scalars att_src . h'_u and att_dst . h'_u of every
- *           vertex.  `features` as in taurus_push_chunk.  Asynchronous on the stream.
+ *   pass 1  taurus_gat_project_chunk for every chunk in ascending, contiguous order: writes the rows pass 3 will
+ *           stream for sources [src_begin, src_end) to hprime_out (DEVICE memory, row i at hprime_out + i * ld,
+ *           ld >= dims[layer+1] floats, dims[layer+1] floats per row) and keeps the two scalars att_src . h'_u and
+ *           att_dst . h'_u of every vertex.  The rows are the transformed rows h'; in a layer that aggregates input
+ *           rows first (see TAURUS_FLAG_PROJECT_FIRST) they are the input rows, zero-padded, and h' is never formed:
+ *           the caller treats them as opaque.  `features` as in taurus_push_chunk.  Asynchronous on the stream.
  *   pass 2  taurus_gat_attention, once all vertices are projected: a topology-only sweep over the CSR that
  *           computes, per destination, the maximum score and the softmax normaliser (no per-edge state is
  *           stored; the coefficients are recomputed from four per-vertex scalars where they are used).
- *   pass 3  taurus_push_chunk / taurus_push_chunk_from_runs for every chunk with the transformed rows as
+ *   pass 3  taurus_push_chunk / taurus_push_chunk_from_runs for every chunk with the rows of pass 1 as
  *           `features` ([n] x dims[layer+1], rows contiguous): the broadcast of Sect. 3.1 with each message
  *           weighted by its attention coefficient; draining and taurus_layer_end as for the other modes.
  * Calls out of this order return TAURUS_ERR_ORDER.

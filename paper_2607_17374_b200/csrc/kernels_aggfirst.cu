@@ -5,7 +5,8 @@
 //     c_in(v) * sum_u c_out(u) (h_u W)  =  (c_in(v) * sum_u c_out(u) h_u) W,
 // and the read-modify-write traffic of the scatter, the pool and every evicted row shrink by d_in / d_out.
 //   push     : S_u = c_out(u) h_u (padded to a multiple of 4 columns) is what the scatter pushes;
-//              GCN / GIN add the self message in input space (c_out(v) h_v, or (1 + eps) h_v: one shared matrix);
+//              GCN / GIN / GAT add the self message in input space (c_out(v) h_v, (1 + eps) h_v, or the attention weight
+//              times h_v: one shared matrix);
 //              SAGE keeps every vertex's input row h_v in a per-vertex store from v's own chunk until v completes
 //              (the scatter pushes the chunk's rows from that store).
 //   finalise : A_i = c_in(v_i) * acc(v_i) gathered for the completed vertices (SAGE: [c_in * acc | h_v]),
@@ -57,6 +58,8 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
       scale = 1.0f / (float)(m > 1 ? m : 1);
     } else if (a.mode == TAURUS_GCN_SYM) {
       scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+    } else if (a.mode == TAURUS_GAT) {
+      scale = 1.0f / a.att_z[v];   // softmax normaliser
     }
     const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
     for (int k = al(); k < vec; k += 32) {
@@ -154,7 +157,8 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
     } else if (sage) {
       launch_gemm_plain_simt(c, c->d_Waf[layer], a.Hout, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);
     } else {
-      launch_gemm_plain_simt(c, c->d_Wcat[layer], a.Hout, a.Hout, c->d_af_A, Ka, c->dims[layer], (int)rows, O, a.Hout, st);
+      launch_gemm_plain_simt(c, c->d_Wcat[layer], taurus_proj_width(c->mode, a.Hout), a.Hout, c->d_af_A, Ka, c->dims[layer], (int)rows, O,
+                             a.Hout, st);
     }
     af_finish_kernel<<<grid, 256, 0, st>>>(a, O, rows);
     c->launches += 1;

@@ -76,6 +76,31 @@ __global__ void gat_edge_sum_kernel(long long V, const long long* __restrict__ r
   }
 }
 
+// Aggregate-first GAT layers: the scores need only s_u = h_u . (W att_src) and t_u = h_u . (W att_dst), so pass 1 is
+// two dot products per row; the (zero-padded) input rows are handed back to the caller for pass 3 in place of the
+// transformed rows.
+__global__ void gat_scores_kernel(const float* __restrict__ X, int ldx, int n, int K, const float* __restrict__ ws,
+                                  const float* __restrict__ wd, long long src_begin, float* __restrict__ rows_out, long long ld,
+                                  int d_out, float* __restrict__ att_s, float* __restrict__ att_t, float* __restrict__ att_max) {
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+    const float* x = X + (size_t)r * ldx;
+    float* o = rows_out + (size_t)r * ld;
+    float s = 0.f, t = 0.f;
+    for (int k = gl(); k < d_out; k += 32) {
+      const float v = k < K ? x[k] : 0.f;
+      if (k < K) { s = fmaf(v, ws[k], s); t = fmaf(v, wd[k], t); }
+      o[k] = v;
+    }
+    for (int off = 16; off; off >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, off); t += __shfl_xor_sync(0xffffffffu, t, off); }
+    if (gl() == 0) {
+      att_s[src_begin + r] = s;
+      att_t[src_begin + r] = t;
+      att_max[src_begin + r] = s;
+    }
+  }
+}
+
 __global__ void gat_repack_kernel(const float* __restrict__ X, int n, int d_out, int Hp, float* __restrict__ PT) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps)
@@ -87,6 +112,14 @@ __global__ void gat_repack_kernel(const float* __restrict__ X, int n, int d_out,
 void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st) {
   gat_split_kernel<<<c->sm_count * 8, 256, 0, st>>>(c->d_PT, Hp + 4, n, Hp, d_out, src_begin, hprime_out, ld, c->d_att_s, c->d_att_t,
                                                     c->d_att_max);
+  c->launches += 1;
+}
+
+void launch_gat_scores(taurus_ctx* c, int layer, const float* X, int ldx, int n, long long src_begin, float* rows_out, long long ld,
+                       cudaStream_t st) {
+  const int K = c->dims[layer];
+  gat_scores_kernel<<<c->sm_count * 8, 256, 0, st>>>(X, ldx, n, K, c->d_att_w[layer], c->d_att_w[layer] + K, src_begin, rows_out, ld,
+                                                     c->dims[layer + 1], c->d_att_s, c->d_att_t, c->d_att_max);
   c->launches += 1;
 }
 

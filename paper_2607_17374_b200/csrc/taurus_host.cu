@@ -74,7 +74,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_X);
-  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) cudaFree(c->d_Waf[l]);
+  for (int l = 0; l < TAURUS_MAX_LAYERS; ++l) { cudaFree(c->d_Waf[l]); cudaFree(c->d_att_w[l]); }
   cudaFree(c->d_att_s); cudaFree(c->d_att_t); cudaFree(c->d_att_max); cudaFree(c->d_att_tm); cudaFree(c->d_att_z);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
   cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
@@ -155,7 +155,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   int af_kmax = 0;
   for (int l = 0; l < c->L; ++l) {
     const int Kp = taurus_round_up(c->dims[l], 4), Hp = taurus_round_up(c->dims[l + 1], 4);
-    bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && c->mode != TAURUS_GAT && 4 * Kp <= 3 * Hp;
+    bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && 4 * Kp <= 3 * Hp;
     if (af && c->mode == TAURUS_SAGE_MEAN && (size_t)V * Kp * sizeof(float) > ((size_t)64 << 30)) af = false;
     c->agg_first[l] = af;
     if (af) af_kmax = std::max(af_kmax, Kp);
@@ -187,6 +187,10 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
         cat[(size_t)k * N + Hp] = (float)ss;
         cat[(size_t)k * N + Hp + 1] = (float)sd;
       }
+      std::vector<float> wv((size_t)2 * K);   // the same two vectors on their own, for layers that never form the transformed rows
+      for (int k = 0; k < K; ++k) { wv[(size_t)k] = cat[(size_t)k * N + Hp]; wv[(size_t)K + k] = cat[(size_t)k * N + Hp + 1]; }
+      ALLOC(c->d_att_w[l], wv.size());
+      CU(cudaMemcpy(c->d_att_w[l], wv.data(), wv.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
     ALLOC(c->d_Wcat[l], cat.size()); ALLOC(c->d_bias[l], b.size());
     CU(cudaMemcpy(c->d_Wcat[l], cat.data(), cat.size() * sizeof(float), cudaMemcpyHostToDevice));
@@ -496,7 +500,14 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   // Aggregate-first layers push the (scaled, padded) input rows instead and transform the finished rows in S7.
   bool x_in_use = false;
   const bool af = c->agg_first[l];
-  if (af) {
+  if (af && gat) {
+    // pass 3 of an aggregate-first GAT layer: the rows handed back by pass 1 are the zero-padded INPUT rows (pitch
+    // dims[l+1]); their first pad4(dims[l]) columns are what the attention-weighted scatter pushes
+    const int Kp = taurus_round_up(c->dims[l], 4);
+    a.Hout = a.Hp; a.Hp = Kp; a.self_rows = 1; a.self_bias = 0;
+    if ((K & 3) == 0 && (reinterpret_cast<uintptr_t>(X) & 15) == 0) { a.PT = X; a.ldpt = K; x_in_use = true; }
+    else { launch_gat_repack(c, X, n, K, Kp, st); a.ldpt = Kp; }
+  } else if (af) {
     const int Kp = taurus_round_up(K, 4);
     a.Hout = a.Hp; a.Hp = Kp; a.ldpt = Kp;
     a.self_rows = c->mode == TAURUS_SAGE_MEAN ? 0 : 1;
@@ -594,6 +605,13 @@ static int gat_project_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, c
   const float* X = nullptr;
   int xbuf = -1;
   { int rc = stage_chunk(c, features, src_runs, src_begin, src_end, K, st, &X, &xbuf); if (rc) return rc; }
+  if (c->agg_first[l]) {   // scores from two dot products per row; the input rows go back to the caller for pass 3
+    launch_gat_scores(c, l, X, K, n, src_begin, hprime_out, ld, st);
+    if (xbuf >= 0) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }
+    CU(cudaGetLastError());
+    c->gat_next_src = src_end;
+    return TAURUS_OK;
+  }
   if (project_tc_usable(c, l, X, K)) {
     int rc = launch_project_tc(c, l, X, K, src_begin, n, st);
     if (rc) return rc;

@@ -148,6 +148,7 @@ struct taurus_ctx {
   float* d_att_t = nullptr;     // [V] att_dst . h'
   float* d_att_max = nullptr;   // [V] running maximum of att_src . h'_u over the neighbourhood
   float2* d_att_tm = nullptr;   // [V] (t, maximum score)
+  float* d_att_w[TAURUS_MAX_LAYERS] = {nullptr};   // per layer: W att_src then W att_dst, dims[l] floats each (scores without the transformed rows)
   float* d_att_z = nullptr;     // [V] normaliser
   long long gat_next_src = 0;   // next source taurus_gat_project_chunk expects
   bool gat_ready = false;       // taurus_gat_attention has run for this layer
@@ -251,6 +252,7 @@ void taurus_note_cuda_error(cudaError_t e, const char* what);   // keeps the tex
 void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp, long long src_begin, float* out, cudaStream_t st);   // out [n x Kp]
 int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long bound, cudaStream_t st);
 // ---- kernels_gat.cu
+void launch_gat_scores(taurus_ctx* c, int layer, const float* X, int ldx, int n, long long src_begin, float* rows_out, long long ld, cudaStream_t st);
 void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st);
 void launch_gat_attention(taurus_ctx* c, cudaStream_t st);
 void launch_gat_repack(taurus_ctx* c, const float* X, int n, int d_out, int Hp, cudaStream_t st);   // X [n x d_out] -> d_PT [n x Hp]
