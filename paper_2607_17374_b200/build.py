@@ -13,7 +13,7 @@ INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_PKG, "libtaurus.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
+              "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-Wno-deprecated-gpu-targets"]
 
 
 def _sources():
