@@ -56,7 +56,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + ".tmp%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart", "-lcuda"])
+    subprocess.check_call([nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", tmp] + objs + ["-lcudart", "-lcuda"])
     os.replace(tmp, LIB)
     return LIB
 
