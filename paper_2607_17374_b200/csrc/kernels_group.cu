@@ -405,8 +405,9 @@ template <int LPE, int VPL>
 static void launch_sg2(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   const uint32_t* gm = c->d_mask_cur ? c->d_gmask : nullptr;
   const bool direct = a.direct && c->hub_count == 0;
-  if (a.mode == TAURUS_GAT) {   // the weighted variants exist for the general (slot-mapped) addressing only
-    if (gm) launch_sg<LPE, VPL, true, false, true>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, true>(c, a, gm, st);
+  if (a.mode == TAURUS_GAT) {   // attention-weighted variants
+    if (gm) { if (direct) launch_sg<LPE, VPL, true, true, true>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, true>(c, a, gm, st); }
+    else    { if (direct) launch_sg<LPE, VPL, false, true, true>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, true>(c, a, gm, st); }
     return;
   }
   if (gm) { if (direct) launch_sg<LPE, VPL, true, true, false>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, false>(c, a, gm, st); }
