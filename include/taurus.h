@@ -9,7 +9,9 @@
  * (Sect. 3.2) into per-destination accumulators, counts down each
  * destination's pending messages (Sect. 3.4), and finalises destinations whose
  * count reached zero into a graduation buffer (Sect. 3.6) that the caller
- * drains.  Accumulators of the highest in-degree vertices are pinned in a
+ * drains.  (Where a layer's input rows are the narrower ones the same sums are
+ * formed from the input rows and the weights are applied to the finished rows:
+ * see TAURUS_FLAG_PROJECT_FIRST.  Results and accounting do not depend on it.)  Accumulators of the highest in-degree vertices are pinned in a
  * GPU-resident hub store (Sect. 3.5.1); all others live in a bounded slot pool
  * (Sect. 3.5.2) whose fewest-pending rows are evicted to pinned host memory
  * when the pool is full (Sect. 3.5.3-3.5.4) and reloaded before they receive
@@ -23,6 +25,7 @@
  *   GCN-sym  : c_out(u) = (dout(u)+1)^-1/2, c_in(v) = (din(v)+1)^-1/2,
  *              c_self = c_out * c_in, W_self = W_neigh
  *   GIN-sum  : c_out = 1, c_in = 1, c_self = 1 + gin_eps, W_self = W_neigh ("GCN/GIN-style aggregation", Sect. 3.9)
+ *   GAT      : attention coefficients in place of c_in * c_out, see taurus_gat_project_chunk
  * M(v) is the multiset of propagated in-edges of v (all of them, or the
  * sampled ones); every CSR entry is one message, duplicates and self-loops
  * included.
