@@ -105,7 +105,12 @@ void launch_group_mask(taurus_ctx* c, cudaStream_t st) {
 
 // ------------------------------------------------------------------------------------------------ classify (S3)
 // Same decisions as the CSR-order classify; adjacent duplicates of a destination are skipped before the
-// epoch stamp is touched (exact layers), and the stamp is tested before the atomic.
+// epoch stamp is touched (exact layers), and the stamp is tested before the atomic.  Every thread handles
+// CG_ITEMS items per round, stage by stage (destinations, stamps, stamp updates, slot and state), so that the
+// scattered per-vertex reads of a round are in flight together and the block-wide list append (two barriers and
+// one round trip to a global counter) is paid once per CG_ITEMS * 256 items: the kernel is bound by that chain
+// of latencies, not by bytes.
+#define CG_ITEMS 4
 __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, const int32_t* __restrict__ g_dst, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
@@ -114,52 +119,75 @@ __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, cons
   __shared__ int s_base[2][2];
   const long long e0 = a.row_ptr[a.src_begin], e1 = a.row_ptr[a.src_end];
   const long long ne = e1 - e0, total = ne + (a.src_end - a.src_begin);
-  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long stride = (long long)gridDim.x * blockDim.x * CG_ITEMS;
   const int warp = threadIdx.x >> 5;
+  const unsigned lt = (1u << lane_id()) - 1;
   int hs = 0, ns = 0, ev = 0, gs = 0, bad = 0, par = 0;
-  for (long long base = (long long)blockIdx.x * blockDim.x; base < total; base += stride, par ^= 1) {
-    long long i = base + threadIdx.x;
-    int v = -1;
-    bool sole = false;   // this item is the only one that can touch v in this chunk: no atomic needed
-    if (i < ne) {
-      long long e = e0 + i;
-      if (gmask == nullptr) {
-        v = g_dst[e];
-        if (i > 0 && g_dst[e - 1] == v) v = -1;   // not the first edge of its destination group
-        // only a vertex of the chunk's own range can also be touched by its self item
-        sole = v < a.src_begin || v >= a.src_end;
-      } else if ((gmask[e >> 5] >> (e & 31)) & 1u) {
-        v = g_dst[e];
+  for (long long base = (long long)blockIdx.x * blockDim.x * CG_ITEMS; base < total; base += stride, par ^= 1) {
+    int v[CG_ITEMS];
+    bool sole[CG_ITEMS];   // this item is the only one that can touch v in this chunk: no atomic needed
+#pragma unroll
+    for (int q = 0; q < CG_ITEMS; ++q) {
+      const long long i = base + q * 256 + threadIdx.x;
+      v[q] = -1;
+      sole[q] = false;
+      if (i < ne) {
+        const long long e = e0 + i;
+        if (gmask == nullptr) {
+          v[q] = g_dst[e];
+          if (i > 0 && g_dst[e - 1] == v[q]) v[q] = -1;   // not the first edge of its destination group
+          // only a vertex of the chunk's own range can also be touched by its self item
+          sole[q] = v[q] < a.src_begin || v[q] >= a.src_end;
+        } else if ((gmask[e >> 5] >> (e & 31)) & 1u) {
+          v[q] = g_dst[e];
+        }
+      } else if (i < total) {
+        v[q] = (int)(a.src_begin + (i - ne));
       }
-    } else if (i < total) {
-      v = (int)(a.src_begin + (i - ne));
+      if (v[q] >= a.V) { bad = 1; v[q] = -1; }
     }
-    bool need = false, first = false;
-    if (v >= a.V) { bad = 1; v = -1; }
-    if (v >= 0 && (sole || a.touch[v] != a.epoch)) {
-      int old;
-      if (sole) { old = 0; a.touch[v] = a.epoch; }
-      else old = atomicMax(&a.touch[v], a.epoch);
-      if (old != a.epoch) {
-        first = true;
-        int l = a.loc[v];
-        int s = a.state[v];
-        if (l >= a.pool_slots) {
+    bool stale[CG_ITEMS];   // the stamp read before any update of this round is not this chunk's
+#pragma unroll
+    for (int q = 0; q < CG_ITEMS; ++q) stale[q] = v[q] >= 0 && (sole[q] || a.touch[v[q]] != a.epoch);
+    bool first[CG_ITEMS];
+#pragma unroll
+    for (int q = 0; q < CG_ITEMS; ++q) {
+      first[q] = false;
+      if (stale[q]) {
+        if (sole[q]) { a.touch[v[q]] = a.epoch; first[q] = true; }
+        else first[q] = atomicMax(&a.touch[v[q]], a.epoch) != a.epoch;
+      }
+    }
+    int l[CG_ITEMS], s[CG_ITEMS];
+#pragma unroll
+    for (int q = 0; q < CG_ITEMS; ++q)
+      if (first[q]) { l[q] = a.loc[v[q]]; s[q] = a.state[v[q]]; }
+    bool need[CG_ITEMS];
+    unsigned mn[CG_ITEMS], mt[CG_ITEMS];
+    int wn = 0, wt = 0;
+#pragma unroll
+    for (int q = 0; q < CG_ITEMS; ++q) {
+      need[q] = false;
+      if (first[q]) {
+        if (l[q] >= a.pool_slots) {
           gs++;
-          if (s == TAURUS_NOT_STARTED) a.state[v] = TAURUS_ON_GPU;
-        } else if (s == TAURUS_IN_BUFFER) {
+          if (s[q] == TAURUS_NOT_STARTED) a.state[v[q]] = TAURUS_ON_GPU;
+        } else if (s[q] == TAURUS_IN_BUFFER) {
           hs++;
-        } else if (s == TAURUS_NOT_STARTED) {
-          ns++; need = true;
-        } else if (s == TAURUS_EVICTED) {
-          ev++; need = true;
+        } else if (s[q] == TAURUS_NOT_STARTED) {
+          ns++; need[q] = true;
+        } else if (s[q] == TAURUS_EVICTED) {
+          ev++; need[q] = true;
         } else {
           bad = 1;
         }
       }
+      mn[q] = __ballot_sync(FULL, need[q]);
+      mt[q] = __ballot_sync(FULL, first[q]);
+      wn += __popc(mn[q]);
+      wt += __popc(mt[q]);
     }
-    const unsigned mn = __ballot_sync(FULL, need), mt = __ballot_sync(FULL, first);
-    if (lane_id() == 0) { s_cnt[par][0][warp] = __popc(mn); s_cnt[par][1][warp] = __popc(mt); }
+    if (lane_id() == 0) { s_cnt[par][0][warp] = wn; s_cnt[par][1][warp] = wt; }
     __syncthreads();
     if (threadIdx.x < 2) {
       int sum = 0;
@@ -167,13 +195,19 @@ __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, cons
       s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &ctl->need_count : &ctl->touched_count, sum) : 0;
     }
     __syncthreads();
-    if (need) {
-      int idx = s_base[par][0] + s_cnt[par][0][warp] + __popc(mn & ((1u << lane_id()) - 1));
-      if (idx < a.pool_slots) a.need_list[idx] = v;
-    }
-    if (first) {
-      int idx = s_base[par][1] + s_cnt[par][1][warp] + __popc(mt & ((1u << lane_id()) - 1));
-      if (idx < a.touched_capacity) a.touched_list[idx] = v; else bad = 1;
+    int on = s_base[par][0] + s_cnt[par][0][warp], ot = s_base[par][1] + s_cnt[par][1][warp];
+#pragma unroll
+    for (int q = 0; q < CG_ITEMS; ++q) {
+      if (need[q]) {
+        const int idx = on + __popc(mn[q] & lt);
+        if (idx < a.pool_slots) a.need_list[idx] = v[q];
+      }
+      if (first[q]) {
+        const int idx = ot + __popc(mt[q] & lt);
+        if (idx < a.touched_capacity) a.touched_list[idx] = v[q]; else bad = 1;
+      }
+      on += __popc(mn[q]);
+      ot += __popc(mt[q]);
     }
   }
   for (int o = 16; o; o >>= 1) {

@@ -296,6 +296,31 @@ __global__ void alloc_kernel(ChunkArgs a) {
   }
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
+  if (a.direct) {
+    // Every vertex owns the slot of its own number and nothing is ever evicted: each entry is a NOT_STARTED vertex
+    // whose row is cleared.  Batches of up to 32 entries per warp, one lane per entry for the list and state
+    // accesses, then the warp clears the rows one after the other.
+    int per = (int)((n + warps - 1) / warps);
+    per = per < 1 ? 1 : per > 32 ? 32 : per;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (long long i0 = (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * per; i0 < n; i0 += warps * per) {
+      const long long mine = i0 + lane_id();
+      int v = -1;
+      if (lane_id() < per && mine < n) {
+        v = a.need_list[mine];
+        if (a.state[v] != TAURUS_NOT_STARTED) { atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL); v = -1; }
+        else a.state[v] = TAURUS_IN_BUFFER;
+      }
+      const int rows = n - i0 < per ? (int)(n - i0) : per;
+      for (int j = 0; j < rows; ++j) {
+        const int vj = __shfl_sync(FULL, v, j);
+        if (vj < 0) continue;
+        float4* __restrict__ row = reinterpret_cast<float4*>(a.acc + (size_t)vj * a.Hp);
+        for (int k = lane_id(); k < vec; k += 32) row[k] = zero;
+      }
+    }
+    return;
+  }
   int reloaded = 0;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
     int v = a.need_list[i];
@@ -381,41 +406,66 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
 // S6: compact the touched vertices whose pending count reached zero (warp ballot + prefix) into done_list.
 // The scatter only decrements the counts with fire-and-forget reductions; completion is read here, after
 // the kernel boundary, when every reduction of the chunk has landed.
+// Each lane takes CD_ITEMS entries per round so that their scattered reads (pending count, slot) are in flight
+// together and one pair of counter round trips serves CD_ITEMS * 32 entries.
+#define CD_ITEMS 4
 __global__ void compact_done_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
   const int n = ctl->touched_count;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const unsigned lt = (1u << lane_id()) - 1;
   int bad = 0;
-  for (long long base = warp0 * 32; base < n; base += warps * 32) {
-    long long i = base + lane_id();
-    int v = -1;
-    bool done = false;
-    if (i < n) {
-      v = a.touched_list[i];
-      int p = a.pend[v];
-      done = p == 0;
-      if (p < 0) bad = 1;
+  for (long long base = warp0 * (32 * CD_ITEMS); base < n; base += warps * (32 * CD_ITEMS)) {
+    int v[CD_ITEMS], l[CD_ITEMS];
+    bool done[CD_ITEMS], rel[CD_ITEMS];
+#pragma unroll
+    for (int q = 0; q < CD_ITEMS; ++q) {
+      const long long i = base + q * 32 + lane_id();
+      v[q] = i < n ? a.touched_list[i] : -1;
     }
-    unsigned m = __ballot_sync(FULL, done);
-    if (m) {
-      int leader = __ffs(m) - 1, idx = 0;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->done_count, __popc(m));
-      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (done) { if (idx < a.grad_cap) a.done_list[idx] = v; else bad = 1; }
+#pragma unroll
+    for (int q = 0; q < CD_ITEMS; ++q) {
+      const int p = v[q] >= 0 ? a.pend[v[q]] : 1;
+      done[q] = p == 0;
+      if (p < 0) bad = 1;
     }
     // the slots of the completed non-hub vertices go back on the free stack (finalise still reads the rows:
     // nothing allocates before the next chunk)
-    const int l = done ? a.loc[v] : 0x7fffffff;
-    const bool rel = done && l < a.pool_slots;
-    m = __ballot_sync(FULL, rel);
-    if (m) {
-      int leader = __ffs(m) - 1;
-      long long f = 0;
-      if (lane_id() == leader) f = (long long)atomicAdd((unsigned long long*)&ctl->free_top, (unsigned long long)__popc(m));
-      f = __shfl_sync(FULL, f, leader) + __popc(m & ((1u << lane_id()) - 1));
-      if (rel && !a.direct) { a.free_stack[f] = l; a.owner[l] = -1; }
+#pragma unroll
+    for (int q = 0; q < CD_ITEMS; ++q) l[q] = done[q] ? a.loc[v[q]] : 0x7fffffff;
+    unsigned md[CD_ITEMS], mr[CD_ITEMS];
+    int cd = 0, cr = 0;
+#pragma unroll
+    for (int q = 0; q < CD_ITEMS; ++q) {
+      rel[q] = done[q] && l[q] < a.pool_slots;
+      md[q] = __ballot_sync(FULL, done[q]);
+      mr[q] = __ballot_sync(FULL, rel[q]);
+      cd += __popc(md[q]);
+      cr += __popc(mr[q]);
+    }
+    int idx = 0;
+    long long f = 0;
+    if (lane_id() == 0) {
+      if (cd) idx = atomicAdd(&ctl->done_count, cd);
+      if (cr) f = (long long)atomicAdd((unsigned long long*)&ctl->free_top, (unsigned long long)cr);
+    }
+    idx = __shfl_sync(FULL, idx, 0);
+    f = __shfl_sync(FULL, f, 0);
+#pragma unroll
+    for (int q = 0; q < CD_ITEMS; ++q) {
+      if (done[q]) {
+        const int at = idx + __popc(md[q] & lt);
+        if (at < a.grad_cap) a.done_list[at] = v[q]; else bad = 1;
+      }
+      if (rel[q] && !a.direct) {
+        const long long at = f + __popc(mr[q] & lt);
+        a.free_stack[at] = l[q];
+        a.owner[l[q]] = -1;
+      }
+      idx += __popc(md[q]);
+      f += __popc(mr[q]);
     }
   }
   if (__any_sync(FULL, bad) && lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
