@@ -41,6 +41,10 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
   const int n = ctl->done_count;
+  if (n > rows) {   // the host sized the transform for fewer rows than completed: its bound was wrong
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+    return;
+  }
   const int vec = a.Hp >> 2;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < rows; i += warps) {
@@ -151,7 +155,18 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
     af_gather_kernel<<<grid, 256, 0, st>>>(a, c->d_af_A, rows, sage ? c->d_af_X : nullptr);
     c->launches += 1;
     void* image = sage ? c->tc_image_af[layer] : c->tc_image[layer];
-    if (gemm_plain_tc_usable(c, image, c->d_af_A, Ka, O, a.Hout)) {
+    const bool tc = gemm_plain_tc_usable(c, image, c->d_af_A, Ka, O, a.Hout);
+    // rows that go straight into the caller's matrix leave the tensor-core kernel finished (bias, activation, state)
+    if (tc && a.dense_direct && a.d_out == a.Hout && (a.dense_ld & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dense_direct) & 15) == 0) {
+      GemmFinish fin;
+      fin.done_list = a.done_list; fin.state = a.state; fin.dense = a.dense_direct; fin.dense_ld = a.dense_ld;
+      fin.bias = a.bias; fin.act = a.act;
+      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, &fin);
+      if (rc) return rc;
+      launch_commit(c, a, st);
+      return TAURUS_OK;
+    }
+    if (tc) {
       int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);
       if (rc) return rc;
     } else if (sage) {

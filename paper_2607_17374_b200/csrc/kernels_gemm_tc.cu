@@ -116,6 +116,8 @@ struct GemmArgs {
   const int32_t* din;
   long long src_begin;
   DevCtl* ctl;
+  int finish;           // epilogue of finished rows: act(row + fin.bias) into fin.dense[fin.done_list[row]], no store to PT
+  GemmFinish fin;
 };
 
 template <bool BF16>
@@ -274,7 +276,13 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     const int tile = w / n_blocks, nb = w % n_blocks;
     const int r = tile * BM + q * 32 + lane;
     float c_out = 1.f, self_mul = 1.f;
-    if (r < g.n) {
+    int vrow = -1;        // finish mode: the vertex this lane's row belongs to
+    if (g.finish) {
+      if (r < g.n && r < g.ctl->done_count && !g.ctl->error) {
+        vrow = g.fin.done_list[r];
+        if (nb == 0) g.fin.state[vrow] = TAURUS_COMPLETED;
+      }
+    } else if (r < g.n) {
       const long long u = g.src_begin + r;
       if (g.mode == TAURUS_GCN_SYM) {
         c_out = (float)(1.0 / sqrt((double)(g.row_ptr[u + 1] - g.row_ptr[u]) + 1.0));
@@ -305,6 +313,30 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         if (cbase >= g.N) continue;           // padding columns of the last block
         // this warp's staging tile: 32 rows (lane = row) x 32 columns, 16-byte chunk c of row r at chunk c ^ (r & 7)
         unsigned char* tile_smem = out_staging + (q * 2 + (out_it & 1)) * OUT_TILE_BYTES;
+        if (g.finish) {
+          // transpose through the staging tile, then the warp writes four rows per step, each as one 128-byte piece of
+          // the row's place in the vertex-ordered matrix
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const int c = cbase + j;
+            const float4 b = c < g.N ? *reinterpret_cast<const float4*>(g.fin.bias + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 o = make_float4(__uint_as_float(v[j]) + b.x, __uint_as_float(v[j + 1]) + b.y, __uint_as_float(v[j + 2]) + b.z,
+                                   __uint_as_float(v[j + 3]) + b.w);
+            if (g.fin.act) { o.x = fmaxf(o.x, 0.f); o.y = fmaxf(o.y, 0.f); o.z = fmaxf(o.z, 0.f); o.w = fmaxf(o.w, 0.f); }
+            *reinterpret_cast<float4*>(tile_smem + lane * 128 + (((j >> 2) ^ (lane & 7)) << 4)) = o;
+          }
+          __syncwarp();
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + (lane >> 3), ch = lane & 7;
+            const int vv = __shfl_sync(0xffffffffu, vrow, rr);
+            const float4 y = *reinterpret_cast<const float4*>(tile_smem + rr * 128 + ((ch ^ (rr & 7)) << 4));
+            if (vv >= 0 && cbase + ch * 4 < g.N)
+              *reinterpret_cast<float4*>(g.fin.dense + (size_t)vv * g.fin.dense_ld + cbase + ch * 4) = y;
+          }
+          __syncwarp();   // the tile is rewritten in the next round
+          continue;
+        }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store that last used this tile has read it
         __syncwarp();
 #pragma unroll
@@ -471,6 +503,7 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   g.b_box_bytes = (w->Np < BN_MAX ? w->Np : BN_MAX) * 128;
   g.Hp = Hp; g.mode = c->mode; g.fanout = c->fanout[layer]; g.bias = c->d_bias[layer];
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = src_begin; g.ctl = c->d_ctl;
+  g.finish = 0; g.fin = GemmFinish();
   const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
   const int n_tiles = (n + BM - 1) / BM;
   const int n_units = n_tiles * ((w->Np + BN_MAX - 1) / BN_MAX);
@@ -499,8 +532,9 @@ bool gemm_plain_tc_usable(const taurus_ctx* c, const void* image, const float* X
 }
 
 int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
-                         cudaStream_t st) {
+                         cudaStream_t st, const GemmFinish* finish) {
   if (n <= 0) return TAURUS_OK;
+  if (finish && ((N & 3) != 0 || (finish->dense_ld & 3) != 0 || (reinterpret_cast<uintptr_t>(finish->dense) & 15) != 0)) return TAURUS_ERR_INTERNAL;
   const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
   WImage* w = static_cast<WImage*>(image);
   const int rows_left = w->Np - col0;                       // image rows (= output columns) from col0 on
@@ -524,6 +558,7 @@ int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const floa
   g.b_box_bytes = bw * 128;
   g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = nullptr;
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = 0; g.ctl = c->d_ctl;
+  g.finish = finish ? 1 : 0; g.fin = finish ? *finish : GemmFinish();
   const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
   const int n_tiles = (n + BM - 1) / BM;
   const int n_units = n_tiles * ((Np + BN_MAX - 1) / BN_MAX);

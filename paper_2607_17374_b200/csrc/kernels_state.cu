@@ -147,9 +147,7 @@ void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
 
 // ------------------------------------------------------------------------------------------------ make room (S4)
 // plan: need, deficit, capacity checks, peak occupancy.
-__global__ void plan_kernel(ChunkArgs a) {
-  DevCtl* ctl = a.ctl;
-  if (threadIdx.x != 0 || ctl->error) return;
+static __device__ void plan_chunk(const ChunkArgs& a, DevCtl* ctl) {   // one thread
   long long need = ctl->need_count;
   if (need > a.pool_slots) { ctl->error = TAURUS_ERR_POOL_TOO_SMALL; return; }
   long long deficit = need - ctl->free_top;
@@ -170,6 +168,11 @@ __global__ void plan_kernel(ChunkArgs a) {
   ctl->host_free_top = H - deficit;      // reloads of this chunk push on top of this
   long long occ = a.pool_slots - ctl->free_top;
   if (occ > ctl->peak_occupancy) ctl->peak_occupancy = occ;
+}
+__global__ void plan_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (threadIdx.x != 0 || ctl->error) return;
+  plan_chunk(a, ctl);
 }
 
 // Victims are the `deficit` smallest keys (pending << 31 | id) among IN_BUFFER vertices the chunk does not
@@ -300,6 +303,9 @@ __global__ void alloc_kernel(ChunkArgs a) {
     // Every vertex owns the slot of its own number and nothing is ever evicted: each entry is a NOT_STARTED vertex
     // whose row is cleared.  Batches of up to 32 entries per warp, one lane per entry for the list and state
     // accesses, then the warp clears the rows one after the other.
+    // No other thread of this kernel reads what the plan writes (there is no deficit and no stack to pop), so one
+    // thread does the chunk's bookkeeping here and the separate plan launch is left out.
+    if (blockIdx.x == 0 && threadIdx.x == 0) plan_chunk(a, ctl);
     int per = (int)((n + warps - 1) / warps);
     per = per < 1 ? 1 : per > 32 ? 32 : per;
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -386,8 +392,10 @@ __global__ void alloc_kernel(ChunkArgs a) {
 
 void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   const int blocks = c->sm_count * 8;
-  plan_kernel<<<1, 32, 0, st>>>(a);
-  c->launches += 1;
+  if (!a.direct) {   // direct-mapped pools plan inside alloc_kernel
+    plan_kernel<<<1, 32, 0, st>>>(a);
+    c->launches += 1;
+  }
   if (c->pool_slots < c->V - c->hub_count) {   // eviction is impossible when every non-hub vertex has a slot
     select_keys_kernel<<<blocks, 256, 0, st>>>(a);
     select_resolve_kernel<<<1, 1024, 0, st>>>(a, 0);

@@ -264,8 +264,19 @@ void launch_gemm_plain_simt(taurus_ctx* c, const float* W, int ldw, int N, const
                             cudaStream_t st);   // out = X . W[:, 0..N), W row-major with pitch ldw
 // ---- kernels_gemm_tc.cu
 bool gemm_plain_tc_usable(const taurus_ctx* c, const void* image, const float* X, int ldx, const float* out, long long ld_out);
+// Optional epilogue of the plain product for finished rows: row i of the product belongs to vertex done_list[i]
+// (i < ctl->done_count); act(row + bias) goes to dense[vertex * dense_ld ...] and the vertex becomes COMPLETED.
+// Needs N % 4 == 0, dense_ld % 4 == 0 and a 16-byte aligned dense base.
+struct GemmFinish {
+  const int32_t* done_list;
+  uint8_t* state;
+  float* dense;
+  long long dense_ld;
+  const float* bias;
+  int act;
+};
 int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
-                         cudaStream_t st);
+                         cudaStream_t st, const GemmFinish* finish = nullptr);
 int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat, int K, int N);   // image of cat [K x N] into *slot
 void free_tc_weights(taurus_ctx* c);
 bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);
