@@ -28,7 +28,8 @@ namespace {
 
 constexpr int BM = 128;            // rows per CTA tile (UMMA M)
 constexpr int BN_MAX = 256;        // output columns per block (UMMA N)
-constexpr int STAGES = 2;
+constexpr int STAGES = 2;            // stages with full-width (256-column) weight tiles: sizes the shared memory
+constexpr int MAX_STAGES = 4;        // narrower weight tiles leave room for more stages in the same memory
 constexpr int TILE_A_BYTES = BM * 128;           // 128 rows x 128 B
 constexpr int TILE_B_BYTES = BN_MAX * 128;       // 256 rows x 128 B
 constexpr unsigned WAIT_LIMIT = 1u << 24;
@@ -37,13 +38,16 @@ constexpr int OUT_TILE_BYTES = 32 * 128;        // epilogue staging tile: 32 row
 constexpr int OUT_STAGING_BYTES = 4 * 2 * OUT_TILE_BYTES;   // 4 epilogue warps x 2 tiles
 
 struct __align__(8) Barriers {
-  unsigned long long full[STAGES], conv[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
+  unsigned long long full[MAX_STAGES], conv[MAX_STAGES], empty[MAX_STAGES], acc_full[2], acc_empty[2];
   unsigned int tmem_base;
   int abort_flag;
 };
 
 // shared memory per stage: fp32 mode  A_hi(raw) 16K | A_lo 16K | B_hi 32K | B_lo 32K       = 96 KB
 //                          bf16 mode  A_raw0 16K | A_raw1 16K | A_bf16 16K | B_bf16 32K     = 80 KB
+// with weight tiles of 256 columns; a launch whose weight tiles are narrower (b_box_bytes < 32K) packs its stages
+// closer and runs as many as fit (GemmArgs::stages, stage_bytes), which hides more of the feature tiles' latency
+// where the product is bound by memory.
 constexpr int STAGE_BYTES_FP32 = 2 * TILE_A_BYTES + 2 * TILE_B_BYTES;
 constexpr int STAGE_BYTES_BF16 = 3 * TILE_A_BYTES + TILE_B_BYTES;
 
@@ -110,6 +114,8 @@ struct GemmArgs {
   int n, N, Np;         // rows, output columns, columns padded to a multiple of 16
   int k_stages;         // K padded / (32 fp32 mode, 64 bf16 mode)
   int b_box_bytes;      // bytes one W-operand TMA box delivers (box rows x 128)
+  int stages;           // operand stages in flight (2 .. MAX_STAGES)
+  int stage_bytes;      // fp32 mode 2 * TILE_A_BYTES + 2 * b_box_bytes, bf16 mode 3 * TILE_A_BYTES + b_box_bytes
   int Hp, mode, fanout;
   const float* bias;
   const long long* row_ptr;
@@ -126,8 +132,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                   const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_out, GemmArgs g) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int STAGE_BYTES = BF16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32;
-  unsigned char* out_staging = smem + STAGES * STAGE_BYTES;
+  constexpr int STAGE_BYTES_MAX = BF16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32;
+  const int STAGE_BYTES = g.stage_bytes;
+  const int n_stages = g.stages;
+  unsigned char* out_staging = smem + STAGES * STAGE_BYTES_MAX;
   Barriers* bars = reinterpret_cast<Barriers*>(out_staging + OUT_STAGING_BYTES);
   volatile int* abort_flag = &bars->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -136,7 +144,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   const int tmem_cols = 512;   // two accumulator buffers of 256 columns; one CTA per SM
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->conv[s], 128); mbar_init(&bars->empty[s], 1); }
+    for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->conv[s], 128); mbar_init(&bars->empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&bars->acc_full[b], 1); mbar_init(&bars->acc_empty[b], 128); }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -161,9 +169,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         const int row0 = tile * BM;
         const int col0 = nb * BN_MAX;
         for (int ks = 0; ks < g.k_stages; ++ks, ++it) {
-          const int s = it % STAGES;
-          const unsigned ph = (it / STAGES) & 1;
-          if (it >= STAGES && !mbar_wait(&bars->empty[s], ph ^ 1, abort_flag)) break;
+          const int s = it % n_stages;
+          const unsigned ph = (it / n_stages) & 1;
+          if (it >= n_stages && !mbar_wait(&bars->empty[s], ph ^ 1, abort_flag)) break;
           unsigned char* st = stage_ptr(s);
           if (BF16) {
             mbar_expect_tx(&bars->full[s], 2 * TILE_A_BYTES + g.b_box_bytes);
@@ -174,7 +182,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             mbar_expect_tx(&bars->full[s], TILE_A_BYTES + 2 * g.b_box_bytes);
             tma_load_2d(st, &map_x, ks * 32, row0, &bars->full[s]);
             tma_load_2d(st + 2 * TILE_A_BYTES, &map_b0, ks * 32, col0, &bars->full[s]);
-            tma_load_2d(st + 2 * TILE_A_BYTES + TILE_B_BYTES, &map_b1, ks * 32, col0, &bars->full[s]);
+            tma_load_2d(st + 2 * TILE_A_BYTES + g.b_box_bytes, &map_b1, ks * 32, col0, &bars->full[s]);
           }
         }
       }
@@ -194,8 +202,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                                ((unsigned)(bw >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
         bool ok = true;
         for (int ks = 0; ks < g.k_stages; ++ks, ++it) {
-          const int s = it % STAGES;
-          const unsigned ph = (it / STAGES) & 1;
+          const int s = it % n_stages;
+          const unsigned ph = (it / n_stages) & 1;
           if (!mbar_wait(&bars->conv[s], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const unsigned base = smem_u32(stage_ptr(s));
@@ -205,7 +213,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             for (int kk = 0; kk < 4; ++kk) umma(tmem_d, da + 2 * kk, db + 2 * kk, idesc, (ks | kk) != 0, false);
           } else {
             const unsigned long long a_hi = umma_desc(base), a_lo = umma_desc(base + TILE_A_BYTES);
-            const unsigned long long b_hi = umma_desc(base + 2 * TILE_A_BYTES), b_lo = umma_desc(base + 2 * TILE_A_BYTES + TILE_B_BYTES);
+            const unsigned long long b_hi = umma_desc(base + 2 * TILE_A_BYTES), b_lo = umma_desc(base + 2 * TILE_A_BYTES + g.b_box_bytes);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) {
               umma(tmem_d, a_lo + 2 * kk, b_hi + 2 * kk, idesc, (ks | kk) != 0, true);
@@ -226,8 +234,8 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     for (int w = blockIdx.x; w < n_tiles * n_blocks && !*abort_flag; w += gridDim.x) {
       bool ok = true;
       for (int ks = 0; ks < g.k_stages; ++ks, ++it) {
-        const int s = it % STAGES;
-        const unsigned ph = (it / STAGES) & 1;
+        const int s = it % n_stages;
+        const unsigned ph = (it / n_stages) & 1;
         if (!mbar_wait(&bars->full[s], ph, abort_flag)) { ok = false; break; }
         unsigned char* st = stage_ptr(s);
         if (BF16) {
@@ -376,7 +384,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     if (threadIdx.x == 0) {
       atomicCAS(&g.ctl->error, 0, TAURUS_ERR_INTERNAL);
       // give copies that may still be in flight a bounded time to land before the shared memory is released
-      for (int s = 0; s < STAGES; ++s)
+      for (int s = 0; s < n_stages; ++s)
         for (unsigned i = 0; i < (1u << 16); ++i)
           if (mbar_try(&bars->full[s], 0) || mbar_try(&bars->full[s], 1)) break;
     }
@@ -421,6 +429,14 @@ bool make_map(CUtensorMap* m, const void* base, CUtensorMapDataType dt, int elem
   cuuint32_t estr[2] = {1, 1};
   return fn(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Stages that fit the shared memory sized for STAGES full-width stages.
+void set_stages(GemmArgs& g, bool bf16) {
+  const int budget = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32);
+  g.stage_bytes = bf16 ? 3 * TILE_A_BYTES + g.b_box_bytes : 2 * TILE_A_BYTES + 2 * g.b_box_bytes;
+  int n = budget / g.stage_bytes;
+  g.stages = n < STAGES ? STAGES : n > MAX_STAGES ? MAX_STAGES : n;
 }
 
 // Per-layer tensor-core images of Wcat, K-major: [Np x Kp].
@@ -501,6 +517,7 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   GemmArgs g;
   g.PT = c->d_PT; g.n = n; g.N = N; g.Np = w->Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
   g.b_box_bytes = (w->Np < BN_MAX ? w->Np : BN_MAX) * 128;
+  set_stages(g, bf16);
   g.Hp = Hp; g.mode = c->mode; g.fanout = c->fanout[layer]; g.bias = c->d_bias[layer];
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = src_begin; g.ctl = c->d_ctl;
   g.finish = 0; g.fin = GemmFinish();
@@ -556,6 +573,7 @@ int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const floa
   GemmArgs g;
   g.PT = out; g.n = n; g.N = N; g.Np = Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
   g.b_box_bytes = bw * 128;
+  set_stages(g, bf16);
   g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = nullptr;
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = 0; g.ctl = c->d_ctl;
   g.finish = finish ? 1 : 0; g.fin = finish ? *finish : GemmFinish();

@@ -359,3 +359,18 @@ def test_maximum_widths_and_fanout(mode):
     for flags in (0, 4):
         lib, _ = _full_check(w, flags=flags)
     assert lib["stats"][0]["evictions"] > 0
+
+
+@pytest.mark.parametrize("mode", [tg.SAGE_MEAN, tg.GCN_SYM, tg.GIN_SUM])
+def test_finished_rows_leave_the_transform_complete(mode):
+    """Layers that aggregate input rows and write into a device-resident dense matrix: the transform of the finished
+    rows applies bias and activation and places every row itself.  Widths whose last 16-column block is partly
+    padding (100, 292), a vertex count that leaves a ragged last row tile, a pool with one slot per vertex and one that
+    evicts; the 30 -> 50 layer has output rows that are not a multiple of 16 bytes and takes the separate finishing kernel."""
+    from dataclasses import replace
+    w = tg.scaled(tg.WORKLOADS["large"], 30_011, chunk=2048)
+    w = replace(w, mode=mode, dims=(20, 100, 292, 36), fanout=(0, 0, 0), pool_slots=30_011, hub_count=0)
+    _full_check(w, dense_output=True)
+    w = replace(w, dims=(20, 100, 30, 50), pool_slots=18_000, hub_count=30)
+    lib, _ = _full_check(w, dense_output=True)
+    assert lib["stats"][0]["evictions"] > 0
