@@ -174,6 +174,7 @@ __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, cons
           if (s[q] == TAURUS_NOT_STARTED) a.state[v[q]] = TAURUS_ON_GPU;
         } else if (s[q] == TAURUS_IN_BUFFER) {
           hs++;
+          if (a.slot_touch) a.slot_touch[l[q]] = a.epoch;
         } else if (s[q] == TAURUS_NOT_STARTED) {
           ns++; need[q] = true;
         } else if (s[q] == TAURUS_EVICTED) {

@@ -99,6 +99,7 @@ __global__ void __launch_bounds__(256) classify_kernel(ChunkArgs a) {
           if (s == TAURUS_NOT_STARTED) a.state[v] = TAURUS_ON_GPU;
         } else if (s == TAURUS_IN_BUFFER) {
           hs++;
+          if (a.slot_touch) a.slot_touch[l] = a.epoch;
         } else if (s == TAURUS_NOT_STARTED) {
           ns++; need = true;
         } else if (s == TAURUS_EVICTED) {
@@ -206,13 +207,13 @@ __global__ void select_keys_kernel(ChunkArgs a) {   // pass 0: gather keys, hist
     int v = a.owner[s];
     unsigned long long key = ~0ull;
     if (v >= 0) {
-      const int t = a.touch[v];
+      const int t = a.slot_touch[s];   // = touch[v]
       if (t != a.epoch) {
         unsigned score;
         if (a.evict_policy == TAURUS_EVICT_FIFO) score = (unsigned)a.slot_epoch[s];
         else if (a.evict_policy == TAURUS_EVICT_LRU) score = (unsigned)t;
         else if (a.evict_policy == TAURUS_EVICT_RANDOM) score = evict_hash(a.seed, (unsigned long long)v, (unsigned long long)(a.epoch - 1));
-        else score = (unsigned)a.pend[v];
+        else score = (unsigned)a.slot_pend[s];   // = pend[v]: v was not touched since the copy was taken
         key = ((unsigned long long)score << 31) | (unsigned long long)v;
       }
     }
@@ -383,7 +384,10 @@ __global__ void alloc_kernel(ChunkArgs a) {
         a.reload_count[v] += 1;
         reloaded++;
       }
-      if (!a.direct) { a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch; }
+      if (!a.direct) {
+        a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch;
+        if (a.slot_touch) a.slot_touch[slot] = a.epoch;   // slot_pend follows in compact_done: v is on the touched list
+      }
       a.state[v] = TAURUS_IN_BUFFER;
     }
   }
@@ -433,16 +437,23 @@ __global__ void compact_done_kernel(ChunkArgs a) {
       const long long i = base + q * 32 + lane_id();
       v[q] = i < n ? a.touched_list[i] : -1;
     }
+    int pq[CD_ITEMS];
 #pragma unroll
     for (int q = 0; q < CD_ITEMS; ++q) {
-      const int p = v[q] >= 0 ? a.pend[v[q]] : 1;
-      done[q] = p == 0;
-      if (p < 0) bad = 1;
+      pq[q] = v[q] >= 0 ? a.pend[v[q]] : 1;
+      done[q] = pq[q] == 0;
+      if (pq[q] < 0) bad = 1;
     }
     // the slots of the completed non-hub vertices go back on the free stack (finalise still reads the rows:
-    // nothing allocates before the next chunk)
+    // nothing allocates before the next chunk); the slots of the others take a copy of the new pending count
+    const bool mirror = a.slot_pend != nullptr;
 #pragma unroll
-    for (int q = 0; q < CD_ITEMS; ++q) l[q] = done[q] ? a.loc[v[q]] : 0x7fffffff;
+    for (int q = 0; q < CD_ITEMS; ++q) l[q] = (done[q] || (mirror && v[q] >= 0)) ? a.loc[v[q]] : 0x7fffffff;
+    if (mirror) {
+#pragma unroll
+      for (int q = 0; q < CD_ITEMS; ++q)
+        if (!done[q] && v[q] >= 0 && l[q] >= 0 && l[q] < a.pool_slots) a.slot_pend[l[q]] = pq[q];
+    }
     unsigned md[CD_ITEMS], mr[CD_ITEMS];
     int cd = 0, cr = 0;
 #pragma unroll

@@ -70,7 +70,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   free_tc_weights(c);
   cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
-  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
+  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_slot_touch); cudaFree(c->d_slot_pend); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_X);
@@ -236,6 +236,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   if (c->pool_slots < V - c->hub_count) {   // a chunk evicts at most what it needs, and it needs at most what it touches
     c->victim_capacity = std::min<long long>(c->pool_slots, c->touched_capacity);
     ALLOC(c->d_victims, c->victim_capacity); ALLOC(c->d_keys, c->pool_slots);
+    ALLOC(c->d_slot_touch, c->pool_slots); ALLOC(c->d_slot_pend, c->pool_slots);
   }
   ALLOC(c->d_host_free, c->host_rows);
   if (c->host_rows > 0) {
@@ -390,6 +391,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.row_ptr = c->d_row_ptr; a.col = c->d_col; a.din = c->d_din; a.mask = c->d_mask_cur;
   a.pend = c->d_pend; a.state = c->d_state; a.loc = c->d_loc; a.touch = c->d_touch; a.reload_count = c->d_reload;
   a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list; a.slot_epoch = c->d_slot_epoch;
+  a.slot_touch = c->d_slot_touch; a.slot_pend = c->d_slot_pend;
   a.touched_list = c->d_touched_list; a.touched_capacity = c->touched_capacity;
   a.victims = c->d_victims; a.victim_capacity = c->victim_capacity; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;

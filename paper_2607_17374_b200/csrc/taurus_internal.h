@@ -61,6 +61,12 @@ struct ChunkArgs {
   float* acc;               // [(pool_slots + hub_count) x Hp]
   int32_t* owner;           // [pool_slots] vertex in the slot, -1 = free
   int32_t* slot_epoch;      // [pool_slots] chunk epoch at which the slot's vertex entered the pool (FIFO policy)
+  // Per-slot copies of the owner's epoch stamp and pending count, kept so that the victim select reads the pool
+  // front to back instead of three scattered per-vertex words per slot; null when nothing can be evicted.
+  // slot_touch[s] is written whenever the owner is touched (hit: classify, hand-out: alloc); slot_pend[s] after
+  // every chunk that touched the owner (compact_done), and the pending count only changes in such chunks.
+  int32_t* slot_touch;
+  int32_t* slot_pend;
   int32_t* free_stack;      // [pool_slots]
   int32_t* need_list;       // [pool_slots]
   int32_t* touched_list;    // [touched_capacity] every vertex the chunk touches, listed at its first touch
@@ -140,6 +146,8 @@ struct taurus_ctx {
   float* d_acc = nullptr;
   int32_t* d_owner = nullptr;
   int32_t* d_slot_epoch = nullptr;
+  int32_t* d_slot_touch = nullptr;
+  int32_t* d_slot_pend = nullptr;
   int evict_policy = 0;
   float gin_eps = 0.f;
   // GAT mode
