@@ -16,7 +16,7 @@
 //
 // Every wait on an mbarrier is bounded: after WAIT_LIMIT polls the kernel raises a CTA-wide abort flag,
 // records TAURUS_ERR_INTERNAL in the control block, waits (bounded) for its TMA copies in flight, frees its
-// TMEM and returns.  No TMA load uses multicast.
+// TMEM and returns.  Every TMA load is a plain load of the issuing CTA alone.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
