@@ -35,8 +35,9 @@ __global__ void af_prep_kernel(const float* __restrict__ X, int ldx, int n, int 
 }
 
 // A[i] = c_in(v_i) * acc(v_i) for the completed vertices (followed by v_i's own input row when `self_store` is given:
-// SAGE), zero rows up to `rows` (the row count the host sized the transform for).  The slot is released by
-// compact_done_kernel; its row stays intact until the next chunk.
+// SAGE).  `rows` is the row count the host sized the transform for; rows behind the completed ones are left as
+// they are (the tensor-core transform skips them, the FFMA one writes products nobody reads).  The slot is released
+// by compact_done_kernel; its row stays intact until the next chunk.
 __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long rows, const float* __restrict__ self_store) {
   DevCtl* ctl = a.ctl;
   if (ctl->error) return;
@@ -47,13 +48,9 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
   }
   const int vec = a.Hp >> 2;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < rows; i += warps) {
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
     const int pitch = self_store ? 2 * a.Hp : a.Hp;
     float4* dst = reinterpret_cast<float4*>(A + (size_t)i * pitch);
-    if (i >= n) {
-      for (int k = al(); k < (pitch >> 2); k += 32) dst[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-      continue;
-    }
     const int v = a.done_list[i];
     const int l = a.loc[v];
     float scale = 1.0f;
@@ -161,13 +158,13 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
       GemmFinish fin;
       fin.done_list = a.done_list; fin.state = a.state; fin.dense = a.dense_direct; fin.dense_ld = a.dense_ld;
       fin.bias = a.bias; fin.act = a.act;
-      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, &fin);
+      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, &fin, true);
       if (rc) return rc;
       launch_commit(c, a, st);
       return TAURUS_OK;
     }
     if (tc) {
-      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);
+      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, nullptr, true);
       if (rc) return rc;
     } else if (sage) {
       launch_gemm_plain_simt(c, c->d_Waf[layer], a.Hout, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);

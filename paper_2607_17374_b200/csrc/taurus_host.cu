@@ -261,6 +261,8 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   if (af_kmax > 0) {
     const bool sage = c->mode == TAURUS_SAGE_MEAN;
     ALLOC(c->d_af_A, (size_t)c->drain_rows * af_kmax * (sage ? 2 : 1));
+    // rows behind a chunk's finished ones are read (and their products dropped) by the last row tile: keep them finite
+    CU(cudaMemset(c->d_af_A, 0, (size_t)c->drain_rows * af_kmax * (sage ? 2 : 1) * sizeof(float)));
     if (sage) ALLOC(c->d_af_X, (size_t)V * af_kmax);
   }
   // sampling

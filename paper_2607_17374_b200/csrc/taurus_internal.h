@@ -284,7 +284,9 @@ struct GemmFinish {
   int act;
 };
 int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
-                         cudaStream_t st, const GemmFinish* finish = nullptr);
+                         cudaStream_t st, const GemmFinish* finish = nullptr, bool rows_from_done_count = false);
+// rows_from_done_count: n is only the host's bound; the kernel works on the first ctl->done_count rows (read on the
+// device at launch) and leaves the others untouched.
 int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat, int K, int N);   // image of cat [K x N] into *slot
 void free_tc_weights(taurus_ctx* c);
 bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);
