@@ -40,9 +40,34 @@ __global__ void group_split_kernel(long long n, long long chunk_begin, const int
   }
 }
 
+// In-list sources from the grouped order.  Chunks are taken in ascending order and a chunk's edges are sorted (stably)
+// by destination, so the edges of one (chunk, destination) group follow the in-list entries of every earlier chunk
+// in ascending source order: entry = csc_ptr[dst] + entries of earlier chunks (cursor[dst]) + rank inside the group.
+__global__ void csc_fill_kernel(long long n, const int32_t* __restrict__ dst_sorted, const unsigned long long* __restrict__ vals,
+                                const long long* __restrict__ csc_ptr, const int32_t* __restrict__ cursor, int32_t* __restrict__ csc_src) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const int d = dst_sorted[i];
+    long long lo = 0, hi = i;   // first edge of the group
+    while (lo < hi) { const long long mid = (lo + hi) >> 1; if (dst_sorted[mid] < d) lo = mid + 1; else hi = mid; }
+    csc_src[csc_ptr[d] + cursor[d] + (i - lo)] = (int32_t)(vals[i] >> 32);
+  }
+}
+__global__ void csc_advance_kernel(long long n, const int32_t* __restrict__ dst_sorted, int32_t* __restrict__ cursor) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const int d = dst_sorted[i];
+    if (i + 1 < n && dst_sorted[i + 1] == d) continue;   // only the last edge of a group advances the cursor
+    long long lo = 0, hi = i;
+    while (lo < hi) { const long long mid = (lo + hi) >> 1; if (dst_sorted[mid] < d) lo = mid + 1; else hi = mid; }
+    cursor[d] += (int32_t)(i - lo + 1);
+  }
+}
+
 // g_dst, g_edge = (destination, source - chunk start) (/ g_eid): per grid chunk, the chunk's CSR edges stably
-// sorted by destination.
-int build_grouped_order(taurus_ctx* c, bool keep_edge_ids) {
+// sorted by destination.  fill_csc_src: the in-list sources csc_src are written along the way (csc_ptr is built,
+// d_vtmp serves as the per-destination cursor).
+int build_grouped_order(taurus_ctx* c, bool keep_edge_ids, bool fill_csc_src) {
   const long long V = c->V, E = c->E, cs = c->chunk_sources;
   const long long n_chunks = (V + cs - 1) / cs;
   std::vector<long long> bounds((size_t)n_chunks + 1);
@@ -69,6 +94,7 @@ int build_grouped_order(taurus_ctx* c, bool keep_edge_ids) {
     if (cudaMalloc(&vals_in, (size_t)max_edges * 8) != cudaSuccess || cudaMalloc(&vals_out, (size_t)max_edges * 8) != cudaSuccess) { rc = TAURUS_ERR_NOMEM; break; }
     cub::DeviceRadixSort::SortPairs(nullptr, tmp_bytes, c->d_col, c->d_gdst, vals_in, vals_out, max_edges, 0, end_bit);
     if (cudaMalloc(&tmp, tmp_bytes > 0 ? tmp_bytes : 16) != cudaSuccess) { rc = TAURUS_ERR_NOMEM; break; }
+    if (fill_csc_src) cudaMemset(c->d_vtmp, 0, (size_t)V * sizeof(int32_t));
     for (long long k = 0; k < n_chunks && rc == TAURUS_OK; ++k) {
       const long long e0 = bounds[(size_t)k], ne = bounds[(size_t)k + 1] - e0;
       if (ne <= 0) continue;
@@ -77,6 +103,10 @@ int build_grouped_order(taurus_ctx* c, bool keep_edge_ids) {
       size_t b = tmp_bytes;
       if (cub::DeviceRadixSort::SortPairs(tmp, b, c->d_col + e0, c->d_gdst + e0, vals_in, vals_out, ne, 0, end_bit) != cudaSuccess) { rc = TAURUS_ERR_CUDA; break; }
       group_split_kernel<<<c->sm_count * 4, 256>>>(ne, s, c->d_gdst + e0, vals_out, c->d_gedge + e0, c->d_geid ? c->d_geid + e0 : nullptr);
+      if (fill_csc_src) {
+        csc_fill_kernel<<<c->sm_count * 8, 256>>>(ne, c->d_gdst + e0, vals_out, c->d_csc_ptr, c->d_vtmp, c->d_csc_src);
+        csc_advance_kernel<<<c->sm_count * 8, 256>>>(ne, c->d_gdst + e0, c->d_vtmp);
+      }
     }
     if (rc == TAURUS_OK && cudaDeviceSynchronize() != cudaSuccess) rc = TAURUS_ERR_CUDA;
   } while (0);

@@ -129,6 +129,44 @@ int build_in_edge_order(taurus_ctx* c) {
   return rc;
 }
 
+// csc_ptr alone (the in-list sources are then filled from the grouped edge order, chunk by chunk).
+int build_csc_ptr(taurus_ctx* c) {
+  const long long V = c->V;
+  void* tmp = nullptr;
+  size_t scan_bytes = 0;
+  int rc = TAURUS_OK;
+  do {
+    if (cudaMalloc(&c->d_csc_ptr, (size_t)(V + 1) * sizeof(long long)) != cudaSuccess) { rc = TAURUS_ERR_NOMEM; break; }
+    widen_kernel<<<c->sm_count * 8, 256>>>(V, c->d_din, c->d_csc_ptr);
+    cudaMemset(c->d_csc_ptr + V, 0, sizeof(long long));
+    cub::DeviceScan::ExclusiveSum(nullptr, scan_bytes, c->d_csc_ptr, c->d_csc_ptr, V + 1);
+    if (cudaMalloc(&tmp, scan_bytes > 0 ? scan_bytes : 16) != cudaSuccess) { rc = TAURUS_ERR_NOMEM; break; }
+    if (cub::DeviceScan::ExclusiveSum(tmp, scan_bytes, c->d_csc_ptr, c->d_csc_ptr, V + 1) != cudaSuccess) { rc = TAURUS_ERR_CUDA; break; }
+    if (cudaDeviceSynchronize() != cudaSuccess) { rc = TAURUS_ERR_CUDA; break; }
+  } while (0);
+  cudaFree(tmp);
+  c->launches += 1;
+  return rc;
+}
+
+// Source of every in-list entry from its CSR edge index: the row whose range holds the index.
+__global__ void csc_src_from_eid_kernel(long long E, long long V, const long long* __restrict__ row_ptr, const uint32_t* __restrict__ csc_eid,
+                                        int32_t* __restrict__ csc_src) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < E; i += stride) {
+    const long long e = csc_eid[i];
+    long long lo = 0, hi = V;   // largest u with row_ptr[u] <= e
+    while (hi - lo > 1) { const long long mid = (lo + hi) >> 1; if (row_ptr[mid] <= e) lo = mid; else hi = mid; }
+    csc_src[i] = (int32_t)lo;
+  }
+}
+
+int build_csc_src_from_eid(taurus_ctx* c) {
+  if (c->E > 0) csc_src_from_eid_kernel<<<c->sm_count * 16, 256>>>(c->E, c->V, c->d_row_ptr, c->d_csc_eid, c->d_csc_src);
+  c->launches += 1;
+  return cudaDeviceSynchronize() == cudaSuccess ? TAURUS_OK : TAURUS_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------------------------------------ inspection
 // One block: the kept edges of one destination, ascending edge index, with their sources.
 __global__ void sampled_edges_kernel(long long dst, const int32_t* din, const long long* csc_ptr, const uint32_t* csc_eid,

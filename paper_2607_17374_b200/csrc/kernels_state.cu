@@ -32,19 +32,22 @@ __global__ void reset_vertices_kernel(long long V, const int32_t* din, int fanou
   }
 }
 
-__global__ void reset_pool_kernel(long long pool_slots, long long host_rows, long long hub_count, const int32_t* hub_ids,
-                                  int32_t* loc, int32_t* owner, int32_t* free_stack, int32_t* host_free, DevCtl* ctl) {
+__global__ void reset_pool_kernel(long long pool_slots, long long n_ext, long long n_buckets, long long hub_count, const int32_t* hub_ids,
+                                  int32_t* loc, int32_t* owner, int32_t* free_stack, int32_t* ext_free, int32_t* ext_live,
+                                  int32_t* bk_tail_ext, int32_t* bk_tail_fill, int32_t* bk_new, DevCtl* ctl) {
   long long stride = (long long)gridDim.x * blockDim.x;
   long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   for (long long i = tid; i < pool_slots; i += stride) {
     owner[i] = -1;
     free_stack[i] = (int32_t)(pool_slots - 1 - i);   // slot 0 is handed out first
   }
-  for (long long i = tid; i < host_rows; i += stride) host_free[i] = (int32_t)(host_rows - 1 - i);
+  for (long long i = tid; i < n_ext; i += stride) { ext_free[i] = (int32_t)(n_ext - 1 - i); ext_live[i] = 0; }
+  for (long long i = tid; i < n_buckets; i += stride) { bk_tail_ext[i] = -1; bk_tail_fill[i] = 0; bk_new[i] = 0; }
   for (long long i = tid; i < hub_count; i += stride) loc[hub_ids[i]] = (int32_t)(pool_slots + i);
   if (tid == 0) {
     ctl->free_top = pool_slots;
-    ctl->host_free_top = host_rows;
+    ctl->ext_free_top = n_ext;
+    ctl->host_live = 0;
   }
 }
 
@@ -53,8 +56,9 @@ void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st) {
   cudaMemsetAsync(c->d_ctl, 0, sizeof(DevCtl), st);
   reset_vertices_kernel<<<blocks, 256, 0, st>>>(c->V, c->d_din, c->fanout[layer], c->d_pend, c->d_state, c->d_loc,
                                                 c->d_touch, c->d_reload, c->pool_slots >= c->V ? 1 : 0);
-  reset_pool_kernel<<<blocks, 256, 0, st>>>(c->pool_slots, c->host_rows, c->hub_count, c->d_hub_ids, c->d_loc, c->d_owner,
-                                            c->d_free_stack, c->d_host_free, c->d_ctl);
+  reset_pool_kernel<<<blocks, 256, 0, st>>>(c->pool_slots, c->n_ext, c->n_ext > 0 ? c->n_buckets : 0, c->hub_count, c->d_hub_ids, c->d_loc,
+                                            c->d_owner, c->d_free_stack, c->d_ext_free, c->d_ext_live, c->d_bk_tail_ext,
+                                            c->d_bk_tail_fill, c->d_bk_new, c->d_ctl);
   // accumulator rows are as wide as what the scatter pushes: input rows in aggregate-first layers, output rows otherwise
   int Hp = taurus_round_up(c->agg_first[layer] ? c->dims[layer] : c->dims[layer + 1], 4);
   if (c->hub_count > 0)
@@ -153,32 +157,37 @@ static __device__ void plan_chunk(const ChunkArgs& a, DevCtl* ctl) {   // one th
   if (need > a.pool_slots) { ctl->error = TAURUS_ERR_POOL_TOO_SMALL; return; }
   long long deficit = need - ctl->free_top;
   if (deficit < 0) deficit = 0;
-  if (deficit > ctl->host_free_top) { ctl->error = TAURUS_ERR_HOST_STORE_FULL; return; }
+  // this chunk's victims leave before its reloads hand their host rows back
+  if (ctl->host_live + deficit > a.host_rows) { ctl->error = TAURUS_ERR_HOST_STORE_FULL; return; }
+  ctl->host_live += deficit - ctl->ev;
   ctl->deficit = (int32_t)deficit;
-  ctl->sel_prefix = 0ull;
-  ctl->sel_k = deficit;
   ctl->victim_count = 0;
-  // Stack positions are handed out by list index, not by per-item atomics: victim i takes host row
-  // host_free[H - 1 - i]; need-list entry i < deficit takes over the slot of victim deficit - 1 - i, entry
-  // i >= deficit pops free_stack[F + deficit - 1 - i].  The counters are brought to their end-of-chunk values here.
-  const long long F = ctl->free_top, H = ctl->host_free_top;
-  ctl->evict_push_base = F;
-  ctl->host_pop_base = H;
+  for (int l = 0; l <= TAURUS_SEL_LEVELS; ++l) { ctl->sel_k[l] = 0; ctl->sel_min[l] = ~0ull; ctl->sel_max[l] = 0ull; ctl->sel_count[l] = 0; }
+  ctl->sel_k[0] = deficit;
+  ctl->sel_final_level = deficit > 0 ? TAURUS_SEL_LEVELS + 1 : -1;
+  // Slots are handed out by list index, not by per-item atomics: need-list entry i < deficit takes over the slot
+  // of victim deficit - 1 - i, entry i >= deficit pops free_stack[F + deficit - 1 - i].  The counter is brought to
+  // its end-of-chunk value here.
+  const long long F = ctl->free_top;
   ctl->alloc_base = F + deficit;
   ctl->free_top = F + deficit - need;
-  ctl->host_free_top = H - deficit;      // reloads of this chunk push on top of this
   long long occ = a.pool_slots - ctl->free_top;
   if (occ > ctl->peak_occupancy) ctl->peak_occupancy = occ;
 }
 __global__ void plan_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
-  if (threadIdx.x != 0 || ctl->error) return;
-  plan_chunk(a, ctl);
+  if (ctl->error) return;
+  for (int i = threadIdx.x; i < 2 * TAURUS_SEL_BINS; i += blockDim.x) (&ctl->hist[0][0])[i] = 0;
+  if (threadIdx.x == 0) plan_chunk(a, ctl);
 }
 
-// Victims are the `deficit` smallest keys (pending << 31 | id) among IN_BUFFER vertices the chunk does not
-// touch.  Keys are unique, so an MSB-first radix select over 6 digits of 11 bits finds the exact
-// threshold key; every key <= threshold is a victim.
+// Victims are the `deficit` smallest keys (score << 31 | id) among IN_BUFFER vertices the chunk does not
+// touch (Sect. 3.5.3: fewest pending messages first).  Keys are unique, so an MSB-first radix select finds
+// them exactly.  Level 0 scans the pool; every level lists the keys below the digit that holds rank k as
+// victims and hands the keys inside that digit to the next level, so deeper levels see a small candidate list.
+// The digit of a level starts at the highest bit in which the keys entering it differ (from their minimum and
+// maximum): pending counts are small numbers, and a fixed digit grid would spend its first passes on bits that
+// are zero in every key.
 // 31-bit score of the random policy: a hash of (seed, vertex, chunk index); constants are part of its definition.
 static __device__ __forceinline__ unsigned long long ev_mix(unsigned long long x) {
   x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
@@ -194,17 +203,36 @@ static __device__ __forceinline__ unsigned evict_hash(unsigned long long seed, u
   return (unsigned)(h >> 33);
 }
 
-static __device__ __forceinline__ int sel_shift(int pass) { return TAURUS_SEL_BITS * (TAURUS_SEL_PASSES - 1 - pass); }
+static __device__ __forceinline__ int sel_shift_of(unsigned long long lo, unsigned long long hi) {
+  const unsigned long long diff = lo ^ hi;
+  if (diff == 0ull) return 0;
+  const int top = 63 - __clzll((long long)diff);
+  return top >= TAURUS_SEL_BITS ? top - (TAURUS_SEL_BITS - 1) : 0;
+}
 
-__global__ void select_keys_kernel(ChunkArgs a) {   // pass 0: gather keys, histogram of the top digit
+// Block-wide minimum / maximum / count of the eligible keys a thread saw, folded into level `lvl` of the control block.
+static __device__ __forceinline__ void sel_fold(DevCtl* ctl, int lvl, unsigned long long kmin, unsigned long long kmax, int cnt) {
+  for (int o = 16; o; o >>= 1) {
+    const unsigned long long m = __shfl_xor_sync(FULL, kmin, o), M = __shfl_xor_sync(FULL, kmax, o);
+    if (m < kmin) kmin = m;
+    if (M > kmax) kmax = M;
+    cnt += __shfl_xor_sync(FULL, cnt, o);
+  }
+  if (lane_id() == 0 && cnt) {
+    atomicMin(&ctl->sel_min[lvl], kmin);
+    atomicMax(&ctl->sel_max[lvl], kmax);
+    atomicAdd(&ctl->sel_count[lvl], cnt);
+  }
+}
+
+__global__ void __launch_bounds__(256) select_keys_kernel(ChunkArgs a) {   // key of every slot; range of the eligible keys
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->deficit == 0) return;
-  __shared__ unsigned int sh[TAURUS_SEL_BINS];
-  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) sh[i] = 0;
-  __syncthreads();
-  long long stride = (long long)gridDim.x * blockDim.x;
+  if (ctl->error || ctl->sel_final_level < 0) return;
+  unsigned long long kmin = ~0ull, kmax = 0ull;
+  int cnt = 0;
+  const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < a.pool_slots; s += stride) {
-    int v = a.owner[s];
+    const int v = a.owner[s];
     unsigned long long key = ~0ull;
     if (v >= 0) {
       const int t = a.slot_touch[s];   // = touch[v]
@@ -215,71 +243,295 @@ __global__ void select_keys_kernel(ChunkArgs a) {   // pass 0: gather keys, hist
         else if (a.evict_policy == TAURUS_EVICT_RANDOM) score = evict_hash(a.seed, (unsigned long long)v, (unsigned long long)(a.epoch - 1));
         else score = (unsigned)a.slot_pend[s];   // = pend[v]: v was not touched since the copy was taken
         key = ((unsigned long long)score << 31) | (unsigned long long)v;
+        if (key < kmin) kmin = key;
+        if (key > kmax) kmax = key;
+        cnt++;
       }
     }
     a.keys[s] = key;
-    if (key != ~0ull) atomicAdd(&sh[(unsigned)(key >> sel_shift(0)) & (TAURUS_SEL_BINS - 1)], 1u);
   }
-  __syncthreads();
-  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x)
-    if (sh[i]) atomicAdd(&ctl->hist[i], sh[i]);
+  sel_fold(ctl, 0, kmin, kmax, cnt);
 }
 
-__global__ void select_hist_kernel(ChunkArgs a, int pass) {   // passes 1..5
+// Histogram of the level's digit over the keys entering the level.  Threads of a warp that hit the same bin add
+// once (most keys of a level often share a bin).
+__global__ void __launch_bounds__(256) select_hist_kernel(ChunkArgs a, int level) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->deficit == 0) return;
+  if (ctl->error || ctl->sel_final_level < level) return;
+  const long long k = ctl->sel_k[level];
+  const long long n = level == 0 ? a.pool_slots : (long long)ctl->sel_count[level];
+  if (ctl->sel_count[level] < k) {   // fewer eligible victims than needed
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(&ctl->error, 0, level == 0 ? TAURUS_ERR_POOL_TOO_SMALL : TAURUS_ERR_INTERNAL);
+    return;
+  }
   __shared__ unsigned int sh[TAURUS_SEL_BINS];
   for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) sh[i] = 0;
   __syncthreads();
-  const int shift = sel_shift(pass);
-  const unsigned long long prefix = ctl->sel_prefix;
-  long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < a.pool_slots; s += stride) {
-    unsigned long long key = a.keys[s];
-    if (key != ~0ull && (key >> (shift + TAURUS_SEL_BITS)) == prefix)
-      atomicAdd(&sh[(unsigned)(key >> shift) & (TAURUS_SEL_BINS - 1)], 1u);
+  const int shift = sel_shift_of(ctl->sel_min[level], ctl->sel_max[level]);
+  const int32_t* __restrict__ cand = level == 0 ? nullptr : a.cand[level & 1];
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long rounds = (n + stride - 1) / stride;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (long long r = 0; r < rounds; ++r, i += stride) {
+    unsigned long long key = ~0ull;
+    if (i < n) key = a.keys[level == 0 ? i : (long long)cand[i]];
+    const bool on = key != ~0ull;
+    const unsigned digit = on ? (unsigned)(key >> shift) & (TAURUS_SEL_BINS - 1) : 0xffffffffu;
+    const unsigned peers = __match_any_sync(FULL, digit);
+    if (on && lane_id() == __ffs(peers) - 1) atomicAdd(&sh[digit], (unsigned)__popc(peers));
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x)
-    if (sh[i]) atomicAdd(&ctl->hist[i], sh[i]);
+  unsigned int* hist = ctl->hist[level & 1];
+  for (int b = threadIdx.x; b < TAURUS_SEL_BINS; b += blockDim.x)
+    if (sh[b]) atomicAdd(&hist[b], sh[b]);
 }
 
-__global__ void select_resolve_kernel(ChunkArgs a, int pass) {   // one block: pick the digit that holds rank k
+// Every block finds the digit that holds rank k from the level's histogram; keys below it are victims, keys inside
+// it go to the next level (or are victims too when the digit holds exactly the ranks still missing).
+__global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int level) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->deficit == 0) return;
+  if (ctl->error || ctl->sel_final_level < level) return;
   __shared__ unsigned int sh[TAURUS_SEL_BINS];
-  for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) { sh[i] = ctl->hist[i]; ctl->hist[i] = 0; }
+  __shared__ unsigned int part[256];
+  __shared__ int s_digit;
+  __shared__ long long s_rest;
+  const unsigned int* hist = ctl->hist[level & 1];
+  const long long k = ctl->sel_k[level];
+  // bins per thread: TAURUS_SEL_BINS / 256 consecutive ones
+  constexpr int PER = TAURUS_SEL_BINS / 256;
+  unsigned int mine[PER], sum = 0;
+#pragma unroll
+  for (int j = 0; j < PER; ++j) { mine[j] = hist[threadIdx.x * PER + j]; sh[threadIdx.x * PER + j] = mine[j]; sum += mine[j]; }
+  part[threadIdx.x] = sum;
+  if (threadIdx.x == 0) s_digit = -1;
   __syncthreads();
   if (threadIdx.x == 0) {
-    long long k = ctl->sel_k, cum = 0;
-    int b = 0;
-    for (; b < TAURUS_SEL_BINS; ++b) {
-      if (cum + sh[b] >= k) break;
-      cum += sh[b];
+    long long cum = 0;
+    int t = 0;
+    for (; t < 256; ++t) { if (cum + part[t] >= k) break; cum += part[t]; }
+    if (t < 256) {
+      int b = t * PER;
+      for (; b < t * PER + PER; ++b) { if (cum + sh[b] >= k) break; cum += sh[b]; }
+      s_digit = b;
+      s_rest = k - cum;
     }
-    if (b == TAURUS_SEL_BINS) { ctl->error = TAURUS_ERR_POOL_TOO_SMALL; return; }   // fewer eligible victims than needed
-    ctl->sel_prefix = (ctl->sel_prefix << TAURUS_SEL_BITS) | (unsigned long long)b;
-    ctl->sel_k = k - cum;
+  }
+  __syncthreads();
+  const int digit_k = s_digit;
+  if (digit_k < 0) {   // the histogram holds fewer keys than k: cannot happen after the count check
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+    return;
+  }
+  const long long rest = s_rest;
+  const bool final = rest == (long long)sh[digit_k];   // the whole digit is victims: nothing left to resolve
+  const int shift = sel_shift_of(ctl->sel_min[level], ctl->sel_max[level]);
+  const long long n = level == 0 ? a.pool_slots : (long long)ctl->sel_count[level];
+  const int32_t* __restrict__ cand = level == 0 ? nullptr : a.cand[level & 1];
+  int32_t* __restrict__ next = a.cand[(level + 1) & 1];
+  if (blockIdx.x == 0) {
+    unsigned int* other = ctl->hist[(level + 1) & 1];   // the next level's histogram (read last by the level above this one)
+    for (int b = threadIdx.x; b < TAURUS_SEL_BINS; b += blockDim.x) other[b] = 0;
+    if (threadIdx.x == 0) {
+      if (final) ctl->sel_final_level = level;
+      else if (level == TAURUS_SEL_LEVELS - 1 || shift == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);   // unique keys always end in a final level
+      else ctl->sel_k[level + 1] = rest;
+    }
+  }
+  unsigned long long kmin = ~0ull, kmax = 0ull;
+  int cnt = 0;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long rounds = (n + stride - 1) / stride;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const unsigned lt = (1u << lane_id()) - 1;
+  for (long long r = 0; r < rounds; ++r, i += stride) {
+    unsigned long long key = ~0ull;
+    int slot = -1;
+    if (i < n) { slot = level == 0 ? (int)i : cand[i]; key = a.keys[slot]; }
+    const bool on = key != ~0ull;
+    const int digit = on ? (int)((unsigned)(key >> shift) & (TAURUS_SEL_BINS - 1)) : TAURUS_SEL_BINS;
+    const bool victim = digit < digit_k || (final && digit == digit_k);
+    const bool keep = !final && digit == digit_k;
+    const unsigned mv = __ballot_sync(FULL, victim), mk = __ballot_sync(FULL, keep);
+    if (mv) {
+      int idx = 0;
+      const int leader = __ffs(mv) - 1;
+      if (lane_id() == leader) idx = atomicAdd(&ctl->victim_count, __popc(mv));
+      idx = __shfl_sync(FULL, idx, leader) + __popc(mv & lt);
+      if (victim && idx < a.victim_capacity) a.victims[idx].x = slot;
+    }
+    if (mk) {
+      int idx = 0;
+      const int leader = __ffs(mk) - 1;
+      if (lane_id() == leader) idx = atomicAdd(&ctl->sel_count[level + 1], __popc(mk));
+      idx = __shfl_sync(FULL, idx, leader) + __popc(mk & lt);
+      if (keep) {
+        next[idx] = slot;   // at most pool_slots keys enter any level
+        if (key < kmin) kmin = key;
+        if (key > kmax) kmax = key;
+        cnt++;
+      }
+    }
+  }
+  // sel_count of the next level is already counted by the appends: fold only the key range
+  for (int o = 16; o; o >>= 1) {
+    const unsigned long long m = __shfl_xor_sync(FULL, kmin, o), M = __shfl_xor_sync(FULL, kmax, o);
+    if (m < kmin) kmin = m;
+    if (M > kmax) kmax = M;
+    cnt += __shfl_xor_sync(FULL, cnt, o);
+  }
+  if (lane_id() == 0 && cnt) {
+    atomicMin(&ctl->sel_min[level + 1], kmin);
+    atomicMax(&ctl->sel_max[level + 1], kmax);
   }
 }
 
-__global__ void evict_list_kernel(ChunkArgs a) {
+// ---- host store: where a victim's row goes
+// Largest in-list position of v whose source is below `src_end` ... the first message still to come decides the
+// bucket: the source of the first propagated in-edge of v at or behind src_end, or v itself while its own chunk (which
+// delivers its self message) has not been pushed.
+static __device__ __forceinline__ long long next_sender(const ChunkArgs& a, int v) {
+  long long lo = a.csc_ptr[v];
+  const long long end = a.csc_ptr[v + 1];
+  long long hi = end;
+  while (lo < hi) {   // first in-list entry with source >= src_end (the in-list is sorted by source)
+    const long long mid = (lo + hi) >> 1;
+    if ((long long)a.csc_src[mid] < a.src_end) lo = mid + 1; else hi = mid;
+  }
+  if (a.mask && a.csc_eid) {
+    while (lo < end) {
+      const uint32_t e = a.csc_eid[lo];
+      if ((a.mask[e >> 5] >> (e & 31)) & 1u) break;
+      ++lo;
+    }
+  }
+  long long ns = lo < end ? (long long)a.csc_src[lo] : a.V;
+  if (v >= a.src_end && v < ns) ns = v;
+  return ns;
+}
+
+__global__ void __launch_bounds__(256) victim_bucket_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
   if (ctl->error || ctl->deficit == 0) return;
-  const unsigned long long thr = ctl->sel_prefix;
-  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  for (long long base = warp0 * 32; base < a.pool_slots; base += warps * 32) {
-    long long s = base + lane_id();
-    bool hit = s < a.pool_slots && a.keys[s] <= thr;   // ~0 (ineligible) is never <= a real key
-    unsigned m = __ballot_sync(FULL, hit);
-    if (m) {
-      int leader = __ffs(m) - 1, idx = 0;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->victim_count, __popc(m));
-      idx = __shfl_sync(FULL, idx, leader) + __popc(m & ((1u << lane_id()) - 1));
-      // victim idx takes the host row host_free[H - 1 - idx]; read here, before this chunk's reloads push rows back
-      if (hit && idx < a.victim_capacity) a.victims[idx] = make_int2((int)s, a.host_free[ctl->host_pop_base - 1 - idx]);
+  const int n = ctl->deficit;
+  if (ctl->victim_count != n) {   // the select must have produced exactly `deficit` victims
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+    return;
+  }
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const int slot = a.victims[i].x;
+    const int v = a.owner[slot];
+    long long ns = next_sender(a, v);
+    if (ns >= a.V) { atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL); ns = a.V - 1; }   // a victim has a message to come
+    const int b = (int)(ns / a.chunk_sources);
+    a.vic_place[i] = make_int2(b, atomicAdd(&a.bk_new[b], 1));
+  }
+}
+
+// One block.  First the tails of the buckets whose grid cell ends inside this push are closed (no victim can be
+// filed there any more: its next sender would lie behind the push); then every bucket that received victims gets
+// the extents it lacks from the free stack.
+__global__ void __launch_bounds__(1024) extent_plan_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error) return;
+  const int E = 1 << a.ext_shift;
+  __shared__ int warp_sum[32];
+  __shared__ long long s_running;
+  __shared__ int s_fail;
+  if (threadIdx.x == 0) { s_running = 0; s_fail = 0; }
+  // phase 1: close tails
+  {
+    const long long first = a.src_begin / a.chunk_sources;
+    const long long b = first + threadIdx.x;
+    if (threadIdx.x < 2 && b < a.n_buckets) {
+      long long cell_end = (b + 1) * a.chunk_sources;
+      if (cell_end > a.V) cell_end = a.V;
+      const int t = a.bk_tail_ext[b];
+      if (cell_end <= a.src_end && t >= 0) {
+        const int unused = E - a.bk_tail_fill[b];
+        if (unused > 0 && atomicSub(&a.ext_live[t], unused) == unused) {   // every row it held is already back in the pool
+          const long long top = (long long)atomicAdd((unsigned long long*)&ctl->ext_free_top, 1ull);
+          a.ext_free[top] = t;
+        }
+        a.bk_tail_ext[b] = -1;
+        a.bk_tail_fill[b] = 0;
+      }
     }
+  }
+  __syncthreads();
+  if (ctl->deficit == 0) return;
+  // phase 2: extents needed per bucket, exclusive prefix over the buckets
+  for (long long base = 0; base < a.n_buckets; base += blockDim.x) {
+    const long long b = base + threadIdx.x;
+    int want = 0;
+    if (b < a.n_buckets) {
+      const int nw = a.bk_new[b];
+      if (nw > 0) {
+        const int t = a.bk_tail_ext[b], f = a.bk_tail_fill[b];
+        a.bk_base[b] = make_int2(t, f);
+        const int room = t >= 0 ? E - f : 0;
+        const int extra = nw > room ? nw - room : 0;
+        want = (extra + E - 1) >> a.ext_shift;
+      }
+    }
+    int x = want;
+    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(FULL, x, o); if (lane_id() >= o) x += y; }
+    if (lane_id() == 31) warp_sum[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      int w = warp_sum[threadIdx.x];
+      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(FULL, w, o); if (lane_id() >= o) w += y; }
+      warp_sum[threadIdx.x] = w;   // inclusive over warps
+    }
+    __syncthreads();
+    const long long before = s_running + ((threadIdx.x >> 5) ? warp_sum[(threadIdx.x >> 5) - 1] : 0) + (x - want);
+    if (b < a.n_buckets && a.bk_new[b] > 0) a.bk_off[b] = (int32_t)before;
+    __syncthreads();
+    if (threadIdx.x == 0) s_running += warp_sum[31];
+    __syncthreads();
+  }
+  const long long total = s_running;
+  if (total > ctl->ext_free_top) {
+    if (threadIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_HOST_STORE_FULL);
+    return;
+  }
+  const long long stack_base = ctl->ext_free_top - total;
+  __syncthreads();
+  if (threadIdx.x == 0) ctl->ext_free_top = stack_base;
+  // phase 3: hand the extents out and move the tails
+  for (long long b = threadIdx.x; b < a.n_buckets; b += blockDim.x) {
+    const int nw = a.bk_new[b];
+    if (nw <= 0) continue;
+    const int2 base = a.bk_base[b];
+    const int room = base.x >= 0 ? E - base.y : 0;
+    const int extra = nw > room ? nw - room : 0;
+    const int want = (extra + E - 1) >> a.ext_shift;
+    const int off = a.bk_off[b];
+    for (int j = 0; j < want; ++j) {
+      const int e = a.ext_free[stack_base + off + j];
+      a.new_ext[off + j] = e;
+      a.ext_live[e] = E;
+    }
+    if (want > 0) { a.bk_tail_ext[b] = a.new_ext[off + want - 1]; a.bk_tail_fill[b] = extra - ((want - 1) << a.ext_shift); }
+    else a.bk_tail_fill[b] = base.y + nw;
+  }
+}
+
+__global__ void __launch_bounds__(256) victim_place_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  if (ctl->error || ctl->deficit == 0) return;
+  const int n = ctl->deficit;
+  const int E = 1 << a.ext_shift;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+    const int2 pl = a.vic_place[i];
+    const int2 base = a.bk_base[pl.x];
+    const int room = base.x >= 0 ? E - base.y : 0;
+    int ext, idx;
+    if (pl.y < room) { ext = base.x; idx = base.y + pl.y; }
+    else { const int q = pl.y - room; ext = a.new_ext[a.bk_off[pl.x] + (q >> a.ext_shift)]; idx = q & (E - 1); }
+    a.victims[i].y = (ext << a.ext_shift) + idx;
+    a.bk_new[pl.x] = 0;   // same value from every victim of the bucket; nothing reads the count after the plan
   }
 }
 
@@ -294,10 +546,6 @@ __global__ void alloc_kernel(ChunkArgs a) {
   if (ctl->error) return;
   const int n = ctl->need_count;
   const int deficit = ctl->deficit;
-  if (deficit > 0 && ctl->victim_count != deficit) {   // the select must have produced exactly `deficit` victims
-    if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
-    return;
-  }
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
   if (a.direct) {
@@ -333,8 +581,7 @@ __global__ void alloc_kernel(ChunkArgs a) {
     int v = a.need_list[i];
     int slot = -1, st = 0, l = 0, out_hrow = -1, victim = -1;
     if (lane_id() == 0) {
-      if (a.direct) slot = v;
-      else if (i < deficit) {
+      if (i < deficit) {
         const int2 vic = a.victims[deficit - 1 - i];
         slot = vic.x; out_hrow = vic.y; victim = a.owner[slot];
       } else { long long f = ctl->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
@@ -379,15 +626,16 @@ __global__ void alloc_kernel(ChunkArgs a) {
         a.state[victim] = TAURUS_EVICTED;
       }
       if (in_hrow >= 0) {
-        long long h = atomicAdd((unsigned long long*)&ctl->host_free_top, 1ull);
-        a.host_free[h] = in_hrow;
+        const int e = in_hrow >> a.ext_shift;
+        if (atomicSub(&a.ext_live[e], 1) == 1) {   // last row of the extent: back on the free stack (popped again by a later chunk's plan)
+          const long long top = (long long)atomicAdd((unsigned long long*)&ctl->ext_free_top, 1ull);
+          a.ext_free[top] = e;
+        }
         a.reload_count[v] += 1;
         reloaded++;
       }
-      if (!a.direct) {
-        a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch;
-        if (a.slot_touch) a.slot_touch[slot] = a.epoch;   // slot_pend follows in compact_done: v is on the touched list
-      }
+      a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch;
+      if (a.slot_touch) a.slot_touch[slot] = a.epoch;   // slot_pend follows in compact_done: v is on the touched list
       a.state[v] = TAURUS_IN_BUFFER;
     }
   }
@@ -397,18 +645,21 @@ __global__ void alloc_kernel(ChunkArgs a) {
 void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   const int blocks = c->sm_count * 8;
   if (!a.direct) {   // direct-mapped pools plan inside alloc_kernel
-    plan_kernel<<<1, 32, 0, st>>>(a);
+    plan_kernel<<<1, 256, 0, st>>>(a);
     c->launches += 1;
   }
   if (c->pool_slots < c->V - c->hub_count) {   // eviction is impossible when every non-hub vertex has a slot
     select_keys_kernel<<<blocks, 256, 0, st>>>(a);
-    select_resolve_kernel<<<1, 1024, 0, st>>>(a, 0);
-    for (int p = 1; p < TAURUS_SEL_PASSES; ++p) {
-      select_hist_kernel<<<blocks, 256, 0, st>>>(a, p);
-      select_resolve_kernel<<<1, 1024, 0, st>>>(a, p);
+    for (int l = 0; l < TAURUS_SEL_LEVELS; ++l) {
+      // deeper levels work on what is left of one digit of the level above: a handful of blocks is enough
+      const int b = l == 0 ? blocks : l == 1 ? c->sm_count * 2 : c->sm_count;
+      select_hist_kernel<<<b, 256, 0, st>>>(a, l);
+      select_split_kernel<<<b, 256, 0, st>>>(a, l);
     }
-    evict_list_kernel<<<blocks, 256, 0, st>>>(a);
-    c->launches += 2 * TAURUS_SEL_PASSES + 1;
+    victim_bucket_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
+    extent_plan_kernel<<<1, 1024, 0, st>>>(a);
+    victim_place_kernel<<<c->sm_count * 2, 256, 0, st>>>(a);
+    c->launches += 2 * TAURUS_SEL_LEVELS + 4;
   }
   alloc_kernel<<<blocks, 256, 0, st>>>(a);
   c->launches += 1;

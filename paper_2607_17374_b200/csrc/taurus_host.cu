@@ -70,7 +70,10 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   free_tc_weights(c);
   cudaFree(c->d_pend); cudaFree(c->d_state); cudaFree(c->d_loc); cudaFree(c->d_touch); cudaFree(c->d_reload);
   cudaFree(c->d_hub); cudaFree(c->d_hub_ids); cudaFree(c->d_acc); cudaFree(c->d_owner); cudaFree(c->d_free_stack);
-  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_slot_touch); cudaFree(c->d_slot_pend); cudaFree(c->d_victims); cudaFree(c->d_keys); cudaFree(c->d_host_free);
+  cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_slot_touch); cudaFree(c->d_slot_pend); cudaFree(c->d_victims); cudaFree(c->d_keys);
+  cudaFree(c->d_cand[0]); cudaFree(c->d_cand[1]); cudaFree(c->d_ext_free); cudaFree(c->d_ext_live); cudaFree(c->d_bk_tail_ext);
+  cudaFree(c->d_bk_tail_fill); cudaFree(c->d_bk_new); cudaFree(c->d_bk_off); cudaFree(c->d_bk_base); cudaFree(c->d_new_ext);
+  cudaFree(c->d_vic_place); cudaFree(c->d_csc_src);
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_X);
@@ -233,14 +236,30 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   ALLOC(c->d_owner, c->pool_slots); ALLOC(c->d_free_stack, c->pool_slots); ALLOC(c->d_need_list, c->pool_slots);
   ALLOC(c->d_slot_epoch, c->pool_slots);   // written at every slot hand-out, also when no eviction can happen
-  if (c->pool_slots < V - c->hub_count) {   // a chunk evicts at most what it needs, and it needs at most what it touches
+  const bool can_evict = c->pool_slots < V - c->hub_count;
+  if (can_evict) {   // a chunk evicts at most what it needs, and it needs at most what it touches
     c->victim_capacity = std::min<long long>(c->pool_slots, c->touched_capacity);
     ALLOC(c->d_victims, c->victim_capacity); ALLOC(c->d_keys, c->pool_slots);
+    ALLOC(c->d_cand[0], c->pool_slots); ALLOC(c->d_cand[1], c->pool_slots);
     ALLOC(c->d_slot_touch, c->pool_slots); ALLOC(c->d_slot_pend, c->pool_slots);
+    ALLOC(c->d_vic_place, c->victim_capacity);
   }
-  ALLOC(c->d_host_free, c->host_rows);
-  if (c->host_rows > 0) {
-    cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->host_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
+  if (can_evict && c->host_rows > 0) {
+    // Host store of evicted rows: extents of 2^ext_shift rows.  Evicted rows are filed by the grid cell of their
+    // vertex's next sender (one open extent per cell), so the store holds up to one partly filled extent per cell on
+    // top of the rows themselves; twice that many spare extents cover pushes that are not whole grid cells.
+    c->n_buckets = (V + c->chunk_sources - 1) / c->chunk_sources;
+    long long per = c->host_rows / (4 * c->n_buckets);
+    c->ext_shift = 3;
+    while (c->ext_shift < 10 && (2ll << c->ext_shift) <= per) c->ext_shift += 1;
+    const long long ext_rows = 1ll << c->ext_shift;
+    c->n_ext = (c->host_rows + ext_rows - 1) / ext_rows + 2 * c->n_buckets + 8;
+    if (c->n_ext * ext_rows >= (1ll << 31) - 2) return TAURUS_ERR_INVALID_ARG;
+    ALLOC(c->d_ext_free, c->n_ext); ALLOC(c->d_ext_live, c->n_ext);
+    ALLOC(c->d_bk_tail_ext, c->n_buckets); ALLOC(c->d_bk_tail_fill, c->n_buckets); ALLOC(c->d_bk_new, c->n_buckets);
+    ALLOC(c->d_bk_off, c->n_buckets); ALLOC(c->d_bk_base, c->n_buckets);
+    ALLOC(c->d_new_ext, (c->victim_capacity >> c->ext_shift) + c->n_buckets + 1);
+    cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->n_ext * ext_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
     if (e != cudaSuccess) { cuda_ok(e, "cudaHostAlloc(evicted-row store)"); c->h_store = nullptr; return TAURUS_ERR_NOMEM; }
     CU(cudaHostGetDevicePointer((void**)&c->d_store_alias, c->h_store, 0));
   }
@@ -265,15 +284,31 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     CU(cudaMemset(c->d_af_A, 0, (size_t)c->drain_rows * af_kmax * (sage ? 2 : 1) * sizeof(float)));
     if (sage) ALLOC(c->d_af_X, (size_t)V * af_kmax);
   }
-  // sampling
-  if (any_sampled) {
+  // In-lists (ascending source id).  Sampled layers pick in-list positions; the host store files an evicted row by the
+  // next sender of its vertex, read from the vertex's in-list.
+  const bool grouping = !(c->flags & TAURUS_FLAG_NO_GROUPING);
+  const bool need_src = c->n_ext > 0;
+  if (any_sampled || (need_src && !grouping)) {
     int rc = build_in_edge_order(c);
     if (rc) { cuda_ok(cudaGetLastError(), "build_in_edge_order"); return rc; }
-    ALLOC(c->d_mask, (E + 31) / 32);
+    if (any_sampled) ALLOC(c->d_mask, (E + 31) / 32);
+  }
+  bool src_from_groups = false;
+  if (need_src) {
+    ALLOC(c->d_csc_src, E);
+    if (c->d_csc_eid) {
+      int rc = build_csc_src_from_eid(c);
+      if (rc) { cuda_ok(cudaGetLastError(), "build_csc_src_from_eid"); return rc; }
+      if (!any_sampled) { cudaFree(c->d_csc_eid); c->d_csc_eid = nullptr; }
+    } else {
+      int rc = build_csc_ptr(c);
+      if (rc) { cuda_ok(cudaGetLastError(), "build_csc_ptr"); return rc; }
+      src_from_groups = true;
+    }
   }
   // destination-grouped edge order of the chunk grid
-  if (!(c->flags & TAURUS_FLAG_NO_GROUPING)) {
-    int rc = build_grouped_order(c, any_sampled);
+  if (grouping) {
+    int rc = build_grouped_order(c, any_sampled, src_from_groups);
     if (rc) { cuda_ok(cudaGetLastError(), "build_grouped_order"); return rc; }
     if (any_sampled) ALLOC(c->d_gmask, (E + 31) / 32);
   }
@@ -395,7 +430,12 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.acc = c->d_acc; a.owner = c->d_owner; a.free_stack = c->d_free_stack; a.need_list = c->d_need_list; a.slot_epoch = c->d_slot_epoch;
   a.slot_touch = c->d_slot_touch; a.slot_pend = c->d_slot_pend;
   a.touched_list = c->d_touched_list; a.touched_capacity = c->touched_capacity;
-  a.victims = c->d_victims; a.victim_capacity = c->victim_capacity; a.keys = c->d_keys; a.host_store = c->d_store_alias; a.host_free = c->d_host_free;
+  a.victims = c->d_victims; a.victim_capacity = c->victim_capacity; a.keys = c->d_keys; a.host_store = c->d_store_alias;
+  a.cand[0] = c->d_cand[0]; a.cand[1] = c->d_cand[1];
+  a.ext_free = c->d_ext_free; a.ext_live = c->d_ext_live; a.bk_tail_ext = c->d_bk_tail_ext; a.bk_tail_fill = c->d_bk_tail_fill;
+  a.bk_new = c->d_bk_new; a.bk_off = c->d_bk_off; a.bk_base = c->d_bk_base; a.new_ext = c->d_new_ext; a.vic_place = c->d_vic_place;
+  a.csc_ptr = c->d_csc_ptr; a.csc_src = c->d_csc_src; a.csc_eid = c->d_csc_eid;
+  a.chunk_sources = c->chunk_sources; a.n_ext = c->n_ext; a.n_buckets = c->n_buckets; a.ext_shift = c->ext_shift;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
   a.Hp = taurus_round_up(c->dims[l + 1], 4);
   a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;   // GAT pass 3 scatters h' rows repacked to pitch Hp

@@ -15,7 +15,7 @@
 #define TAURUS_MAX_TIMED_PUSHES 16384
 #define TAURUS_SEL_BITS 11                      // radix-select digit width
 #define TAURUS_SEL_BINS (1 << TAURUS_SEL_BITS)
-#define TAURUS_SEL_PASSES 6                     // 6 x 11 = 66 bits >= the 62-bit (pending, id) key
+#define TAURUS_SEL_LEVELS 6                     // 6 x 11 = 66 bits >= the 62-bit (score, id) key
 
 // Device-resident control block: counters the kernels of one chunk hand to one another, so that
 // no step of a push needs the host.  One per context.
@@ -29,15 +29,18 @@ struct DevCtl {
   int32_t hs, ns, ev, gs; // touched vertices by state at chunk start
   int32_t reloaded;       // reloads this chunk
   long long free_top;       // entries on the free-slot stack
-  long long host_free_top;  // entries on the free-host-row stack
+  long long ext_free_top;   // entries on the free-extent stack of the host store
+  long long host_live;      // rows currently held by the host store
   long long grad_count;     // rows waiting in the graduation buffer
   long long out_count[2];   // dense-output mode: rows finalise left in each half of the graduation buffer
   long long alloc_base;       // this chunk: need-list entry i takes free_stack[alloc_base - 1 - i]
-  long long evict_push_base;  // this chunk: free-stack height before the chunk (victims' slots go straight to the vertices that need them)
-  long long host_pop_base;    // this chunk: victim i's row goes to host row host_free[host_pop_base - 1 - i]
-  unsigned long long sel_prefix;  // radix select: digits fixed so far (high bits)
-  long long sel_k;                // radix select: rank still to resolve inside the prefix bucket
-  unsigned int hist[TAURUS_SEL_BINS];
+  // Victim select, level by level (level 0 scans the pool, deeper levels the candidates the level above left):
+  long long sel_k[TAURUS_SEL_LEVELS + 1];               // rank still to resolve among the keys entering the level
+  unsigned long long sel_min[TAURUS_SEL_LEVELS + 1];    // smallest / largest key entering the level: the digit of a level
+  unsigned long long sel_max[TAURUS_SEL_LEVELS + 1];    //   starts at the highest bit in which they differ
+  int32_t sel_count[TAURUS_SEL_LEVELS + 1];             // keys entering the level
+  int32_t sel_final_level;                              // level that listed the last victims; kernels of deeper levels return
+  unsigned int hist[2][TAURUS_SEL_BINS];                // digit histogram, alternating between levels
   // layer totals
   long long evictions, reloads, peak_occupancy, hub_messages, total_messages, completed;
   long long sum_hs, sum_ns, sum_ev, sum_gs, chunks;
@@ -74,8 +77,26 @@ struct ChunkArgs {
   int2* victims;            // [victim_capacity] (slot, pinned host row) of this chunk's victims
   long long victim_capacity;
   unsigned long long* keys; // [pool_slots]
-  float* host_store;        // device alias of the pinned host rows [host_evict_rows x Hp]
-  int32_t* host_free;       // [host_evict_rows]
+  int32_t* cand[2];         // [pool_slots] each: slots still in the running for the last victims, alternating between levels
+  // Host store of evicted rows (pinned, mapped): extents of (1 << ext_shift) rows handed out from a free stack.  A
+  // victim's row is filed under the grid cell of the source that sends its vertex the next message ("bucket"), so
+  // the rows a chunk reloads sit together and the rows it evicts are appended to a few hundred open extents.
+  float* host_store;        // device alias of the pinned host rows [(n_ext << ext_shift) x Hp]
+  int32_t* ext_free;        // [n_ext] stack of free extents
+  int32_t* ext_live;        // [n_ext] rows of the extent not yet reloaded, plus its rows not yet handed out
+  int32_t* bk_tail_ext;     // [buckets] extent the bucket appends to, -1 none
+  int32_t* bk_tail_fill;    // [buckets] rows handed out of that extent
+  int32_t* bk_new;          // [buckets] this chunk: victims filed under the bucket
+  int32_t* bk_off;          // [buckets] this chunk: first of the bucket's new extents in new_ext
+  int2* bk_base;            // [buckets] this chunk: (tail extent, tail fill) before the chunk's victims
+  int32_t* new_ext;         // [victim_capacity >> ext_shift + buckets] this chunk: extents taken from the stack
+  int2* vic_place;          // [victim_capacity] this chunk: (bucket, rank among the chunk's victims of that bucket)
+  const long long* csc_ptr; // [V + 1] in-lists (ascending source id): offsets,
+  const int32_t* csc_src;   // [E]       sources,
+  const uint32_t* csc_eid;  // [E]       CSR edge indices (sampled layers: the mask is looked up through them), else NULL
+  long long chunk_sources;  // width of a grid cell in sources
+  long long n_ext, n_buckets;
+  int32_t ext_shift;
   // graduation buffer
   long long* grad_ids;
   float* grad_rows;         // [drain_rows x Hp]
@@ -173,9 +194,21 @@ struct taurus_ctx {
   int2* d_victims = nullptr;
   long long victim_capacity = 0;
   unsigned long long* d_keys = nullptr;
+  int32_t* d_cand[2] = {nullptr, nullptr};
   float* h_store = nullptr;      // pinned, mapped
   float* d_store_alias = nullptr;
-  int32_t* d_host_free = nullptr;
+  int32_t* d_ext_free = nullptr;
+  int32_t* d_ext_live = nullptr;
+  int32_t* d_bk_tail_ext = nullptr;
+  int32_t* d_bk_tail_fill = nullptr;
+  int32_t* d_bk_new = nullptr;
+  int32_t* d_bk_off = nullptr;
+  int2* d_bk_base = nullptr;
+  int32_t* d_new_ext = nullptr;
+  int2* d_vic_place = nullptr;
+  int32_t* d_csc_src = nullptr;   // in-list sources, built when rows can be evicted
+  long long n_ext = 0, n_buckets = 0;
+  int ext_shift = 0;
   long long* d_grad_ids = nullptr;
   float* d_grad_rows = nullptr;
   int32_t* d_done_list = nullptr;
@@ -292,12 +325,14 @@ void free_tc_weights(taurus_ctx* c);
 bool project_tc_usable(const taurus_ctx* c, int layer, const float* X, int ldx);
 int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st);
 // ---- kernels_group.cu
-int build_grouped_order(taurus_ctx* c, bool keep_edge_ids);
+int build_grouped_order(taurus_ctx* c, bool keep_edge_ids, bool fill_csc_src);   // fill_csc_src: also writes csc_src (needs csc_ptr)
 void launch_group_mask(taurus_ctx* c, cudaStream_t st);
 void launch_classify_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 // ---- kernels_sample.cu
 int build_in_edge_order(taurus_ctx* c);                                      // csc_ptr, csc_eid
+int build_csc_ptr(taurus_ctx* c);                                            // csc_ptr alone
+int build_csc_src_from_eid(taurus_ctx* c);                                   // csc_src from csc_eid (both in in-list order)
 void launch_sample_mask(taurus_ctx* c, int layer, cudaStream_t st);
 int sampled_edges_of(taurus_ctx* c, int layer, long long dst, long long* out_eids, int32_t* out_src, int cap, int* n);
 void launch_sample_digest(taurus_ctx* c, unsigned long long* d_digest, cudaStream_t st);   // d_digest [2V], zeroed by the caller
