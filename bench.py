@@ -336,14 +336,14 @@ def run_ours(args):
     launches = ctx.launch_count() - launches0
     sampler.stop_flag.set()
     sampler.join()
-    phases = ctx.get_phase_ms()   # [pushes, 5]
+    phases = ctx.get_phase_ms()   # [pushes, 6]
     ms_max = max_over_ranks(ms, world, dev)
     value = whole_job_value(msgs_per_step, args.steps, world, ms_max)
 
     # ---- roofline of the dominant kernel (the scatter), from the events recorded inside the timed region
     n_push = len(chunks) * L * args.steps
-    ph = phases[:n_push].reshape(args.steps, L, len(chunks), 5)
-    scatter_ms = ph[..., 3]
+    ph = phases[:n_push].reshape(args.steps, L, len(chunks), 6)
+    scatter_ms = ph[..., 4]
     # Algorithmic bytes of the scatter: per accumulator-row reduction a read-modify-write of
     # the row (2 * 4 Hp) plus slot and pending-count words (8); per propagated edge its (destination, source)
     # words (8); per source its projected row read once (4 Hp) and its self message (row read 4 Hp + RMW 2 * 4 Hp + 8).
@@ -390,7 +390,7 @@ def run_ours(args):
                                     groups=int(groups_per_layer[l]), accumulator_floats=acc_width[l], aggregate_first=bool(agg_first[l]),
                                     gteps_scatter_only=edges_per_layer[l] / (per_layer_ms[l] * 1e-3) / 1e9)
                                for l in range(L)])
-    phase_ms = dict(zip(["copy_in", "projection", "classify_make_room", "scatter", "finalise"],
+    phase_ms = dict(zip(["copy_in", "projection", "classify_select", "row_moves", "scatter", "finalise"],
                         [float(x) / args.steps for x in ph.sum(axis=(0, 1, 2))]))
 
     # ---- end to end through the C ABI with host buffers: every step streams the layer-0 features from pinned host

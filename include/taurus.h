@@ -130,8 +130,10 @@ enum {
                                    applies the weights to the finished rows instead (exact by linearity, Sect. 3.6 / 3.9): the
                                    accumulators, the scatter traffic and every evicted row shrink by d_in / d_out.  SAGE layers
                                    keep every vertex's input row on the device until the vertex completes (its self term goes
-                                   through W_self with the transform) and do so only while that store (V x d_in floats) stays
-                                   below 64 GiB */
+                                   through W_self with the transform): V x d_in floats of device memory that stay allocated
+                                   for the life of the context.  They take this order only while that store fits in the
+                                   device memory free at taurus_graph_init beside an estimate of everything else the context
+                                   allocates; taurus_get_layer_plan tells which order a layer got */
 };
 
 /* Integer accounting of one layer pass (Sect. 4.4-4.7 report these quantities). */
@@ -300,7 +302,9 @@ int taurus_completion_bound(taurus_ctx* ctx, int64_t src_begin, int64_t src_end,
  * max(v, largest source among the propagated in-edges of v) lies in [64 b, 64 b + 64): the vertices a
  * push of those 64 sources completes (Sect. 3.8, c(v)).  edge_mask is the layer's propagated-edge mask in
  * the format of taurus_get_edge_mask, or NULL when every edge is propagated.  *out_bad_index is set to 1
- * if a destination outside [0, V) was met (such edges are skipped), else 0.
+ * if a destination outside [0, V) was met (such edges are skipped) or if a row of row_ptr does not lie
+ * inside [0, E] in ascending order (the row is cut to the part inside [0, E], so col_idx and edge_mask are
+ * never read beyond their E entries, and the counts are then not meaningful), else 0.
  *
  * Arguments: row_ptr [V+1], col_idx [E], edge_mask [ceil(E/32)] or NULL, out_counts [ceil(V/64)] and
  * out_bad_index [1] are DEVICE pointers owned by the caller; the work is enqueued on cuda_stream
@@ -423,13 +427,20 @@ int taurus_relabel_csr(int64_t V, int64_t E, const int64_t* row_ptr, const int32
 int taurus_permute_rows(int64_t V, int32_t width, const float* in_rows, int64_t ld_in, const int32_t* rank, float* out_rows,
                         int64_t ld_out, void* cuda_stream);
 
+/* Which order layer `layer` runs in: *out_aggregate_first = 1 when it aggregates (scaled) input rows and applies the
+ * weights to the finished rows (see TAURUS_FLAG_PROJECT_FIRST), 0 when it projects every chunk first;
+ * *out_row_floats = floats per accumulator row (and per evicted row) of that layer.  Either pointer may be NULL.
+ * Decided at taurus_graph_init; no device work. */
+int taurus_get_layer_plan(const taurus_ctx* ctx, int32_t layer, int32_t* out_aggregate_first, int32_t* out_row_floats);
+
 /* Kernels launched by this context since init (for launch accounting in benchmarks). */
 int64_t taurus_launch_count(const taurus_ctx* ctx);
 
 /* Per-push device times.  taurus_set_timing(ctx, 1) starts a recording window: every later push (up to
  * 16384) brackets its phases with CUDA events on the push's stream.  taurus_get_phase_ms (blocking) returns,
- * for each recorded push p, out[p * 5 + k] in milliseconds: k = 0 copy-in, 1 projection, 2 classify..reload,
- * 3 scatter, 4 finalise; *out_pushes = pushes written (at most capacity_pushes). */
+ * for each recorded push p, out[p * 6 + k] in milliseconds: k = 0 copy-in, 1 projection, 2 classify and victim
+ * selection, 3 row moves (evicted rows out, reloaded rows in, new rows cleared), 4 scatter, 5 finalise;
+ * *out_pushes = pushes written (at most capacity_pushes). */
 int taurus_set_timing(taurus_ctx* ctx, int32_t on);
 int taurus_get_phase_ms(taurus_ctx* ctx, float* out, int64_t capacity_pushes, int64_t* out_pushes);
 

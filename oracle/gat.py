@@ -24,9 +24,14 @@ import numpy as np
 
 
 def gat_layer_forward(ms, h: np.ndarray, W: np.ndarray, a_src: np.ndarray, a_dst: np.ndarray, bias: np.ndarray, act: int,
-                      slope: float = 0.2, dst: Optional[np.ndarray] = None) -> np.ndarray:
-    """out_v for v in dst (default: all).  ms is the layer's MessageSets (ptr, src)."""
+                      slope: float = 0.2, dst: Optional[np.ndarray] = None, magnitude: bool = False):
+    """out_v for v in dst (default: all).  ms is the layer's MessageSets (ptr, src).
+
+    magnitude=True returns (out, mag): mag_v = sum_u alpha_uv (|h_u| |W|) + |b|, the same weighted sum with every
+    product of the transform replaced by its absolute value (the scale against which a rounding error of the sum is
+    measured); `out` is unchanged by the flag."""
     hp = np.asarray(h, dtype=np.float64) @ np.asarray(W, dtype=np.float64)
+    hp_abs = np.abs(np.asarray(h, dtype=np.float64)) @ np.abs(np.asarray(W, dtype=np.float64)) if magnitude else None
     s = hp @ np.asarray(a_src, dtype=np.float64)
     t = hp @ np.asarray(a_dst, dtype=np.float64)
     b = np.asarray(bias, dtype=np.float64)
@@ -34,6 +39,7 @@ def gat_layer_forward(ms, h: np.ndarray, W: np.ndarray, a_src: np.ndarray, a_dst
     if dst is None:
         dst = np.arange(V, dtype=np.int64)
     out = np.empty((len(dst), hp.shape[1]), np.float64)
+    mag = np.empty_like(out) if magnitude else None
     for i, v in enumerate(dst):
         v = int(v)
         nb = np.concatenate([ms.src[ms.ptr[v]:ms.ptr[v + 1]].astype(np.int64), [v]])
@@ -43,4 +49,6 @@ def gat_layer_forward(ms, h: np.ndarray, W: np.ndarray, a_src: np.ndarray, a_dst
         alpha = w / w.sum()
         z = alpha @ hp[nb] + b
         out[i] = np.maximum(z, 0.0) if act else z
-    return out
+        if magnitude:
+            mag[i] = alpha @ hp_abs[nb] + np.abs(b)
+    return (out, mag) if magnitude else out

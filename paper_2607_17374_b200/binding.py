@@ -84,7 +84,7 @@ class _RunsConfig(ctypes.Structure):
 EXPORTS = [
     "taurus_graph_init", "taurus_layer_begin", "taurus_push_chunk", "taurus_drain_completed", "taurus_drain_dense",
     "taurus_layer_end", "taurus_get_stats", "taurus_get_chunk_log", "taurus_get_vertex_array",
-    "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count",
+    "taurus_get_sampled_edges", "taurus_get_edge_mask", "taurus_completion_bound", "taurus_launch_count", "taurus_get_layer_plan",
     "taurus_set_timing", "taurus_get_phase_ms", "taurus_destroy", "taurus_strerror", "taurus_last_cuda_error",
     "taurus_completion_counts_noalloc", "taurus_layer_set_dense_output", "taurus_reorder",
     "taurus_runs_create", "taurus_runs_append", "taurus_runs_flush", "taurus_runs_read_chunk", "taurus_runs_info",
@@ -139,6 +139,7 @@ def load_library():
     lib.taurus_gat_project_chunk_from_runs.argtypes = [vp, i64, i64, vp, vp, i64, vp]
     lib.taurus_relabel_csr.argtypes = [i64, i64, vp, vp, vp, vp, vp, vp, vp]
     lib.taurus_permute_rows.argtypes = [i64, i32, vp, i64, vp, vp, i64, vp]
+    lib.taurus_get_layer_plan.argtypes = [vp, ctypes.c_int32, vp, vp]
     lib.taurus_launch_count.argtypes = [vp]
     lib.taurus_launch_count.restype = i64
     lib.taurus_set_timing.argtypes = [vp, i32]
@@ -407,6 +408,13 @@ class Context:
         self._check(self._lib.taurus_completion_bound(self._h, src_begin, src_end, ctypes.byref(n)), "taurus_completion_bound")
         return int(n.value)
 
+    def layer_plan(self, layer: int):
+        """(aggregate_first, floats per accumulator row) of a layer, as decided at init."""
+        af, width = ctypes.c_int32(0), ctypes.c_int32(0)
+        self._check(self._lib.taurus_get_layer_plan(self._h, layer, ctypes.addressof(af), ctypes.addressof(width)),
+                    "taurus_get_layer_plan")
+        return bool(af.value), int(width.value)
+
     def launch_count(self) -> int:
         return int(self._lib.taurus_launch_count(self._h))
 
@@ -414,8 +422,9 @@ class Context:
         self._check(self._lib.taurus_set_timing(self._h, 1 if on else 0), "taurus_set_timing")
 
     def get_phase_ms(self, capacity_pushes: int = 16384) -> np.ndarray:
-        """float32 [pushes, 5]: copy-in, projection, classify..reload, scatter, finalise (ms) per recorded push."""
-        out = np.zeros((capacity_pushes, 5), np.float32)
+        """float32 [pushes, 6]: copy-in, projection, classify + victim selection, row moves (evict / reload / clear),
+        scatter, finalise (ms) per recorded push."""
+        out = np.zeros((capacity_pushes, 6), np.float32)
         n = ctypes.c_int64(0)
         self._check(self._lib.taurus_get_phase_ms(self._h, out.ctypes.data, capacity_pushes, ctypes.byref(n)),
                     "taurus_get_phase_ms")

@@ -138,14 +138,8 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
     if (a.dense_direct) O = c->d_grad_rows;
     else if (a.dense_half >= 0) O = c->d_grad_rows + (size_t)a.grad_off * a.Hout;
     else {
-      if (!c->d_af_O) {   // the place in the graduation buffer is known only on the device: transform into a scratch matrix
-        if (cudaMalloc((void**)&c->d_af_O, (size_t)c->drain_rows * c->Hmax * sizeof(float)) != cudaSuccess) {
-          cudaGetLastError();
-          c->d_af_O = nullptr;
-          return TAURUS_ERR_NOMEM;
-        }
-      }
-      O = c->d_af_O;
+      if (!c->d_af_O) return TAURUS_ERR_INTERNAL;   // allocated by the push before it enqueues anything
+      O = c->d_af_O;   // the place in the graduation buffer is known only on the device: transform into a scratch matrix
     }
     const bool sage = c->mode == TAURUS_SAGE_MEAN;
     const int Ka = sage ? 2 * a.Hp : a.Hp;               // columns of the gathered matrix

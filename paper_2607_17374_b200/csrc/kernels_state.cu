@@ -642,7 +642,7 @@ __global__ void alloc_kernel(ChunkArgs a) {
   if (lane_id() == 0 && reloaded) atomicAdd(&ctl->reloaded, reloaded);
 }
 
-void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEvent_t before_moves) {
   const int blocks = c->sm_count * 8;
   if (!a.direct) {   // direct-mapped pools plan inside alloc_kernel
     plan_kernel<<<1, 256, 0, st>>>(a);
@@ -661,6 +661,7 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
     victim_place_kernel<<<c->sm_count * 2, 256, 0, st>>>(a);
     c->launches += 2 * TAURUS_SEL_LEVELS + 4;
   }
+  if (before_moves) cudaEventRecord(before_moves, st);
   alloc_kernel<<<blocks, 256, 0, st>>>(a);
   c->launches += 1;
 }

@@ -24,12 +24,19 @@ static __global__ void na_rank_init_kernel(long long V, int32_t* rank) {
   for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) rank[v] = (int32_t)v;
 }
 
-static __global__ void na_rank_max_kernel(long long V, const long long* row_ptr, const int32_t* col, const uint32_t* mask,
+// A row range that leaves [0, E] or runs backwards is reported through *bad and clamped, so that neither the
+// destination array nor the edge mask is ever read outside its E entries.
+static __global__ void na_rank_max_kernel(long long V, long long E, const long long* row_ptr, const int32_t* col, const uint32_t* mask,
                                           int32_t* rank, int* bad) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int lane = threadIdx.x & 31;
   for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
     long long b = row_ptr[u], e = row_ptr[u + 1];
+    if (b < 0 || e > E || b > e) {
+      if (lane == 0) *bad = 1;
+      b = b < 0 ? 0 : b;
+      e = e > E ? E : e;
+    }
     for (long long k = b + lane; k < e; k += 32) {
       if (mask != nullptr && !((mask[k >> 5] >> (k & 31)) & 1u)) continue;
       int v = col[k];
@@ -67,7 +74,7 @@ extern "C" int taurus_completion_counts_noalloc(int64_t V, int64_t E, const int6
       cudaMemsetAsync(out_bad_index, 0, sizeof(int32_t), st) != cudaSuccess) { cudaGetLastError(); return TAURUS_ERR_CUDA; }
   const int grid = 148 * 8;
   na_rank_init_kernel<<<grid, 256, 0, st>>>(V, rank);
-  na_rank_max_kernel<<<grid, 256, 0, st>>>(V, reinterpret_cast<const long long*>(row_ptr), col_idx, edge_mask, rank, out_bad_index);
+  na_rank_max_kernel<<<grid, 256, 0, st>>>(V, E, reinterpret_cast<const long long*>(row_ptr), col_idx, edge_mask, rank, out_bad_index);
   na_rank_hist_kernel<<<grid, 256, 0, st>>>(V, rank, out_counts);
   if (cudaGetLastError() != cudaSuccess) return TAURUS_ERR_CUDA;
   return TAURUS_OK;

@@ -81,7 +81,7 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_att_s); cudaFree(c->d_att_t); cudaFree(c->d_att_max); cudaFree(c->d_att_tm); cudaFree(c->d_att_z);
   cudaFree(c->d_csc_ptr); cudaFree(c->d_csc_eid); cudaFree(c->d_mask); cudaFree(c->d_vtmp); cudaFree(c->d_rank_hist);
   cudaFree(c->d_gdst); cudaFree(c->d_gedge); cudaFree(c->d_geid); cudaFree(c->d_gmask);
-  cudaFree(c->d_ctl); cudaFree(c->d_chunk_log);
+  cudaFree(c->d_ctl); cudaFree(c->d_chunk_log); cudaFree(c->d_reload_hist);
   if (c->h_ctl) cudaFreeHost(c->h_ctl);
   if (c->order_event) cudaEventDestroy(c->order_event);
   for (int i = 0; i < 2; ++i) {
@@ -156,10 +156,17 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   // aggregate-first layers: input rows at most 3/4 as wide as output rows.  SAGE keeps every vertex's input row until
   // the vertex completes (its self term goes through W_self with the transform): only while that store stays small.
   int af_kmax = 0;
+  size_t free_b = 0, total_b = 0;
+  CU(cudaMemGetInfo(&free_b, &total_b));
+  // what the context still allocates besides that store, roughly: pool and hub rows, the grouped edge order (12 B per
+  // edge, 20 B while it is sorted), in-lists where rows can be evicted or layers are sampled, per-vertex words
+  const double other = (double)(c->pool_slots + c->hub_count) * c->Hmax * 4.0 + (double)E * 28.0 + (double)V * 64.0 +
+                       (double)c->pool_slots * 40.0 + (double)c->drain_rows * c->Hmax * 8.0;
   for (int l = 0; l < c->L; ++l) {
     const int Kp = taurus_round_up(c->dims[l], 4), Hp = taurus_round_up(c->dims[l + 1], 4);
     bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && 4 * Kp <= 3 * Hp;
-    if (af && c->mode == TAURUS_SAGE_MEAN && (size_t)V * Kp * sizeof(float) > ((size_t)64 << 30)) af = false;
+    // SAGE keeps V input rows on the device for such a layer: only while they fit beside everything else
+    if (af && c->mode == TAURUS_SAGE_MEAN && (double)V * Kp * sizeof(float) + other > 0.92 * (double)free_b) af = false;
     c->agg_first[l] = af;
     if (af) af_kmax = std::max(af_kmax, Kp);
   }
@@ -314,6 +321,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   }
   // control
   ALLOC(c->d_ctl, 1);
+  ALLOC(c->d_reload_hist, 18);
   CU(cudaMemset(c->d_ctl, 0, sizeof(DevCtl)));
   CU(cudaHostAlloc((void**)&c->h_ctl, sizeof(DevCtl), cudaHostAllocDefault));
   memset(c->h_ctl, 0, sizeof(DevCtl));
@@ -516,19 +524,25 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   if (halves ? bound > c->drain_rows / 2 : (direct_dense ? bound : c->ub_since_drain + bound) > c->drain_rows) return TAURUS_ERR_DRAIN_FULL;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   CU(cudaSetDevice(c->device));
+  const int l = c->layer;
+  if (c->agg_first[l] && !direct_dense && !halves && !c->d_af_O) {
+    // rows drained by the caller: their place in the graduation buffer is a device-side count, so the transform of
+    // the finished rows writes a scratch matrix first.  Allocated here, before anything of the chunk is enqueued, so
+    // that a failure leaves the layer untouched.
+    ALLOC(c->d_af_O, (size_t)c->drain_rows * c->Hmax);
+  }
   if (st != c->last_stream) {   // keep chunk order across streams
     CU(cudaEventRecord(c->order_event, c->last_stream));
     CU(cudaStreamWaitEvent(st, c->order_event, 0));
     c->last_stream = st;
   }
-  const int l = c->layer;
   const int K = gat ? c->dims[l + 1] : c->dims[l];
   const int n = (int)(src_end - src_begin);
   cudaEvent_t* pev = nullptr;
   if (c->timing && c->timed_pushes < TAURUS_MAX_TIMED_PUSHES) {
-    const size_t need = (size_t)(c->timed_pushes + 1) * 6;
+    const size_t need = (size_t)(c->timed_pushes + 1) * 7;
     while (c->phase_ev.size() < need) { cudaEvent_t e; CU(cudaEventCreate(&e)); c->phase_ev.push_back(e); }
-    pev = &c->phase_ev[(size_t)c->timed_pushes * 6];
+    pev = &c->phase_ev[(size_t)c->timed_pushes * 7];
     c->timed_pushes += 1;
   }
   const bool timing = pev != nullptr;
@@ -582,17 +596,17 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   const bool grouped = c->d_gdst != nullptr && src_begin % c->chunk_sources == 0 &&
                        src_end == std::min<long long>(c->V, src_begin + c->chunk_sources);
   if (grouped) launch_classify_grouped(c, a, st); else launch_classify(c, a, st);
-  launch_make_room(c, a, st);
-  if (timing) cudaEventRecord(pev[3], st);
+  launch_make_room(c, a, st, timing ? pev[3] : nullptr);   // pev[3]: victims chosen and placed, rows not yet moved
+  if (timing) cudaEventRecord(pev[4], st);
   // S5, S5', S6
   if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
   if (xbuf >= 0 && x_in_use) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }   // the scatter read the staged rows in place
-  if (timing) cudaEventRecord(pev[4], st);
+  if (timing) cudaEventRecord(pev[5], st);
   // S7
   if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
   if (af) {
     int rc = launch_af_finalise(c, a, l, std::min<long long>(bound, a.grad_cap), st);
-    if (rc) return rc;
+    if (rc) { c->h_ctl->error = rc; return rc; }   // the chunk is half applied: the layer has to be begun again
   } else {
     launch_finalise(c, a, st);
   }
@@ -620,7 +634,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
       if (!run_rc) c->run_pending_half = h;
     }
   }
-  if (timing) cudaEventRecord(pev[5], st);
+  if (timing) cudaEventRecord(pev[6], st);
   CU(cudaGetLastError());
   c->next_src = src_end;
   c->chunk_seq += 1;
@@ -796,13 +810,10 @@ extern "C" int taurus_layer_set_dense_output(taurus_ctx* c, float* dense_rows, i
 static int fill_stats(taurus_ctx* c, taurus_stats* s) {
   const DevCtl* h = c->h_ctl;
   memset(s, 0, sizeof(*s));
-  long long* d_hist = nullptr;
-  ALLOC(d_hist, 18);
-  launch_reload_histogram(c, d_hist, c->last_stream);
+  launch_reload_histogram(c, c->d_reload_hist, c->last_stream);
   long long hist[18];
-  cudaError_t e = cudaMemcpy(hist, d_hist, sizeof(hist), cudaMemcpyDeviceToHost);
-  cudaFree(d_hist);
-  CU(e);
+  CU(cudaMemcpyAsync(hist, c->d_reload_hist, sizeof(hist), cudaMemcpyDeviceToHost, c->last_stream));
+  CU(cudaStreamSynchronize(c->last_stream));
   long long nonzero = 0;
   for (int i = 1; i < 17; ++i) { s->reload_histogram[i] = hist[i]; nonzero += hist[i]; }
   s->reload_histogram[0] = c->V - nonzero;
@@ -905,6 +916,14 @@ extern "C" int taurus_get_sample_digest(taurus_ctx* c, uint64_t* out_digest) {
 
 extern "C" int64_t taurus_launch_count(const taurus_ctx* c) { return c ? c->launches : 0; }
 
+extern "C" int taurus_get_layer_plan(const taurus_ctx* c, int32_t layer, int32_t* out_aggregate_first, int32_t* out_row_floats) {
+  if (!c || layer < 0 || layer >= c->L) return TAURUS_ERR_INVALID_ARG;
+  const bool af = c->agg_first[layer];
+  if (out_aggregate_first) *out_aggregate_first = af ? 1 : 0;
+  if (out_row_floats) *out_row_floats = taurus_round_up(af ? c->dims[layer] : c->dims[layer + 1], 4);
+  return TAURUS_OK;
+}
+
 extern "C" int taurus_set_timing(taurus_ctx* c, int32_t on) {
   if (!c) return TAURUS_ERR_INVALID_ARG;
   c->timing = on ? 1 : 0;
@@ -918,8 +937,8 @@ extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out, int64_t capacity_p
   CU(cudaStreamSynchronize(c->last_stream));
   long long n = std::min<long long>(c->timed_pushes, capacity_pushes);
   for (long long p = 0; p < n; ++p)
-    for (int i = 0; i < 5; ++i)
-      CU(cudaEventElapsedTime(&out[p * 5 + i], c->phase_ev[(size_t)p * 6 + i], c->phase_ev[(size_t)p * 6 + i + 1]));
+    for (int i = 0; i < 6; ++i)
+      CU(cudaEventElapsedTime(&out[p * 6 + i], c->phase_ev[(size_t)p * 7 + i], c->phase_ev[(size_t)p * 7 + i + 1]));
   *out_pushes = n;
   return TAURUS_OK;
 }

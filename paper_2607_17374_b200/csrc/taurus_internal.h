@@ -238,6 +238,7 @@ struct taurus_ctx {
   int32_t* d_vtmp = nullptr;     // [V] scratch for layer_begin
   int32_t* d_rank_hist = nullptr;
   DevCtl* d_ctl = nullptr;
+  long long* d_reload_hist = nullptr;   // 18 words for the reload histogram of taurus_get_stats
   DevCtl* h_ctl = nullptr;       // pinned
   long long* d_chunk_log = nullptr;
   long long log_capacity = 0;
@@ -251,7 +252,7 @@ struct taurus_ctx {
   cudaEvent_t order_event = nullptr;
   long long launches = 0;
   int timing = 0;
-  std::vector<cudaEvent_t> phase_ev;   // 6 events per timed push, created on demand
+  std::vector<cudaEvent_t> phase_ev;   // 7 events per timed push, created on demand
   long long timed_pushes = 0;          // pushes recorded since timing was switched on
   std::vector<std::vector<long long>> rank_cum_cache;   // per layer: rank_cum computed at the first layer_begin
   int sm_count = 148;
@@ -264,7 +265,7 @@ static inline int taurus_proj_width(int mode, int Hp) { return mode == TAURUS_SA
 // ---- kernels_state.cu
 void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st);
 void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
-void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);   // plan, select, evict, alloc/reload
+void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEvent_t before_moves = nullptr);   // plan, select, placement, [event], row moves
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // compact + finalise + commit
 void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);

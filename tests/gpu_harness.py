@@ -107,7 +107,7 @@ def run_oracle(w, g, model, x0, evict_policy=0):
     din, dout = np.diff(inl.ptr), np.diff(g.row_ptr)
     hub = oracle.hub_set(g.in_degree, w.hub_count)
     h = x0.astype(np.float64)
-    out = dict(outs=[], sims=[], msets=[], hub=hub)
+    out = dict(outs=[], sims=[], msets=[], hub=hub, din=din, dout=dout)
     for l in range(w.L):
         ms = oracle.message_sets(inl, w.fanout[l], w.seed, l)
         if w.mode == tg.GAT:
@@ -121,6 +121,36 @@ def run_oracle(w, g, model, x0, evict_policy=0):
         out["sims"].append(oracle.simulate(g.V, g.row_ptr, g.col_idx, ms, hub, w.chunk, w.pool_slots, evict_policy, w.seed))
         out["msets"].append(ms)
     return out
+
+
+def layer_on_input(w, model, orc, l, h_in):
+    """Layer l evaluated by the oracle on the rows h_in (those the library consumed for that layer).  Returns
+    (ref, mag): ref is the layer's definition in fp64; mag is the same expression with every term replaced by its
+    absolute value,  c_in sum c_out |h_u| |W_neigh| + c_self |h_v| |W_self| + |b|  (GAT: attention weights times
+    |h_u| |W|): the sum of the magnitudes of everything that is added up for an output element."""
+    ms = orc["msets"][l]
+    h = np.asarray(h_in, dtype=np.float64)
+    if w.mode == tg.GAT:
+        from oracle import gat
+        return gat.gat_layer_forward(ms, h, model.W_neigh[l], model.att_src[l], model.att_dst[l], model.bias[l], model.act[l],
+                                     w.leaky_slope, magnitude=True)
+    ref = oracle.layer_forward(ms, w.mode, orc["din"], orc["dout"], h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l],
+                               gin_eps=w.gin_eps)
+    mag = oracle.layer_forward(ms, w.mode, orc["din"], orc["dout"], np.abs(h), np.abs(model.W_neigh[l]), np.abs(model.W_self[l]),
+                               np.abs(model.bias[l]), 0, gin_eps=w.gin_eps)   # 1 + eps > 0 for every eps the tests draw
+    return ref, mag
+
+
+def forward_error(got, ref, mag):
+    """max over rows of ||g_v - r_v||_inf / ||mag_v||_inf: the error of a row measured against the magnitude of what
+    was summed for it.  A computation that rounds every product and partial sum to a relative u ends below
+    (number of terms) * u on this scale, whatever the cancellation in the row; a dropped, doubled or misplaced term
+    ends near 1.  (The activation does not increase an error: |relu(a) - relu(b)| <= |a - b|.)"""
+    diff = np.abs(got.astype(np.float64) - ref).max(axis=1)
+    scale = np.abs(mag).max(axis=1)
+    exact = scale == 0
+    assert (diff[exact] == 0).all()          # nothing was summed: the row is exactly zero on both sides
+    return float((diff[~exact] / scale[~exact]).max()) if (~exact).any() else 0.0
 
 
 def row_error(got, ref):

@@ -43,3 +43,13 @@ def test_missing_library_fails_loudly(monkeypatch):
         assert "no CPU fallback" in str(e)
     else:
         raise AssertionError("expected a RuntimeError")
+
+
+def test_noalloc_entry_point_checks_its_sizes_before_touching_the_device():
+    """Size and pointer checks of the allocation-free entry point come before its first CUDA call, so they can be
+    exercised without a GPU."""
+    assert tb.completion_counts_noalloc(0, 0, 1, 1, None, 1, 1) == tb.ERROR_CODES["INVALID_ARG"]
+    assert tb.completion_counts_noalloc(10, -1, 1, 1, None, 1, 1) == tb.ERROR_CODES["INVALID_ARG"]
+    assert tb.completion_counts_noalloc(10, 5, 1, None, None, 1, 1) == tb.ERROR_CODES["INVALID_ARG"]     # edges but no destinations
+    assert tb.completion_counts_noalloc(10, 0, None, None, None, 1, 1) == tb.ERROR_CODES["INVALID_ARG"]
+    assert tb.completion_counts_noalloc(tb.NOALLOC_MAX_VERTICES + 1, 0, 1, None, None, 1, 1) == tb.ERROR_CODES["UNSUPPORTED"]

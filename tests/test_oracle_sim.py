@@ -9,6 +9,29 @@ import taurus_gen as tg
 from helpers import random_multigraph
 
 
+_M64 = (1 << 64) - 1
+
+
+def _random_score(seed, vertex, chunk):
+    """The random policy's 31-bit score restated with Python integers: start 0x452821E638D01377, absorb seed, vertex and
+    chunk index in turn (h <- mix(h xor 0x9E3779B97F4A7C15 * (x + 1)); mix = shifts 30 / 27 / 31 with the two 64-bit
+    multipliers), keep the top 31 bits."""
+    def mix(x):
+        x ^= x >> 30; x = (x * 0xBF58476D1CE4E5B9) & _M64
+        x ^= x >> 27; x = (x * 0x94D049BB133111EB) & _M64
+        return x ^ (x >> 31)
+    h = 0x452821E638D01377
+    for x in (seed, vertex, chunk):
+        h = mix(h ^ ((0x9E3779B97F4A7C15 * (x + 1)) & _M64))
+    return h >> 33
+
+
+def test_random_score_restatement_matches_the_oracle():
+    for seed, v, c in [(0, 0, 0), (1, 2, 3), (7, 123456, 99), (2 ** 40 + 5, 2 ** 31 - 1, 1693)]:
+        assert _random_score(seed, v, c) == int(oracle._lib().to_evict_hash(seed, v, c))
+        assert 0 <= _random_score(seed, v, c) < 2 ** 31
+
+
 def second_simulator(V, row_ptr, col, prop, m, is_hub, chunk, pool, policy=0, seed=0):
     """Independent restatement with Python sets; victims by a full sort of (pending, id)."""
     pend = {v: int(m[v]) + 1 for v in range(V)}
@@ -34,7 +57,7 @@ def second_simulator(V, row_ptr, col, prop, m, is_hub, chunk, pool, policy=0, se
         n_ev = 0
         if deficit > 0:
             score = {0: lambda v: pend[v], 1: lambda v: entered[v], 2: lambda v: touched_at[v],
-                     3: lambda v: int(oracle._lib().to_evict_hash(seed, v, c))}[policy]
+                     3: lambda v: _random_score(seed, v, c)}[policy]
             order = sorted((score(v), v) for v in in_pool - T)
             if len(order) < deficit:
                 return None

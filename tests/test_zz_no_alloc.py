@@ -60,8 +60,46 @@ def test_noalloc_matches_layer_begin_on_two_calls_in_a_row():
     assert (got_big == want_big).all()
     assert (got_small == want_small).all()
     assert got_big.sum() == g_big.V and got_small.sum() == g_small.V
+    # and against the oracle's closed form of the completion rank, max(v, largest propagated in-neighbour), per 64 ranks
+    import oracle
+    for g, w, layer, got in [(g_big, big, 1, got_big), (g_small, small, 0, got_small)]:
+        ms = oracle.message_sets(oracle.build_in_lists(g.V, g.row_ptr, g.col_idx), w.fanout[layer], w.seed, layer)
+        want = np.bincount(oracle.complete_chunk_closed_form(ms, 64), minlength=(g.V + 63) // 64)
+        assert (got == want).all()
     # and once more in the other order
     assert (_counts_noalloc(g_big, mask_big) == want_big).all()
+
+
+def test_noalloc_flags_malformed_row_offsets_without_reading_past_the_edges():
+    """Row offsets that leave [0, E] or run backwards are reported and cut to the valid part; a graph without edges and
+    a null destination array is fine."""
+    import torch
+    import paper_2607_17374_b200 as tb
+    dev = torch.device("cuda:0")
+    g = tg.make_graph(tg.WORKLOADS["tiny"])
+
+    def call(row_ptr, E, col):
+        out = torch.zeros(((g.V + 63) // 64,), dtype=torch.int32, device=dev)
+        bad = torch.zeros((1,), dtype=torch.int32, device=dev)
+        assert tb.completion_counts_noalloc(g.V, E, torch.from_numpy(row_ptr).to(dev), col, None, out, bad) == 0
+        torch.cuda.synchronize()
+        return out.cpu().numpy().astype(np.int64), int(bad.item())
+
+    col = torch.from_numpy(g.col_idx).to(dev)
+    counts, bad = call(g.row_ptr, g.E, col)
+    assert bad == 0 and counts.sum() == g.V
+    # the caller says E is smaller than the offsets claim: rows are cut at E (the array still holds g.E entries)
+    counts, bad = call(g.row_ptr, g.E - 1000, col)
+    assert bad == 1 and counts.sum() == g.V
+    backwards = g.row_ptr.copy()
+    backwards[100] = backwards[101] + 5
+    assert call(backwards, g.E, col)[1] == 1
+    negative = g.row_ptr.copy()
+    negative[0] = -3
+    assert call(negative, g.E, col)[1] == 1
+    # no edges at all: every vertex completes with its own chunk
+    counts, bad = call(np.zeros(g.V + 1, np.int64), 0, None)
+    assert bad == 0 and (counts[:-1] == 64).all() and counts.sum() == g.V
 
 
 def test_noalloc_rejects_sizes_beyond_the_static_scratch():
