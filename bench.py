@@ -1,24 +1,35 @@
 """Benchmark of the source-centric broadcast step (libtaurus) on synthetic graphs.
 
-A step is one full pass of the hot path over the workload: every layer, every chunk (copy-in, projection,
-classify, make-room, scatter, finalise, drain).  The metric is propagated edges per second (GTEPS,
-self messages not counted) over the whole step.
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large] [--impl ours|reference]
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mid] [--impl ours|reference]
+The metric is propagated edges per second (GTEPS, self messages not counted).
 
-N > 1 (under torchrun): the path has no exchange step, so every rank runs an independent replica of the
-workload on its own GPU ("replicas only", weak scaling); the value is the sum over ranks / max time.
---impl reference times the CPU oracle (a deliberately plain program) on a bounded sample of the same workload.
+Workloads whose accumulator pool holds every vertex ("mid", "tiny"): a step is one full pass of the hot path over
+the workload, every layer and every chunk (copy-in, projection, classify, make-room, scatter, finalise, output).
+
+Workloads with a bounded pool ("large", "sampled", "stress"; a full pass takes tens of seconds): a step is a
+window of --window consecutive chunks of one layer pass in steady state.  The layer (--layer, default the first
+hidden-to-hidden layer) is begun, --prefill chunks fill the pool (untimed), then W warm-up windows and K timed
+windows follow in the same pass; every window ends with a drain of the rows it completed.  The layer's input rows
+are generated rows of the right width (the paper's convention of dummy inputs of matching dimensions for later
+layers, Sect. 4.2).  The full layer time is printed as an estimate from the timed windows, marked as such.
+
+The default run times "large" (the eviction-bound configuration) and then "mid" as a secondary entry in the same
+JSON line.  N > 1 (under torchrun): the path has no exchange step, so every rank runs an independent replica
+("replicas only", weak scaling); value = sum over ranks / max time.
+--impl reference times the CPU oracle (a deliberately plain program) on bounded destination samples of the workload.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
 import sys
 import threading
 import time
+from dataclasses import replace
 
 import numpy as np
 
@@ -27,10 +38,23 @@ sys.path.insert(0, ROOT)
 
 import taurus_gen as tg  # noqa: E402
 
+METRIC = "edges/sec per GNN layer (GTEPS)"
 
-# DRAM bytes (read + write) per accumulator-row reduction of scatter_grouped_kernel<32,2>, from the ncu capture
-# summarised in profiles/scatter_grouped_kernel_mid_1200k.md (2.67 GB per launch / 0.98 M groups).
+# DRAM bytes (read + write) per accumulator-row reduction of the 256-float scatter_grouped_kernel instance, from the ncu
+# capture summarised in profiles/scatter_grouped_kernel_mid_1200k.md.  The figure belongs to the kernel source with
+# the digest below (sha256 of csrc/kernels_group.cu, first 16 hex digits); when the source has changed since the
+# capture the bench prints traffic = null instead of a stale number.
 SCATTER_TRAFFIC_PER_GROUP_BYTES = 2720.0
+SCATTER_CAPTURE_SOURCE = "0000000000000000"
+# PCIe bytes (both directions) per row moved by alloc_kernel, from profiles/alloc_kernel_large_1500k.md, same rule
+# (sha256 of csrc/kernels_state.cu).
+ALLOC_CAPTURE_SOURCE = "0000000000000000"
+ALLOC_PCIE_BYTES_PER_ROW_BYTE = None
+
+
+def source_digest(name: str) -> str:
+    path = os.path.join(ROOT, "paper_2607_17374_b200", "csrc", name)
+    return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
 
 
 def parse_args():
@@ -38,9 +62,14 @@ def parse_args():
     p.add_argument("--gpus", type=int, default=1)
     p.add_argument("--steps", type=int, default=3)
     p.add_argument("--warmup", type=int, default=3)
-    p.add_argument("--workload", default="mid")
+    p.add_argument("--workload", default="large")
+    p.add_argument("--secondary", default="mid", help="a second workload timed after the first and added to the JSON line "
+                   "under 'secondary' (single-GPU runs only); 'none' switches it off")
     p.add_argument("--vertices", type=int, default=0, help="scale the workload to this many vertices (0 = full size)")
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--window", type=int, default=32, help="bounded-pool workloads: chunks per step")
+    p.add_argument("--prefill", type=int, default=384, help="bounded-pool workloads: untimed chunks that fill the pool first")
+    p.add_argument("--layer", type=int, default=1, help="bounded-pool workloads: the layer whose pass is timed")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--simt-gemm", action="store_true", help="use the plain FFMA projection kernel")
@@ -54,23 +83,26 @@ def parse_args():
     p.add_argument("--model", default="", choices=["", "sage", "gcn", "gin", "gat"],
                    help="aggregation of every layer (default: the workload's); gat runs its three passes per layer")
     p.add_argument("--output", default="dense", choices=["dense", "runs-device", "runs-host"],
-                   help="where a layer's rows go: a dense matrix in HBM (default), or sorted runs (in HBM / pinned host "
-                        "memory) that the next layer reads back by merge-on-read")
+                   help="full-pass workloads: where a layer's rows go: a dense matrix in HBM (default), or sorted runs (in HBM / "
+                        "pinned host memory) that the next layer reads back by merge-on-read")
     return p.parse_args()
 
 
-def workload_of(args):
-    w = tg.WORKLOADS[args.workload]
+def workload_of(args, name=None):
+    w = tg.WORKLOADS[name or args.workload]
     if args.vertices:
         w = tg.scaled(w, args.vertices)
     if args.pool_fraction > 0:
-        from dataclasses import replace
         w = replace(w, pool_slots=max(1, int(w.V * args.pool_fraction)))
     if args.model:
-        from dataclasses import replace
         w = replace(w, mode={"sage": tg.SAGE_MEAN, "gcn": tg.GCN_SYM, "gin": tg.GIN_SUM, "gat": tg.GAT}[args.model],
                     gemm_mode=tg.GEMM_FP32 if args.model == "gat" else w.gemm_mode)
     return w
+
+
+def windowed(w) -> bool:
+    """Bounded pool: rows can be evicted, and a step is a window of chunks."""
+    return w.pool_slots < w.V - w.hub_count
 
 
 def peaks():
@@ -131,7 +163,9 @@ class ClockSampler(threading.Thread):
                 pass
             self.stop_flag.wait(0.01 if self.nvml is not None else 0.2)
 
-    def summary(self):
+    def finish(self):
+        self.stop_flag.set()
+        self.join()
         if not self.mhz:
             return dict(sm_mhz=None, sm_max_mhz=self.max_mhz, reasons=[], samples=0, source=self.source)
         mhz = sorted(self.mhz)
@@ -141,55 +175,104 @@ class ClockSampler(threading.Thread):
 
 # ----------------------------------------------------------------------------------------------- reference arm / CPU baseline
 
-def oracle_sample(w, g, budget_s=12.0, inl=None):
-    """Times the oracle (as it stands) on a bounded destination sample of layer 0.  Returns (edges/s, info)."""
-    import oracle
-    t0 = time.time()
-    inl = inl or oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
-    t_inl = time.time() - t0
-    ms = oracle.message_sets(inl, w.fanout[0], w.seed, 0)
-    model = tg.make_model(w)
-    rng = np.random.default_rng(0)
-    n_dst = min(g.V, 4096)
-    rate, used, edges, total_t = 0.0, 0, 0, 0.0
-    x = tg.features(w.seed, 0, 0, g.V, w.dims[0]).astype(np.float64)
-    din, dout = np.diff(inl.ptr), np.diff(g.row_ptr)
-    while True:
-        dst = np.sort(rng.choice(g.V, size=n_dst, replace=False)).astype(np.int64)
-        t1 = time.time()
-        oracle.layer_forward(ms, w.mode, din, dout, x, model.W_neigh[0], model.W_self[0], model.bias[0], model.act[0], dst)
-        dt = time.time() - t1
-        e = int(ms.m[dst].sum())
-        edges += e; total_t += dt; used += n_dst
-        rate = e / dt
-        if total_t >= budget_s or n_dst >= g.V:
-            break
-        n_dst = int(min(g.V, max(n_dst * 2, n_dst * (budget_s - total_t) / max(dt, 1e-3) * 0.7)))
-    info = dict(cores=oracle.cores_used(), kind="oracle",
-                sample="layer 0 (%d -> %d), %d sampled destinations, %d in-edges pulled in %.1f s; in-list build %.1f s not counted"
-                       % (w.dims[0], w.dims[1], used, edges, total_t, t_inl))
-    return edges / total_t, info, inl
+class OracleSampler:
+    """Times the oracle (as it stands) on bounded destination samples of a workload.
+
+    One scan of the CSR collects the in-lists of all sampled destinations (not timed: it replaces the whole-graph
+    in-list builder, which at 1.6 B edges would not fit the budget).  A batch is then timed as the oracle runs it:
+    the layer's message sets (the sampler where the layer is sampled), the fp64 aggregation of the input rows, the fp64
+    transform, bias and activation.  Layer l reads generated N(0,1) rows of its input width (layer 0: the workload's
+    features), keyed by vertex; generating them is not timed."""
+
+    def __init__(self, w, g, layers, n_batches, batch_dst):
+        import oracle
+        self.o, self.w, self.g, self.layers = oracle, w, g, list(layers)
+        rng = np.random.default_rng(0)
+        total = min(g.V, n_batches * batch_dst)
+        t0 = time.time()
+        self.dsts = np.sort(rng.choice(g.V, size=total, replace=False)).astype(np.int64)
+        self.ptr, self.src, self.eid = oracle.subset_in_lists(g.V, g.row_ptr, g.col_idx, self.dsts)
+        self.scan_s = time.time() - t0
+        self.batches = [(i * total // n_batches, (i + 1) * total // n_batches) for i in range(n_batches)]
+        self.model = tg.make_model(w)
+        self.dout = np.diff(g.row_ptr)
+        self.cores = oracle.cores_used()
+
+    def run_batch(self, b):
+        """Every listed layer on batch b.  Returns (in-edges pulled, seconds of oracle work)."""
+        o, w, g = self.o, self.w, self.g
+        lo, hi = self.batches[b % len(self.batches)]
+        dsts = self.dsts[lo:hi]
+        ptr = self.ptr[lo:hi + 1] - self.ptr[lo]
+        src = self.src[self.ptr[lo]:self.ptr[hi]]
+        eid = self.eid[self.ptr[lo]:self.ptr[hi]]
+        edges, secs = 0, 0.0
+        for l in self.layers:
+            t0 = time.time()
+            kp, ks, _ = (ptr, src, eid) if w.fanout[l] == 0 else o.subset_message_sets(ptr, src, eid, dsts, w.fanout[l], w.seed, l)
+            need = np.unique(np.concatenate([ks, dsts]))
+            t1 = time.time()
+            h = tg.features_rows(w.seed, l, need, w.dims[l])          # inputs: not part of the oracle's work
+            t2 = time.time()
+            o.subset_forward(w.mode if w.mode != tg.GAT else o.SAGE_MEAN, dsts, kp, ks, g.in_degree[dsts], self.dout[dsts], need,
+                             self.dout[need], h, self.model.W_neigh[l], self.model.W_self[l], self.model.bias[l], self.model.act[l])
+            t3 = time.time()
+            edges += int(kp[-1])
+            secs += (t1 - t0) + (t3 - t2)
+        return edges, secs
+
+    def describe(self, batches_run, edges, secs):
+        return dict(cores=self.cores, kind="oracle",
+                    sample="layers %s, %d batch(es) of %d sampled destinations each (dims %s), %d in-edges pulled in %.1f s of oracle "
+                           "work; one CSR scan for the sampled in-lists (%.1f s) and input-row generation not counted"
+                           % (self.layers, batches_run, self.batches[0][1] - self.batches[0][0],
+                              [(self.w.dims[l], self.w.dims[l + 1]) for l in self.layers], edges, secs, self.scan_s))
+
+
+def batch_size_for(w, layers):
+    """Destinations per batch: bounded by the fp64 input rows a batch gathers (about 3 GB)."""
+    widest = max(w.dims[l] for l in layers)
+    mean_deg = max(1.0, w.E / w.V)
+    fan = [min(mean_deg, w.fanout[l]) if w.fanout[l] else mean_deg for l in layers]
+    return int(max(1024, min(400_000, 3e9 / (8.0 * widest * (max(fan) + 1)))))
+
+
+def timed_layers(args, w):
+    return [min(max(args.layer, 0), w.L - 1)] if windowed(w) else list(range(w.L))
+
+
+def cpu_baseline(args, w, g, budget_s=12.0):
+    layers = timed_layers(args, w)
+    smp = OracleSampler(w, g, layers, 8, batch_size_for(w, layers))
+    edges, secs, n = 0, 0.0, 0
+    while n < 8 and (n == 0 or secs < budget_s):
+        e, s = smp.run_batch(n)
+        edges += e; secs += s; n += 1
+    return dict(value=edges / secs / 1e9, unit="GTEPS", **smp.describe(n, edges, secs))
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
     w = workload_of(args)
     g = tg.make_graph(w)
-    inl = None
-    for _ in range(max(args.warmup, 0) and 1):
-        _, _, inl = oracle_sample(w, g, 2.0, inl)
-    vals, info = [], None
-    t0 = time.time()
-    for _ in range(args.steps):
-        v, info, inl = oracle_sample(w, g, 8.0, inl)
-        vals.append(v)
-    value = float(np.mean(vals)) / 1e9
-    line = dict(impl="reference", metric="edges/sec per GNN layer (GTEPS)", value=value, unit="GTEPS", n_gpus=args.gpus,
-                steps=args.steps, warmup=args.warmup, ms_per_step=(time.time() - t0) * 1e3 / max(args.steps, 1),
-                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=w.name, V=g.V, E=g.E, dims=list(w.dims), l2="inputs larger than L2"),
+    layers = timed_layers(args, w)
+    n = max(args.steps, 1) + max(args.warmup, 0)
+    smp = OracleSampler(w, g, layers, min(n, 8), batch_size_for(w, layers))
+    for i in range(max(args.warmup, 0)):
+        smp.run_batch(i)
+    edges, secs = 0, 0.0
+    for i in range(args.steps):
+        e, s = smp.run_batch(args.warmup + i)
+        edges += e; secs += s
+    value = edges / secs / 1e9
+    info = smp.describe(args.steps, edges, secs)
+    line = dict(impl="reference", metric=METRIC, value=value, unit="GTEPS", n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=secs * 1e3 / max(args.steps, 1), higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic",
+                config=dict(workload=w.name, V=g.V, E=g.E, dims=list(w.dims), layers_timed=layers, fanout=list(w.fanout),
+                            step="one batch of sampled destinations through the listed layers",
+                            l2="inputs larger than L2"),
                 cpu_baseline=dict(value=value, unit="GTEPS", **info),
                 e2e=dict(value=value, unit="GTEPS", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
@@ -213,46 +296,248 @@ def whole_job_value(units_per_rank_step: float, steps: int, world: int, ms_max: 
     return world * units_per_rank_step * steps / (ms_max * 1e-3) / 1e9
 
 
-# ----------------------------------------------------------------------------------------------- our arm
+class Env:
+    """Device, rank and barrier of this process."""
 
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
+    def __init__(self):
+        import torch
+        import torch.distributed as dist
+        self.torch, self.dist = torch, dist
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=self.dev)
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def make_context(args, w, g, model, host_evict, drain_rows):
     import paper_2607_17374_b200 as tb
+    flags = (tb.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (tb.FLAG_NO_GROUPING if args.no_grouping else 0) | \
+        (tb.FLAG_PROJECT_FIRST if args.project_first else 0)
+    return tb.Context(g.V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
+                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags,
+                      {"fewest": 0, "fifo": 1, "lru": 2, "random": 3}[args.evict_policy], w.gin_eps, model.att_src, model.att_dst,
+                      w.leaky_slope)
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+PHASES = ["copy_in", "projection", "classify_select", "row_moves", "scatter", "finalise"]
 
-    w = workload_of(args)
+
+def scatter_bytes(groups, edges, n_src, width, self_row):
+    """Algorithmic bytes of the scatter: per accumulator-row reduction a read-modify-write of the row (2 * 4 width)
+    plus slot and pending-count words (8); per propagated edge its (destination, source) words (8); per source its
+    row read once (4 width) and its self message (row read 4 width + read-modify-write 2 * 4 width + 8)."""
+    return groups * (8 * width + 8) + edges * 8 + n_src * (4 * width + (12 * width if self_row else 0) + 8)
+
+
+def link_peaks(env, mb=256, reps=3):
+    """Pinned-memory copy bandwidth of this machine, GB/s: host -> device alone, device -> host alone, and both at once on
+    two streams (per direction).  Plain asynchronous copies of `mb` MB, best of `reps`."""
+    torch = env.torch
+    n = mb << 20
+    h_in, h_out = torch.empty(n, dtype=torch.uint8).pin_memory(), torch.empty(n, dtype=torch.uint8).pin_memory()
+    d_in, d_out = torch.empty(n, dtype=torch.uint8, device=env.dev), torch.zeros(n, dtype=torch.uint8, device=env.dev)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    best = [0.0, 0.0, 0.0]
+    for _ in range(reps + 1):
+        for mode in range(3):
+            torch.cuda.synchronize()
+            a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            a.record(s1)
+            s2.wait_event(a)
+            if mode in (0, 2):
+                with torch.cuda.stream(s1):
+                    d_in.copy_(h_in, non_blocking=True)
+            if mode in (1, 2):
+                with torch.cuda.stream(s2):
+                    h_out.copy_(d_out, non_blocking=True)
+            c.record(s2)
+            s1.wait_event(c)
+            b.record(s1)
+            torch.cuda.synchronize()
+            best[mode] = max(best[mode], n / (a.elapsed_time(b) * 1e-3) / 1e9)
+    return dict(h2d_alone_gbs=best[0], d2h_alone_gbs=best[1], both_per_direction_gbs=best[2],
+                how="cudaMemcpyAsync of %d MB pinned buffers, both directions at once on two streams, best of %d" % (mb, reps))
+
+
+# ----------------------------------------------------------------------------------------------- bounded-pool workloads
+
+def run_windowed(args, env, w):
+    """Steps = windows of chunks of one layer pass in steady state (see the module docstring)."""
+    import paper_2607_17374_b200 as tb
+    torch, dev = env.torch, env.dev
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    V, chunk = g.V, w.chunk
+    chunks = [(s, min(s + chunk, V)) for s in range(0, V, chunk)]
+    l = timed_layers(args, w)[0]
+    d_in, d_out = w.dims[l], w.dims[l + 1]
+    K, W = max(args.steps, 1), max(args.warmup, 0)
+    window, prefill = max(args.window, 1), max(args.prefill, 0)
+    while prefill + (W + K) * window > len(chunks) and window > 1:
+        window -= 1
+    prefill = max(0, min(prefill, len(chunks) - (W + K) * window))
+    if (W + K) * window > len(chunks):
+        raise SystemExit("workload too small for %d windows" % (W + K))
+    cap = 3 * window * chunk                       # graduation buffer: drained once per window, earlier when it could overflow
+    host_evict = min(V - w.hub_count, 56_000_000)   # rows evicted at once stay below this on the three bounded-pool workloads
+    ctx = make_context(args, w, g, model, host_evict, cap)
+    agg_first, acc_width = ctx.layer_plan(l)
+    R = 8                                          # distinct generated input chunks, reused in turn
+    x_host = [torch.empty((chunk, d_in), dtype=torch.float32).pin_memory() for _ in range(R)]
+    for i in range(R):
+        tg.features(w.seed, l, i * chunk, (i + 1) * chunk, d_in, out=x_host[i].numpy())
+    x_dev = [x.to(dev) for x in x_host]
+    ids_dev = torch.empty(cap, dtype=torch.int64, device=dev)
+    rows_dev = torch.empty((cap, d_out), dtype=torch.float32, device=dev)
+    ids_host = torch.empty(cap, dtype=torch.int64).pin_memory()
+    rows_host = torch.empty((cap, d_out), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream()
+    link = link_peaks(env)
+    pk = peaks()
+
+    def run_chunks(c0, c1, feats, ids, rows, drain_every):
+        """Chunks [c0, c1); a drain after every `drain_every` chunks.  Returns rows drained."""
+        drained = 0
+        for c in range(c0, c1):
+            s, e = chunks[c]
+            x = feats[c % R][: e - s]
+            if ctx.push_chunk(s, e, x, stream, raise_on_drain_full=False) != 0:
+                drained += ctx.drain_completed(ids, rows, cap)
+                ctx.push_chunk(s, e, x, stream)
+            if (c - c0 + 1) % drain_every == 0:
+                drained += ctx.drain_completed(ids, rows, cap)
+        return drained
+
+    def one_pass(feats, ids, rows, timing):
+        """Prefill, warm-up windows, timed windows.  Returns (ms of the timed windows, stats before, stats after, rows drained,
+        phase times, launches, clocks, wall ms)."""
+        ctx.layer_begin(l, stream)
+        run_chunks(0, prefill, feats, ids, rows, window)
+        ctx.drain_completed(ids, rows, cap)
+        c = prefill
+        run_chunks(c, c + W * window, feats, ids, rows, window)
+        c += W * window
+        st0 = ctx.get_stats()
+        env.barrier()
+        sampler = ClockSampler(env.local)
+        sampler.start()
+        if timing:
+            ctx.set_timing(True)
+        launches0 = ctx.launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        ev0.record(stream)
+        drained = run_chunks(c, c + K * window, feats, ids, rows, window)
+        ev1.record(stream)
+        env.barrier()
+        wall = (time.time() - t0) * 1e3
+        ms = ev0.elapsed_time(ev1)
+        launches = ctx.launch_count() - launches0
+        clocks = sampler.finish()
+        ph = None
+        if timing:
+            ph = ctx.get_phase_ms()
+            ctx.set_timing(False)
+        st1 = ctx.get_stats()
+        return ms, st0, st1, drained, ph, launches, clocks, wall
+
+    # ---- inputs resident in HBM, rows drained into HBM
+    ms, st0, st1, drained, ph, launches, clocks, _ = one_pass(x_dev, ids_dev, rows_dev, True)
+    msgs = st1["total_messages"] - st0["total_messages"]
+    evicted, reloaded = st1["evictions"] - st0["evictions"], st1["reloads"] - st0["reloads"]
+    groups = st1["scatter_groups"] - st0["scatter_groups"]
+    ms_max = max_over_ranks(ms, env.world, dev)
+    value = whole_job_value(msgs / K, K, env.world, ms_max)
+    phase = ph[: K * window].sum(axis=0).astype(np.float64)            # ms over the timed windows
+    phase_ms = dict(zip(PHASES, [float(x) / K for x in phase]))
+    row_bytes = 4 * acc_width
+    move_s = phase[3] * 1e-3
+    out_gbs, in_gbs = evicted * row_bytes / move_s / 1e9, reloaded * row_bytes / move_s / 1e9
+    n_src = chunks[prefill + (W + K) * window - 1][1] - chunks[prefill + W * window][0]
+    sc_bytes = scatter_bytes(groups, msgs, n_src, acc_width, not (agg_first and w.mode == tg.SAGE_MEAN))
+    sc_s = phase[4] * 1e-3
+    moves_share = phase[3] / ms
+    # the dominant kernel: the row moves between the pool and pinned host memory (alloc_kernel), bound by the host link
+    roofline = dict(bound="pcie", kernel="alloc_kernel (evicted rows out, reloaded rows in, %d-byte rows)" % row_bytes,
+                    achieved=(out_gbs + in_gbs) / 2, peak=link["both_per_direction_gbs"], unit="GB/s per direction",
+                    frac=(out_gbs + in_gbs) / 2 / link["both_per_direction_gbs"], peak_source="measured in this run: " + link["how"],
+                    device_to_host_gbs=out_gbs, host_to_device_gbs=in_gbs, link=link,
+                    rows_out_per_step=evicted / K, rows_in_per_step=reloaded / K, launches_per_step=window,
+                    avg_launch_ms=float(phase[3]) / (K * window), algorithmic_bytes_per_launch=(evicted + reloaded) * row_bytes / (K * window),
+                    share_of_step=float(moves_share), traffic=None,
+                    traffic_note="no counter capture at this size (110 GB resident); PCIe counters of the same kernel on a 1.5 M-vertex "
+                                 "instance are in profiles/alloc_kernel_large_1500k.md")
+    roofline_hbm = dict(bound="hbm", kernel="scatter_grouped_kernel (accumulator rows of %d floats)" % acc_width,
+                        achieved=sc_bytes / sc_s / 1e9, peak=pk["hbm_gbs"], unit="GB/s", frac=sc_bytes / sc_s / 1e9 / pk["hbm_gbs"],
+                        peak_source=pk["source"], groups_per_step=groups / K, avg_launch_ms=float(phase[4]) / (K * window),
+                        algorithmic_bytes_per_launch=sc_bytes / (K * window), share_of_step=float(phase[4] / ms),
+                        gteps_scatter_only=msgs / sc_s / 1e9)
+
+    # ---- end to end through the C ABI with host buffers: every chunk's input rows come from pinned host memory (one
+    # host -> device copy per chunk inside push_chunk) and every window's finished rows and ids are drained into pinned
+    # host memory (taurus_drain_completed), all inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        ms2, s0, s1, drained2, _, _, _, wall2 = one_pass(x_host, ids_host, rows_host, False)
+        msgs2 = s1["total_messages"] - s0["total_messages"]
+        e2e_ms = max_over_ranks(max(ms2, wall2), env.world, dev)
+        e2e = dict(value=whole_job_value(msgs2 / K, K, env.world, e2e_ms), unit="GTEPS", ms_per_step=e2e_ms / K,
+                   h2d_bytes_per_step=int(4 * d_in * n_src / K), d2h_bytes_per_step=int(drained2 * (4 * d_out + 8) / K),
+                   note="input rows of every chunk host -> device inside taurus_push_chunk; finished rows and ids device -> host "
+                        "through taurus_drain_completed once per window; evicted rows travel over the same link")
+    cpu = None
+    if env.rank == 0 and env.world == 1 and not args.no_cpu_baseline and w.mode != tg.GAT:
+        cpu = cpu_baseline(args, w, g)
+    free, total = torch.cuda.mem_get_info()
+    line = dict(metric=METRIC, value=value, unit="GTEPS", n_gpus=env.world, steps=K, warmup=W, ms_per_step=ms_max / K,
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if w.gemm_mode == tg.GEMM_BF16 else "f32",
+                data="synthetic",
+                config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=chunk, chunks_per_layer=len(chunks),
+                            pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
+                            mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], evict_policy=args.evict_policy,
+                            step="window of %d chunks of layer %d (%d -> %d) in steady state; %d prefill chunks and %d warm-up windows "
+                                 "before the timed ones, same layer pass; rows drained once per window" % (window, l, d_in, d_out, prefill, W),
+                            layer=l, window_chunks=window, prefill_chunks=prefill, aggregate_first=bool(agg_first),
+                            accumulator_floats=acc_width, messages_per_step=msgs / K, evictions_per_step=evicted / K,
+                            reloads_per_step=reloaded / K, rows_drained_per_step=drained / K,
+                            layer_time_estimate_ms=ms_max / (K * window) * len(chunks),
+                            layer_time_note="extrapolated linearly from the timed windows to the layer's %d chunks" % len(chunks),
+                            l2="inputs larger than L2 (pool %.1f GB, one chunk's rows %.0f MB)" %
+                               (w.pool_slots * 4 * acc_width / 1e9, chunk * 4 * max(d_in, d_out) / 1e6),
+                            device_memory_in_use_gb=(total - free) / 1e9,
+                            parallelism="replicas only" if env.world > 1 else "1 gpu", phase_ms=phase_ms),
+                clocks=clocks, roofline=roofline, roofline_hbm=roofline_hbm, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
+    ctx.destroy()
+    return line
+
+
+# ----------------------------------------------------------------------------------------------- full-pass workloads
+
+def run_full_pass(args, env, w):
+    import paper_2607_17374_b200 as tb
+    torch, dev, world, rank = env.torch, env.dev, env.world, env.rank
     g = tg.make_graph(w)
     model = tg.make_model(w)
     V, L = g.V, w.L
     chunks = [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
-    ctx_bound = V   # upper bound on the rows one chunk can complete
     # two graduation halves; badly ordered graphs complete a large share of V in the last chunks
-    drain_rows = 2 * max(ctx_bound, w.chunk)
+    drain_rows = 2 * max(V, w.chunk)
     host_evict = 0 if w.pool_slots >= V - w.hub_count else V - w.hub_count
-    flags = (tb.FLAG_SIMT_GEMM if args.simt_gemm else 0) | (tb.FLAG_NO_GROUPING if args.no_grouping else 0) | \
-        (tb.FLAG_PROJECT_FIRST if args.project_first else 0)
-    pad4 = lambda x: (x + 3) // 4 * 4
-    # the library's rule: a layer whose input rows are at most 3/4 as wide as its output rows aggregates input rows and
-    # transforms the finished rows (SAGE: while its per-vertex store of input rows stays below 64 GiB)
-    agg_first = [(not args.project_first) and 4 * pad4(w.dims[l]) <= 3 * pad4(w.dims[l + 1]) and
-                 (w.mode != tg.SAGE_MEAN or V * pad4(w.dims[l]) * 4 <= (64 << 30)) for l in range(L)]
-    ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
-                     model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, drain_rows, w.gemm_mode, flags,
-                     {"fewest": 0, "fifo": 1, "lru": 2, "random": 3}[args.evict_policy], w.gin_eps, model.att_src, model.att_dst,
-                     w.leaky_slope)
+    ctx = make_context(args, w, g, model, host_evict, drain_rows)
+    plan = [ctx.layer_plan(l) for l in range(L)]
+    agg_first, acc_width = [p[0] for p in plan], [p[1] for p in plan]
     gat = w.mode == tg.GAT
     use_runs = args.output != "dense"
     hprime = torch.zeros((V, max(w.dims[1:])), dtype=torch.float32, device=dev) if gat else None
@@ -313,29 +598,28 @@ def run_ours(args):
         return feat
 
     # warm-up (also collects the per-layer message counts)
-    barrier()
+    env.barrier()
     for i in range(max(args.warmup, 1)):
         step(x_dev, out_dev, collect_stats=(i == 0))
     torch.cuda.synchronize()
     msgs_per_step = int(sum(edges_per_layer))
 
     # ---- device-resident timing
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(env.local)
     sampler.start()
     ctx.set_timing(True)
     launches0 = ctx.launch_count()
-    barrier()
+    env.barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
     for _ in range(args.steps):
         step(x_dev, out_dev)
     ev1.record(stream)
-    barrier()
+    env.barrier()
     ms = ev0.elapsed_time(ev1)
     ctx.set_timing(False)
     launches = ctx.launch_count() - launches0
-    sampler.stop_flag.set()
-    sampler.join()
+    clocks = sampler.finish()
     phases = ctx.get_phase_ms()   # [pushes, 6]
     ms_max = max_over_ranks(ms, world, dev)
     value = whole_job_value(msgs_per_step, args.steps, world, ms_max)
@@ -344,19 +628,13 @@ def run_ours(args):
     n_push = len(chunks) * L * args.steps
     ph = phases[:n_push].reshape(args.steps, L, len(chunks), 6)
     scatter_ms = ph[..., 4]
-    # Algorithmic bytes of the scatter: per accumulator-row reduction a read-modify-write of
-    # the row (2 * 4 Hp) plus slot and pending-count words (8); per propagated edge its (destination, source)
-    # words (8); per source its projected row read once (4 Hp) and its self message (row read 4 Hp + RMW 2 * 4 Hp + 8).
-    # In CSR order a "group" is one edge.  The per-edge cold-miss model (12 + 2 * 4 Hp per edge) is kept beside it.
+    # In CSR order a "group" is one edge.  The per-edge cold-miss model (12 + 2 * 4 width per edge) is kept beside it.
     layer_bytes, edge_model_bytes = [], []
-    n_src = V
-    acc_width = [pad4(w.dims[l]) if agg_first[l] else pad4(w.dims[l + 1]) for l in range(L)]   # floats per accumulator row
     for l in range(L):
         Wd = acc_width[l]
         self_row = not (agg_first[l] and w.mode == tg.SAGE_MEAN)   # aggregate-first SAGE adds its self term after the transform
-        layer_bytes.append(groups_per_layer[l] * (8 * Wd + 8) + edges_per_layer[l] * 8 +
-                           n_src * (4 * Wd + (12 * Wd if self_row else 0) + 8))
-        edge_model_bytes.append(edges_per_layer[l] * (12 + 8 * Wd) + n_src * (4 * Wd + 8))
+        layer_bytes.append(scatter_bytes(groups_per_layer[l], edges_per_layer[l], V, Wd, self_row))
+        edge_model_bytes.append(edges_per_layer[l] * (12 + 8 * Wd) + V * (4 * Wd + 8))
     alg_bytes_step = float(sum(layer_bytes))
     scatter_total_ms = float(scatter_ms.sum()) / args.steps
     pk = peaks()
@@ -374,12 +652,14 @@ def run_ours(args):
     dom_bytes = float(sum(layer_bytes[l] for l in dom))
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     kname = ("scatter_grouped_kernel" if grouped else "scatter_kernel") + " (accumulator rows of %d floats, layers %s)" % (dom_w, dom)
+    capture_valid = grouped and dom_w == 256 and source_digest("kernels_group.cu") == SCATTER_CAPTURE_SOURCE
     roofline = dict(bound="hbm", kernel=kname, achieved=achieved,
                     peak=pk["hbm_gbs"], unit="GB/s", frac=achieved / pk["hbm_gbs"], peak_source=pk["source"],
                     traffic=SCATTER_TRAFFIC_PER_GROUP_BYTES * sum(groups_per_layer[l] for l in dom) / (len(dom) * len(chunks))
-                    if grouped and dom_w == 256 else None,
-                    traffic_note="ncu dram read+write per launch of the 256-float kernel, scaled by groups per launch "
-                                 "(profiles/scatter_grouped_kernel_mid_1200k.md)" if grouped and dom_w == 256 else None,
+                    if capture_valid else None,
+                    traffic_note=("ncu dram read+write per launch of the 256-float kernel, scaled by groups per launch "
+                                  "(profiles/scatter_grouped_kernel_mid_1200k.md)") if capture_valid else
+                                 "no capture of this kernel source (profiles/scatter_grouped_kernel_mid_1200k.md names the source it measured)",
                     launches_per_step=len(chunks) * len(dom), avg_launch_ms=dom_ms / (len(chunks) * len(dom)),
                     algorithmic_bytes_per_launch=dom_bytes / (len(chunks) * len(dom)),
                     share_of_step=dom_ms / (ms_max / args.steps),
@@ -390,8 +670,7 @@ def run_ours(args):
                                     groups=int(groups_per_layer[l]), accumulator_floats=acc_width[l], aggregate_first=bool(agg_first[l]),
                                     gteps_scatter_only=edges_per_layer[l] / (per_layer_ms[l] * 1e-3) / 1e9)
                                for l in range(L)])
-    phase_ms = dict(zip(["copy_in", "projection", "classify_select", "row_moves", "scatter", "finalise"],
-                        [float(x) / args.steps for x in ph.sum(axis=(0, 1, 2))]))
+    phase_ms = dict(zip(PHASES, [float(x) / args.steps for x in ph.sum(axis=(0, 1, 2))]))
 
     # ---- end to end through the C ABI with host buffers: every step streams the layer-0 features from pinned host
     # memory (one host -> device copy per chunk, inside push_chunk) and brings the last layer's rows back to pinned
@@ -422,7 +701,7 @@ def run_ours(args):
         for b in range(2):
             d2h_done[b].record(stream)
         e2e_step(0)
-        barrier()
+        env.barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.time()
         e0.record(stream)
@@ -431,7 +710,7 @@ def run_ours(args):
         for b in range(2):
             stream.wait_event(d2h_done[b])
         e1.record(stream)
-        barrier()
+        env.barrier()
         wall = (time.time() - t0) * 1e3
         e2e_ms = max_over_ranks(max(e0.elapsed_time(e1), wall), world, dev)
         e2e = dict(value=whole_job_value(msgs_per_step, args.steps, world, e2e_ms), unit="GTEPS",
@@ -439,32 +718,43 @@ def run_ours(args):
                    h2d_bytes_per_step=int(4 * V * w.dims[0]), d2h_bytes_per_step=int(4 * V * w.dims[-1]),
                    note="layer-0 features host -> device per chunk; last layer's rows device -> host in one copy per step on a "
                         "side stream, overlapping the next step's first layer; intermediate layers in HBM")
-        out_host = outs_host
-        del out_host
+        del outs_host
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not gat:
-        v, info, _ = oracle_sample(w, g, 12.0)
-        cpu = dict(value=v / 1e9, unit="GTEPS", **info)
+        cpu = cpu_baseline(args, w, g)
 
-    if rank == 0:
-        line = dict(metric="edges/sec per GNN layer (GTEPS)", value=value, unit="GTEPS", n_gpus=world, steps=args.steps,
-                    warmup=args.warmup, ms_per_step=ms_max / args.steps, higher_is_better=True, scaling="weak",
-                    vs_baseline=None, dtype="f32", data="synthetic",
-                    config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=w.chunk, chunks_per_layer=len(chunks),
-                                pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
-                                mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], output=args.output, evict_policy=args.evict_policy,
-                                messages_per_step=msgs_per_step,
-                                l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
-                                parallelism="replicas only" if world > 1 else "1 gpu",
-                                layer_ms=[float(ph[:, l].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
-                    clocks=sampler.summary(), roofline=roofline, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
-        print(json.dumps(line))
+    line = dict(metric=METRIC, value=value, unit="GTEPS", n_gpus=world, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms_max / args.steps, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="bf16" if w.gemm_mode == tg.GEMM_BF16 else "f32", data="synthetic",
+                config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=w.chunk, chunks_per_layer=len(chunks),
+                            pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
+                            mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], output=args.output, evict_policy=args.evict_policy,
+                            step="one pass over every layer and chunk of the workload",
+                            messages_per_step=msgs_per_step,
+                            l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
+                            parallelism="replicas only" if world > 1 else "1 gpu",
+                            layer_ms=[float(ph[:, l].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
+                clocks=clocks, roofline=roofline, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
     for r in runs or []:
         r.destroy()
     ctx.destroy()
-    if world > 1:
-        dist.destroy_process_group()
+    return line
+
+
+def run_ours(args):
+    env = Env()
+    w = workload_of(args)
+    line = run_windowed(args, env, w) if windowed(w) else run_full_pass(args, env, w)
+    if args.secondary not in ("none", "", w.name.split("@")[0]) and env.world == 1:
+        import gc
+        gc.collect()
+        env.torch.cuda.empty_cache()
+        w2 = workload_of(args, args.secondary)
+        line["secondary"] = {args.secondary: run_windowed(args, env, w2) if windowed(w2) else run_full_pass(args, env, w2)}
+    if env.rank == 0:
+        print(json.dumps(line))
+    env.close()
 
 
 def main():

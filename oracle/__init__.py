@@ -211,6 +211,56 @@ def layer_forward(ms: MessageSets, mode: int, din: np.ndarray, dout: np.ndarray,
     return np.maximum(z, 0.0) if act else z
 
 
+# ----------------------------------------------------------------------------- a destination subset of a large graph
+# Where the whole graph is out of reach, the same definition is evaluated for a listed subset of destinations:
+# their in-lists come from one scan of the CSR, everything else is the code above.
+
+def subset_in_lists(V: int, row_ptr: np.ndarray, col: np.ndarray, dsts: np.ndarray):
+    """In-lists (ascending source id, duplicates in CSR order) of the sorted, distinct destinations dsts.
+    Returns (ptr int64 [len(dsts) + 1], src int64, eid int64)."""
+    dsts = np.asarray(dsts, dtype=np.int64)
+    wanted = np.zeros(V, dtype=bool)
+    wanted[dsts] = True
+    sel = np.flatnonzero(wanted[col])                          # ascending CSR edge index = (source, position) order
+    d = col[sel]
+    order = np.argsort(d, kind="stable")
+    sel, d = sel[order], d[order]
+    ptr = np.zeros(dsts.size + 1, np.int64)
+    np.cumsum(np.bincount(np.searchsorted(dsts, d), minlength=dsts.size), out=ptr[1:])
+    src = np.searchsorted(row_ptr, sel, side="right") - 1      # the row whose range holds the edge
+    return ptr, src.astype(np.int64), sel.astype(np.int64)
+
+
+def subset_message_sets(ptr: np.ndarray, src: np.ndarray, eid: np.ndarray, dsts: np.ndarray, fanout: int, seed: int, layer: int):
+    """M(v) of the listed destinations from their in-lists: all entries, or the sampled positions (Sect. 3.9).
+    Returns (keep_ptr, keep_src, keep_eid), kept entries in ascending in-list position."""
+    keep_ptr, keep_src, keep_eid = [0], [], []
+    for i, v in enumerate(dsts):
+        lo, hi = int(ptr[i]), int(ptr[i + 1])
+        p = np.sort(sample_positions(seed, layer, int(v), hi - lo, fanout))
+        keep_src.append(src[lo:hi][p]); keep_eid.append(eid[lo:hi][p])
+        keep_ptr.append(keep_ptr[-1] + p.size)
+    cat = lambda xs: np.concatenate(xs) if xs else np.zeros(0, np.int64)
+    return np.asarray(keep_ptr, np.int64), cat(keep_src), cat(keep_eid)
+
+
+def subset_forward(mode: int, dsts: np.ndarray, keep_ptr: np.ndarray, keep_src: np.ndarray, din_dst: np.ndarray, dout_dst: np.ndarray,
+                   need: np.ndarray, dout_need: np.ndarray, h_need: np.ndarray, W_neigh: np.ndarray, W_self: np.ndarray,
+                   bias: np.ndarray, act: int, gin_eps: float = 0.0) -> np.ndarray:
+    """Eq. 1-2 for the destinations dsts.  need = sorted distinct ids of every kept source and every destination,
+    h_need their input rows, dout_need their out-degrees (GCN); din_dst / dout_dst the degrees of the destinations."""
+    m = np.diff(keep_ptr).astype(np.int32)
+    ms = MessageSets(keep_ptr, np.searchsorted(need, keep_src).astype(np.int32), None, None, m)
+    c_out, c_in, c_self = coefficients(mode, m, din_dst, dout_dst, gin_eps)
+    c_out_src = (dout_need.astype(np.float64) + 1.0) ** -0.5 if mode == GCN_SYM else None
+    h = np.asarray(h_need, dtype=np.float64)
+    agg = aggregate(ms, np.arange(dsts.size), c_out_src, h)
+    Wn = np.asarray(W_neigh, dtype=np.float64)
+    Ws = np.asarray(W_self, dtype=np.float64) if mode == SAGE_MEAN else Wn
+    z = c_in[:, None] * (agg @ Wn) + c_self[:, None] * (h[np.searchsorted(need, dsts)] @ Ws) + np.asarray(bias, dtype=np.float64)[None, :]
+    return np.maximum(z, 0.0) if act else z
+
+
 def forward(V: int, row_ptr: np.ndarray, col: np.ndarray, x: np.ndarray, mode: int, W_neigh: Sequence[np.ndarray],
             W_self: Sequence[np.ndarray], bias: Sequence[np.ndarray], act: Sequence[int],
             fanout: Sequence[int], seed: int, inl: Optional[InLists] = None, gin_eps: float = 0.0) -> List[np.ndarray]:

@@ -189,3 +189,30 @@ def test_in_lists_are_sorted_by_source_with_duplicates_in_csr_order():
         assert (np.diff(e) > 0).all()               # CSR order == (source, position) order
         assert (col[e] == v).all() and (src_of_edge[e] == s).all()
     assert (np.diff(inl.ptr) == np.bincount(col, minlength=V)).all()
+
+
+@pytest.mark.parametrize("mode", [oracle.SAGE_MEAN, oracle.GCN_SYM, oracle.GIN_SUM])
+@pytest.mark.parametrize("fanout", [0, 3])
+def test_subset_evaluation_equals_the_full_layer_on_those_rows(mode, fanout):
+    """The destination-subset path (in-lists by a CSR scan) against the whole-graph path restricted to the same rows."""
+    from helpers import random_multigraph
+    V, E, F, H = 300, 2500, 12, 7
+    row_ptr, col = random_multigraph(V, E, 5)
+    rng = np.random.default_rng(2)
+    h = rng.standard_normal((V, F))
+    Wn, Ws, b = rng.standard_normal((F, H)), rng.standard_normal((F, H)), rng.standard_normal(H)
+    inl = oracle.build_in_lists(V, row_ptr, col)
+    ms = oracle.message_sets(inl, fanout, 9, 1)
+    din, dout = np.diff(inl.ptr), np.diff(row_ptr)
+    full = oracle.layer_forward(ms, mode, din, dout, h, Wn, Ws, b, 1, gin_eps=0.25)
+    dsts = np.unique(rng.integers(0, V, 40)).astype(np.int64)
+    ptr, src, eid = oracle.subset_in_lists(V, row_ptr, col, dsts)
+    for i, v in enumerate(dsts):                      # the scan finds exactly the in-list of the whole-graph builder
+        assert (src[ptr[i]:ptr[i + 1]] == inl.src[inl.ptr[v]:inl.ptr[v + 1]]).all()
+        assert (eid[ptr[i]:ptr[i + 1]] == inl.eid[inl.ptr[v]:inl.ptr[v + 1]]).all()
+    kp, ks, ke = oracle.subset_message_sets(ptr, src, eid, dsts, fanout, 9, 1)
+    for i, v in enumerate(dsts):
+        assert sorted(ke[kp[i]:kp[i + 1]].tolist()) == sorted(ms.eid[ms.ptr[v]:ms.ptr[v + 1]].tolist())
+    need = np.unique(np.concatenate([ks, dsts]))
+    sub = oracle.subset_forward(mode, dsts, kp, ks, din[dsts], dout[dsts], need, dout[need], h[need], Wn, Ws, b, 1, gin_eps=0.25)
+    assert np.abs(sub - full[dsts]).max() <= 1e-12
