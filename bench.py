@@ -331,7 +331,10 @@ def make_context(args, w, g, model, host_evict, drain_rows):
                       w.leaky_slope)
 
 
-PHASES = ["copy_in", "projection", "classify_select", "row_moves", "scatter", "finalise"]
+# per push, from taurus_get_phase_ms: seven consecutive spans of the compute stream, the chunk's own finalise (which, with a
+# bounded pool, runs inside the NEXT chunk's fourth span) and the chunk's row transfers on the library's transfer stream
+PHASES = ["copy_in", "projection", "classify_select", "transfer_wait_and_previous_finalise", "slot_handout", "scatter",
+          "completion_list", "finalise", "row_transfers"]
 
 
 def scatter_bytes(groups, edges, n_src, width, self_row):
@@ -463,26 +466,30 @@ def run_windowed(args, env, w):
     phase = ph[: K * window].sum(axis=0).astype(np.float64)            # ms over the timed windows
     phase_ms = dict(zip(PHASES, [float(x) / K for x in phase]))
     row_bytes = 4 * acc_width
-    move_s = phase[3] * 1e-3
+    move_s = phase[8] * 1e-3                                           # transfer kernels, timed on their own stream
     out_gbs, in_gbs = evicted * row_bytes / move_s / 1e9, reloaded * row_bytes / move_s / 1e9
     n_src = chunks[prefill + (W + K) * window - 1][1] - chunks[prefill + W * window][0]
     sc_bytes = scatter_bytes(groups, msgs, n_src, acc_width, not (agg_first and w.mode == tg.SAGE_MEAN))
-    sc_s = phase[4] * 1e-3
-    moves_share = phase[3] / ms
+    sc_s = phase[5] * 1e-3
+    moves_share = phase[8] / ms
     # the dominant kernel: the row moves between the pool and pinned host memory (alloc_kernel), bound by the host link
-    roofline = dict(bound="pcie", kernel="alloc_kernel (evicted rows out, reloaded rows in, %d-byte rows)" % row_bytes,
+    roofline = dict(bound="pcie", kernel="transfer_kernel (evicted rows out, reloaded rows in, %d-byte rows)" % row_bytes,
                     achieved=(out_gbs + in_gbs) / 2, peak=link["both_per_direction_gbs"], unit="GB/s per direction",
                     frac=(out_gbs + in_gbs) / 2 / link["both_per_direction_gbs"], peak_source="measured in this run: " + link["how"],
                     device_to_host_gbs=out_gbs, host_to_device_gbs=in_gbs, link=link,
                     rows_out_per_step=evicted / K, rows_in_per_step=reloaded / K, launches_per_step=window,
-                    avg_launch_ms=float(phase[3]) / (K * window), algorithmic_bytes_per_launch=(evicted + reloaded) * row_bytes / (K * window),
-                    share_of_step=float(moves_share), traffic=None,
+                    avg_launch_ms=float(phase[8]) / (K * window), algorithmic_bytes_per_launch=(evicted + reloaded) * row_bytes / (K * window),
+                    share_of_step=float(moves_share),
+                    share_note="the transfers run on their own stream beside the compute stream: their share of the step is how "
+                               "much of the step the host link is busy",
+                    traffic=None,
                     traffic_note="no counter capture at this size (110 GB resident); PCIe counters of the same kernel on a 1.5 M-vertex "
                                  "instance are in profiles/alloc_kernel_large_1500k.md")
     roofline_hbm = dict(bound="hbm", kernel="scatter_grouped_kernel (accumulator rows of %d floats)" % acc_width,
                         achieved=sc_bytes / sc_s / 1e9, peak=pk["hbm_gbs"], unit="GB/s", frac=sc_bytes / sc_s / 1e9 / pk["hbm_gbs"],
-                        peak_source=pk["source"], groups_per_step=groups / K, avg_launch_ms=float(phase[4]) / (K * window),
-                        algorithmic_bytes_per_launch=sc_bytes / (K * window), share_of_step=float(phase[4] / ms),
+                        peak_source=pk["source"], groups_per_step=groups / K, avg_launch_ms=float(phase[5]) / (K * window),
+                        algorithmic_bytes_per_launch=sc_bytes / (K * window), share_of_step=float(phase[5] / ms),
+
                         gteps_scatter_only=msgs / sc_s / 1e9)
 
     # ---- end to end through the C ABI with host buffers: every chunk's input rows come from pinned host memory (one
@@ -620,14 +627,14 @@ def run_full_pass(args, env, w):
     ctx.set_timing(False)
     launches = ctx.launch_count() - launches0
     clocks = sampler.finish()
-    phases = ctx.get_phase_ms()   # [pushes, 6]
+    phases = ctx.get_phase_ms()   # [pushes, 9]
     ms_max = max_over_ranks(ms, world, dev)
     value = whole_job_value(msgs_per_step, args.steps, world, ms_max)
 
     # ---- roofline of the dominant kernel (the scatter), from the events recorded inside the timed region
     n_push = len(chunks) * L * args.steps
-    ph = phases[:n_push].reshape(args.steps, L, len(chunks), 6)
-    scatter_ms = ph[..., 4]
+    ph = phases[:n_push].reshape(args.steps, L, len(chunks), 9)
+    scatter_ms = ph[..., 5]
     # In CSR order a "group" is one edge.  The per-edge cold-miss model (12 + 2 * 4 width per edge) is kept beside it.
     layer_bytes, edge_model_bytes = [], []
     for l in range(L):
@@ -734,7 +741,7 @@ def run_full_pass(args, env, w):
                             messages_per_step=msgs_per_step,
                             l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
                             parallelism="replicas only" if world > 1 else "1 gpu",
-                            layer_ms=[float(ph[:, l].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
+                            layer_ms=[float(ph[:, l, :, :8].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
                 clocks=clocks, roofline=roofline, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
     for r in runs or []:
         r.destroy()

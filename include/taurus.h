@@ -437,10 +437,12 @@ int taurus_get_layer_plan(const taurus_ctx* ctx, int32_t layer, int32_t* out_agg
 int64_t taurus_launch_count(const taurus_ctx* ctx);
 
 /* Per-push device times.  taurus_set_timing(ctx, 1) starts a recording window: every later push (up to
- * 16384) brackets its phases with CUDA events on the push's stream.  taurus_get_phase_ms (blocking) returns,
- * for each recorded push p, out[p * 6 + k] in milliseconds: k = 0 copy-in, 1 projection, 2 classify and victim
- * selection, 3 row moves (evicted rows out, reloaded rows in, new rows cleared), 4 scatter, 5 finalise;
- * *out_pushes = pushes written (at most capacity_pushes). */
+ * 16384) brackets its phases with CUDA events.  taurus_get_phase_ms (blocking) returns, for each recorded push p,
+ * out[p * 9 + k] in milliseconds: k = 0 copy-in, 1 projection, 2 classify and victim selection, 3 the wait for the
+ * previous chunk's row transfers plus that chunk's finalise (bounded pools; else about zero), 4 slot hand-out (victims'
+ * rows staged, new rows cleared), 5 scatter, 6 completion list, 7 the chunk's own finalise, 8 the chunk's row
+ * transfers over the host link (evicted rows out, reloaded rows in; on the library's transfer stream, beside
+ * k = 5, 6 of this chunk and k = 0..2 of the next); *out_pushes = pushes written (at most capacity_pushes). */
 int taurus_set_timing(taurus_ctx* ctx, int32_t on);
 int taurus_get_phase_ms(taurus_ctx* ctx, float* out, int64_t capacity_pushes, int64_t* out_pushes);
 

@@ -422,9 +422,10 @@ class Context:
         self._check(self._lib.taurus_set_timing(self._h, 1 if on else 0), "taurus_set_timing")
 
     def get_phase_ms(self, capacity_pushes: int = 16384) -> np.ndarray:
-        """float32 [pushes, 6]: copy-in, projection, classify + victim selection, row moves (evict / reload / clear),
-        scatter, finalise (ms) per recorded push."""
-        out = np.zeros((capacity_pushes, 6), np.float32)
+        """float32 [pushes, 9] (ms per recorded push): copy-in, projection, classify + victim selection, wait for the
+        previous chunk's transfers + its finalise, slot hand-out, scatter, completion list, own finalise, row
+        transfers over the host link (side stream)."""
+        out = np.zeros((capacity_pushes, 9), np.float32)
         n = ctypes.c_int64(0)
         self._check(self._lib.taurus_get_phase_ms(self._h, out.ctypes.data, capacity_pushes, ctypes.byref(n)),
                     "taurus_get_phase_ms")

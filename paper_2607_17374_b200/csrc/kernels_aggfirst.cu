@@ -40,8 +40,9 @@ __global__ void af_prep_kernel(const float* __restrict__ X, int ldx, int n, int 
 // by compact_done_kernel; its row stays intact until the next chunk.
 __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long rows, const float* __restrict__ self_store) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
-  const int n = ctl->done_count;
+  const int n = pc->done_count;
   if (n > rows) {   // the host sized the transform for fewer rows than completed: its bound was wrong
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
     return;
@@ -79,8 +80,9 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
 // O has pitch a.Hout; rows of the graduation buffer too.
 __global__ void af_finish_kernel(ChunkArgs a, const float* __restrict__ O, long long rows) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
-  const int n = ctl->done_count;
+  const int n = pc->done_count;
   if (n > rows) {   // the host sized the transform for fewer rows than completed: its bound was wrong
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
     return;
@@ -128,10 +130,9 @@ void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp
   c->launches += 1;
 }
 
-// S6 + S7 of an aggregate-first layer: compact, gather, transform, finish, commit.  `rows` is the host's bound on the
-// vertices this chunk completes (the transform is sized for it; rows beyond the actual count are zero).
+// S7 of an aggregate-first layer (after launch_compact_done): gather, transform, finish, commit.  `rows` is the host's
+// bound on the vertices this chunk completes (the transform is sized for it; rows beyond the actual count are zero).
 int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long rows, cudaStream_t st) {
-  launch_compact_done(c, a, st);
   if (rows > 0) {
     const int grid = c->sm_count * 8;
     float* O;
@@ -152,13 +153,13 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
       GemmFinish fin;
       fin.done_list = a.done_list; fin.state = a.state; fin.dense = a.dense_direct; fin.dense_ld = a.dense_ld;
       fin.bias = a.bias; fin.act = a.act;
-      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, &fin, true);
+      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, &fin, &a.pc->done_count);
       if (rc) return rc;
       launch_commit(c, a, st);
       return TAURUS_OK;
     }
     if (tc) {
-      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, nullptr, true);
+      int rc = launch_gemm_plain_tc(c, image, 0, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st, nullptr, &a.pc->done_count);
       if (rc) return rc;
     } else if (sage) {
       launch_gemm_plain_simt(c, c->d_Waf[layer], a.Hout, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);

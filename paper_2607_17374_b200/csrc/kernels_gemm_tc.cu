@@ -122,7 +122,7 @@ struct GemmArgs {
   const int32_t* din;
   long long src_begin;
   DevCtl* ctl;
-  int rows_from_ctl;    // the rows that matter are the first ctl->done_count ones: row tiles behind them are skipped
+  const int32_t* done_count;   // non-null: the rows that matter are the first *done_count ones (read on the device): row tiles behind them are skipped
   int finish;           // epilogue of finished rows: act(row + fin.bias) into fin.dense[fin.done_list[row]], no store to PT
   GemmFinish fin;
 };
@@ -141,7 +141,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   volatile int* abort_flag = &bars->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int n_rows = g.n;
-  if (g.rows_from_ctl) { const int nd = g.ctl->done_count; n_rows = nd < g.n ? nd : g.n; }   // same value in every thread
+  if (g.done_count) { const int nd = *g.done_count; n_rows = nd < g.n ? nd : g.n; }   // same value in every thread
   const int n_tiles = (n_rows + BM - 1) / BM;
   const int n_blocks = (g.Np + BN_MAX - 1) / BN_MAX;
   const int tmem_cols = 512;   // two accumulator buffers of 256 columns; one CTA per SM
@@ -289,7 +289,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     float c_out = 1.f, self_mul = 1.f;
     int vrow = -1;        // finish mode: the vertex this lane's row belongs to
     if (g.finish) {
-      if (r < g.n && r < g.ctl->done_count && !g.ctl->error) {
+      if (r < g.n && r < *g.done_count && !g.ctl->error) {
         vrow = g.fin.done_list[r];
         if (nb == 0) g.fin.state[vrow] = TAURUS_COMPLETED;
       }
@@ -523,7 +523,7 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   set_stages(g, bf16);
   g.Hp = Hp; g.mode = c->mode; g.fanout = c->fanout[layer]; g.bias = c->d_bias[layer];
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = src_begin; g.ctl = c->d_ctl;
-  g.finish = 0; g.fin = GemmFinish(); g.rows_from_ctl = 0;
+  g.finish = 0; g.fin = GemmFinish(); g.done_count = nullptr;
   const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
   const int n_tiles = (n + BM - 1) / BM;
   const int n_units = n_tiles * ((w->Np + BN_MAX - 1) / BN_MAX);
@@ -552,7 +552,7 @@ bool gemm_plain_tc_usable(const taurus_ctx* c, const void* image, const float* X
 }
 
 int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
-                         cudaStream_t st, const GemmFinish* finish, bool rows_from_done_count) {
+                         cudaStream_t st, const GemmFinish* finish, const int32_t* done_count) {
   if (n <= 0) return TAURUS_OK;
   if (finish && ((N & 3) != 0 || (finish->dense_ld & 3) != 0 || (reinterpret_cast<uintptr_t>(finish->dense) & 15) != 0)) return TAURUS_ERR_INTERNAL;
   const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
@@ -580,7 +580,7 @@ int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const floa
   g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = nullptr;
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = 0; g.ctl = c->d_ctl;
   g.finish = finish ? 1 : 0; g.fin = finish ? *finish : GemmFinish();
-  g.rows_from_ctl = rows_from_done_count ? 1 : 0;
+  g.done_count = done_count;
   const int smem = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32) + OUT_STAGING_BYTES + (int)sizeof(Barriers) + 1024;
   const int n_tiles = (n + BM - 1) / BM;
   const int n_units = n_tiles * ((Np + BN_MAX - 1) / BN_MAX);

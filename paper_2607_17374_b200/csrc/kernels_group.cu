@@ -143,6 +143,7 @@ void launch_group_mask(taurus_ctx* c, cudaStream_t st) {
 #define CG_ITEMS 4
 __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, const int32_t* __restrict__ g_dst, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
   // list appends are aggregated per block: single-address atomics are the throughput limit of this kernel
   __shared__ int s_cnt[2][2][8];   // [parity][need / touched][warp]
@@ -223,7 +224,7 @@ __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, cons
     if (threadIdx.x < 2) {
       int sum = 0;
       for (int w = 0; w < 8; ++w) { int c = s_cnt[par][threadIdx.x][w]; s_cnt[par][threadIdx.x][w] = sum; sum += c; }
-      s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &ctl->need_count : &ctl->touched_count, sum) : 0;
+      s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &pc->need_count : &pc->touched_count, sum) : 0;
     }
     __syncthreads();
     int on = s_base[par][0] + s_cnt[par][0][warp], ot = s_base[par][1] + s_cnt[par][1][warp];
@@ -247,10 +248,10 @@ __global__ void __launch_bounds__(256) classify_grouped_kernel(ChunkArgs a, cons
     bad |= __shfl_xor_sync(FULL, bad, o);
   }
   if (lane_id() == 0) {
-    if (hs) atomicAdd(&ctl->hs, hs);
-    if (ns) atomicAdd(&ctl->ns, ns);
-    if (ev) atomicAdd(&ctl->ev, ev);
-    if (gs) atomicAdd(&ctl->gs, gs);
+    if (hs) atomicAdd(&pc->hs, hs);
+    if (ns) atomicAdd(&pc->ns, ns);
+    if (ev) atomicAdd(&pc->ev, ev);
+    if (gs) atomicAdd(&pc->gs, gs);
     if (bad) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
   }
 }
@@ -275,6 +276,7 @@ template <int LPE, int VPL, bool SAMPLED, bool DIRECT, bool GAT>
 __global__ void __launch_bounds__(256, (VPL <= 2 ? 3 : VPL == 3 ? 2 : 1))
 scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
   constexpr int EPS = 32 / LPE;                 // sub-groups per warp
   constexpr int STRETCH = SPAN_EDGES / EPS;     // edges one sub-group walks per span

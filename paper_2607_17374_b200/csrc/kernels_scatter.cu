@@ -39,6 +39,7 @@ static __device__ __forceinline__ long long warp_find_source(const long long* ro
 template <int LPE, int VPL>
 __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
   constexpr int EPS = 32 / LPE;                 // edges handled per warp step
   const int lane = lane_id();

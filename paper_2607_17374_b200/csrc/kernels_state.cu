@@ -72,6 +72,7 @@ void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st) {
 // loc encoding: -1 none, [0, pool_slots) pool slot, >= pool_slots hub row, <= -2 host row (-2 - loc).
 __global__ void __launch_bounds__(256) classify_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
   // list appends are aggregated per block: single-address atomics are the throughput limit of this kernel
   __shared__ int s_cnt[2][2][8];   // [parity][need / touched][warp]
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(256) classify_kernel(ChunkArgs a) {
     if (threadIdx.x < 2) {
       int sum = 0;
       for (int w = 0; w < 8; ++w) { int c = s_cnt[par][threadIdx.x][w]; s_cnt[par][threadIdx.x][w] = sum; sum += c; }
-      s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &ctl->need_count : &ctl->touched_count, sum) : 0;
+      s_base[par][threadIdx.x] = sum ? atomicAdd(threadIdx.x == 0 ? &pc->need_count : &pc->touched_count, sum) : 0;
     }
     __syncthreads();
     if (need) {
@@ -137,10 +138,10 @@ __global__ void __launch_bounds__(256) classify_kernel(ChunkArgs a) {
     bad |= __shfl_xor_sync(FULL, bad, o);
   }
   if (lane_id() == 0) {
-    if (hs) atomicAdd(&ctl->hs, hs);
-    if (ns) atomicAdd(&ctl->ns, ns);
-    if (ev) atomicAdd(&ctl->ev, ev);
-    if (gs) atomicAdd(&ctl->gs, gs);
+    if (hs) atomicAdd(&pc->hs, hs);
+    if (ns) atomicAdd(&pc->ns, ns);
+    if (ev) atomicAdd(&pc->ev, ev);
+    if (gs) atomicAdd(&pc->gs, gs);
     if (bad) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
   }
 }
@@ -152,33 +153,34 @@ void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
 
 // ------------------------------------------------------------------------------------------------ make room (S4)
 // plan: need, deficit, capacity checks, peak occupancy.
-static __device__ void plan_chunk(const ChunkArgs& a, DevCtl* ctl) {   // one thread
-  long long need = ctl->need_count;
+static __device__ void plan_chunk(const ChunkArgs& a, DevCtl* ctl, ChunkCtl* pc) {   // one thread
+  long long need = pc->need_count;
   if (need > a.pool_slots) { ctl->error = TAURUS_ERR_POOL_TOO_SMALL; return; }
   long long deficit = need - ctl->free_top;
   if (deficit < 0) deficit = 0;
   // this chunk's victims leave before its reloads hand their host rows back
   if (ctl->host_live + deficit > a.host_rows) { ctl->error = TAURUS_ERR_HOST_STORE_FULL; return; }
-  ctl->host_live += deficit - ctl->ev;
-  ctl->deficit = (int32_t)deficit;
-  ctl->victim_count = 0;
-  for (int l = 0; l <= TAURUS_SEL_LEVELS; ++l) { ctl->sel_k[l] = 0; ctl->sel_min[l] = ~0ull; ctl->sel_max[l] = 0ull; ctl->sel_count[l] = 0; }
-  ctl->sel_k[0] = deficit;
-  ctl->sel_final_level = deficit > 0 ? TAURUS_SEL_LEVELS + 1 : -1;
+  ctl->host_live += deficit - pc->ev;
+  pc->deficit = (int32_t)deficit;
+  pc->victim_count = 0;
+  for (int l = 0; l <= TAURUS_SEL_LEVELS; ++l) { pc->sel_k[l] = 0; pc->sel_min[l] = ~0ull; pc->sel_max[l] = 0ull; pc->sel_count[l] = 0; }
+  pc->sel_k[0] = deficit;
+  pc->sel_final_level = deficit > 0 ? TAURUS_SEL_LEVELS + 1 : -1;
   // Slots are handed out by list index, not by per-item atomics: need-list entry i < deficit takes over the slot
   // of victim deficit - 1 - i, entry i >= deficit pops free_stack[F + deficit - 1 - i].  The counter is brought to
   // its end-of-chunk value here.
   const long long F = ctl->free_top;
-  ctl->alloc_base = F + deficit;
+  pc->alloc_base = F + deficit;
   ctl->free_top = F + deficit - need;
   long long occ = a.pool_slots - ctl->free_top;
   if (occ > ctl->peak_occupancy) ctl->peak_occupancy = occ;
 }
 __global__ void plan_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
-  for (int i = threadIdx.x; i < 2 * TAURUS_SEL_BINS; i += blockDim.x) (&ctl->hist[0][0])[i] = 0;
-  if (threadIdx.x == 0) plan_chunk(a, ctl);
+  for (int i = threadIdx.x; i < 2 * TAURUS_SEL_BINS; i += blockDim.x) (&pc->hist[0][0])[i] = 0;
+  if (threadIdx.x == 0) plan_chunk(a, ctl, pc);
 }
 
 // Victims are the `deficit` smallest keys (score << 31 | id) among IN_BUFFER vertices the chunk does not
@@ -211,7 +213,7 @@ static __device__ __forceinline__ int sel_shift_of(unsigned long long lo, unsign
 }
 
 // Block-wide minimum / maximum / count of the eligible keys a thread saw, folded into level `lvl` of the control block.
-static __device__ __forceinline__ void sel_fold(DevCtl* ctl, int lvl, unsigned long long kmin, unsigned long long kmax, int cnt) {
+static __device__ __forceinline__ void sel_fold(ChunkCtl* pc, int lvl, unsigned long long kmin, unsigned long long kmax, int cnt) {
   for (int o = 16; o; o >>= 1) {
     const unsigned long long m = __shfl_xor_sync(FULL, kmin, o), M = __shfl_xor_sync(FULL, kmax, o);
     if (m < kmin) kmin = m;
@@ -219,15 +221,16 @@ static __device__ __forceinline__ void sel_fold(DevCtl* ctl, int lvl, unsigned l
     cnt += __shfl_xor_sync(FULL, cnt, o);
   }
   if (lane_id() == 0 && cnt) {
-    atomicMin(&ctl->sel_min[lvl], kmin);
-    atomicMax(&ctl->sel_max[lvl], kmax);
-    atomicAdd(&ctl->sel_count[lvl], cnt);
+    atomicMin(&pc->sel_min[lvl], kmin);
+    atomicMax(&pc->sel_max[lvl], kmax);
+    atomicAdd(&pc->sel_count[lvl], cnt);
   }
 }
 
 __global__ void __launch_bounds__(256) select_keys_kernel(ChunkArgs a) {   // key of every slot; range of the eligible keys
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->sel_final_level < 0) return;
+  ChunkCtl* pc = a.pc;
+  if (ctl->error || pc->sel_final_level < 0) return;
   unsigned long long kmin = ~0ull, kmax = 0ull;
   int cnt = 0;
   const long long stride = (long long)gridDim.x * blockDim.x;
@@ -250,24 +253,25 @@ __global__ void __launch_bounds__(256) select_keys_kernel(ChunkArgs a) {   // ke
     }
     a.keys[s] = key;
   }
-  sel_fold(ctl, 0, kmin, kmax, cnt);
+  sel_fold(pc, 0, kmin, kmax, cnt);
 }
 
 // Histogram of the level's digit over the keys entering the level.  Threads of a warp that hit the same bin add
 // once (most keys of a level often share a bin).
 __global__ void __launch_bounds__(256) select_hist_kernel(ChunkArgs a, int level) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->sel_final_level < level) return;
-  const long long k = ctl->sel_k[level];
-  const long long n = level == 0 ? a.pool_slots : (long long)ctl->sel_count[level];
-  if (ctl->sel_count[level] < k) {   // fewer eligible victims than needed
+  ChunkCtl* pc = a.pc;
+  if (ctl->error || pc->sel_final_level < level) return;
+  const long long k = pc->sel_k[level];
+  const long long n = level == 0 ? a.pool_slots : (long long)pc->sel_count[level];
+  if (pc->sel_count[level] < k) {   // fewer eligible victims than needed
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(&ctl->error, 0, level == 0 ? TAURUS_ERR_POOL_TOO_SMALL : TAURUS_ERR_INTERNAL);
     return;
   }
   __shared__ unsigned int sh[TAURUS_SEL_BINS];
   for (int i = threadIdx.x; i < TAURUS_SEL_BINS; i += blockDim.x) sh[i] = 0;
   __syncthreads();
-  const int shift = sel_shift_of(ctl->sel_min[level], ctl->sel_max[level]);
+  const int shift = sel_shift_of(pc->sel_min[level], pc->sel_max[level]);
   const int32_t* __restrict__ cand = level == 0 ? nullptr : a.cand[level & 1];
   const long long stride = (long long)gridDim.x * blockDim.x;
   const long long rounds = (n + stride - 1) / stride;
@@ -281,7 +285,7 @@ __global__ void __launch_bounds__(256) select_hist_kernel(ChunkArgs a, int level
     if (on && lane_id() == __ffs(peers) - 1) atomicAdd(&sh[digit], (unsigned)__popc(peers));
   }
   __syncthreads();
-  unsigned int* hist = ctl->hist[level & 1];
+  unsigned int* hist = pc->hist[level & 1];
   for (int b = threadIdx.x; b < TAURUS_SEL_BINS; b += blockDim.x)
     if (sh[b]) atomicAdd(&hist[b], sh[b]);
 }
@@ -290,13 +294,14 @@ __global__ void __launch_bounds__(256) select_hist_kernel(ChunkArgs a, int level
 // it go to the next level (or are victims too when the digit holds exactly the ranks still missing).
 __global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int level) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->sel_final_level < level) return;
+  ChunkCtl* pc = a.pc;
+  if (ctl->error || pc->sel_final_level < level) return;
   __shared__ unsigned int sh[TAURUS_SEL_BINS];
   __shared__ unsigned int part[256];
   __shared__ int s_digit;
   __shared__ long long s_rest;
-  const unsigned int* hist = ctl->hist[level & 1];
-  const long long k = ctl->sel_k[level];
+  const unsigned int* hist = pc->hist[level & 1];
+  const long long k = pc->sel_k[level];
   // bins per thread: TAURUS_SEL_BINS / 256 consecutive ones
   constexpr int PER = TAURUS_SEL_BINS / 256;
   unsigned int mine[PER], sum = 0;
@@ -324,17 +329,17 @@ __global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int leve
   }
   const long long rest = s_rest;
   const bool final = rest == (long long)sh[digit_k];   // the whole digit is victims: nothing left to resolve
-  const int shift = sel_shift_of(ctl->sel_min[level], ctl->sel_max[level]);
-  const long long n = level == 0 ? a.pool_slots : (long long)ctl->sel_count[level];
+  const int shift = sel_shift_of(pc->sel_min[level], pc->sel_max[level]);
+  const long long n = level == 0 ? a.pool_slots : (long long)pc->sel_count[level];
   const int32_t* __restrict__ cand = level == 0 ? nullptr : a.cand[level & 1];
   int32_t* __restrict__ next = a.cand[(level + 1) & 1];
   if (blockIdx.x == 0) {
-    unsigned int* other = ctl->hist[(level + 1) & 1];   // the next level's histogram (read last by the level above this one)
+    unsigned int* other = pc->hist[(level + 1) & 1];   // the next level's histogram (read last by the level above this one)
     for (int b = threadIdx.x; b < TAURUS_SEL_BINS; b += blockDim.x) other[b] = 0;
     if (threadIdx.x == 0) {
-      if (final) ctl->sel_final_level = level;
+      if (final) pc->sel_final_level = level;
       else if (level == TAURUS_SEL_LEVELS - 1 || shift == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);   // unique keys always end in a final level
-      else ctl->sel_k[level + 1] = rest;
+      else pc->sel_k[level + 1] = rest;
     }
   }
   unsigned long long kmin = ~0ull, kmax = 0ull;
@@ -355,14 +360,14 @@ __global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int leve
     if (mv) {
       int idx = 0;
       const int leader = __ffs(mv) - 1;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->victim_count, __popc(mv));
+      if (lane_id() == leader) idx = atomicAdd(&pc->victim_count, __popc(mv));
       idx = __shfl_sync(FULL, idx, leader) + __popc(mv & lt);
       if (victim && idx < a.victim_capacity) a.victims[idx].x = slot;
     }
     if (mk) {
       int idx = 0;
       const int leader = __ffs(mk) - 1;
-      if (lane_id() == leader) idx = atomicAdd(&ctl->sel_count[level + 1], __popc(mk));
+      if (lane_id() == leader) idx = atomicAdd(&pc->sel_count[level + 1], __popc(mk));
       idx = __shfl_sync(FULL, idx, leader) + __popc(mk & lt);
       if (keep) {
         next[idx] = slot;   // at most pool_slots keys enter any level
@@ -380,8 +385,8 @@ __global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int leve
     cnt += __shfl_xor_sync(FULL, cnt, o);
   }
   if (lane_id() == 0 && cnt) {
-    atomicMin(&ctl->sel_min[level + 1], kmin);
-    atomicMax(&ctl->sel_max[level + 1], kmax);
+    atomicMin(&pc->sel_min[level + 1], kmin);
+    atomicMax(&pc->sel_max[level + 1], kmax);
   }
 }
 
@@ -411,9 +416,10 @@ static __device__ __forceinline__ long long next_sender(const ChunkArgs& a, int 
 
 __global__ void __launch_bounds__(256) victim_bucket_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->deficit == 0) return;
-  const int n = ctl->deficit;
-  if (ctl->victim_count != n) {   // the select must have produced exactly `deficit` victims
+  ChunkCtl* pc = a.pc;
+  if (ctl->error || pc->deficit == 0) return;
+  const int n = pc->deficit;
+  if (pc->victim_count != n) {   // the select must have produced exactly `deficit` victims
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
     return;
   }
@@ -433,12 +439,25 @@ __global__ void __launch_bounds__(256) victim_bucket_kernel(ChunkArgs a) {
 // the extents it lacks from the free stack.
 __global__ void __launch_bounds__(1024) extent_plan_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
   const int E = 1 << a.ext_shift;
   __shared__ int warp_sum[32];
   __shared__ long long s_running;
   __shared__ int s_fail;
   if (threadIdx.x == 0) { s_running = 0; s_fail = 0; }
+  // phase 0: the extents emptied by the transfers of the last chunk of this parity go back on the free stack.  Those
+  // transfers are complete (the chunk in between waited for them before it moved its own rows); the transfers of the
+  // chunk in between may still be running and append to the other list.
+  {
+    const int par = a.epoch & 1;
+    const int n_ret = ctl->ext_ret_count[par];
+    const long long top = ctl->ext_free_top;
+    for (int i = threadIdx.x; i < n_ret; i += blockDim.x) a.ext_free[top + i] = a.ext_ret[par][i];
+    __syncthreads();
+    if (threadIdx.x == 0) { ctl->ext_free_top = top + n_ret; ctl->ext_ret_count[par] = 0; }
+    __syncthreads();
+  }
   // phase 1: close tails
   {
     const long long first = a.src_begin / a.chunk_sources;
@@ -459,7 +478,7 @@ __global__ void __launch_bounds__(1024) extent_plan_kernel(ChunkArgs a) {
     }
   }
   __syncthreads();
-  if (ctl->deficit == 0) return;
+  if (pc->deficit == 0) return;
   // phase 2: extents needed per bucket, exclusive prefix over the buckets
   for (long long base = 0; base < a.n_buckets; base += blockDim.x) {
     const long long b = base + threadIdx.x;
@@ -519,8 +538,9 @@ __global__ void __launch_bounds__(1024) extent_plan_kernel(ChunkArgs a) {
 
 __global__ void __launch_bounds__(256) victim_place_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
-  if (ctl->error || ctl->deficit == 0) return;
-  const int n = ctl->deficit;
+  ChunkCtl* pc = a.pc;
+  if (ctl->error || pc->deficit == 0) return;
+  const int n = pc->deficit;
   const int E = 1 << a.ext_shift;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
@@ -543,9 +563,10 @@ __global__ void __launch_bounds__(256) victim_place_kernel(ChunkArgs a) {
 // the vertex is IN_BUFFER afterwards.
 __global__ void alloc_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
-  const int n = ctl->need_count;
-  const int deficit = ctl->deficit;
+  const int n = pc->need_count;
+  const int deficit = pc->deficit;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
   if (a.direct) {
@@ -554,7 +575,7 @@ __global__ void alloc_kernel(ChunkArgs a) {
     // accesses, then the warp clears the rows one after the other.
     // No other thread of this kernel reads what the plan writes (there is no deficit and no stack to pop), so one
     // thread does the chunk's bookkeeping here and the separate plan launch is left out.
-    if (blockIdx.x == 0 && threadIdx.x == 0) plan_chunk(a, ctl);
+    if (blockIdx.x == 0 && threadIdx.x == 0) plan_chunk(a, ctl, pc);
     int per = (int)((n + warps - 1) / warps);
     per = per < 1 ? 1 : per > 32 ? 32 : per;
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -576,7 +597,13 @@ __global__ void alloc_kernel(ChunkArgs a) {
     }
     return;
   }
+  // Bounded pool.  Need-list entry i < deficit takes over the slot of victim deficit - 1 - i: the victim's row is
+  // copied to the staging buffer (it leaves for its pinned host row in transfer_kernel) and the victim becomes
+  // EVICTED; entry i >= deficit pops the free stack.  Either way the slot is cleared and handed to the vertex, which
+  // is IN_BUFFER afterwards; the partial sum of a vertex that was EVICTED is ADDED into the slot by transfer_kernel
+  // (sums commute: the scatter may already be adding this chunk's messages to the same row).
   int reloaded = 0;
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
   for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
     int v = a.need_list[i];
     int slot = -1, st = 0, l = 0, out_hrow = -1, victim = -1;
@@ -584,53 +611,31 @@ __global__ void alloc_kernel(ChunkArgs a) {
       if (i < deficit) {
         const int2 vic = a.victims[deficit - 1 - i];
         slot = vic.x; out_hrow = vic.y; victim = a.owner[slot];
-      } else { long long f = ctl->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
+      } else { long long f = pc->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
       st = a.state[v];
       l = a.loc[v];
     }
     slot = __shfl_sync(FULL, slot, 0);
-    st = __shfl_sync(FULL, st, 0);
-    l = __shfl_sync(FULL, l, 0);
     out_hrow = __shfl_sync(FULL, out_hrow, 0);
     if (slot < 0) {
       if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
       continue;
     }
     float4* __restrict__ row = reinterpret_cast<float4*>(a.acc + (size_t)slot * a.Hp);
-    float4* __restrict__ host_out = out_hrow >= 0 ? reinterpret_cast<float4*>(a.host_store + (size_t)out_hrow * a.Hp) : nullptr;
-    const int in_hrow = st == TAURUS_EVICTED ? -2 - l : -1;
-    const float4* __restrict__ host_in = in_hrow >= 0 ? reinterpret_cast<const float4*>(a.host_store + (size_t)in_hrow * a.Hp) : nullptr;
-    for (int k0 = 0; k0 < vec; k0 += 128) {   // four float4 per lane and direction in flight
-      float4 keep[4], in[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int k = k0 + q * 32 + lane_id();
-        in[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (k < vec) {
-          if (host_out) keep[q] = row[k];
-          if (host_in) in[q] = host_in[k];
-        }
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int k = k0 + q * 32 + lane_id();
-        if (k < vec) {
-          if (host_out) host_out[k] = keep[q];
-          row[k] = in[q];
-        }
-      }
+    if (out_hrow >= 0) {
+      float4* __restrict__ keep = reinterpret_cast<float4*>(a.stage_out + (size_t)i * a.Hp);
+      for (int k = lane_id(); k < vec; k += 32) { keep[k] = row[k]; row[k] = zero; }
+    } else {
+      for (int k = lane_id(); k < vec; k += 32) row[k] = zero;
     }
     if (lane_id() == 0) {
+      const int in_hrow = st == TAURUS_EVICTED ? -2 - l : -1;
+      if (a.xfer_list) a.xfer_list[i] = make_int4(slot, in_hrow, out_hrow, 0);
       if (out_hrow >= 0) {
         a.loc[victim] = -2 - out_hrow;
         a.state[victim] = TAURUS_EVICTED;
       }
       if (in_hrow >= 0) {
-        const int e = in_hrow >> a.ext_shift;
-        if (atomicSub(&a.ext_live[e], 1) == 1) {   // last row of the extent: back on the free stack (popped again by a later chunk's plan)
-          const long long top = (long long)atomicAdd((unsigned long long*)&ctl->ext_free_top, 1ull);
-          a.ext_free[top] = e;
-        }
         a.reload_count[v] += 1;
         reloaded++;
       }
@@ -639,7 +644,53 @@ __global__ void alloc_kernel(ChunkArgs a) {
       a.state[v] = TAURUS_IN_BUFFER;
     }
   }
-  if (lane_id() == 0 && reloaded) atomicAdd(&ctl->reloaded, reloaded);
+  if (lane_id() == 0 && reloaded) atomicAdd(&pc->reloaded, reloaded);
+}
+
+// The rows of one chunk across the host link, one warp per need-list entry: the staged row of the victim whose slot the
+// entry took over goes to its pinned host row (device -> host), and the host row of a vertex that was EVICTED is added
+// into its new slot (host -> device), so both directions of the link are busy at once.  An extent whose last row has
+// come back is listed for the free stack (taken back two chunks later by extent_plan_kernel).
+__global__ void transfer_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
+  if (ctl->error) return;
+  const int n = pc->need_count;
+  const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const int vec = a.Hp >> 2;
+  const int par = a.epoch & 1;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+    const int4 x = a.xfer_list[i];   // same address for the whole warp
+    const int slot = x.x, in_hrow = x.y, out_hrow = x.z;
+    if (in_hrow < 0 && out_hrow < 0) continue;
+    float* __restrict__ row = a.acc + (size_t)slot * a.Hp;
+    const float4* __restrict__ staged = reinterpret_cast<const float4*>(a.stage_out + (size_t)i * a.Hp);
+    float4* __restrict__ host_out = out_hrow >= 0 ? reinterpret_cast<float4*>(a.host_store + (size_t)out_hrow * a.Hp) : nullptr;
+    const float4* __restrict__ host_in = in_hrow >= 0 ? reinterpret_cast<const float4*>(a.host_store + (size_t)in_hrow * a.Hp) : nullptr;
+    for (int k0 = 0; k0 < vec; k0 += 128) {   // four float4 per lane and direction in flight
+      float4 keep[4], in[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = k0 + q * 32 + lane_id();
+        if (k < vec) {
+          if (host_out) keep[q] = staged[k];
+          if (host_in) in[q] = host_in[k];
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = k0 + q * 32 + lane_id();
+        if (k < vec) {
+          if (host_out) host_out[k] = keep[q];
+          if (host_in) asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(row + 4 * k), "f"(in[q].x), "f"(in[q].y), "f"(in[q].z), "f"(in[q].w) : "memory");
+        }
+      }
+    }
+    if (lane_id() == 0 && in_hrow >= 0) {
+      const int e = in_hrow >> a.ext_shift;
+      if (atomicSub(&a.ext_live[e], 1) == 1) a.ext_ret[par][atomicAdd(&ctl->ext_ret_count[par], 1)] = e;   // last row of the extent
+    }
+  }
 }
 
 void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEvent_t before_moves) {
@@ -662,7 +713,19 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEv
     c->launches += 2 * TAURUS_SEL_LEVELS + 4;
   }
   if (before_moves) cudaEventRecord(before_moves, st);
-  alloc_kernel<<<blocks, 256, 0, st>>>(a);
+}
+
+// Slots handed out, victims' rows staged, new rows cleared (S4, device side).
+void launch_alloc(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  alloc_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
+  c->launches += 1;
+}
+// Rows across the host link (bounded pools only).
+void launch_transfer(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+  // One block per SM.  The warps spend their time waiting for the host link; measured on the "large" workload, fewer
+  // blocks leave the link short of requests (64 blocks: 36 + 33 GB/s, 148: 38 + 34, 1 184: 39 + 35), more blocks only
+  // take thread slots from the scatter and select kernels that run beside the transfers on the compute stream.
+  transfer_kernel<<<c->sm_count, 256, 0, st>>>(a);
   c->launches += 1;
 }
 
@@ -675,8 +738,9 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEv
 #define CD_ITEMS 4
 __global__ void compact_done_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
-  const int n = ctl->touched_count;
+  const int n = pc->touched_count;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const unsigned lt = (1u << lane_id()) - 1;
@@ -719,7 +783,7 @@ __global__ void compact_done_kernel(ChunkArgs a) {
     int idx = 0;
     long long f = 0;
     if (lane_id() == 0) {
-      if (cd) idx = atomicAdd(&ctl->done_count, cd);
+      if (cd) idx = atomicAdd(&pc->done_count, cd);
       if (cr) f = (long long)atomicAdd((unsigned long long*)&ctl->free_top, (unsigned long long)cr);
     }
     idx = __shfl_sync(FULL, idx, 0);
@@ -748,8 +812,9 @@ __global__ void compact_done_kernel(ChunkArgs a) {
 // caller's vertex-ordered matrix (Sect. 3.6); the slot is released by compact_done_kernel.
 __global__ void finalise_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (ctl->error) return;
-  const int n = ctl->done_count;
+  const int n = pc->done_count;
   const long long base = a.dense_half >= 0 ? a.grad_off : ctl->grad_count;
   const long long limit = a.dense_half >= 0 ? a.grad_off + a.grad_cap : a.drain_rows;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -817,43 +882,54 @@ __global__ void finalise_kernel(ChunkArgs a) {
   }
 }
 
-// One thread: fold the chunk's counters into the layer totals, write the chunk record, reset.
-__global__ void commit_kernel(ChunkArgs a) {
+// One thread, after the chunk's completions are listed: fold the chunk's counters into the layer totals, write the chunk
+// record.
+__global__ void commit_counts_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
   if (threadIdx.x != 0 || ctl->error) return;
   long long c = ctl->chunks;
   if (c < a.log_capacity) {
     long long* r = a.chunk_log + c * TAURUS_CK_COLUMNS;
-    r[TAURUS_CK_HS] = ctl->hs; r[TAURUS_CK_NS] = ctl->ns; r[TAURUS_CK_EV] = ctl->ev; r[TAURUS_CK_GS] = ctl->gs;
-    r[TAURUS_CK_NEED] = ctl->need_count; r[TAURUS_CK_EVICTED] = ctl->deficit; r[TAURUS_CK_RELOADED] = ctl->reloaded;
-    r[TAURUS_CK_COMPLETED] = ctl->done_count; r[TAURUS_CK_OCCUPANCY] = a.pool_slots - ctl->free_top;
+    r[TAURUS_CK_HS] = pc->hs; r[TAURUS_CK_NS] = pc->ns; r[TAURUS_CK_EV] = pc->ev; r[TAURUS_CK_GS] = pc->gs;
+    r[TAURUS_CK_NEED] = pc->need_count; r[TAURUS_CK_EVICTED] = pc->deficit; r[TAURUS_CK_RELOADED] = pc->reloaded;
+    r[TAURUS_CK_COMPLETED] = pc->done_count; r[TAURUS_CK_OCCUPANCY] = a.pool_slots - ctl->free_top;
   }
-  ctl->sum_hs += ctl->hs; ctl->sum_ns += ctl->ns; ctl->sum_ev += ctl->ev; ctl->sum_gs += ctl->gs;
-  ctl->evictions += ctl->deficit;
-  ctl->reloads += ctl->reloaded;
-  ctl->completed += ctl->done_count;
-  if (a.dense_direct) { /* rows already sit in the caller's matrix */ }
-  else if (a.dense_half >= 0) ctl->out_count[a.dense_half] = ctl->done_count;
-  else ctl->grad_count += ctl->done_count;
+  ctl->sum_hs += pc->hs; ctl->sum_ns += pc->ns; ctl->sum_ev += pc->ev; ctl->sum_gs += pc->gs;
+  ctl->evictions += pc->deficit;
+  ctl->reloads += pc->reloaded;
+  ctl->completed += pc->done_count;
   ctl->chunks = c + 1;
-  ctl->hs = ctl->ns = ctl->ev = ctl->gs = 0;
-  ctl->need_count = 0; ctl->done_count = 0; ctl->touched_count = 0; ctl->deficit = 0; ctl->victim_count = 0; ctl->reloaded = 0;
+}
+// One thread, after the chunk's rows are finalised: the graduation buffer's row count, and the chunk's counters are
+// cleared for the chunk after next.
+__global__ void commit_kernel(ChunkArgs a) {
+  DevCtl* ctl = a.ctl;
+  ChunkCtl* pc = a.pc;
+  if (threadIdx.x != 0 || ctl->error) return;
+  if (a.dense_direct) { /* rows already sit in the caller's matrix */ }
+  else if (a.dense_half >= 0) ctl->out_count[a.dense_half] = pc->done_count;
+  else ctl->grad_count += pc->done_count;
+  pc->hs = pc->ns = pc->ev = pc->gs = 0;
+  pc->need_count = 0; pc->done_count = 0; pc->touched_count = 0; pc->deficit = 0; pc->victim_count = 0; pc->reloaded = 0;
 }
 
+// S6: completions listed, slots released, chunk record written.
 void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   compact_done_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
-  c->launches += 1;
+  commit_counts_kernel<<<1, 32, 0, st>>>(a);
+  c->launches += 2;
 }
 void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   commit_kernel<<<1, 32, 0, st>>>(a);
   c->launches += 1;
 }
 
+// S7 of a project-first layer (after launch_compact_done): rows finalised, graduation bookkeeping.
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
-  compact_done_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
   finalise_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
   commit_kernel<<<1, 32, 0, st>>>(a);
-  c->launches += 3;
+  c->launches += 2;
 }
 
 // ------------------------------------------------------------------------------------------------ drain helpers

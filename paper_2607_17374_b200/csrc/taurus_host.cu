@@ -73,7 +73,12 @@ extern "C" void taurus_destroy(taurus_ctx* c) {
   cudaFree(c->d_touched_list); cudaFree(c->d_need_list); cudaFree(c->d_slot_epoch); cudaFree(c->d_slot_touch); cudaFree(c->d_slot_pend); cudaFree(c->d_victims); cudaFree(c->d_keys);
   cudaFree(c->d_cand[0]); cudaFree(c->d_cand[1]); cudaFree(c->d_ext_free); cudaFree(c->d_ext_live); cudaFree(c->d_bk_tail_ext);
   cudaFree(c->d_bk_tail_fill); cudaFree(c->d_bk_new); cudaFree(c->d_bk_off); cudaFree(c->d_bk_base); cudaFree(c->d_new_ext);
-  cudaFree(c->d_vic_place); cudaFree(c->d_csc_src);
+  cudaFree(c->d_vic_place); cudaFree(c->d_csc_src); cudaFree(c->d_ext_ret[0]); cudaFree(c->d_ext_ret[1]); cudaFree(c->d_xfer_list);
+  cudaFree(c->d_stage_out);
+  if (c->moves_ready) cudaEventDestroy(c->moves_ready);
+  if (c->xfer_done) cudaEventDestroy(c->xfer_done);
+  if (c->xfer_stream) cudaStreamDestroy(c->xfer_stream);
+  delete c->pend_chunk;
   if (c->h_store) cudaFreeHost(c->h_store);
   cudaFree(c->d_grad_ids); cudaFree(c->d_grad_rows); cudaFree(c->d_done_list); cudaFree(c->d_X[0]); cudaFree(c->d_X[1]); cudaFree(c->d_PT);
   cudaFree(c->d_af_A); cudaFree(c->d_af_O); cudaFree(c->d_af_X);
@@ -260,12 +265,20 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     c->ext_shift = 3;
     while (c->ext_shift < 10 && (2ll << c->ext_shift) <= per) c->ext_shift += 1;
     const long long ext_rows = 1ll << c->ext_shift;
-    c->n_ext = (c->host_rows + ext_rows - 1) / ext_rows + 2 * c->n_buckets + 8;
+    // ... and the extents emptied by one chunk's reloads wait for two chunks before they return to the free stack
+    c->n_ext = (c->host_rows + ext_rows - 1) / ext_rows + 2 * c->n_buckets + 8 + 2 * ((c->victim_capacity >> c->ext_shift) + 1);
     if (c->n_ext * ext_rows >= (1ll << 31) - 2) return TAURUS_ERR_INVALID_ARG;
     ALLOC(c->d_ext_free, c->n_ext); ALLOC(c->d_ext_live, c->n_ext);
     ALLOC(c->d_bk_tail_ext, c->n_buckets); ALLOC(c->d_bk_tail_fill, c->n_buckets); ALLOC(c->d_bk_new, c->n_buckets);
     ALLOC(c->d_bk_off, c->n_buckets); ALLOC(c->d_bk_base, c->n_buckets);
     ALLOC(c->d_new_ext, (c->victim_capacity >> c->ext_shift) + c->n_buckets + 1);
+    ALLOC(c->d_ext_ret[0], c->n_ext); ALLOC(c->d_ext_ret[1], c->n_ext);
+    ALLOC(c->d_xfer_list, c->pool_slots);   // one entry per need-list entry
+    ALLOC(c->d_stage_out, (size_t)c->victim_capacity * c->Hmax);
+    CU(cudaStreamCreateWithFlags(&c->xfer_stream, cudaStreamNonBlocking));
+    CU(cudaEventCreateWithFlags(&c->moves_ready, cudaEventDisableTiming));
+    CU(cudaEventCreateWithFlags(&c->xfer_done, cudaEventDisableTiming));
+    c->pipelined = true;
     cudaError_t e = cudaHostAlloc((void**)&c->h_store, (size_t)c->n_ext * ext_rows * c->Hmax * sizeof(float), cudaHostAllocMapped);
     if (e != cudaSuccess) { cuda_ok(e, "cudaHostAlloc(evicted-row store)"); c->h_store = nullptr; return TAURUS_ERR_NOMEM; }
     CU(cudaHostGetDevicePointer((void**)&c->d_store_alias, c->h_store, 0));
@@ -361,6 +374,8 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
   if (r->pool_slots + r->hub_count >= (1ll << 31)) return TAURUS_ERR_INVALID_ARG;
   taurus_ctx* c = new (std::nothrow) taurus_ctx();
   if (!c) return TAURUS_ERR_NOMEM;
+  c->pend_chunk = new (std::nothrow) PendingChunk();
+  if (!c->pend_chunk) { delete c; return TAURUS_ERR_NOMEM; }
   int rc;
   try { rc = init_impl(c, g, m, r); } catch (const std::bad_alloc&) { rc = TAURUS_ERR_NOMEM; }
   if (rc != TAURUS_OK) { taurus_destroy(c); return rc; }
@@ -369,7 +384,9 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
 }
 
 // Reads the device control block (after synchronising `st`) and returns its sticky error.
+static int finish_chunk(taurus_ctx* c, cudaStream_t st);
 static int read_ctl(taurus_ctx* c, cudaStream_t st) {
+  { int rc = finish_chunk(c, st); if (rc) return rc; }   // the last chunk's finalise may still be waiting for a successor
   CU(cudaStreamSynchronize(st));
   CU(cudaStreamSynchronize(c->out_stream));
   CU(cudaMemcpy(c->h_ctl, c->d_ctl, sizeof(DevCtl), cudaMemcpyDeviceToHost));
@@ -383,6 +400,8 @@ extern "C" int taurus_layer_begin(taurus_ctx* c, int32_t layer, void* cuda_strea
   if (c->last_stream != st) CU(cudaStreamSynchronize(c->last_stream));
   CU(cudaStreamSynchronize(c->copy_stream));
   CU(cudaStreamSynchronize(c->out_stream));
+  if (c->xfer_stream) CU(cudaStreamSynchronize(c->xfer_stream));
+  c->pending = false;   // an abandoned layer's last chunk is dropped with it
   c->layer = layer;
   c->dense_out = nullptr; c->dense_ld = 0;
   c->run_out = nullptr; c->run_pending_half = -1;
@@ -443,13 +462,14 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.ext_free = c->d_ext_free; a.ext_live = c->d_ext_live; a.bk_tail_ext = c->d_bk_tail_ext; a.bk_tail_fill = c->d_bk_tail_fill;
   a.bk_new = c->d_bk_new; a.bk_off = c->d_bk_off; a.bk_base = c->d_bk_base; a.new_ext = c->d_new_ext; a.vic_place = c->d_vic_place;
   a.csc_ptr = c->d_csc_ptr; a.csc_src = c->d_csc_src; a.csc_eid = c->d_csc_eid;
+  a.ext_ret[0] = c->d_ext_ret[0]; a.ext_ret[1] = c->d_ext_ret[1]; a.xfer_list = c->d_xfer_list; a.stage_out = c->d_stage_out;
   a.chunk_sources = c->chunk_sources; a.n_ext = c->n_ext; a.n_buckets = c->n_buckets; a.ext_shift = c->ext_shift;
   a.grad_ids = c->d_grad_ids; a.grad_rows = c->d_grad_rows; a.done_list = c->d_done_list;
   a.Hp = taurus_round_up(c->dims[l + 1], 4);
   a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;   // GAT pass 3 scatters h' rows repacked to pitch Hp
   a.att_s = c->d_att_s; a.att_tm = c->d_att_tm; a.att_z = c->d_att_z; a.leaky = c->leaky;
   a.bias = c->d_bias[l];
-  a.ctl = c->d_ctl; a.chunk_log = c->d_chunk_log; a.log_capacity = c->log_capacity;
+  a.ctl = c->d_ctl; a.pc = &c->d_ctl->pc[c->chunk_seq & 1]; a.chunk_log = c->d_chunk_log; a.log_capacity = c->log_capacity;
   a.V = c->V; a.pool_slots = c->pool_slots; a.hub_count = c->hub_count; a.host_rows = c->host_rows; a.drain_rows = c->drain_rows;
   a.src_begin = s; a.src_end = e;
   a.epoch = (int32_t)(c->chunk_seq + 1);
@@ -478,6 +498,51 @@ static int finish_run_append(taurus_ctx* c) {
   CU(cudaEventRecord(c->out_done[h], c->out_stream));
   c->half_used[h] = true;
   return TAURUS_OK;
+}
+
+static int finish_chunk(taurus_ctx* c, cudaStream_t st) {
+  if (!c->pending) return TAURUS_OK;
+  c->pending = false;
+  const PendingChunk& p = *c->pend_chunk;
+  const ChunkArgs& a = p.a;
+  const int l = p.layer;
+  cudaEvent_t* pev = p.timed_index >= 0 ? &c->phase_ev[(size_t)p.timed_index * TAURUS_PUSH_EVENTS] : nullptr;
+  if (c->pipelined) CU(cudaStreamWaitEvent(st, c->xfer_done, 0));   // reloaded partial sums have been added to the chunk's rows
+  if (pev) cudaEventRecord(pev[8], st);
+  if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
+  if (p.af) {
+    int rc = launch_af_finalise(c, a, l, std::min<long long>(p.bound, a.grad_cap), st);
+    if (rc) { c->h_ctl->error = rc; return rc; }   // the chunk is half applied: the layer has to be begun again
+  } else {
+    launch_finalise(c, a, st);
+  }
+  int run_rc = TAURUS_OK;
+  if (a.dense_half >= 0 && c->dense_out) {   // hand this chunk's rows to the output stream (matrix in pinned host memory)
+    const int h = a.dense_half, d_out = c->dims[l + 1];
+    CU(cudaEventRecord(c->fin_done[h], st));
+    CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
+    launch_place_half(c, h, d_out, a.Hout, c->out_stream);
+    CU(cudaEventRecord(c->out_done[h], c->out_stream));
+    c->half_used[h] = true;
+  } else if (a.dense_half >= 0) {
+    // Run-output mode.  The previous chunk's rows are already grouped by id range and its per-range counts are
+    // on their way to the host: now that this chunk's kernels are queued behind it, wait for them (the device
+    // stays busy), move those rows into the partition buffers and flush the full ones; then group this chunk's
+    // rows once its finalise has run.
+    const int h = a.dense_half;
+    CU(cudaEventRecord(c->fin_done[h], st));
+    run_rc = finish_run_append(c);
+    if (!run_rc) {
+      CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
+      const long long off = a.grad_off;
+      run_rc = runs_phase1(c->run_out, c->d_grad_ids + off, c->d_grad_rows + (size_t)off * a.Hout, a.Hout, std::min(p.bound, a.grad_cap),
+                           &c->d_ctl->out_count[h], 0, c->out_stream);
+      if (!run_rc) c->run_pending_half = h;
+    }
+  }
+  if (pev) cudaEventRecord(pev[9], st);
+  CU(cudaGetLastError());
+  return run_rc;
 }
 
 // S1: features of sources [s, e) ([n x K], rows contiguous) to the device.  Host chunks are copied on the library's
@@ -540,9 +605,9 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   const int n = (int)(src_end - src_begin);
   cudaEvent_t* pev = nullptr;
   if (c->timing && c->timed_pushes < TAURUS_MAX_TIMED_PUSHES) {
-    const size_t need = (size_t)(c->timed_pushes + 1) * 7;
+    const size_t need = (size_t)(c->timed_pushes + 1) * TAURUS_PUSH_EVENTS;
     while (c->phase_ev.size() < need) { cudaEvent_t e; CU(cudaEventCreate(&e)); c->phase_ev.push_back(e); }
-    pev = &c->phase_ev[(size_t)c->timed_pushes * 7];
+    pev = &c->phase_ev[(size_t)c->timed_pushes * TAURUS_PUSH_EVENTS];
     c->timed_pushes += 1;
   }
   const bool timing = pev != nullptr;
@@ -597,44 +662,34 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
                        src_end == std::min<long long>(c->V, src_begin + c->chunk_sources);
   if (grouped) launch_classify_grouped(c, a, st); else launch_classify(c, a, st);
   launch_make_room(c, a, st, timing ? pev[3] : nullptr);   // pev[3]: victims chosen and placed, rows not yet moved
+  // The chunk before this one: its rows have been crossing the host link since its slots were handed out.  Its
+  // finalise runs now, before this chunk takes over the slots it released.
+  int run_rc = finish_chunk(c, st);
   if (timing) cudaEventRecord(pev[4], st);
+  launch_alloc(c, a, st);
+  if (timing) cudaEventRecord(pev[5], st);
+  if (c->pipelined) {
+    CU(cudaEventRecord(c->moves_ready, st));
+    CU(cudaStreamWaitEvent(c->xfer_stream, c->moves_ready, 0));
+    if (timing) cudaEventRecord(pev[10], c->xfer_stream);
+    launch_transfer(c, a, c->xfer_stream);
+    if (timing) cudaEventRecord(pev[11], c->xfer_stream);
+    CU(cudaEventRecord(c->xfer_done, c->xfer_stream));
+  } else if (timing) {
+    cudaEventRecord(pev[10], st);
+    cudaEventRecord(pev[11], st);
+  }
   // S5, S5', S6
   if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
   if (xbuf >= 0 && x_in_use) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }   // the scatter read the staged rows in place
-  if (timing) cudaEventRecord(pev[5], st);
-  // S7
-  if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
-  if (af) {
-    int rc = launch_af_finalise(c, a, l, std::min<long long>(bound, a.grad_cap), st);
-    if (rc) { c->h_ctl->error = rc; return rc; }   // the chunk is half applied: the layer has to be begun again
-  } else {
-    launch_finalise(c, a, st);
-  }
-  int run_rc = TAURUS_OK;
-  if (a.dense_half >= 0 && c->dense_out) {   // hand this chunk's rows to the output stream (matrix in pinned host memory)
-    const int h = a.dense_half, d_out = c->dims[l + 1];
-    CU(cudaEventRecord(c->fin_done[h], st));
-    CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
-    launch_place_half(c, h, d_out, a.Hout, c->out_stream);
-    CU(cudaEventRecord(c->out_done[h], c->out_stream));
-    c->half_used[h] = true;
-  } else if (a.dense_half >= 0) {
-    // Run-output mode.  The previous chunk's rows are already grouped by id range and its per-range counts are
-    // on their way to the host: now that this chunk's kernels are queued behind it, wait for them (the device
-    // stays busy), move those rows into the partition buffers and flush the full ones; then group this chunk's
-    // rows once its finalise has run.
-    const int h = a.dense_half;
-    CU(cudaEventRecord(c->fin_done[h], st));
-    run_rc = finish_run_append(c);
-    if (!run_rc) {
-      CU(cudaStreamWaitEvent(c->out_stream, c->fin_done[h], 0));
-      const long long off = a.grad_off;
-      run_rc = runs_phase1(c->run_out, c->d_grad_ids + off, c->d_grad_rows + (size_t)off * a.Hout, a.Hout, std::min(bound, a.grad_cap),
-                           &c->d_ctl->out_count[h], 0, c->out_stream);
-      if (!run_rc) c->run_pending_half = h;
-    }
-  }
   if (timing) cudaEventRecord(pev[6], st);
+  launch_compact_done(c, a, st);
+  if (timing) cudaEventRecord(pev[7], st);
+  // S7: deferred behind the next chunk's select when rows cross the host link, else at once
+  c->pend_chunk->a = a; c->pend_chunk->layer = l; c->pend_chunk->af = af; c->pend_chunk->bound = bound;
+  c->pend_chunk->timed_index = timing ? c->timed_pushes - 1 : -1;
+  c->pending = true;
+  if (!c->pipelined) { int rc = finish_chunk(c, st); if (!run_rc) run_rc = rc; }
   CU(cudaGetLastError());
   c->next_src = src_end;
   c->chunk_seq += 1;
@@ -838,6 +893,7 @@ extern "C" int taurus_layer_end(taurus_ctx* c, taurus_stats* stats) {
   if (!c) return TAURUS_ERR_INVALID_ARG;
   if (c->layer < 0) return TAURUS_ERR_ORDER;
   CU(cudaSetDevice(c->device));
+  { int rc = finish_chunk(c, c->last_stream); if (rc) return rc; }
   if (c->run_out) {   // last chunk's rows, then every partition buffer leaves as a run
     int rc = finish_run_append(c);
     if (!rc) rc = runs_flush_all(c->run_out, c->out_stream);
@@ -865,6 +921,7 @@ extern "C" int taurus_get_chunk_log(taurus_ctx* c, int64_t* out, int64_t capacit
 extern "C" int taurus_get_vertex_array(taurus_ctx* c, int32_t which, void* out_host) {
   if (!c || !out_host || which < 0 || which > 3) return TAURUS_ERR_INVALID_ARG;
   CU(cudaSetDevice(c->device));
+  { int rc = finish_chunk(c, c->last_stream); if (rc) return rc; }
   CU(cudaStreamSynchronize(c->last_stream));
   const void* src = which == 0 ? (const void*)c->d_state : which == 1 ? (const void*)c->d_pend
                     : which == 2 ? (const void*)c->d_reload : (const void*)c->d_hub;
@@ -934,11 +991,15 @@ extern "C" int taurus_set_timing(taurus_ctx* c, int32_t on) {
 extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out, int64_t capacity_pushes, int64_t* out_pushes) {
   if (!c || !out || !out_pushes || capacity_pushes < 0) return TAURUS_ERR_INVALID_ARG;
   CU(cudaSetDevice(c->device));
+  { int rc = finish_chunk(c, c->last_stream); if (rc) return rc; }
   CU(cudaStreamSynchronize(c->last_stream));
+  if (c->xfer_stream) CU(cudaStreamSynchronize(c->xfer_stream));
   long long n = std::min<long long>(c->timed_pushes, capacity_pushes);
+  static const int from[TAURUS_PHASES] = {0, 1, 2, 3, 4, 5, 6, 8, 10};
   for (long long p = 0; p < n; ++p)
-    for (int i = 0; i < 6; ++i)
-      CU(cudaEventElapsedTime(&out[p * 6 + i], c->phase_ev[(size_t)p * 7 + i], c->phase_ev[(size_t)p * 7 + i + 1]));
+    for (int i = 0; i < TAURUS_PHASES; ++i)
+      CU(cudaEventElapsedTime(&out[p * TAURUS_PHASES + i], c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + from[i]],
+                              c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + from[i] + 1]));
   *out_pushes = n;
   return TAURUS_OK;
 }

@@ -13,27 +13,24 @@
 #define TAURUS_MAX_DIM 1024
 #define TAURUS_MAX_FANOUT 64
 #define TAURUS_MAX_TIMED_PUSHES 16384
+#define TAURUS_PUSH_EVENTS 12                   // CUDA events per timed push
+#define TAURUS_PHASES 9                         // durations reported per timed push
 #define TAURUS_SEL_BITS 11                      // radix-select digit width
 #define TAURUS_SEL_BINS (1 << TAURUS_SEL_BITS)
 #define TAURUS_SEL_LEVELS 6                     // 6 x 11 = 66 bits >= the 62-bit (score, id) key
 
-// Device-resident control block: counters the kernels of one chunk hand to one another, so that
-// no step of a push needs the host.  One per context.
-struct DevCtl {
-  int32_t error;          // sticky TAURUS_ERR_* found on the device
-  int32_t need_count;     // touched vertices that need a slot (NOT_STARTED or EVICTED), this chunk
-  int32_t done_count;     // vertices whose pending count reached zero, this chunk
-  int32_t touched_count;  // vertices touched by this chunk (first touches), this chunk
-  int32_t deficit;        // slots to free by eviction, this chunk
-  int32_t victim_count;   // victims listed so far, this chunk
+// Counters of ONE chunk that its kernels hand to one another.  Two of them alternate (chunk sequence number & 1): with a
+// bounded pool the finalise step of chunk k runs after the classify / select steps of chunk k + 1 (while chunk k's rows
+// are still crossing the host link), so the two chunks' counters are alive together.
+struct ChunkCtl {
+  int32_t need_count;     // touched vertices that need a slot (NOT_STARTED or EVICTED)
+  int32_t done_count;     // vertices whose pending count reached zero
+  int32_t touched_count;  // vertices touched by this chunk (first touches)
+  int32_t deficit;        // slots to free by eviction
+  int32_t victim_count;   // victims listed so far
   int32_t hs, ns, ev, gs; // touched vertices by state at chunk start
-  int32_t reloaded;       // reloads this chunk
-  long long free_top;       // entries on the free-slot stack
-  long long ext_free_top;   // entries on the free-extent stack of the host store
-  long long host_live;      // rows currently held by the host store
-  long long grad_count;     // rows waiting in the graduation buffer
-  long long out_count[2];   // dense-output mode: rows finalise left in each half of the graduation buffer
-  long long alloc_base;       // this chunk: need-list entry i takes free_stack[alloc_base - 1 - i]
+  int32_t reloaded;       // reloads
+  long long alloc_base;   // need-list entry i takes free_stack[alloc_base - 1 - i]
   // Victim select, level by level (level 0 scans the pool, deeper levels the candidates the level above left):
   long long sel_k[TAURUS_SEL_LEVELS + 1];               // rank still to resolve among the keys entering the level
   unsigned long long sel_min[TAURUS_SEL_LEVELS + 1];    // smallest / largest key entering the level: the digit of a level
@@ -41,10 +38,23 @@ struct DevCtl {
   int32_t sel_count[TAURUS_SEL_LEVELS + 1];             // keys entering the level
   int32_t sel_final_level;                              // level that listed the last victims; kernels of deeper levels return
   unsigned int hist[2][TAURUS_SEL_BINS];                // digit histogram, alternating between levels
+};
+
+// Device-resident control block: counters the kernels hand to one another, so that no step of a push needs
+// the host.  One per context.
+struct DevCtl {
+  int32_t error;            // sticky TAURUS_ERR_* found on the device
+  int32_t ext_ret_count[2]; // extents emptied by the row transfers of the chunks of each parity, waiting to go back on the free stack
+  long long free_top;       // entries on the free-slot stack
+  long long ext_free_top;   // entries on the free-extent stack of the host store
+  long long host_live;      // rows currently held by the host store
+  long long grad_count;     // rows waiting in the graduation buffer
+  long long out_count[2];   // dense-output mode: rows finalise left in each half of the graduation buffer
   // layer totals
   long long evictions, reloads, peak_occupancy, hub_messages, total_messages, completed;
   long long sum_hs, sum_ns, sum_ev, sum_gs, chunks;
   long long scatter_groups; // accumulator-row reductions issued by the scatter (self messages not counted)
+  ChunkCtl pc[2];
 };
 
 // Everything the per-chunk kernels need, passed by value.
@@ -91,6 +101,10 @@ struct ChunkArgs {
   int2* bk_base;            // [buckets] this chunk: (tail extent, tail fill) before the chunk's victims
   int32_t* new_ext;         // [victim_capacity >> ext_shift + buckets] this chunk: extents taken from the stack
   int2* vic_place;          // [victim_capacity] this chunk: (bucket, rank among the chunk's victims of that bucket)
+  int32_t* ext_ret[2];      // [n_ext] each: extents emptied by the transfers of the chunks of each parity
+  // Row transfers of the chunk: entry i = (slot, host row to add into it or -1, host row that takes stage_out[i] or -1)
+  int4* xfer_list;          // [need capacity]
+  float* stage_out;         // [victim_capacity x Hp] victims' rows on their way to the host store
   const long long* csc_ptr; // [V + 1] in-lists (ascending source id): offsets,
   const int32_t* csc_src;   // [E]       sources,
   const uint32_t* csc_eid;  // [E]       CSR edge indices (sampled layers: the mask is looked up through them), else NULL
@@ -106,6 +120,7 @@ struct ChunkArgs {
   int32_t ldpt;
   const float* bias;        // [Hp]
   DevCtl* ctl;
+  ChunkCtl* pc;             // this chunk's counters: &ctl->pc[chunk sequence number & 1]
   long long* chunk_log;     // [log_capacity x TAURUS_CK_COLUMNS]
   long long log_capacity;
   long long V, pool_slots, hub_count, host_rows, drain_rows;
@@ -133,6 +148,17 @@ struct ChunkArgs {
   int32_t Hout;             // padded output width (= Hp for project-first layers)
   int32_t self_rows;        // 1: the scatter adds a self row; 0: it only counts the self message (the self term is added after the transform)
   int32_t self_bias;        // 1: the self row carries the bias (project-first); 0: the bias is added after the transform
+};
+
+// What is still to be enqueued for the chunk pushed last: S7 (finalise) and the hand-off of its rows.  With a bounded
+// pool this waits until the next chunk has chosen its victims, so that the chunk's rows cross the host link in the
+// meantime (Sect. 3.6 runs graduation beside aggregation in the same way); otherwise it follows the push at once.
+struct PendingChunk {
+  ChunkArgs a;
+  int layer = 0;
+  bool af = false;
+  long long bound = 0;
+  long long timed_index = -1;   // index of the push among the timed ones (its events live in a vector that may grow), -1 = not timed
 };
 
 struct taurus_ctx {
@@ -206,6 +232,14 @@ struct taurus_ctx {
   int2* d_bk_base = nullptr;
   int32_t* d_new_ext = nullptr;
   int2* d_vic_place = nullptr;
+  int32_t* d_ext_ret[2] = {nullptr, nullptr};
+  int4* d_xfer_list = nullptr;
+  float* d_stage_out = nullptr;
+  cudaStream_t xfer_stream = nullptr;   // rows cross the host link here while the compute stream goes on
+  cudaEvent_t moves_ready = nullptr, xfer_done = nullptr;
+  bool pipelined = false;               // bounded pool with a host store: finalise of chunk k is deferred behind chunk k + 1's select
+  bool pending = false;                 // a chunk's finalise (and what follows it) is still to be enqueued
+  struct PendingChunk* pend_chunk = nullptr;
   int32_t* d_csc_src = nullptr;   // in-list sources, built when rows can be evicted
   long long n_ext = 0, n_buckets = 0;
   int ext_shift = 0;
@@ -252,7 +286,7 @@ struct taurus_ctx {
   cudaEvent_t order_event = nullptr;
   long long launches = 0;
   int timing = 0;
-  std::vector<cudaEvent_t> phase_ev;   // 7 events per timed push, created on demand
+  std::vector<cudaEvent_t> phase_ev;   // TAURUS_PUSH_EVENTS events per timed push, created on demand
   long long timed_pushes = 0;          // pushes recorded since timing was switched on
   std::vector<std::vector<long long>> rank_cum_cache;   // per layer: rank_cum computed at the first layer_begin
   int sm_count = 148;
@@ -265,9 +299,11 @@ static inline int taurus_proj_width(int mode, int Hp) { return mode == TAURUS_SA
 // ---- kernels_state.cu
 void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st);
 void launch_classify(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
-void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEvent_t before_moves = nullptr);   // plan, select, placement, [event], row moves
-void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // compact + finalise + commit
-void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
+void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEvent_t before_moves = nullptr);   // plan, select, placement, [event]
+void launch_alloc(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);       // slots handed out, victims' rows staged, new rows cleared
+void launch_transfer(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // staged rows to the host store, reloaded rows added into their slots
+void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // finalise + commit (after launch_compact_done)
+void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);   // completions listed, chunk record written
 void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st);
 void launch_place_half(taurus_ctx* c, int half, int d_out, int Hp, cudaStream_t st);   // dense-output mode
@@ -318,8 +354,8 @@ struct GemmFinish {
   int act;
 };
 int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const float* X, int ldx, int K, int n, float* out, long long ld_out,
-                         cudaStream_t st, const GemmFinish* finish = nullptr, bool rows_from_done_count = false);
-// rows_from_done_count: n is only the host's bound; the kernel works on the first ctl->done_count rows (read on the
+                         cudaStream_t st, const GemmFinish* finish = nullptr, const int32_t* done_count = nullptr);
+// done_count (device pointer): n is only the host's bound; the kernel works on the first *done_count rows (read on the
 // device at launch) and leaves the others untouched.
 int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat, int K, int N);   // image of cat [K x N] into *slot
 void free_tc_weights(taurus_ctx* c);

@@ -142,9 +142,10 @@ def test_full_config(name):
         dt = time.time() - t1
         ph = ctx.get_phase_ms().sum(axis=0)
         ctx.set_timing(False)
-        print("%s layer %d: device time %.0f ms (copy-in %.0f, projection %.0f, classify + select %.0f, row moves %.0f, scatter %.0f, "
-              "finalise %.0f) = %.2f G messages/s on the device" % (name, l, ph.sum(), ph[0], ph[1], ph[2], ph[3], ph[4], ph[5],
-                                                    st["total_messages"] / max(ph.sum(), 1e-9) / 1e6), flush=True)
+        print("%s layer %d: device time %.0f ms on the compute stream (copy-in %.0f, projection %.0f, classify + select %.0f, wait for "
+              "transfers + previous finalise %.0f, slot hand-out %.0f, scatter %.0f, completion list %.0f, finalise %.0f; row transfers on "
+              "their own stream %.0f) = %.2f G messages/s on the device" % (name, l, ph[:7].sum(), ph[0], ph[1], ph[2], ph[3], ph[4], ph[5], ph[6], ph[7], ph[8],
+                                                    st["total_messages"] / max(ph[:7].sum(), 1e-9) / 1e6), flush=True)
         print("%s layer %d: %.1f s, %.3f G messages/s incl. host feature generation; evictions %d reloads %d peak occupancy %d "
               "max reloads of one vertex %d hub messages %.1f %%" %
               (name, l, dt, st["total_messages"] / dt / 1e9, st["evictions"], st["reloads"], st["peak_occupancy"],
