@@ -882,12 +882,8 @@ __global__ void finalise_kernel(ChunkArgs a) {
   }
 }
 
-// One thread, after the chunk's completions are listed: fold the chunk's counters into the layer totals, write the chunk
-// record.
-__global__ void commit_counts_kernel(ChunkArgs a) {
-  DevCtl* ctl = a.ctl;
-  ChunkCtl* pc = a.pc;
-  if (threadIdx.x != 0 || ctl->error) return;
+// After the chunk's completions are listed: fold the chunk's counters into the layer totals, write the chunk record.
+static __device__ void commit_counts(const ChunkArgs& a, DevCtl* ctl, ChunkCtl* pc) {   // one thread
   long long c = ctl->chunks;
   if (c < a.log_capacity) {
     long long* r = a.chunk_log + c * TAURUS_CK_COLUMNS;
@@ -901,12 +897,18 @@ __global__ void commit_counts_kernel(ChunkArgs a) {
   ctl->completed += pc->done_count;
   ctl->chunks = c + 1;
 }
+__global__ void commit_counts_kernel(ChunkArgs a) {
+  if (threadIdx.x != 0 || a.ctl->error) return;
+  commit_counts(a, a.ctl, a.pc);
+}
 // One thread, after the chunk's rows are finalised: the graduation buffer's row count, and the chunk's counters are
-// cleared for the chunk after next.
-__global__ void commit_kernel(ChunkArgs a) {
+// cleared for the chunk after next.  with_counts: the chunk record has not been written yet (no transfers in flight:
+// finalise followed the completion list directly).
+__global__ void commit_kernel(ChunkArgs a, int with_counts) {
   DevCtl* ctl = a.ctl;
   ChunkCtl* pc = a.pc;
   if (threadIdx.x != 0 || ctl->error) return;
+  if (with_counts) commit_counts(a, ctl, pc);
   if (a.dense_direct) { /* rows already sit in the caller's matrix */ }
   else if (a.dense_half >= 0) ctl->out_count[a.dense_half] = pc->done_count;
   else ctl->grad_count += pc->done_count;
@@ -915,20 +917,20 @@ __global__ void commit_kernel(ChunkArgs a) {
 }
 
 // S6: completions listed, slots released, chunk record written.
-void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
+void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, bool write_record) {
   compact_done_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
-  commit_counts_kernel<<<1, 32, 0, st>>>(a);
-  c->launches += 2;
+  if (write_record) commit_counts_kernel<<<1, 32, 0, st>>>(a);
+  c->launches += write_record ? 2 : 1;
 }
 void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
-  commit_kernel<<<1, 32, 0, st>>>(a);
+  commit_kernel<<<1, 32, 0, st>>>(a, c->pipelined ? 0 : 1);
   c->launches += 1;
 }
 
 // S7 of a project-first layer (after launch_compact_done): rows finalised, graduation bookkeeping.
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   finalise_kernel<<<c->sm_count * 8, 256, 0, st>>>(a);
-  commit_kernel<<<1, 32, 0, st>>>(a);
+  commit_kernel<<<1, 32, 0, st>>>(a, c->pipelined ? 0 : 1);
   c->launches += 2;
 }
 

@@ -507,8 +507,10 @@ static int finish_chunk(taurus_ctx* c, cudaStream_t st) {
   const ChunkArgs& a = p.a;
   const int l = p.layer;
   cudaEvent_t* pev = p.timed_index >= 0 ? &c->phase_ev[(size_t)p.timed_index * TAURUS_PUSH_EVENTS] : nullptr;
-  if (c->pipelined) CU(cudaStreamWaitEvent(st, c->xfer_done, 0));   // reloaded partial sums have been added to the chunk's rows
-  if (pev) cudaEventRecord(pev[8], st);
+  if (c->pipelined) {
+    CU(cudaStreamWaitEvent(st, c->xfer_done, 0));   // reloaded partial sums have been added to the chunk's rows
+    if (pev) cudaEventRecord(pev[8], st);           // (without transfers the finalise follows event 7 directly)
+  }
   if (a.dense_half >= 0 && c->half_used[a.dense_half]) CU(cudaStreamWaitEvent(st, c->out_done[a.dense_half], 0));
   if (p.af) {
     int rc = launch_af_finalise(c, a, l, std::min<long long>(p.bound, a.grad_cap), st);
@@ -665,7 +667,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   // The chunk before this one: its rows have been crossing the host link since its slots were handed out.  Its
   // finalise runs now, before this chunk takes over the slots it released.
   int run_rc = finish_chunk(c, st);
-  if (timing) cudaEventRecord(pev[4], st);
+  if (timing && c->pipelined) cudaEventRecord(pev[4], st);
   launch_alloc(c, a, st);
   if (timing) cudaEventRecord(pev[5], st);
   if (c->pipelined) {
@@ -675,15 +677,12 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
     launch_transfer(c, a, c->xfer_stream);
     if (timing) cudaEventRecord(pev[11], c->xfer_stream);
     CU(cudaEventRecord(c->xfer_done, c->xfer_stream));
-  } else if (timing) {
-    cudaEventRecord(pev[10], st);
-    cudaEventRecord(pev[11], st);
   }
   // S5, S5', S6
   if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
   if (xbuf >= 0 && x_in_use) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }   // the scatter read the staged rows in place
   if (timing) cudaEventRecord(pev[6], st);
-  launch_compact_done(c, a, st);
+  launch_compact_done(c, a, st, c->pipelined);   // with transfers in flight the chunk record is written now, else by the commit after finalise
   if (timing) cudaEventRecord(pev[7], st);
   // S7: deferred behind the next chunk's select when rows cross the host link, else at once
   c->pend_chunk->a = a; c->pend_chunk->layer = l; c->pend_chunk->af = af; c->pend_chunk->bound = bound;
@@ -995,11 +994,19 @@ extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out, int64_t capacity_p
   CU(cudaStreamSynchronize(c->last_stream));
   if (c->xfer_stream) CU(cudaStreamSynchronize(c->xfer_stream));
   long long n = std::min<long long>(c->timed_pushes, capacity_pushes);
-  static const int from[TAURUS_PHASES] = {0, 1, 2, 3, 4, 5, 6, 8, 10};
+  // event pairs of the nine durations; without row transfers events 4, 8, 10 and 11 are not recorded: no wait, the
+  // slot hand-out runs from event 3, the finalise from event 7
+  static const int from_x[TAURUS_PHASES] = {0, 1, 2, 3, 4, 5, 6, 8, 10}, to_x[TAURUS_PHASES] = {1, 2, 3, 4, 5, 6, 7, 9, 11};
+  static const int from_d[TAURUS_PHASES] = {0, 1, 2, -1, 3, 5, 6, 7, -1}, to_d[TAURUS_PHASES] = {1, 2, 3, -1, 5, 6, 7, 9, -1};
+  const int* from = c->pipelined ? from_x : from_d;
+  const int* to = c->pipelined ? to_x : to_d;
   for (long long p = 0; p < n; ++p)
-    for (int i = 0; i < TAURUS_PHASES; ++i)
-      CU(cudaEventElapsedTime(&out[p * TAURUS_PHASES + i], c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + from[i]],
-                              c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + from[i] + 1]));
+    for (int i = 0; i < TAURUS_PHASES; ++i) {
+      out[p * TAURUS_PHASES + i] = 0.f;
+      if (from[i] >= 0)
+        CU(cudaEventElapsedTime(&out[p * TAURUS_PHASES + i], c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + from[i]],
+                                c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + to[i]]));
+    }
   *out_pushes = n;
   return TAURUS_OK;
 }

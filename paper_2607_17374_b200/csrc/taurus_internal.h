@@ -303,7 +303,7 @@ void launch_make_room(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, cudaEv
 void launch_alloc(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);       // slots handed out, victims' rows staged, new rows cleared
 void launch_transfer(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // staged rows to the host store, reloaded rows added into their slots
 void launch_finalise(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);    // finalise + commit (after launch_compact_done)
-void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);   // completions listed, chunk record written
+void launch_compact_done(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st, bool write_record);   // completions listed (and the chunk record written)
 void launch_commit(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st);
 void launch_place_rows(taurus_ctx* c, float* dense, long long ld, int d_out, int Hp, long long count, cudaStream_t st);
 void launch_place_half(taurus_ctx* c, int half, int d_out, int Hp, cudaStream_t st);   // dense-output mode
