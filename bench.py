@@ -45,11 +45,7 @@ METRIC = "edges/sec per GNN layer (GTEPS)"
 # the digest below (sha256 of csrc/kernels_group.cu, first 16 hex digits); when the source has changed since the
 # capture the bench prints traffic = null instead of a stale number.
 SCATTER_TRAFFIC_PER_GROUP_BYTES = 2720.0
-SCATTER_CAPTURE_SOURCE = "0000000000000000"
-# PCIe bytes (both directions) per row moved by alloc_kernel, from profiles/alloc_kernel_large_1500k.md, same rule
-# (sha256 of csrc/kernels_state.cu).
-ALLOC_CAPTURE_SOURCE = "0000000000000000"
-ALLOC_PCIE_BYTES_PER_ROW_BYTE = None
+SCATTER_CAPTURE_SOURCE = "19efb17de4f02d04"
 
 
 def source_digest(name: str) -> str:
@@ -472,7 +468,7 @@ def run_windowed(args, env, w):
     sc_bytes = scatter_bytes(groups, msgs, n_src, acc_width, not (agg_first and w.mode == tg.SAGE_MEAN))
     sc_s = phase[5] * 1e-3
     moves_share = phase[8] / ms
-    # the dominant kernel: the row moves between the pool and pinned host memory (alloc_kernel), bound by the host link
+    # the dominant kernel: the row transfers between the pool and pinned host memory, bound by the host link
     roofline = dict(bound="pcie", kernel="transfer_kernel (evicted rows out, reloaded rows in, %d-byte rows)" % row_bytes,
                     achieved=(out_gbs + in_gbs) / 2, peak=link["both_per_direction_gbs"], unit="GB/s per direction",
                     frac=(out_gbs + in_gbs) / 2 / link["both_per_direction_gbs"], peak_source="measured in this run: " + link["how"],
@@ -484,7 +480,7 @@ def run_windowed(args, env, w):
                                "much of the step the host link is busy",
                     traffic=None,
                     traffic_note="no counter capture at this size (110 GB resident); PCIe counters of the same kernel on a 1.5 M-vertex "
-                                 "instance are in profiles/alloc_kernel_large_1500k.md")
+                                 "instance are in profiles/transfer_kernel_large_1500k.md")
     roofline_hbm = dict(bound="hbm", kernel="scatter_grouped_kernel (accumulator rows of %d floats)" % acc_width,
                         achieved=sc_bytes / sc_s / 1e9, peak=pk["hbm_gbs"], unit="GB/s", frac=sc_bytes / sc_s / 1e9 / pk["hbm_gbs"],
                         peak_source=pk["source"], groups_per_step=groups / K, avg_launch_ms=float(phase[5]) / (K * window),

@@ -647,49 +647,54 @@ __global__ void alloc_kernel(ChunkArgs a) {
   if (lane_id() == 0 && reloaded) atomicAdd(&pc->reloaded, reloaded);
 }
 
-// The rows of one chunk across the host link, one warp per need-list entry: the staged row of the victim whose slot the
-// entry took over goes to its pinned host row (device -> host), and the host row of a vertex that was EVICTED is added
-// into its new slot (host -> device), so both directions of the link are busy at once.  An extent whose last row has
-// come back is listed for the free stack (taken back two chunks later by extent_plan_kernel).
-__global__ void transfer_kernel(ChunkArgs a) {
+// The rows of one chunk across the host link: the staged row of the victim whose slot a need-list entry took over
+// goes to its pinned host row (device -> host), and the host row of a vertex that was EVICTED is added into its new
+// slot (host -> device), so both directions of the link are busy at once.  A warp takes R entries per round, R chosen so
+// that it has four float4 per lane and direction in flight whatever the row width (R = 4 for rows of up to 32 float4,
+// 2 up to 64, else 1): the link is fed by bytes in flight, and narrow rows otherwise leave it short.  An extent whose
+// last row has come back is listed for the free stack (taken back two chunks later by extent_plan_kernel).
+template <int R>
+__global__ void __launch_bounds__(256) transfer_kernel(ChunkArgs a) {
   DevCtl* ctl = a.ctl;
   ChunkCtl* pc = a.pc;
   if (ctl->error) return;
+  constexpr int QPR = 4 / R;   // float4 steps of one row per round
   const int n = pc->need_count;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   const int vec = a.Hp >> 2;
   const int par = a.epoch & 1;
-  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    const int4 x = a.xfer_list[i];   // same address for the whole warp
-    const int slot = x.x, in_hrow = x.y, out_hrow = x.z;
-    if (in_hrow < 0 && out_hrow < 0) continue;
-    float* __restrict__ row = a.acc + (size_t)slot * a.Hp;
-    const float4* __restrict__ staged = reinterpret_cast<const float4*>(a.stage_out + (size_t)i * a.Hp);
-    float4* __restrict__ host_out = out_hrow >= 0 ? reinterpret_cast<float4*>(a.host_store + (size_t)out_hrow * a.Hp) : nullptr;
-    const float4* __restrict__ host_in = in_hrow >= 0 ? reinterpret_cast<const float4*>(a.host_store + (size_t)in_hrow * a.Hp) : nullptr;
-    for (int k0 = 0; k0 < vec; k0 += 128) {   // four float4 per lane and direction in flight
+  for (long long i0 = (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * R; i0 < n; i0 += warps * R) {
+    int4 x[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) x[r] = i0 + r < n ? a.xfer_list[i0 + r] : make_int4(0, -1, -1, 0);   // same address for the whole warp
+    for (int k0 = 0; k0 < vec; k0 += 32 * QPR) {
       float4 keep[4], in[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int k = k0 + q * 32 + lane_id();
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int r = s4 / QPR, k = k0 + (s4 % QPR) * 32 + lane_id();
         if (k < vec) {
-          if (host_out) keep[q] = staged[k];
-          if (host_in) in[q] = host_in[k];
+          if (x[r].z >= 0) keep[s4] = reinterpret_cast<const float4*>(a.stage_out + (size_t)(i0 + r) * a.Hp)[k];
+          if (x[r].y >= 0) in[s4] = reinterpret_cast<const float4*>(a.host_store + (size_t)x[r].y * a.Hp)[k];
         }
       }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int k = k0 + q * 32 + lane_id();
+      for (int s4 = 0; s4 < 4; ++s4) {
+        const int r = s4 / QPR, k = k0 + (s4 % QPR) * 32 + lane_id();
         if (k < vec) {
-          if (host_out) host_out[k] = keep[q];
-          if (host_in) asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(row + 4 * k), "f"(in[q].x), "f"(in[q].y), "f"(in[q].z), "f"(in[q].w) : "memory");
+          if (x[r].z >= 0) reinterpret_cast<float4*>(a.host_store + (size_t)x[r].z * a.Hp)[k] = keep[s4];
+          if (x[r].y >= 0) {
+            float* row = a.acc + (size_t)x[r].x * a.Hp + 4 * k;
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(row), "f"(in[s4].x), "f"(in[s4].y), "f"(in[s4].z), "f"(in[s4].w) : "memory");
+          }
         }
       }
     }
-    if (lane_id() == 0 && in_hrow >= 0) {
-      const int e = in_hrow >> a.ext_shift;
-      if (atomicSub(&a.ext_live[e], 1) == 1) a.ext_ret[par][atomicAdd(&ctl->ext_ret_count[par], 1)] = e;   // last row of the extent
-    }
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+      if (lane_id() == r && x[r].y >= 0) {
+        const int e = x[r].y >> a.ext_shift;
+        if (atomicSub(&a.ext_live[e], 1) == 1) a.ext_ret[par][atomicAdd(&ctl->ext_ret_count[par], 1)] = e;   // last row of the extent
+      }
   }
 }
 
@@ -725,7 +730,10 @@ void launch_transfer(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   // One block per SM.  The warps spend their time waiting for the host link; measured on the "large" workload, fewer
   // blocks leave the link short of requests (64 blocks: 36 + 33 GB/s, 148: 38 + 34, 1 184: 39 + 35), more blocks only
   // take thread slots from the scatter and select kernels that run beside the transfers on the compute stream.
-  transfer_kernel<<<c->sm_count, 256, 0, st>>>(a);
+  const int vec = a.Hp >> 2;
+  if (vec <= 32) transfer_kernel<4><<<c->sm_count, 256, 0, st>>>(a);
+  else if (vec <= 64) transfer_kernel<2><<<c->sm_count, 256, 0, st>>>(a);
+  else transfer_kernel<1><<<c->sm_count, 256, 0, st>>>(a);
   c->launches += 1;
 }
 
