@@ -62,6 +62,7 @@ def parse_args():
     p.add_argument("--secondary", default="mid", help="a second workload timed after the first and added to the JSON line "
                    "under 'secondary' (single-GPU runs only); 'none' switches it off")
     p.add_argument("--vertices", type=int, default=0, help="scale the workload to this many vertices (0 = full size)")
+    p.add_argument("--chunk", type=int, default=0, help="sources per pushed chunk (0 = the workload's own, 65 536 for all but 'tiny')")
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--window", type=int, default=32, help="bounded-pool workloads: chunks per step")
     p.add_argument("--prefill", type=int, default=384, help="bounded-pool workloads: untimed chunks that fill the pool first")
@@ -88,12 +89,21 @@ def workload_of(args, name=None):
     w = tg.WORKLOADS[name or args.workload]
     if args.vertices:
         w = tg.scaled(w, args.vertices)
+    if args.chunk > 0:
+        w = replace(w, chunk=args.chunk)
     if args.pool_fraction > 0:
         w = replace(w, pool_slots=max(1, int(w.V * args.pool_fraction)))
     if args.model:
         w = replace(w, mode={"sage": tg.SAGE_MEAN, "gcn": tg.GCN_SYM, "gin": tg.GIN_SUM, "gat": tg.GAT}[args.model],
                     gemm_mode=tg.GEMM_FP32 if args.model == "gat" else w.gemm_mode)
     return w
+
+
+def graph_of(args, w):
+    """The workload's graph.  --chunk changes how the sources are cut into pushes, not the graph: the generator's band
+    width stays the one of the workload's own chunk size."""
+    base = tg.WORKLOADS[w.name.split("@")[0]]
+    return tg.make_graph(replace(w, chunk=base.chunk) if args.chunk > 0 else w)
 
 
 def windowed(w) -> bool:
@@ -251,7 +261,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     w = workload_of(args)
-    g = tg.make_graph(w)
+    g = graph_of(args, w)
     layers = timed_layers(args, w)
     n = max(args.steps, 1) + max(args.warmup, 0)
     smp = OracleSampler(w, g, layers, min(n, 8), batch_size_for(w, layers))
@@ -376,7 +386,7 @@ def run_windowed(args, env, w):
     """Steps = windows of chunks of one layer pass in steady state (see the module docstring)."""
     import paper_2607_17374_b200 as tb
     torch, dev = env.torch, env.dev
-    g = tg.make_graph(w)
+    g = graph_of(args, w)
     model = tg.make_model(w)
     V, chunk = g.V, w.chunk
     chunks = [(s, min(s + chunk, V)) for s in range(0, V, chunk)]
@@ -531,7 +541,7 @@ def run_windowed(args, env, w):
 def run_full_pass(args, env, w):
     import paper_2607_17374_b200 as tb
     torch, dev, world, rank = env.torch, env.dev, env.world, env.rank
-    g = tg.make_graph(w)
+    g = graph_of(args, w)
     model = tg.make_model(w)
     V, L = g.V, w.L
     chunks = [(s, min(s + w.chunk, V)) for s in range(0, V, w.chunk)]
