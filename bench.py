@@ -80,8 +80,9 @@ def parse_args():
     p.add_argument("--model", default="", choices=["", "sage", "gcn", "gin", "gat"],
                    help="aggregation of every layer (default: the workload's); gat runs its three passes per layer")
     p.add_argument("--output", default="dense", choices=["dense", "runs-device", "runs-host"],
-                   help="full-pass workloads: where a layer's rows go: a dense matrix in HBM (default), or sorted runs (in HBM / "
-                        "pinned host memory) that the next layer reads back by merge-on-read")
+                   help="where a layer's rows go: a dense matrix in HBM (full-pass workloads) or the caller's drain buffers (bounded-pool "
+                        "workloads) by default, or sorted runs (in HBM / pinned host memory) that the next layer reads back by "
+                        "merge-on-read")
     return p.parse_args()
 
 
@@ -402,6 +403,15 @@ def run_windowed(args, env, w):
     cap = 3 * window * chunk                       # graduation buffer: drained once per window, earlier when it could overflow
     host_evict = min(V - w.hub_count, 56_000_000)   # rows evicted at once stay below this on the three bounded-pool workloads
     ctx = make_context(args, w, g, model, host_evict, cap)
+    runs = None
+    if args.output != "dense":
+        # Finished rows leave as sorted runs (embedding writer of Sect. 3.7) instead of being drained: 64 id ranges with
+        # partition buffers of 65 536 rows in HBM, the run store in HBM or in pinned host memory, sized for the rows the
+        # pass can complete (the pass stops after the timed windows).
+        n_used = prefill + (W + K) * window
+        kind = tb.RUNS_DEVICE if args.output == "runs-device" else tb.RUNS_HOST
+        runs = tb.Runs(V, w.dims[timed_layers(args, w)[0] + 1], 64, 65536, store_rows=min(V, int(1.25 * n_used * chunk) + 64 * 65536),
+                       max_append_rows=cap, max_chunk_rows=chunk, store_kind=kind)
     agg_first, acc_width = ctx.layer_plan(l)
     R = 8                                          # distinct generated input chunks, reused in turn
     x_host = [torch.empty((chunk, d_in), dtype=torch.float32).pin_memory() for _ in range(R)]
@@ -422,6 +432,9 @@ def run_windowed(args, env, w):
         for c in range(c0, c1):
             s, e = chunks[c]
             x = feats[c % R][: e - s]
+            if runs is not None:                      # rows go to the run store on the library's output stream
+                ctx.push_chunk(s, e, x, stream)
+                continue
             if ctx.push_chunk(s, e, x, stream, raise_on_drain_full=False) != 0:
                 drained += ctx.drain_completed(ids, rows, cap)
                 ctx.push_chunk(s, e, x, stream)
@@ -433,8 +446,12 @@ def run_windowed(args, env, w):
         """Prefill, warm-up windows, timed windows.  Returns (ms of the timed windows, stats before, stats after, rows drained,
         phase times, launches, clocks, wall ms)."""
         ctx.layer_begin(l, stream)
+        if runs is not None:
+            runs.reset()
+            ctx.layer_set_run_output(runs)
         run_chunks(0, prefill, feats, ids, rows, window)
-        ctx.drain_completed(ids, rows, cap)
+        if runs is None:
+            ctx.drain_completed(ids, rows, cap)
         c = prefill
         run_chunks(c, c + W * window, feats, ids, rows, window)
         c += W * window
@@ -460,6 +477,8 @@ def run_windowed(args, env, w):
             ph = ctx.get_phase_ms()
             ctx.set_timing(False)
         st1 = ctx.get_stats()
+        if runs is not None:
+            drained = st1["completed"] - st0["completed"]
         return ms, st0, st1, drained, ph, launches, clocks, wall
 
     # ---- inputs resident in HBM, rows drained into HBM
@@ -519,7 +538,7 @@ def run_windowed(args, env, w):
                 data="synthetic",
                 config=dict(workload=w.name, V=V, E=g.E, dims=list(w.dims), chunk=chunk, chunks_per_layer=len(chunks),
                             pool_slots=w.pool_slots, hub_count=w.hub_count, fanout=list(w.fanout),
-                            mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], evict_policy=args.evict_policy,
+                            mode=["sage_mean", "gcn_sym", "gin_sum", "gat"][w.mode], evict_policy=args.evict_policy, output=args.output,
                             step="window of %d chunks of layer %d (%d -> %d) in steady state; %d prefill chunks and %d warm-up windows "
                                  "before the timed ones, same layer pass; rows drained once per window" % (window, l, d_in, d_out, prefill, W),
                             layer=l, window_chunks=window, prefill_chunks=prefill, aggregate_first=bool(agg_first),
@@ -532,6 +551,8 @@ def run_windowed(args, env, w):
                             device_memory_in_use_gb=(total - free) / 1e9,
                             parallelism="replicas only" if env.world > 1 else "1 gpu", phase_ms=phase_ms),
                 clocks=clocks, roofline=roofline, roofline_hbm=roofline_hbm, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
+    if runs is not None:
+        runs.destroy()
     ctx.destroy()
     return line
 

@@ -28,10 +28,18 @@ namespace {
 
 constexpr int BM = 128;            // rows per CTA tile (UMMA M)
 constexpr int BN_MAX = 256;        // output columns per block (UMMA N)
-constexpr int STAGES = 2;            // stages with full-width (256-column) weight tiles: sizes the shared memory
-constexpr int MAX_STAGES = 4;        // narrower weight tiles leave room for more stages in the same memory
+constexpr int STAGES = 2;            // stages of 128-byte operand rows with full-width (256-column) weight tiles: sizes the shared memory
+constexpr int MAX_STAGES = 8;        // shorter operand rows and narrower weight tiles leave room for more stages in the same memory
 constexpr int TILE_A_BYTES = BM * 128;           // 128 rows x 128 B
 constexpr int TILE_B_BYTES = BN_MAX * 128;       // 256 rows x 128 B
+// fp32 mode: K columns per stage, 32 (128-byte operand rows, 128-byte swizzle) or 16 (64-byte rows and swizzle: stages half
+// as large, twice as many in flight).  Both are exact and measure the same (projection of the "mid" workload 6.1 against
+// 6.3 ms per step): the three TF32 MMAs of a K step read their operands from shared memory without reuse between them
+// (12 KB per 128 x 256 x 8 MMA, one MMA per 134 cycles at the pipe's rate = 92 B per cycle), and with the TMA fill and the
+// operand split on top the SM's 128 B per cycle of shared memory are the limit, not the depth of the pipeline.
+constexpr int KS32 = 32;
+constexpr int ROW32 = KS32 * 4;                  // operand row bytes in fp32 mode
+constexpr int A32_BYTES = BM * ROW32;            // one fp32-mode feature tile (raw / hi, or lo)
 constexpr unsigned WAIT_LIMIT = 1u << 24;
 constexpr int NUM_THREADS = 320;
 constexpr int OUT_TILE_BYTES = 32 * 128;        // epilogue staging tile: 32 rows x 32 fp32, 128B-swizzled
@@ -43,11 +51,10 @@ struct __align__(8) Barriers {
   int abort_flag;
 };
 
-// shared memory per stage: fp32 mode  A_hi(raw) 16K | A_lo 16K | B_hi 32K | B_lo 32K       = 96 KB
-//                          bf16 mode  A_raw0 16K | A_raw1 16K | A_bf16 16K | B_bf16 32K     = 80 KB
-// with weight tiles of 256 columns; a launch whose weight tiles are narrower (b_box_bytes < 32K) packs its stages
-// closer and runs as many as fit (GemmArgs::stages, stage_bytes), which hides more of the feature tiles' latency
-// where the product is bound by memory.
+// shared memory per stage: fp32 mode  A_hi(raw) 16K | A_lo 16K | B_hi 32K | B_lo 32K       = 96 KB (32 K-columns)
+//                          bf16 mode  A_raw0 16K | A_raw1 16K | A_bf16 16K | B_bf16 32K     = 80 KB (64 K-columns)
+// with weight tiles of 256 columns; the memory is sized for two such stages, and a launch whose weight tiles are
+// narrower runs as many stages as fit (GemmArgs::stages, stage_bytes).
 constexpr int STAGE_BYTES_FP32 = 2 * TILE_A_BYTES + 2 * TILE_B_BYTES;
 constexpr int STAGE_BYTES_BF16 = 3 * TILE_A_BYTES + TILE_B_BYTES;
 
@@ -83,14 +90,16 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
                ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
-// K-major operand tile, 128-byte rows, 128B swizzle, 8-row groups 1024 B apart.
+// K-major operand tile with ROW-byte rows (128: 128-byte swizzle; 64: 64-byte swizzle), 8-row groups 8 * ROW bytes apart.
+template <int ROW>
 __device__ __forceinline__ unsigned long long umma_desc(unsigned smem_addr) {
+  static_assert(ROW == 128 || ROW == 64, "operand rows of 128 or 64 bytes");
   unsigned long long d = 0;
   d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);   // start address
   d |= 1ull << 16;                                           // leading byte offset (unused for swizzled K-major)
-  d |= (unsigned long long)(1024 >> 4) << 32;                // stride byte offset: next 8-row group
+  d |= (unsigned long long)((8 * ROW) >> 4) << 32;           // stride byte offset: next 8-row group
   d |= 1ull << 46;                                           // descriptor version of this architecture
-  d |= 2ull << 61;                                           // SWIZZLE_128B
+  d |= (ROW == 128 ? 2ull : 4ull) << 61;                     // SWIZZLE_128B / SWIZZLE_64B
   return d;
 }
 
@@ -112,10 +121,10 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 struct GemmArgs {
   float* PT;            // [n x N]
   int n, N, Np;         // rows, output columns, columns padded to a multiple of 16
-  int k_stages;         // K padded / (32 fp32 mode, 64 bf16 mode)
-  int b_box_bytes;      // bytes one W-operand TMA box delivers (box rows x 128)
+  int k_stages;         // K padded / (KS32 fp32 mode, 64 bf16 mode)
+  int b_box_bytes;      // bytes one W-operand TMA box delivers (box rows x operand row bytes)
   int stages;           // operand stages in flight (2 .. MAX_STAGES)
-  int stage_bytes;      // fp32 mode 2 * TILE_A_BYTES + 2 * b_box_bytes, bf16 mode 3 * TILE_A_BYTES + b_box_bytes
+  int stage_bytes;      // fp32 mode 2 * A32_BYTES + 2 * b_box_bytes, bf16 mode 3 * TILE_A_BYTES + b_box_bytes
   int Hp, mode, fanout;
   const float* bias;
   const long long* row_ptr;
@@ -182,10 +191,10 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             tma_load_2d(st + TILE_A_BYTES, &map_x, ks * 64 + 32, row0, &bars->full[s]);
             tma_load_2d(st + 3 * TILE_A_BYTES, &map_b0, ks * 64, col0, &bars->full[s]);
           } else {
-            mbar_expect_tx(&bars->full[s], TILE_A_BYTES + 2 * g.b_box_bytes);
-            tma_load_2d(st, &map_x, ks * 32, row0, &bars->full[s]);
-            tma_load_2d(st + 2 * TILE_A_BYTES, &map_b0, ks * 32, col0, &bars->full[s]);
-            tma_load_2d(st + 2 * TILE_A_BYTES + g.b_box_bytes, &map_b1, ks * 32, col0, &bars->full[s]);
+            mbar_expect_tx(&bars->full[s], A32_BYTES + 2 * g.b_box_bytes);
+            tma_load_2d(st, &map_x, ks * KS32, row0, &bars->full[s]);
+            tma_load_2d(st + 2 * A32_BYTES, &map_b0, ks * KS32, col0, &bars->full[s]);
+            tma_load_2d(st + 2 * A32_BYTES + g.b_box_bytes, &map_b1, ks * KS32, col0, &bars->full[s]);
           }
         }
       }
@@ -211,14 +220,14 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
           tc_fence_after();
           const unsigned base = smem_u32(stage_ptr(s));
           if (BF16) {
-            const unsigned long long da = umma_desc(base + 2 * TILE_A_BYTES), db = umma_desc(base + 3 * TILE_A_BYTES);
+            const unsigned long long da = umma_desc<128>(base + 2 * TILE_A_BYTES), db = umma_desc<128>(base + 3 * TILE_A_BYTES);
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk) umma(tmem_d, da + 2 * kk, db + 2 * kk, idesc, (ks | kk) != 0, false);
           } else {
-            const unsigned long long a_hi = umma_desc(base), a_lo = umma_desc(base + TILE_A_BYTES);
-            const unsigned long long b_hi = umma_desc(base + 2 * TILE_A_BYTES), b_lo = umma_desc(base + 2 * TILE_A_BYTES + g.b_box_bytes);
+            const unsigned long long a_hi = umma_desc<ROW32>(base), a_lo = umma_desc<ROW32>(base + A32_BYTES);
+            const unsigned long long b_hi = umma_desc<ROW32>(base + 2 * A32_BYTES), b_lo = umma_desc<ROW32>(base + 2 * A32_BYTES + g.b_box_bytes);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk) {
+            for (int kk = 0; kk < KS32 / 8; ++kk) {
               umma(tmem_d, a_lo + 2 * kk, b_hi + 2 * kk, idesc, (ks | kk) != 0, true);
               umma(tmem_d, a_hi + 2 * kk, b_lo + 2 * kk, idesc, 1u, true);
               umma(tmem_d, a_hi + 2 * kk, b_hi + 2 * kk, idesc, 1u, true);
@@ -262,9 +271,9 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         } else {
           // element-wise and layout-preserving: the swizzle does not matter
           float4* hi = reinterpret_cast<float4*>(st);
-          float4* lo = reinterpret_cast<float4*>(st + TILE_A_BYTES);
+          float4* lo = reinterpret_cast<float4*>(st + A32_BYTES);
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < A32_BYTES / 16 / 128; ++i) {
             const int idx = t + i * 128;
             float4 x = hi[idx], h4, l4;
             h4.x = __uint_as_float(__float_as_uint(x.x) & 0xFFFFE000u); l4.x = x.x - h4.x;
@@ -430,14 +439,15 @@ bool make_map(CUtensorMap* m, const void* base, CUtensorMapDataType dt, int elem
   cuuint64_t strides[1] = {(cuuint64_t)ld_elems * elem};
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle swz = box_cols * elem == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B;   // box rows of 64 or 128 bytes
   return fn(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Stages that fit the shared memory sized for STAGES full-width stages.
 void set_stages(GemmArgs& g, bool bf16) {
   const int budget = STAGES * (bf16 ? STAGE_BYTES_BF16 : STAGE_BYTES_FP32);
-  g.stage_bytes = bf16 ? 3 * TILE_A_BYTES + g.b_box_bytes : 2 * TILE_A_BYTES + 2 * g.b_box_bytes;
+  g.stage_bytes = bf16 ? 3 * TILE_A_BYTES + g.b_box_bytes : 2 * A32_BYTES + 2 * g.b_box_bytes;
   int n = budget / g.stage_bytes;
   g.stages = n < STAGES ? STAGES : n > MAX_STAGES ? MAX_STAGES : n;
 }
@@ -457,7 +467,7 @@ int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat
   WImage* w = new WImage();
   *slot = w;
   w->Np = taurus_round_up(N, 16);
-  w->Kp = taurus_round_up(K, bf16 ? 64 : 32);
+  w->Kp = taurus_round_up(K, bf16 ? 64 : KS32);
   const size_t cnt = (size_t)w->Np * w->Kp;
   const int bw = w->Np < BN_MAX ? w->Np : BN_MAX;
   if (bf16) {
@@ -483,8 +493,8 @@ int prepare_tc_weights(taurus_ctx* c, void** slot, const std::vector<float>& cat
     if (cudaMalloc(&w->hi, cnt * 4) != cudaSuccess || cudaMalloc(&w->lo, cnt * 4) != cudaSuccess) return TAURUS_ERR_NOMEM;
     if (cudaMemcpy(w->hi, hi.data(), cnt * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemcpy(w->lo, lo.data(), cnt * 4, cudaMemcpyHostToDevice) != cudaSuccess) return TAURUS_ERR_CUDA;
-    if (!make_map(&w->map_hi, w->hi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w->Np, w->Kp, w->Kp, bw, 32) ||
-        !make_map(&w->map_lo, w->lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w->Np, w->Kp, w->Kp, bw, 32)) return TAURUS_ERR_CUDA;
+    if (!make_map(&w->map_hi, w->hi, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w->Np, w->Kp, w->Kp, bw, KS32) ||
+        !make_map(&w->map_lo, w->lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w->Np, w->Kp, w->Kp, bw, KS32)) return TAURUS_ERR_CUDA;
   }
   return TAURUS_OK;
 }
@@ -514,12 +524,12 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   const int K = c->dims[layer], Hp = taurus_round_up(c->dims[layer + 1], 4);
   const int N = taurus_proj_width(c->mode, Hp);
   CUtensorMap map_x;
-  if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, 32)) return TAURUS_ERR_CUDA;
+  if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, bf16 ? 32 : KS32)) return TAURUS_ERR_CUDA;
   CUtensorMap map_out;
   if (!make_map(&map_out, c->d_PT, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, N, N, 32, 32)) return TAURUS_ERR_CUDA;
   GemmArgs g;
-  g.PT = c->d_PT; g.n = n; g.N = N; g.Np = w->Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
-  g.b_box_bytes = (w->Np < BN_MAX ? w->Np : BN_MAX) * 128;
+  g.PT = c->d_PT; g.n = n; g.N = N; g.Np = w->Np; g.k_stages = w->Kp / (bf16 ? 64 : KS32);
+  g.b_box_bytes = (w->Np < BN_MAX ? w->Np : BN_MAX) * (bf16 ? 128 : ROW32);
   set_stages(g, bf16);
   g.Hp = Hp; g.mode = c->mode; g.fanout = c->fanout[layer]; g.bias = c->d_bias[layer];
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = src_begin; g.ctl = c->d_ctl;
@@ -562,20 +572,20 @@ int launch_gemm_plain_tc(taurus_ctx* c, void* image, int col0, int N, const floa
   const int bw = Np < BN_MAX ? Np : BN_MAX;
   const int elem = bf16 ? 2 : 4;
   CUtensorMap map_x, map_out, map_hi, map_lo;
-  if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, 32)) return TAURUS_ERR_CUDA;
+  if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, bf16 ? 32 : KS32)) return TAURUS_ERR_CUDA;
   if (!make_map(&map_out, out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, N, ld_out, 32, 32)) return TAURUS_ERR_CUDA;
   const char* hi = static_cast<const char*>(w->hi) + (size_t)col0 * w->Kp * elem;
   if (!make_map(&map_hi, hi, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, elem, rows_left, w->Kp, w->Kp, bw,
-                bf16 ? 64 : 32))
+                bf16 ? 64 : KS32))
     return TAURUS_ERR_CUDA;
   map_lo = map_hi;
   if (!bf16) {
     const char* lo = static_cast<const char*>(w->lo) + (size_t)col0 * w->Kp * elem;
-    if (!make_map(&map_lo, lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, rows_left, w->Kp, w->Kp, bw, 32)) return TAURUS_ERR_CUDA;
+    if (!make_map(&map_lo, lo, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, rows_left, w->Kp, w->Kp, bw, KS32)) return TAURUS_ERR_CUDA;
   }
   GemmArgs g;
-  g.PT = out; g.n = n; g.N = N; g.Np = Np; g.k_stages = w->Kp / (bf16 ? 64 : 32);
-  g.b_box_bytes = bw * 128;
+  g.PT = out; g.n = n; g.N = N; g.Np = Np; g.k_stages = w->Kp / (bf16 ? 64 : KS32);
+  g.b_box_bytes = bw * (bf16 ? 128 : ROW32);
   set_stages(g, bf16);
   g.Hp = N; g.mode = TAURUS_GIN_SUM; g.fanout = 0; g.bias = nullptr;
   g.row_ptr = c->d_row_ptr; g.din = c->d_din; g.src_begin = 0; g.ctl = c->d_ctl;
