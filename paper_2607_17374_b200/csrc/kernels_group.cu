@@ -361,7 +361,21 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
       if (lane_on[k]) row[k] = *reinterpret_cast<const float4*>(p + k * LPE * 16);
   };
 
-  for (long long span = warp0; span < spans; span += warps) {
+  // Where row transfers of the previous chunk may be running beside this kernel (bounded pool), spans are handed out
+  // from a counter rather than by warp number: SMs that also host transfer warps get through fewer of them (measured on
+  // "large": scatter 105 -> 34 ms per 32-chunk window).  A span is requested only when the warp is ready for it: a chunk
+  // has about two spans per warp there, and a warp that asked ahead would sit on a span while it is slow.  Elsewhere the
+  // spans are dealt by warp number: same-address atomics cost about 3 ns each, 75 us per launch at the 25 k spans of a
+  // "mid" chunk.
+  const bool dyn = a.dynamic_spans != 0;
+  for (long long it = 0;; ++it) {
+    long long span = warp0 + it * warps;
+    if (dyn) {
+      unsigned int got = 0;
+      if (lane == 0) got = atomicAdd(&pc->span_next, 1u);
+      span = (long long)__shfl_sync(FULL, got, 0);
+    }
+    if (span >= spans) break;
     long long x = e0 + span * SPAN_EDGES + (long long)sub * STRETCH;
     const long long x_end = (x + STRETCH < e1) ? x + STRETCH : e1;
     const int2* ge = g_edge + x;
@@ -398,7 +412,14 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
   if (c4 != 0) { msgs = 0; hub_msgs = 0; groups = 0; }
 
   // self messages (one per chunk vertex)
-  for (long long t = warp0; t < self_tiles; t += warps) {
+  for (long long it = 0;; ++it) {
+    long long t = warp0 + it * warps;
+    if (dyn) {
+      unsigned int got = 0;
+      if (lane == 0) got = atomicAdd(&pc->self_next, 1u);
+      t = (long long)__shfl_sync(FULL, got, 0);
+    }
+    if (t >= self_tiles) break;
     const long long u = a.src_begin + t * 32 + lane;
     int v = u < a.src_end ? (int)u : -1;
     int l = -1;

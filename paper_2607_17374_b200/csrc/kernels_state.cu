@@ -227,14 +227,33 @@ static __device__ __forceinline__ void sel_fold(ChunkCtl* pc, int lvl, unsigned 
   }
 }
 
+// The passes over the pool work on tiles of SEL_TILE slots.  A block takes the tiles of its own number, or, where row
+// transfers may run beside the kernel (dynamic_spans), the next tile of a counter: blocks on SMs that also host transfer
+// warps are several times slower, and with a fixed deal the pass would wait for them.
+#define SEL_ITEMS 8
+#define SEL_TILE (256 * SEL_ITEMS)
+static __device__ __forceinline__ long long next_tile(bool dyn, unsigned int* counter, long long it, long long* s_tile) {
+  if (!dyn) return (long long)blockIdx.x + it * gridDim.x;
+  __syncthreads();   // every thread has read the previous value
+  if (threadIdx.x == 0) *s_tile = (long long)atomicAdd(counter, 1u);
+  __syncthreads();
+  return *s_tile;
+}
+
 __global__ void __launch_bounds__(256) select_keys_kernel(ChunkArgs a) {   // key of every slot; range of the eligible keys
   DevCtl* ctl = a.ctl;
   ChunkCtl* pc = a.pc;
   if (ctl->error || pc->sel_final_level < 0) return;
   unsigned long long kmin = ~0ull, kmax = 0ull;
   int cnt = 0;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x; s < a.pool_slots; s += stride) {
+  __shared__ long long s_tile;
+  for (long long it = 0;; ++it) {
+    const long long base = next_tile(a.dynamic_spans != 0, &pc->tile_next[0], it, &s_tile) * SEL_TILE;
+    if (base >= a.pool_slots) break;
+#pragma unroll
+  for (int j = 0; j < SEL_ITEMS; ++j) {
+    const long long s = base + j * 256 + threadIdx.x;
+    if (s >= a.pool_slots) break;
     const int v = a.owner[s];
     unsigned long long key = ~0ull;
     if (v >= 0) {
@@ -252,6 +271,7 @@ __global__ void __launch_bounds__(256) select_keys_kernel(ChunkArgs a) {   // ke
       }
     }
     a.keys[s] = key;
+  }
   }
   sel_fold(pc, 0, kmin, kmax, cnt);
 }
@@ -273,16 +293,21 @@ __global__ void __launch_bounds__(256) select_hist_kernel(ChunkArgs a, int level
   __syncthreads();
   const int shift = sel_shift_of(pc->sel_min[level], pc->sel_max[level]);
   const int32_t* __restrict__ cand = level == 0 ? nullptr : a.cand[level & 1];
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  const long long rounds = (n + stride - 1) / stride;
-  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  for (long long r = 0; r < rounds; ++r, i += stride) {
-    unsigned long long key = ~0ull;
-    if (i < n) key = a.keys[level == 0 ? i : (long long)cand[i]];
-    const bool on = key != ~0ull;
-    const unsigned digit = on ? (unsigned)(key >> shift) & (TAURUS_SEL_BINS - 1) : 0xffffffffu;
-    const unsigned peers = __match_any_sync(FULL, digit);
-    if (on && lane_id() == __ffs(peers) - 1) atomicAdd(&sh[digit], (unsigned)__popc(peers));
+  __shared__ long long s_tile;
+  const bool dyn = level == 0 && a.dynamic_spans != 0;   // deeper levels see short candidate lists
+  for (long long it = 0;; ++it) {
+    const long long base = next_tile(dyn, &pc->tile_next[1], it, &s_tile) * SEL_TILE;
+    if (base >= n) break;
+#pragma unroll
+    for (int j = 0; j < SEL_ITEMS; ++j) {
+      const long long i = base + j * 256 + threadIdx.x;
+      unsigned long long key = ~0ull;
+      if (i < n) key = a.keys[level == 0 ? i : (long long)cand[i]];
+      const bool on = key != ~0ull;
+      const unsigned digit = on ? (unsigned)(key >> shift) & (TAURUS_SEL_BINS - 1) : 0xffffffffu;
+      const unsigned peers = __match_any_sync(FULL, digit);
+      if (on && lane_id() == __ffs(peers) - 1) atomicAdd(&sh[digit], (unsigned)__popc(peers));
+    }
   }
   __syncthreads();
   unsigned int* hist = pc->hist[level & 1];
@@ -344,11 +369,15 @@ __global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int leve
   }
   unsigned long long kmin = ~0ull, kmax = 0ull;
   int cnt = 0;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  const long long rounds = (n + stride - 1) / stride;
-  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const unsigned lt = (1u << lane_id()) - 1;
-  for (long long r = 0; r < rounds; ++r, i += stride) {
+  __shared__ long long s_tile;
+  const bool dyn = level == 0 && a.dynamic_spans != 0;
+  for (long long it = 0;; ++it) {
+    const long long base = next_tile(dyn, &pc->tile_next[2], it, &s_tile) * SEL_TILE;
+    if (base >= n) break;
+#pragma unroll 2
+  for (int j = 0; j < SEL_ITEMS; ++j) {
+    const long long i = base + j * 256 + threadIdx.x;
     unsigned long long key = ~0ull;
     int slot = -1;
     if (i < n) { slot = level == 0 ? (int)i : cand[i]; key = a.keys[slot]; }
@@ -376,6 +405,7 @@ __global__ void __launch_bounds__(256) select_split_kernel(ChunkArgs a, int leve
         cnt++;
       }
     }
+  }
   }
   // sel_count of the next level is already counted by the appends: fold only the key range
   for (int o = 16; o; o >>= 1) {
@@ -922,6 +952,8 @@ __global__ void commit_kernel(ChunkArgs a, int with_counts) {
   else ctl->grad_count += pc->done_count;
   pc->hs = pc->ns = pc->ev = pc->gs = 0;
   pc->need_count = 0; pc->done_count = 0; pc->touched_count = 0; pc->deficit = 0; pc->victim_count = 0; pc->reloaded = 0;
+  pc->span_next = 0; pc->self_next = 0;
+  pc->tile_next[0] = pc->tile_next[1] = pc->tile_next[2] = pc->tile_next[3] = 0;
 }
 
 // S6: completions listed, slots released, chunk record written.

@@ -476,6 +476,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.mode = c->mode; a.act = c->act[l]; a.fanout = c->fanout[l]; a.evict_policy = c->evict_policy; a.seed = c->seed;
   a.gin_self = 1.0f + c->gin_eps;
   a.direct = c->pool_slots >= c->V ? 1 : 0;
+  a.dynamic_spans = c->pipelined ? 1 : 0;
   const bool direct_dense = c->dense_out && c->dense_is_device;
   const bool halves = (c->dense_out && !direct_dense) || c->run_out;   // the graduation buffer alternates between two halves
   a.dense_direct = direct_dense ? c->dense_out : nullptr;

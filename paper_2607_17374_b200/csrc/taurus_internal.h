@@ -30,6 +30,9 @@ struct ChunkCtl {
   int32_t victim_count;   // victims listed so far
   int32_t hs, ns, ev, gs; // touched vertices by state at chunk start
   int32_t reloaded;       // reloads
+  unsigned int span_next; // scatter: next span of the chunk's edge list to hand to a warp
+  unsigned int self_next; // scatter: next tile of 32 self messages to hand to a warp
+  unsigned int tile_next[4];  // pool passes of the victim select: next tile of slots to hand to a block
   long long alloc_base;   // need-list entry i takes free_stack[alloc_base - 1 - i]
   // Victim select, level by level (level 0 scans the pool, deeper levels the candidates the level above left):
   long long sel_k[TAURUS_SEL_LEVELS + 1];               // rank still to resolve among the keys entering the level
@@ -140,6 +143,7 @@ struct ChunkArgs {
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
   int32_t dense_half;       // -1: graduation buffer drained by the caller; 0 / 1: half used by this chunk
   int32_t direct;           // pool_slots >= V: vertex v owns slot v, no free stack, no eviction
+  int32_t dynamic_spans;    // the scatter hands its spans out from a counter (row transfers may run beside it)
   float* dense_direct;      // dense-output mode with the matrix in device memory: finalise writes row v at dense_direct + v * dense_ld
   long long dense_ld;
   int32_t d_out;            // unpadded output width
