@@ -632,48 +632,55 @@ __global__ void alloc_kernel(ChunkArgs a) {
   // EVICTED; entry i >= deficit pops the free stack.  Either way the slot is cleared and handed to the vertex, which
   // is IN_BUFFER afterwards; the partial sum of a vertex that was EVICTED is ADDED into the slot by transfer_kernel
   // (sums commute: the scatter may already be adding this chunk's messages to the same row).
+  // Batches of up to 32 entries per warp: each lane follows the chain of dependent reads of one entry (vertex, victim,
+  // slot, state) and writes its metadata, then the warp walks the batch row by row.
   int reloaded = 0;
   const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    int v = a.need_list[i];
-    int slot = -1, st = 0, l = 0, out_hrow = -1, victim = -1;
-    if (lane_id() == 0) {
+  int per = (int)((n + warps - 1) / warps);
+  per = per < 1 ? 1 : per > 32 ? 32 : per;
+  for (long long i0 = (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * per; i0 < n; i0 += warps * per) {
+    const long long i = i0 + lane_id();
+    int slot = -1, out_hrow = -1;
+    if (lane_id() < per && i < n) {
+      const int v = a.need_list[i];
+      int victim = -1;
       if (i < deficit) {
         const int2 vic = a.victims[deficit - 1 - i];
         slot = vic.x; out_hrow = vic.y; victim = a.owner[slot];
-      } else { long long f = pc->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
-      st = a.state[v];
-      l = a.loc[v];
-    }
-    slot = __shfl_sync(FULL, slot, 0);
-    out_hrow = __shfl_sync(FULL, out_hrow, 0);
-    if (slot < 0) {
-      if (lane_id() == 0) atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
-      continue;
-    }
-    float4* __restrict__ row = reinterpret_cast<float4*>(a.acc + (size_t)slot * a.Hp);
-    if (out_hrow >= 0) {
-      float4* __restrict__ keep = reinterpret_cast<float4*>(a.stage_out + (size_t)i * a.Hp);
-      for (int k = lane_id(); k < vec; k += 32) { keep[k] = row[k]; row[k] = zero; }
-    } else {
-      for (int k = lane_id(); k < vec; k += 32) row[k] = zero;
-    }
-    if (lane_id() == 0) {
-      const int in_hrow = st == TAURUS_EVICTED ? -2 - l : -1;
-      if (a.xfer_list) a.xfer_list[i] = make_int4(slot, in_hrow, out_hrow, 0);
-      if (out_hrow >= 0) {
-        a.loc[victim] = -2 - out_hrow;
-        a.state[victim] = TAURUS_EVICTED;
+      } else { const long long f = pc->alloc_base - 1 - i; slot = f >= 0 ? a.free_stack[f] : -1; }
+      if (slot < 0) {
+        atomicCAS(&ctl->error, 0, TAURUS_ERR_INTERNAL);
+      } else {
+        const int in_hrow = a.state[v] == TAURUS_EVICTED ? -2 - a.loc[v] : -1;
+        if (a.xfer_list) a.xfer_list[i] = make_int4(slot, in_hrow, out_hrow, 0);
+        if (out_hrow >= 0) {
+          a.loc[victim] = -2 - out_hrow;
+          a.state[victim] = TAURUS_EVICTED;
+        }
+        if (in_hrow >= 0) {
+          a.reload_count[v] += 1;
+          reloaded++;
+        }
+        a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch;
+        if (a.slot_touch) a.slot_touch[slot] = a.epoch;   // slot_pend follows in compact_done: v is on the touched list
+        a.state[v] = TAURUS_IN_BUFFER;
       }
-      if (in_hrow >= 0) {
-        a.reload_count[v] += 1;
-        reloaded++;
+    }
+    const int rows = n - i0 < per ? (int)(n - i0) : per;
+    for (int j = 0; j < rows; ++j) {
+      const int sj = __shfl_sync(FULL, slot, j);
+      const int oj = __shfl_sync(FULL, out_hrow, j);
+      if (sj < 0) continue;
+      float4* __restrict__ row = reinterpret_cast<float4*>(a.acc + (size_t)sj * a.Hp);
+      if (oj >= 0) {
+        float4* __restrict__ keep = reinterpret_cast<float4*>(a.stage_out + (size_t)(i0 + j) * a.Hp);
+        for (int k = lane_id(); k < vec; k += 32) { keep[k] = row[k]; row[k] = zero; }
+      } else {
+        for (int k = lane_id(); k < vec; k += 32) row[k] = zero;
       }
-      a.loc[v] = slot; a.owner[slot] = v; a.slot_epoch[slot] = a.epoch;
-      if (a.slot_touch) a.slot_touch[slot] = a.epoch;   // slot_pend follows in compact_done: v is on the touched list
-      a.state[v] = TAURUS_IN_BUFFER;
     }
   }
+  for (int o = 16; o; o >>= 1) reloaded += __shfl_xor_sync(FULL, reloaded, o);
   if (lane_id() == 0 && reloaded) atomicAdd(&pc->reloaded, reloaded);
 }
 
