@@ -16,7 +16,8 @@ layers, Sect. 4.2).  The full layer time is printed as an estimate from the time
 
 The default run times "large" (the eviction-bound configuration) and then "mid" as a secondary entry in the same
 JSON line.  N > 1 (under torchrun): the path has no exchange step, so every rank runs an independent replica
-("replicas only", weak scaling); value = sum over ranks / max time.
+("replicas only", weak scaling); value = sum over ranks / max time.  Every replica of "large" holds the 8 GB graph and
+pins 65 GB of host memory for its evicted rows: N replicas need N times that on the node.
 --impl reference times the CPU oracle (a deliberately plain program) on bounded destination samples of the workload.
 """
 from __future__ import annotations
