@@ -49,29 +49,43 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
   }
   const int vec = a.Hp >> 2;
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
-  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
-    const int pitch = self_store ? 2 * a.Hp : a.Hp;
-    float4* dst = reinterpret_cast<float4*>(A + (size_t)i * pitch);
-    const int v = a.done_list[i];
-    const int l = a.loc[v];
+  const int pitch = self_store ? 2 * a.Hp : a.Hp;
+  // Batches of up to 32 finished vertices per warp: each lane follows the dependent reads of one vertex (list entry,
+  // slot, degree), then the warp walks the batch row by row.
+  int per = (int)((n + warps - 1) / warps);
+  per = per < 1 ? 1 : per > 32 ? 32 : per;
+  for (long long i0 = (((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * per; i0 < n; i0 += warps * per) {
+    const long long mine = i0 + al();
+    int v = -1, l = 0;
     float scale = 1.0f;
-    if (a.mode == TAURUS_SAGE_MEAN) {
-      const int m = af_messages(a.din[v], a.fanout);
-      scale = 1.0f / (float)(m > 1 ? m : 1);
-    } else if (a.mode == TAURUS_GCN_SYM) {
-      scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
-    } else if (a.mode == TAURUS_GAT) {
-      scale = 1.0f / a.att_z[v];   // softmax normaliser
+    if (al() < per && mine < n) {
+      v = a.done_list[mine];
+      l = a.loc[v];
+      if (a.mode == TAURUS_SAGE_MEAN) {
+        const int m = af_messages(a.din[v], a.fanout);
+        scale = 1.0f / (float)(m > 1 ? m : 1);
+      } else if (a.mode == TAURUS_GCN_SYM) {
+        scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
+      } else if (a.mode == TAURUS_GAT) {
+        scale = 1.0f / a.att_z[v];   // softmax normaliser
+      }
     }
-    const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)l * a.Hp);
-    for (int k = al(); k < vec; k += 32) {
-      float4 x = src[k];
-      x.x *= scale; x.y *= scale; x.z *= scale; x.w *= scale;
-      dst[k] = x;
-    }
-    if (self_store) {
-      const float4* own = reinterpret_cast<const float4*>(self_store + (size_t)v * a.Hp);
-      for (int k = al(); k < vec; k += 32) dst[vec + k] = own[k];
+    const int rows_here = n - i0 < per ? (int)(n - i0) : per;
+    for (int j = 0; j < rows_here; ++j) {
+      const int vj = __shfl_sync(0xffffffffu, v, j);
+      const int lj = __shfl_sync(0xffffffffu, l, j);
+      const float sj = __shfl_sync(0xffffffffu, scale, j);
+      float4* dst = reinterpret_cast<float4*>(A + (size_t)(i0 + j) * pitch);
+      const float4* src = reinterpret_cast<const float4*>(a.acc + (size_t)lj * a.Hp);
+      for (int k = al(); k < vec; k += 32) {
+        float4 x = src[k];
+        x.x *= sj; x.y *= sj; x.z *= sj; x.w *= sj;
+        dst[k] = x;
+      }
+      if (self_store) {
+        const float4* own = reinterpret_cast<const float4*>(self_store + (size_t)vj * a.Hp);
+        for (int k = al(); k < vec; k += 32) dst[vec + k] = own[k];
+      }
     }
   }
 }
