@@ -67,6 +67,9 @@ def _lib():
         lib.to_message_sets.argtypes = [i64, vp, vp, vp, i32, u64, i32, vp, vp, vp, vp]
         lib.to_aggregate.argtypes = [i64, vp, vp, vp, vp, vp, i32, vp]
         lib.to_simulate.argtypes = [i64, vp, vp, vp, vp, vp, i64, i64, i32, u64, vp, vp, vp, vp, vp]
+        lib.to_completion_rank_exact.argtypes = [i64, vp, vp, vp]
+        lib.to_scan_in_edges.restype = i64
+        lib.to_scan_in_edges.argtypes = [i64, vp, vp, vp, vp, vp, i64]
         lib.to_evict_hash.restype = ctypes.c_uint32
         lib.to_evict_hash.argtypes = [u64, u64, u64]
         _handle = lib
@@ -219,16 +222,21 @@ def subset_in_lists(V: int, row_ptr: np.ndarray, col: np.ndarray, dsts: np.ndarr
     """In-lists (ascending source id, duplicates in CSR order) of the sorted, distinct destinations dsts.
     Returns (ptr int64 [len(dsts) + 1], src int64, eid int64)."""
     dsts = np.asarray(dsts, dtype=np.int64)
-    wanted = np.zeros(V, dtype=bool)
-    wanted[dsts] = True
-    sel = np.flatnonzero(wanted[col])                          # ascending CSR edge index = (source, position) order
+    wanted = np.zeros(V, dtype=np.uint8)
+    wanted[dsts] = 1
+    row_ptr = np.ascontiguousarray(row_ptr, dtype=np.int64)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    n = int(_lib().to_scan_in_edges(V, _p(row_ptr), _p(col), _p(wanted), None, None, 0))
+    sel = np.empty(n, np.int64)                                # ascending CSR edge index = (source, position) order
+    src = np.empty(n, np.int64)
+    if int(_lib().to_scan_in_edges(V, _p(row_ptr), _p(col), _p(wanted), _p(sel), _p(src), n)) != n:
+        raise MemoryError
     d = col[sel]
     order = np.argsort(d, kind="stable")
-    sel, d = sel[order], d[order]
+    sel, src, d = sel[order], src[order], d[order]
     ptr = np.zeros(dsts.size + 1, np.int64)
     np.cumsum(np.bincount(np.searchsorted(dsts, d), minlength=dsts.size), out=ptr[1:])
-    src = np.searchsorted(row_ptr, sel, side="right") - 1      # the row whose range holds the edge
-    return ptr, src.astype(np.int64), sel.astype(np.int64)
+    return ptr, src, sel
 
 
 def subset_message_sets(ptr: np.ndarray, src: np.ndarray, eid: np.ndarray, dsts: np.ndarray, fanout: int, seed: int, layer: int):
@@ -298,6 +306,16 @@ def complete_chunk_closed_form(ms: MessageSets, chunk_sources: int) -> np.ndarra
         mx = np.maximum.reduceat(ms.src.astype(np.int64), ms.ptr[nz])
         last[nz] = np.maximum(last[nz], mx)
     return (last // chunk_sources).astype(np.int32)
+
+
+def completion_rank_exact(V: int, row_ptr: np.ndarray, col: np.ndarray) -> np.ndarray:
+    """max(v, largest in-neighbour of v) for every v of an exact layer, straight from the CSR (no in-lists needed): the
+    rank whose chunk completes v (Sect. 3.8, c(v))."""
+    rank = np.empty(V, np.int32)
+    row_ptr = np.ascontiguousarray(row_ptr, dtype=np.int64)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    _lib().to_completion_rank_exact(V, _p(row_ptr), _p(col), _p(rank))
+    return rank
 
 
 def first_touch_chunk(ms: MessageSets, chunk_sources: int) -> np.ndarray:

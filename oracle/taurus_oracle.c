@@ -18,6 +18,9 @@
  * No function in this file is "parity unpinned".
  */
 #include <stdint.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 #include <stdlib.h>
 #include <string.h>
 
@@ -43,6 +46,58 @@ int to_build_in_lists(int64_t V, int64_t E, const int64_t* row_ptr, const int32_
     }
   free(cur);
   return 0;
+}
+
+/* In-edges of a marked subset of destinations: every CSR edge (u -> v) with wanted[v] != 0, in ascending edge index
+ * (= ascending source, CSR order among equal sources).  Rows are cut into one contiguous block per thread; the blocks
+ * are counted, then filled at their offsets, so the output order does not depend on the thread count.
+ * out_eid / out_src may be NULL (count only).  Returns the number of such edges, or -1 if it exceeds `capacity`
+ * when filling. */
+int64_t to_scan_in_edges(int64_t V, const int64_t* row_ptr, const int32_t* col, const uint8_t* wanted,
+                         int64_t* out_eid, int64_t* out_src, int64_t capacity) {
+  int T = 1;
+#ifdef _OPENMP
+  T = omp_get_max_threads();
+#endif
+  int64_t* cnt = (int64_t*)calloc((size_t)T + 1, sizeof(int64_t));
+  if (!cnt) return -1;
+#pragma omp parallel for schedule(static, 1)
+  for (int t = 0; t < T; ++t) {
+    const int64_t u0 = V * t / T, u1 = V * (t + 1) / T;
+    int64_t n = 0;
+    for (int64_t e = row_ptr[u0]; e < row_ptr[u1]; ++e) n += wanted[col[e]] != 0;
+    cnt[t + 1] = n;
+  }
+  for (int t = 0; t < T; ++t) cnt[t + 1] += cnt[t];
+  const int64_t total = cnt[T];
+  if (out_eid && out_src) {
+    if (total > capacity) { free(cnt); return -1; }
+#pragma omp parallel for schedule(static, 1)
+    for (int t = 0; t < T; ++t) {
+      const int64_t u0 = V * t / T, u1 = V * (t + 1) / T;
+      int64_t p = cnt[t];
+      for (int64_t u = u0; u < u1; ++u)
+        for (int64_t e = row_ptr[u]; e < row_ptr[u + 1]; ++e)
+          if (wanted[col[e]]) { out_eid[p] = e; out_src[p] = u; ++p; }
+    }
+  }
+  free(cnt);
+  return total;
+}
+
+/* Completion rank of every vertex for an exact layer: max(v, largest in-neighbour of v) (Sect. 3.8, c(v) with the self
+ * message).  One pass over the CSR; the maximum is taken with a compare-and-swap so that the rows can be split among
+ * threads. */
+void to_completion_rank_exact(int64_t V, const int64_t* row_ptr, const int32_t* col, int32_t* rank /*[V]*/) {
+#pragma omp parallel for schedule(static)
+  for (int64_t v = 0; v < V; ++v) rank[v] = (int32_t)v;
+#pragma omp parallel for schedule(static, 4096)
+  for (int64_t u = 0; u < V; ++u)
+    for (int64_t e = row_ptr[u]; e < row_ptr[u + 1]; ++e) {
+      int32_t* p = &rank[col[e]];
+      int32_t old = __atomic_load_n(p, __ATOMIC_RELAXED);
+      while (old < (int32_t)u && !__atomic_compare_exchange_n(p, &old, (int32_t)u, 1, __ATOMIC_RELAXED, __ATOMIC_RELAXED)) {}
+    }
 }
 
 /* ------------------------------------------------------------------ sampling

@@ -236,3 +236,13 @@ def test_fewest_pending_reloads_less_than_fifo_and_random():
                for p in (oracle.EVICT_FEWEST_PENDING, oracle.EVICT_FIFO, oracle.EVICT_LRU, oracle.EVICT_RANDOM)}
     assert reloads[oracle.EVICT_FEWEST_PENDING] < reloads[oracle.EVICT_FIFO]
     assert reloads[oracle.EVICT_FEWEST_PENDING] < reloads[oracle.EVICT_RANDOM]
+
+
+def test_completion_rank_from_the_csr_equals_the_closed_form_over_the_in_lists():
+    V, E = 700, 6000
+    row_ptr, col, inl, ms, hub = _setup(V, E, 11)
+    rank = oracle.completion_rank_exact(V, row_ptr, col)
+    for chunk in (1, 7, 64):
+        assert (rank // chunk == oracle.complete_chunk_closed_form(ms, chunk)).all()
+    for v in range(0, V, 13):      # written out
+        assert rank[v] == max([v] + inl.src[inl.ptr[v]:inl.ptr[v + 1]].tolist())

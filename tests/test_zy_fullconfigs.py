@@ -1,9 +1,10 @@
 """The 'large', 'sampled' and 'stress' workloads at their FULL sizes (111 M / 269 M vertices, 1.6 B / 4 B edges).
 
-'large' and 'sampled' run by default, late in the collection order (two to four minutes each, about 100 GB of host
-memory and 130 GB of device memory); a machine with less prints why and skips.  TAURUS_FULL_CONFIGS selects other
-sets: a comma-separated list of workload names ("large,sampled,stress"; 'stress' takes five more minutes and
-160 GB of host memory, so it stays opt-in), or "none".
+All three run by default, late in the collection order (two to four minutes each, 110-165 GB of host memory and
+125-145 GB of device memory); a machine with less prints why and skips.  'large' and 'sampled' run their first and
+last layer; 'stress' runs its last layer by default and its first one (512 input columns: the host needs two and a
+half minutes to generate the 551 GB of feature rows) as well with TAURUS_FULL_STRESS_LAYERS=all.  TAURUS_FULL_CONFIGS
+selects a subset: a comma-separated list of workload names, or "none".
 
 At these sizes the full oracle is out of reach, so the checks are
   * output rows of a destination sample (random vertices + the largest hubs) against the oracle's pull-based
@@ -26,7 +27,7 @@ import taurus_gen as tg
 
 pytestmark = pytest.mark.gpu
 
-WANTED = [x for x in os.environ.get("TAURUS_FULL_CONFIGS", "large,sampled").split(",") if x]
+WANTED = [x for x in os.environ.get("TAURUS_FULL_CONFIGS", "large,sampled,stress").split(",") if x]
 HOST_GB = {"large": 110, "sampled": 130, "stress": 165}      # host memory (graph, check arrays, pinned evicted-row store)
 DEVICE_GB = {"large": 125, "sampled": 140, "stress": 145}
 
@@ -74,22 +75,19 @@ def test_full_config(name):
     V, chunk = g.V, w.chunk
     print("%s: V %d E %d max in-degree %d built in %.0f s" % (name, V, g.E, int(g.in_degree.max()), time.time() - t0), flush=True)
     model = tg.make_model(w, bias_scale=0.2)
-    src_of_edge = np.repeat(np.arange(V, dtype=np.int32), np.diff(g.row_ptr))
-    # closed form of the completion chunk for exact layers (edges are stored in ascending source order, so the last
-    # assignment to a destination is its largest in-neighbour)
-    last = np.arange(V, dtype=np.int32)
-    last[g.col_idx] = src_of_edge
-    np.maximum(last, np.arange(V, dtype=np.int32), out=last)
+    # closed form of the completion chunk for exact layers: max(v, largest in-neighbour)
+    last = oracle.completion_rank_exact(V, g.row_ptr, g.col_idx)
     rng = np.random.default_rng(0)
     n_hubs = 2 if w.dims[0] >= 512 else 16      # the hubs' in-neighbour rows must fit in host memory as fp64
-    dsts = np.unique(np.concatenate([np.argsort(-g.in_degree)[:n_hubs], rng.integers(0, V, 4096)])).astype(np.int64)
+    top = np.argpartition(-g.in_degree, n_hubs)[:n_hubs]
+    dsts = np.unique(np.concatenate([top, rng.integers(0, V, 4096)])).astype(np.int64)
     ptr, src, eid = oracle.subset_in_lists(V, g.row_ptr, g.col_idx, dsts)
     assert (np.diff(ptr) == g.in_degree[dsts]).all()
     has = np.diff(ptr) > 0        # the closed form against the in-lists of the sample: largest in-neighbour = last entry
     assert (last[dsts[has]] == np.maximum(dsts[has], src[ptr[1:][has] - 1])).all() and (last[dsts[~has]] == dsts[~has]).all()
     n_chunks = (V + chunk - 1) // chunk
     completed_closed_form = np.bincount(last // chunk, minlength=n_chunks)
-    del last, src_of_edge
+    del last
     print("subset in-lists: %d destinations, %d in-edges, %.0f s" % (dsts.size, src.size, time.time() - t0), flush=True)
     full_inl = None
     if any(f > 0 for f in w.fanout):     # the oracle's own in-lists of the whole graph, for the full-mask comparison
@@ -105,6 +103,8 @@ def test_full_config(name):
     dsts_dev = torch.from_numpy(dsts).to(dev)
     tol = 2e-2 if w.gemm_mode == tg.GEMM_BF16 else 1e-4
     layers = [0, w.L - 1]
+    if base == "stress" and os.environ.get("TAURUS_FULL_STRESS_LAYERS", "last") != "all":
+        layers = [w.L - 1]
     stream = torch.cuda.current_stream()
     for l in layers:
         d_in, d_out = w.dims[l], w.dims[l + 1]
