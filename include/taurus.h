@@ -96,6 +96,9 @@ typedef struct {
   const float* const* att_src; /* TAURUS_GAT only: [L] each dims[l+1], the half of the attention vector applied to the source */
   const float* const* att_dst; /* TAURUS_GAT only: [L] each dims[l+1], the half applied to the destination      */
   float leaky_slope;           /* TAURUS_GAT only: negative slope of the LeakyReLU on the scores, in [0, 1]     */
+  int32_t gat_heads;           /* TAURUS_GAT only: attention heads, 0 or 1 = one.  Head i owns columns [i d, (i+1) d) of
+                                  W_neigh[l], att_src[l], att_dst[l], bias[l] and of the layer's output, d = dims[l+1] / heads
+                                  (every dims[l+1] must be a multiple of 4 * heads); the heads' outputs are concatenated */
 } taurus_model;
 
 typedef struct {
@@ -189,8 +192,9 @@ int taurus_layer_begin(taurus_ctx* ctx, int32_t layer, void* cuda_stream);
 int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream);
 
 /*
- * GATConv in three sequential passes (GATConv paragraph of Sect. 3.9); contexts created with TAURUS_GAT, one
- * attention head (several heads are several contexts), fp32 projection only.  With h' = h W,
+ * GATConv in three sequential passes (GATConv paragraph of Sect. 3.9); contexts created with TAURUS_GAT, fp32
+ * projection only.  One head or several (taurus_model.gat_heads: "the same procedure applies per head"; one pass over
+ * the topology serves all heads, each head weighting its own block of columns).  Per head, with h' = h W,
  *     e_uv = LeakyReLU(att_src . h'_u + att_dst . h'_v),  alpha_uv = softmax over u in N(v) of e_uv,
  *     out_v = act(sum_{u in N(v)} alpha_uv h'_u + b),
  * where N(v) is the propagated in-multiset of v (all in-edges, or the layer's sampled ones) plus v itself:
@@ -198,7 +202,7 @@ int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const
  *   pass 1  taurus_gat_project_chunk for every chunk in ascending, contiguous order: writes the rows pass 3 will
  *           stream for sources [src_begin, src_end) to hprime_out (DEVICE memory, row i at hprime_out + i * ld,
  *           ld >= dims[layer+1] floats, dims[layer+1] floats per row) and keeps the two scalars att_src . h'_u and
- *           att_dst . h'_u of every vertex.  The rows are the transformed rows h'; in a layer that aggregates input
+ *           att_dst . h'_u of every vertex (per head).  The rows are the transformed rows h'; in a layer that aggregates input
  *           rows first (see TAURUS_FLAG_PROJECT_FIRST) they are the input rows, zero-padded, and h' is never formed:
  *           the caller treats them as opaque.  `features` as in taurus_push_chunk.  Asynchronous on the stream.
  *   pass 2  taurus_gat_attention, once all vertices are projected: a topology-only sweep over the CSR that

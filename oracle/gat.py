@@ -9,7 +9,9 @@ The definition, pull-based and in fp64, one destination at a time:
 
 N(v) is the propagated in-multiset M(v) (all in-edges, or the sampled ones; a multi-edge counts once per
 copy) together with v itself: every vertex aggregates a self message (Sect. 3.8), so a vertex without
-in-edges keeps act(h'_v + b).  One attention head; several heads are several calls.
+in-edges keeps act(h'_v + b).  gat_layer_forward is one attention head; gat_layer_forward_heads applies the same
+procedure per head ("the same procedure applies per head", Sect. 3.9) to column blocks of W, a_src, a_dst and b and
+concatenates the heads' outputs.
 
 Pins (tests/test_oracle_gat.py): two hand-worked examples (tests/golden/gat_example.txt), a dense masked
 softmax on tiny multigraphs, uniform attention when a = 0 (a plain mean, checked against the C aggregator),
@@ -52,3 +54,17 @@ def gat_layer_forward(ms, h: np.ndarray, W: np.ndarray, a_src: np.ndarray, a_dst
         if magnitude:
             mag[i] = alpha @ hp_abs[nb] + np.abs(b)
     return (out, mag) if magnitude else out
+
+
+def gat_layer_forward_heads(ms, h: np.ndarray, W: np.ndarray, a_src: np.ndarray, a_dst: np.ndarray, bias: np.ndarray, act: int,
+                            heads: int, slope: float = 0.2, dst: Optional[np.ndarray] = None, magnitude: bool = False):
+    """Several heads: head i owns columns [i * d, (i + 1) * d) of W, a_src, a_dst and bias (d = columns / heads) and is
+    one call of gat_layer_forward; the outputs are concatenated in head order."""
+    W = np.asarray(W)
+    d = W.shape[1] // heads
+    assert d * heads == W.shape[1]
+    outs = [gat_layer_forward(ms, h, W[:, i * d:(i + 1) * d], np.asarray(a_src)[i * d:(i + 1) * d], np.asarray(a_dst)[i * d:(i + 1) * d],
+                              np.asarray(bias)[i * d:(i + 1) * d], act, slope, dst, magnitude) for i in range(heads)]
+    if magnitude:
+        return np.concatenate([o[0] for o in outs], axis=1), np.concatenate([o[1] for o in outs], axis=1)
+    return np.concatenate(outs, axis=1)

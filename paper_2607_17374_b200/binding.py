@@ -49,7 +49,7 @@ class _Model(ctypes.Structure):
                 ("bias", ctypes.POINTER(ctypes.c_void_p)), ("act", ctypes.POINTER(ctypes.c_int32)),
                 ("gemm_mode", ctypes.c_int32), ("gin_eps", ctypes.c_float),
                 ("att_src", ctypes.POINTER(ctypes.c_void_p)), ("att_dst", ctypes.POINTER(ctypes.c_void_p)),
-                ("leaky_slope", ctypes.c_float)]
+                ("leaky_slope", ctypes.c_float), ("gat_heads", ctypes.c_int32)]
 
 
 class _Run(ctypes.Structure):
@@ -287,7 +287,7 @@ class Context:
                  bias, act: Sequence[int], chunk_sources: int, pool_slots: int, hub_count: int = 0,
                  fanout: Optional[Sequence[int]] = None, seed: int = 1, host_evict_rows: int = 0, drain_rows: int = 0,
                  gemm_mode: int = GEMM_FP32, flags: int = 0, evict_policy: int = 0, gin_eps: float = 0.0,
-                 att_src=None, att_dst=None, leaky_slope: float = 0.2):
+                 att_src=None, att_dst=None, leaky_slope: float = 0.2, gat_heads: int = 1):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         L = len(dims) - 1
@@ -302,7 +302,7 @@ class Context:
         c_as = (ctypes.c_void_p * L)(*[_ptr(a) for a in att_src]) if att_src is not None else None
         c_ad = (ctypes.c_void_p * L)(*[_ptr(a) for a in att_dst]) if att_dst is not None else None
         keep += [att_src, att_dst]
-        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode, gin_eps, c_as, c_ad, leaky_slope)
+        m = _Model(mode, L, c_dims, c_wn, c_ws, c_b, c_act, gemm_mode, gin_eps, c_as, c_ad, leaky_slope, gat_heads)
         c_f = (ctypes.c_int32 * L)(*[int(f) for f in fanout]) if fanout is not None else None
         r = _Run(chunk_sources, pool_slots, hub_count, c_f, seed, host_evict_rows, drain_rows or chunk_sources, flags, evict_policy)
         rc = self._lib.taurus_graph_init(ctypes.byref(self._h), ctypes.byref(g), ctypes.byref(m), ctypes.byref(r))

@@ -178,7 +178,7 @@ int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long r
     } else if (sage) {
       launch_gemm_plain_simt(c, c->d_Waf[layer], a.Hout, a.Hout, c->d_af_A, Ka, Ka, (int)rows, O, a.Hout, st);
     } else {
-      launch_gemm_plain_simt(c, c->d_Wcat[layer], taurus_proj_width(c->mode, a.Hout), a.Hout, c->d_af_A, Ka, c->dims[layer], (int)rows, O,
+      launch_gemm_plain_simt(c, c->d_Wcat[layer], taurus_proj_width(c->mode, a.Hout, c->heads), a.Hout, c->d_af_A, Ka, c->dims[layer], (int)rows, O,
                              a.Hout, st);
     }
     af_finish_kernel<<<grid, 256, 0, st>>>(a, O, rows);

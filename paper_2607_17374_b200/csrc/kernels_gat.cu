@@ -21,7 +21,8 @@ __device__ __forceinline__ void atomic_max_float(float* addr, float v) {
   else atomicMin(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
 }
 
-__global__ void gat_split_kernel(const float* __restrict__ PT, int ldpt, int n, int Hp, int d_out, long long src_begin,
+// The per-vertex scalars are stored [V x heads]: head h of vertex v at v * heads + h.
+__global__ void gat_split_kernel(const float* __restrict__ PT, int ldpt, int n, int Hp, int d_out, int heads, long long src_begin,
                                  float* __restrict__ hprime, long long ld, float* __restrict__ att_s, float* __restrict__ att_t,
                                  float* __restrict__ att_max) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -29,29 +30,32 @@ __global__ void gat_split_kernel(const float* __restrict__ PT, int ldpt, int n, 
     const float* src = PT + (size_t)r * ldpt;
     float* dst = hprime + (size_t)r * ld;
     for (int k = gl(); k < d_out; k += 32) dst[k] = src[k];
-    if (gl() == 0) {
-      const float s = src[Hp], t = src[Hp + 1];
-      att_s[src_begin + r] = s;
-      att_t[src_begin + r] = t;
-      att_max[src_begin + r] = s;   // the self message takes part in the maximum
+    if (gl() < heads) {
+      const float s = src[Hp + 2 * gl()], t = src[Hp + 2 * gl() + 1];
+      const size_t at = (size_t)(src_begin + r) * heads + gl();
+      att_s[at] = s;
+      att_t[at] = t;
+      att_max[at] = s;   // the self message takes part in the maximum
     }
   }
 }
 
 // max over propagated in-edges (u -> v) of s_u, one warp per source row
-__global__ void gat_edge_max_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
+__global__ void gat_edge_max_kernel(long long V, int heads, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
                                     const uint32_t* __restrict__ mask, const float* __restrict__ att_s, float* __restrict__ att_max) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
-    const float s = att_s[u];
     for (long long e = row_ptr[u] + gl(); e < row_ptr[u + 1]; e += 32)
-      if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) atomic_max_float(&att_max[col[e]], s);
+      if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) {
+        const size_t v = (size_t)col[e] * heads;
+        for (int h = 0; h < heads; ++h) atomic_max_float(&att_max[v + h], att_s[(size_t)u * heads + h]);
+      }
   }
 }
 
 // tm[v] = (t_v, LeakyReLU(max_u s_u + t_v));  z[v] starts with the self term
 __global__ void gat_tm_kernel(long long V, const float* __restrict__ att_s, const float* __restrict__ att_t,
-                              const float* __restrict__ att_max, float slope, float2* __restrict__ tm, float* __restrict__ z) {
+                              const float* __restrict__ att_max, float slope, float2* __restrict__ tm, float* __restrict__ z) {   // V = vertices x heads
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
     const float t = att_t[v];
@@ -61,17 +65,18 @@ __global__ void gat_tm_kernel(long long V, const float* __restrict__ att_s, cons
   }
 }
 
-__global__ void gat_edge_sum_kernel(long long V, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
+__global__ void gat_edge_sum_kernel(long long V, int heads, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
                                     const uint32_t* __restrict__ mask, const float* __restrict__ att_s,
                                     const float2* __restrict__ tm, float slope, float* __restrict__ z) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
-    const float s = att_s[u];
     for (long long e = row_ptr[u] + gl(); e < row_ptr[u + 1]; e += 32)
       if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) {
-        const int v = col[e];
-        const float2 x = tm[v];
-        atomicAdd(&z[v], __expf(lrelu(s + x.x, slope) - x.y));
+        const size_t v = (size_t)col[e] * heads;
+        for (int h = 0; h < heads; ++h) {
+          const float2 x = tm[v + h];
+          atomicAdd(&z[v + h], __expf(lrelu(att_s[(size_t)u * heads + h] + x.x, slope) - x.y));
+        }
       }
   }
 }
@@ -110,8 +115,8 @@ __global__ void gat_repack_kernel(const float* __restrict__ X, int n, int d_out,
 }  // namespace
 
 void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st) {
-  gat_split_kernel<<<c->sm_count * 8, 256, 0, st>>>(c->d_PT, Hp + 4, n, Hp, d_out, src_begin, hprime_out, ld, c->d_att_s, c->d_att_t,
-                                                    c->d_att_max);
+  gat_split_kernel<<<c->sm_count * 8, 256, 0, st>>>(c->d_PT, taurus_proj_width(TAURUS_GAT, Hp, c->heads), n, Hp, d_out, c->heads, src_begin,
+                                                    hprime_out, ld, c->d_att_s, c->d_att_t, c->d_att_max);
   c->launches += 1;
 }
 
@@ -125,9 +130,9 @@ void launch_gat_scores(taurus_ctx* c, int layer, const float* X, int ldx, int n,
 
 void launch_gat_attention(taurus_ctx* c, cudaStream_t st) {
   const int grid = c->sm_count * 8;
-  gat_edge_max_kernel<<<grid, 256, 0, st>>>(c->V, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_max);
-  gat_tm_kernel<<<grid, 256, 0, st>>>(c->V, c->d_att_s, c->d_att_t, c->d_att_max, c->leaky, c->d_att_tm, c->d_att_z);
-  gat_edge_sum_kernel<<<grid, 256, 0, st>>>(c->V, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_tm, c->leaky, c->d_att_z);
+  gat_edge_max_kernel<<<grid, 256, 0, st>>>(c->V, c->heads, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_max);
+  gat_tm_kernel<<<grid, 256, 0, st>>>(c->V * c->heads, c->d_att_s, c->d_att_t, c->d_att_max, c->leaky, c->d_att_tm, c->d_att_z);
+  gat_edge_sum_kernel<<<grid, 256, 0, st>>>(c->V, c->heads, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_tm, c->leaky, c->d_att_z);
   c->launches += 3;
 }
 

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(256) project_simt_kernel(const float* __restri
 
 void launch_project_simt(taurus_ctx* c, int layer, const float* X, int ldx, long long src_begin, int n, cudaStream_t st) {
   const int Hp = taurus_round_up(c->dims[layer + 1], 4);
-  const int N = taurus_proj_width(c->mode, Hp);
+  const int N = taurus_proj_width(c->mode, Hp, c->heads);
   dim3 grid((N + BN - 1) / BN, (n + BM - 1) / BM);
   project_simt_kernel<<<grid, 256, 0, st>>>(X, ldx, c->dims[layer], c->d_Wcat[layer], N, N, c->d_PT, N, n, Hp, c->mode,
                                             c->d_bias[layer], c->d_row_ptr, c->d_din, c->fanout[layer], src_begin);

@@ -522,7 +522,7 @@ int launch_project_tc(taurus_ctx* c, int layer, const float* X, int ldx, long lo
   const bool bf16 = c->gemm_mode == TAURUS_GEMM_BF16;
   WImage* w = static_cast<WImage*>(c->tc_image[layer]);
   const int K = c->dims[layer], Hp = taurus_round_up(c->dims[layer + 1], 4);
-  const int N = taurus_proj_width(c->mode, Hp);
+  const int N = taurus_proj_width(c->mode, Hp, c->heads);
   CUtensorMap map_x;
   if (!make_map(&map_x, X, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, n, K, ldx, BM, bf16 ? 32 : KS32)) return TAURUS_ERR_CUDA;
   CUtensorMap map_out;

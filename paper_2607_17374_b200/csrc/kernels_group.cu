@@ -272,7 +272,9 @@ void launch_classify_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st)
 
 // With GAT every message is weighted by exp(LeakyReLU(s_u + t_v) - max_v), recomputed from per-vertex scalars
 // (the 1 / normaliser factor is applied at finalise).
-template <int LPE, int VPL, bool SAMPLED, bool DIRECT, bool GAT>
+// GAT: 0 no attention, 1 one head (one weight per message), 2 several heads (each lane weights its float4 columns by the
+// coefficient of the head they belong to; the per-vertex scalars are [V x heads]).
+template <int LPE, int VPL, bool SAMPLED, bool DIRECT, int GAT>
 __global__ void __launch_bounds__(256, (VPL <= 2 ? 3 : VPL == 3 ? 2 : 1))
 scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint32_t* __restrict__ gmask) {
   DevCtl* ctl = a.ctl;
@@ -299,7 +301,11 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
 
   int cur = -1, cnt = 0, cur_loc = -1;
   float2 cur_tm = make_float2(0.f, 0.f);
-  const float* const att_s_chunk = GAT ? a.att_s + a.src_begin : nullptr;
+  float2 head_tm[VPL];     // several heads: (t, maximum score) of the current destination for the head of each float4 of this lane
+  int hk[VPL];             //                head of each float4 of this lane
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) { hk[k] = GAT == 2 ? (c4 + k * LPE) / a.head_vec : 0; if (hk[k] >= a.heads) hk[k] = a.heads - 1; head_tm[k] = make_float2(0.f, 0.f); }
+  const float* const att_s_chunk = GAT ? a.att_s + (size_t)a.src_begin * (GAT == 2 ? a.heads : 1) : nullptr;
   float4 sum[VPL];
   // byte addressing with 32-bit x 32-bit -> 64-bit products keeps the address arithmetic to one instruction
   const char* const Pb = reinterpret_cast<const char*>(a.PT) + c4 * 16;
@@ -325,12 +331,23 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
     const float e = att_s_chunk[src_rel] + cur_tm.x;
     return __expf((e > 0.f ? e : a.leaky * e) - cur_tm.y);
   };
+  auto weight_of_head = [&](int src_rel, int k) {   // the same for the head of this lane's k-th float4
+    const float e = att_s_chunk[(size_t)src_rel * a.heads + hk[k]] + head_tm[k].x;
+    return __expf((e > 0.f ? e : a.leaky * e) - head_tm[k].y);
+  };
   auto take = [&](int d, int src_rel, const float4 (&row)[VPL]) {
     if (d != cur) {
       if (cur >= 0) flush();
       cur = d; cnt = 1;
       if (!DIRECT) cur_loc = a.loc[d];
-      if (GAT) {
+      if (GAT == 2) {
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          head_tm[k] = a.att_tm[(size_t)d * a.heads + hk[k]];
+          const float w = weight_of_head(src_rel, k);
+          sum[k] = make_float4(w * row[k].x, w * row[k].y, w * row[k].z, w * row[k].w);
+        }
+      } else if (GAT) {
         cur_tm = a.att_tm[d];
         const float w = weight(src_rel);
 #pragma unroll
@@ -341,7 +358,14 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
       }
     } else {
       cnt++;
-      if (GAT) {
+      if (GAT == 2) {
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          const float w = weight_of_head(src_rel, k);
+          sum[k].x = fmaf(w, row[k].x, sum[k].x); sum[k].y = fmaf(w, row[k].y, sum[k].y);
+          sum[k].z = fmaf(w, row[k].z, sum[k].z); sum[k].w = fmaf(w, row[k].w, sum[k].w);
+        }
+      } else if (GAT) {
         const float w = weight(src_rel);
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
@@ -446,7 +470,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
         float ps = 1.0f, sc = 1.0f;
         if (a.mode == TAURUS_GIN_SUM) ps = a.gin_self;
         else if (a.mode == TAURUS_GCN_SYM) sc = (float)sqrt((double)a.din[vj] + 1.0);
-        else {
+        else if (GAT != 2) {
           const float2 tm = a.att_tm[vj];
           const float e = a.att_s[vj] + tm.x;
           ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
@@ -456,6 +480,13 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
 #pragma unroll
         for (int k = 0; k < VPL; ++k)
           if (c4 + k * LPE < nvec) {
+            if (GAT == 2) {                     // the head of these columns
+              const size_t at = (size_t)vj * a.heads + hk[k];
+              const float2 tm = a.att_tm[at];
+              const float e = a.att_s[at] + tm.x;
+              ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
+              sc = a.self_bias ? a.att_z[at] : 0.f;
+            }
             float4 xx = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
             float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];
             red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(xx.x * ps + b.x * sc, xx.y * ps + b.y * sc, xx.z * ps + b.z * sc, xx.w * ps + b.w * sc));
@@ -478,7 +509,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
   }
 }
 
-template <int LPE, int VPL, bool SAMPLED, bool DIRECT, bool GAT>
+template <int LPE, int VPL, bool SAMPLED, bool DIRECT, int GAT>
 static void launch_sg(taurus_ctx* c, const ChunkArgs& a, const uint32_t* gm, cudaStream_t st) {
   static int blocks_per_sm = 0;
   if (blocks_per_sm == 0) {
@@ -493,13 +524,18 @@ template <int LPE, int VPL>
 static void launch_sg2(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {
   const uint32_t* gm = c->d_mask_cur ? c->d_gmask : nullptr;
   const bool direct = a.direct && c->hub_count == 0;
-  if (a.mode == TAURUS_GAT) {   // attention-weighted variants
-    if (gm) { if (direct) launch_sg<LPE, VPL, true, true, true>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, true>(c, a, gm, st); }
-    else    { if (direct) launch_sg<LPE, VPL, false, true, true>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, true>(c, a, gm, st); }
+  if (a.mode == TAURUS_GAT && a.heads > 1) {   // attention-weighted, one coefficient per head
+    if (gm) { if (direct) launch_sg<LPE, VPL, true, true, 2>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, 2>(c, a, gm, st); }
+    else    { if (direct) launch_sg<LPE, VPL, false, true, 2>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, 2>(c, a, gm, st); }
     return;
   }
-  if (gm) { if (direct) launch_sg<LPE, VPL, true, true, false>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, false>(c, a, gm, st); }
-  else    { if (direct) launch_sg<LPE, VPL, false, true, false>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, false>(c, a, gm, st); }
+  if (a.mode == TAURUS_GAT) {   // attention-weighted variants
+    if (gm) { if (direct) launch_sg<LPE, VPL, true, true, 1>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, 1>(c, a, gm, st); }
+    else    { if (direct) launch_sg<LPE, VPL, false, true, 1>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, 1>(c, a, gm, st); }
+    return;
+  }
+  if (gm) { if (direct) launch_sg<LPE, VPL, true, true, 0>(c, a, gm, st); else launch_sg<LPE, VPL, true, false, 0>(c, a, gm, st); }
+  else    { if (direct) launch_sg<LPE, VPL, false, true, 0>(c, a, gm, st); else launch_sg<LPE, VPL, false, false, 0>(c, a, gm, st); }
 }
 
 void launch_scatter_grouped(taurus_ctx* c, const ChunkArgs& a, cudaStream_t st) {

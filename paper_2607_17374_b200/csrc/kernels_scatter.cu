@@ -100,7 +100,8 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
       }
       // GAT: weight of this lane's message, exp(LeakyReLU(s_u + t_v) - max_v)
       float wgt = 1.f;
-      if (a.mode == TAURUS_GAT && v >= 0 && !self_run) {
+      const bool multi = a.mode == TAURUS_GAT && a.heads > 1;   // several heads: the weights are taken per float4 column below
+      if (a.mode == TAURUS_GAT && !multi && v >= 0 && !self_run) {
         const float2 tm = a.att_tm[v];
         const float e = a.att_s[src] + tm.x;
         wgt = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
@@ -126,6 +127,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
         const int lj = __shfl_sync(FULL, l, j);
         const long long sj = __shfl_sync(FULL, src, j);
         const float wj = __shfl_sync(FULL, wgt, j);
+        const int vj = __shfl_sync(FULL, v, j);
         if (lj < 0) continue;
         if (self_run && !a.self_rows) continue;   // aggregate-first SAGE: the self message is only counted
         if (sj != held) {
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
               float ps = 1.0f, s = 1.0f;
               if (a.mode == TAURUS_GIN_SUM) ps = a.gin_self;
               else if (a.mode == TAURUS_GCN_SYM) s = (float)sqrt((double)a.din[sj] + 1.0);
-              else {
+              else if (!multi) {
                 const float2 tm = a.att_tm[sj];
                 const float e = a.att_s[sj] + tm.x;
                 ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
@@ -153,6 +155,13 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
 #pragma unroll
               for (int k = 0; k < VPL; ++k)
                 if (c4 + k * LPE < nvec) {
+                  if (multi) {                    // the head of these columns
+                    const size_t at = (size_t)sj * a.heads + (c4 + k * LPE) / a.head_vec;
+                    const float2 tm = a.att_tm[at];
+                    const float e = a.att_s[at] + tm.x;
+                    ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
+                    s = a.self_bias ? a.att_z[at] : 0.f;
+                  }
                   float4 x = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
                   float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];
                   row[k] = make_float4(x.x * ps + b.x * s, x.y * ps + b.y * s, x.z * ps + b.z * s, x.w * ps + b.w * s);
@@ -165,7 +174,17 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
           }
         }
         float* dst = a.acc + (size_t)lj * a.Hp;
-        if (a.mode == TAURUS_GAT && !self_run) {
+        if (multi && !self_run) {
+#pragma unroll
+          for (int k = 0; k < VPL; ++k)
+            if (c4 + k * LPE < nvec) {
+              const int hd = (c4 + k * LPE) / a.head_vec;
+              const float2 tm = a.att_tm[(size_t)vj * a.heads + hd];
+              const float e = a.att_s[(size_t)sj * a.heads + hd] + tm.x;
+              const float wk = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
+              red_add_v4(dst + 4 * (c4 + k * LPE), make_float4(row[k].x * wk, row[k].y * wk, row[k].z * wk, row[k].w * wk));
+            }
+        } else if (a.mode == TAURUS_GAT && !self_run) {
 #pragma unroll
           for (int k = 0; k < VPL; ++k)
             if (c4 + k * LPE < nvec)

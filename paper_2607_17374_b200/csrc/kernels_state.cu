@@ -910,7 +910,9 @@ __global__ void finalise_kernel(ChunkArgs a) {
           const int k = k0 + q * 32 + lane_id();
           if (k >= vec) continue;
           float4 y = x[q];
-          y.x *= sj; y.y *= sj; y.z *= sj; y.w *= sj;
+          float sk = sj;
+          if (a.mode == TAURUS_GAT && a.heads > 1) sk = 1.0f / a.att_z[(size_t)vj * a.heads + k / a.head_vec];   // normaliser of the column's head
+          y.x *= sk; y.y *= sk; y.z *= sk; y.w *= sk;
           if (a.act) { y.x = fmaxf(y.x, 0.f); y.y = fmaxf(y.y, 0.f); y.z = fmaxf(y.z, 0.f); y.w = fmaxf(y.w, 0.f); }
           const int c0 = k << 2;
           if (!a.dense_direct || (vec_ok && c0 + 3 < a.d_out)) {

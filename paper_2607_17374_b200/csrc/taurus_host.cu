@@ -112,6 +112,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   c->seed = r->seed;
   c->gin_eps = m->gin_eps;
   c->leaky = m->leaky_slope;
+  c->heads = (m->mode == TAURUS_GAT && m->gat_heads > 1) ? m->gat_heads : 1;
   c->chunk_sources = r->chunk_sources; c->pool_slots = r->pool_slots; c->hub_count = r->hub_count;
   c->host_rows = r->host_evict_rows; c->drain_rows = r->drain_rows; c->evict_policy = r->evict_policy;
   bool any_sampled = false;
@@ -170,6 +171,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   for (int l = 0; l < c->L; ++l) {
     const int Kp = taurus_round_up(c->dims[l], 4), Hp = taurus_round_up(c->dims[l + 1], 4);
     bool af = !(c->flags & TAURUS_FLAG_PROJECT_FIRST) && 4 * Kp <= 3 * Hp;
+    if (c->heads > 1) af = false;   // every head weights the messages differently: the sums cannot be shared in input space
     // SAGE keeps V input rows on the device for such a layer: only while they fit beside everything else
     if (af && c->mode == TAURUS_SAGE_MEAN && (double)V * Kp * sizeof(float) + other > 0.92 * (double)free_b) af = false;
     c->agg_first[l] = af;
@@ -179,7 +181,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
   // weights: Wcat = [W_neigh | W_self] with both halves padded to Hp columns
   for (int l = 0; l < c->L; ++l) {
     const int K = c->dims[l], d_out = c->dims[l + 1], Hp = taurus_round_up(d_out, 4);
-    const int N = taurus_proj_width(c->mode, Hp);
+    const int N = taurus_proj_width(c->mode, Hp, c->heads);
     std::vector<float> wn((size_t)K * d_out), ws, b((size_t)Hp, 0.f), cat((size_t)K * N, 0.f);
     CU(cudaMemcpy(wn.data(), m->W_neigh[l], wn.size() * sizeof(float), cudaMemcpyDefault));
     if (c->mode == TAURUS_SAGE_MEAN) {
@@ -192,16 +194,18 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
         cat[(size_t)k * N + j] = wn[(size_t)k * d_out + j];
         if (c->mode == TAURUS_SAGE_MEAN) cat[(size_t)k * N + Hp + j] = ws[(size_t)k * d_out + j];
       }
-    if (c->mode == TAURUS_GAT) {   // two more columns, W att_src and W att_dst: the attention scalars come out of the same GEMM
+    if (c->mode == TAURUS_GAT) {   // two more columns per head, W att_src and W att_dst over the head's block: the attention scalars come out of the same GEMM
       std::vector<float> as((size_t)d_out), ad((size_t)d_out);
       CU(cudaMemcpy(as.data(), m->att_src[l], as.size() * sizeof(float), cudaMemcpyDefault));
       CU(cudaMemcpy(ad.data(), m->att_dst[l], ad.size() * sizeof(float), cudaMemcpyDefault));
-      for (int k = 0; k < K; ++k) {
-        double ss = 0.0, sd = 0.0;
-        for (int j = 0; j < d_out; ++j) { ss += (double)wn[(size_t)k * d_out + j] * as[(size_t)j]; sd += (double)wn[(size_t)k * d_out + j] * ad[(size_t)j]; }
-        cat[(size_t)k * N + Hp] = (float)ss;
-        cat[(size_t)k * N + Hp + 1] = (float)sd;
-      }
+      const int dh = d_out / c->heads;
+      for (int k = 0; k < K; ++k)
+        for (int hd = 0; hd < c->heads; ++hd) {
+          double ss = 0.0, sd = 0.0;
+          for (int j = hd * dh; j < (hd + 1) * dh; ++j) { ss += (double)wn[(size_t)k * d_out + j] * as[(size_t)j]; sd += (double)wn[(size_t)k * d_out + j] * ad[(size_t)j]; }
+          cat[(size_t)k * N + Hp + 2 * hd] = (float)ss;
+          cat[(size_t)k * N + Hp + 2 * hd + 1] = (float)sd;
+        }
       std::vector<float> wv((size_t)2 * K);   // the same two vectors on their own, for layers that never form the transformed rows
       for (int k = 0; k < K; ++k) { wv[(size_t)k] = cat[(size_t)k * N + Hp]; wv[(size_t)K + k] = cat[(size_t)k * N + Hp + 1]; }
       ALLOC(c->d_att_w[l], wv.size());
@@ -296,7 +300,10 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     CU(cudaEventCreateWithFlags(&c->out_done[i], cudaEventDisableTiming));
   }
   ALLOC(c->d_PT, (size_t)c->chunk_sources * 2 * c->Hmax);
-  if (c->mode == TAURUS_GAT) { ALLOC(c->d_att_s, V); ALLOC(c->d_att_t, V); ALLOC(c->d_att_max, V); ALLOC(c->d_att_tm, V); ALLOC(c->d_att_z, V); }
+  if (c->mode == TAURUS_GAT) {
+    const size_t nh = (size_t)V * c->heads;
+    ALLOC(c->d_att_s, nh); ALLOC(c->d_att_t, nh); ALLOC(c->d_att_max, nh); ALLOC(c->d_att_tm, nh); ALLOC(c->d_att_z, nh);
+  }
   if (af_kmax > 0) {
     const bool sage = c->mode == TAURUS_SAGE_MEAN;
     ALLOC(c->d_af_A, (size_t)c->drain_rows * af_kmax * (sage ? 2 : 1));
@@ -356,6 +363,10 @@ extern "C" int taurus_graph_init(taurus_ctx** out, const taurus_graph* g, const 
   if (m->mode == TAURUS_GAT) {
     if (!m->att_src || !m->att_dst || !(m->leaky_slope >= 0.f && m->leaky_slope <= 1.f)) return TAURUS_ERR_INVALID_ARG;
     if (m->gemm_mode != TAURUS_GEMM_FP32) return TAURUS_ERR_UNSUPPORTED;   // the scores need the fp32-accurate projection
+    if (m->gat_heads < 0 || m->gat_heads > 16) return TAURUS_ERR_INVALID_ARG;
+    if (m->gat_heads > 1)
+      for (int l = 0; l < m->L; ++l)
+        if (m->dims[l + 1] % (4 * m->gat_heads) != 0) return TAURUS_ERR_INVALID_ARG;   // a head is a whole number of float4
     for (int l = 0; l < m->L; ++l)
       if (!m->att_src[l] || !m->att_dst[l]) return TAURUS_ERR_INVALID_ARG;
   }
@@ -468,6 +479,7 @@ static ChunkArgs make_args(taurus_ctx* c, long long s, long long e) {
   a.Hp = taurus_round_up(c->dims[l + 1], 4);
   a.PT = c->d_PT; a.ldpt = c->mode == TAURUS_SAGE_MEAN ? 2 * a.Hp : a.Hp;   // GAT pass 3 scatters h' rows repacked to pitch Hp
   a.att_s = c->d_att_s; a.att_tm = c->d_att_tm; a.att_z = c->d_att_z; a.leaky = c->leaky;
+  a.heads = c->heads; a.head_vec = (taurus_round_up(c->dims[l + 1], 4) / c->heads) >> 2;
   a.bias = c->d_bias[l];
   a.ctl = c->d_ctl; a.pc = &c->d_ctl->pc[c->chunk_seq & 1]; a.chunk_log = c->d_chunk_log; a.log_capacity = c->log_capacity;
   a.V = c->V; a.pool_slots = c->pool_slots; a.hub_count = c->hub_count; a.host_rows = c->host_rows; a.drain_rows = c->drain_rows;

@@ -138,6 +138,8 @@ struct ChunkArgs {
   const float2* att_tm;     // [V] (att_dst . h'_v, maximum score of v's neighbourhood)
   const float* att_z;       // [V] softmax normaliser
   float leaky;              // LeakyReLU slope
+  int32_t heads;            // GAT: attention heads (the per-vertex scalars are [V x heads])
+  int32_t head_vec;         // GAT: float4 per head (d_head / 4)
   unsigned long long seed;
   long long grad_off;       // dense-output mode: first row of this chunk's half of the graduation buffer
   long long grad_cap;       // rows the chunk may write (drain_rows, or half of it in dense-output mode)
@@ -203,6 +205,7 @@ struct taurus_ctx {
   float gin_eps = 0.f;
   // GAT mode
   float leaky = 0.2f;
+  int heads = 1;                // GAT: attention heads
   float* d_att_s = nullptr;     // [V] att_src . h'
   float* d_att_t = nullptr;     // [V] att_dst . h'
   float* d_att_max = nullptr;   // [V] running maximum of att_src . h'_u over the neighbourhood
@@ -297,8 +300,10 @@ struct taurus_ctx {
 };
 
 static inline int taurus_round_up(int x, int m) { return (x + m - 1) / m * m; }
-// Columns of the projection output: [P | T] for SAGE, [h' | att_src.h' att_dst.h' 0 0] for GAT, P otherwise.
-static inline int taurus_proj_width(int mode, int Hp) { return mode == TAURUS_SAGE_MEAN ? 2 * Hp : mode == TAURUS_GAT ? Hp + 4 : Hp; }
+// Columns of the projection output: [P | T] for SAGE, [h' | (att_src.h', att_dst.h') per head, padded to 4] for GAT, P otherwise.
+static inline int taurus_proj_width(int mode, int Hp, int heads = 1) {
+  return mode == TAURUS_SAGE_MEAN ? 2 * Hp : mode == TAURUS_GAT ? Hp + taurus_round_up(2 * heads, 4) : Hp;
+}
 
 // ---- kernels_state.cu
 void launch_layer_reset(taurus_ctx* c, int layer, cudaStream_t st);
@@ -335,7 +340,7 @@ void launch_af_prep(taurus_ctx* c, const float* X, int ldx, int n, int K, int Kp
 int launch_af_finalise(taurus_ctx* c, const ChunkArgs& a, int layer, long long bound, cudaStream_t st);
 // ---- kernels_gat.cu
 void launch_gat_scores(taurus_ctx* c, int layer, const float* X, int ldx, int n, long long src_begin, float* rows_out, long long ld, cudaStream_t st);
-void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st);
+void launch_gat_split(taurus_ctx* c, int n, int Hp, int d_out, long long src_begin, float* hprime_out, long long ld, cudaStream_t st);   // c->heads heads
 void launch_gat_attention(taurus_ctx* c, cudaStream_t st);
 void launch_gat_repack(taurus_ctx* c, const float* X, int n, int d_out, int Hp, cudaStream_t st);   // X [n x d_out] -> d_PT [n x Hp]
 // ---- kernels_scatter.cu

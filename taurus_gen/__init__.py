@@ -102,6 +102,7 @@ class Workload:
     seed: int = 1
     gin_eps: float = 0.0        # GIN_SUM only: the self weight is 1 + gin_eps
     leaky_slope: float = 0.2    # GAT only: negative slope of the LeakyReLU on the attention scores
+    gat_heads: int = 1          # GAT only: attention heads; head i owns columns [i d, (i + 1) d) of every layer's output
 
     @property
     def L(self) -> int:

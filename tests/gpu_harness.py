@@ -22,7 +22,7 @@ def run_library(w, g, model, x0, *, drain_each_chunk=True, flags=0, host_feature
     ctx = tb.Context(V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict,
                      drain_rows or (2 * V if (dense_output or run_output) else V), w.gemm_mode if gemm_mode is None else gemm_mode, flags, evict_policy, w.gin_eps,
-                     model.att_src, model.att_dst, w.leaky_slope)
+                     model.att_src, model.att_dst, w.leaky_slope, w.gat_heads)
     res = dict(outs=[], completed=[], stats=[], chunk_log=[], reload_count=[], masks=[], ctx=ctx)
     if host_features:
         feat = torch.from_numpy(np.ascontiguousarray(x0)).pin_memory()
@@ -112,8 +112,8 @@ def run_oracle(w, g, model, x0, evict_policy=0):
         ms = oracle.message_sets(inl, w.fanout[l], w.seed, l)
         if w.mode == tg.GAT:
             from oracle import gat
-            h = gat.gat_layer_forward(ms, h, model.W_neigh[l], model.att_src[l], model.att_dst[l], model.bias[l], model.act[l],
-                                      w.leaky_slope)
+            h = gat.gat_layer_forward_heads(ms, h, model.W_neigh[l], model.att_src[l], model.att_dst[l], model.bias[l], model.act[l],
+                                            w.gat_heads, w.leaky_slope)
         else:
             h = oracle.layer_forward(ms, w.mode, din, dout, h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l],
                                      gin_eps=w.gin_eps)
@@ -132,8 +132,8 @@ def layer_on_input(w, model, orc, l, h_in):
     h = np.asarray(h_in, dtype=np.float64)
     if w.mode == tg.GAT:
         from oracle import gat
-        return gat.gat_layer_forward(ms, h, model.W_neigh[l], model.att_src[l], model.att_dst[l], model.bias[l], model.act[l],
-                                     w.leaky_slope, magnitude=True)
+        return gat.gat_layer_forward_heads(ms, h, model.W_neigh[l], model.att_src[l], model.att_dst[l], model.bias[l], model.act[l],
+                                           w.gat_heads, w.leaky_slope, magnitude=True)
     ref = oracle.layer_forward(ms, w.mode, orc["din"], orc["dout"], h, model.W_neigh[l], model.W_self[l], model.bias[l], model.act[l],
                                gin_eps=w.gin_eps)
     mag = oracle.layer_forward(ms, w.mode, orc["din"], orc["dout"], np.abs(h), np.abs(model.W_neigh[l]), np.abs(model.W_self[l]),

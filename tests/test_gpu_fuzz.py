@@ -25,8 +25,12 @@ def random_config(seed):
     mode = int(rng.choice([tg.SAGE_MEAN, tg.GCN_SYM, tg.GIN_SUM, tg.GAT]))
     fanout = tuple(int(rng.choice([0, 0, 1, 2, 5, 9])) for _ in range(L))
     hub_count = int(rng.choice([0, 0, 1, 7, V // 50, V // 3]))
+    heads = 1
+    if mode == tg.GAT:     # several heads where every layer's output width splits into whole float4 per head
+        ok = [hd for hd in (1, 1, 2, 4, 8) if all(d % (4 * hd) == 0 for d in dims[1:])]
+        heads = int(rng.choice(ok)) if ok else 1
     w = replace(w, dims=dims, mode=mode, fanout=fanout, hub_count=hub_count, gemm_mode=tg.GEMM_FP32, gin_eps=float(rng.uniform(-0.5, 0.5)),
-                leaky_slope=float(rng.choice([0.0, 0.2, 1.0])), seed=int(rng.integers(1, 1 << 30)))
+                leaky_slope=float(rng.choice([0.0, 0.2, 1.0])), seed=int(rng.integers(1, 1 << 30)), gat_heads=heads)
     g = tg.make_graph(w)
     # a pool between "just feasible" and "never evicts": grow it until the oracle's simulator accepts every layer
     inl = oracle.build_in_lists(g.V, g.row_ptr, g.col_idx)
@@ -75,8 +79,8 @@ def random_config(seed):
 @pytest.mark.parametrize("seed", range(int(os.environ.get("TAURUS_FUZZ_SEEDS", "32"))))   # more seeds: set TAURUS_FUZZ_SEEDS
 def test_random_configuration(seed):
     w, g, kw = random_config(seed)
-    print("config %d: %s V=%d E=%d mode=%d dims=%s chunk=%d pool=%d hubs=%d fanout=%s %s" %
-          (seed, w.name, g.V, g.E, w.mode, w.dims, w.chunk, w.pool_slots, w.hub_count, w.fanout, kw))
+    print("config %d: %s V=%d E=%d mode=%d heads=%d dims=%s chunk=%d pool=%d hubs=%d fanout=%s %s" %
+          (seed, w.name, g.V, g.E, w.mode, w.gat_heads, w.dims, w.chunk, w.pool_slots, w.hub_count, w.fanout, kw))
     model = tg.make_model(w, bias_scale=0.3)
     if w.mode == tg.GAT:
         model.att_src = [(a * 3).astype(np.float32) for a in model.att_src]

@@ -57,6 +57,40 @@ def test_gat_dense_output_mode_simt_projection():
     _check(w, flags=2)                       # FFMA projection
 
 
+def test_gat_several_heads_in_one_context():
+    """Heads weight their own column blocks; one pass over the topology serves all of them.  Checked against the oracle
+    (one single-head evaluation per head, concatenated) and, head by head, against single-head contexts of this library
+    built from the head's own columns."""
+    import paper_2607_17374_b200 as tb
+    w = tg.scaled(tg.WORKLOADS["large"], 30_000, chunk=2048)
+    w = replace(w, mode=tg.GAT, dims=(64, 96, 32), fanout=(0, 4), pool_slots=20_000, hub_count=30, gat_heads=4)
+    lib, orc = _check(w)                       # grouped scatter, eviction, hubs, a sampled layer
+    assert lib["stats"][0]["evictions"] > 0
+    _check(w, flags=4)                         # CSR-order scatter
+    _check(replace(w, dims=(256, 128, 64), gat_heads=2, pool_slots=30_000), dense_output=True)
+    # head by head: layer 0 of a 4-head context = four 1-head contexts on the head's columns
+    g = tg.make_graph(w)
+    model = tg.make_model(w, bias_scale=0.3)
+    model.att_src = [(a * 4).astype(np.float32) for a in model.att_src]
+    model.att_dst = [(a * 4).astype(np.float32) for a in model.att_dst]
+    x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
+    d = w.dims[1] // w.gat_heads
+    for hd in range(w.gat_heads):
+        w1 = replace(w, dims=(w.dims[0], d), fanout=(0,), gat_heads=1)
+        m1 = replace(tg.make_model(w1), W_neigh=[np.ascontiguousarray(model.W_neigh[0][:, hd * d:(hd + 1) * d])],
+                     W_self=[np.ascontiguousarray(model.W_neigh[0][:, hd * d:(hd + 1) * d])],
+                     bias=[np.ascontiguousarray(model.bias[0][hd * d:(hd + 1) * d])], act=(model.act[0],),
+                     att_src=[np.ascontiguousarray(model.att_src[0][hd * d:(hd + 1) * d])],
+                     att_dst=[np.ascontiguousarray(model.att_dst[0][hd * d:(hd + 1) * d])])
+        one = run_library(w1, g, m1, x0)
+        diff = np.abs(one["outs"][0] - lib["outs"][0][:, hd * d:(hd + 1) * d]).max()
+        print("head %d: single-head context against the head's block of the 4-head context: max abs difference %.3e" % (hd, diff))
+        assert diff <= 2e-5
+    # widths that a head cannot own as whole float4 are refused
+    with pytest.raises(tb.TaurusError):
+        run_library(replace(w, dims=(64, 100, 32)), g, tg.make_model(replace(w, dims=(64, 100, 32))), x0)
+
+
 def test_gat_call_order_and_arguments():
     import torch
     import paper_2607_17374_b200 as tb

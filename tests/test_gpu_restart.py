@@ -19,7 +19,7 @@ def make(w, **kw):
     host_evict = 0 if w.pool_slots >= g.V - w.hub_count else g.V - w.hub_count
     ctx = tb.Context(g.V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias,
                      model.act, w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, 2 * g.V, w.gemm_mode, 0, 0,
-                     w.gin_eps, model.att_src, model.att_dst, w.leaky_slope)
+                     w.gin_eps, model.att_src, model.att_dst, w.leaky_slope, w.gat_heads)
     return g, model, ctx
 
 

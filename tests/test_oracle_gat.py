@@ -122,3 +122,28 @@ def test_vertex_without_in_edges_and_large_fanout():
     assert np.allclose(out[0], np.maximum(h[0] @ W + b, 0))
     big = oracle.message_sets(inl, 64, 1, 0)
     assert np.array_equal(gat.gat_layer_forward(big, h, W, a_s, a_d, b, 1), out)
+
+
+def test_several_heads_are_the_single_head_layer_per_column_block():
+    """gat_layer_forward_heads against its definition written out: each head is the one-head layer on its own columns of
+    W, a_src, a_dst and b; with one head it is the one-head layer itself."""
+    from oracle import gat
+    from helpers import random_multigraph
+    V, E, F, H, heads = 60, 300, 5, 12, 3
+    row_ptr, col = random_multigraph(V, E, 4)
+    ms = oracle.message_sets(oracle.build_in_lists(V, row_ptr, col), 0, 1, 0)
+    rng = np.random.default_rng(8)
+    h, W = rng.standard_normal((V, F)), rng.standard_normal((F, H))
+    a_s, a_d, b = rng.standard_normal(H), rng.standard_normal(H), rng.standard_normal(H)
+    out = gat.gat_layer_forward_heads(ms, h, W, a_s, a_d, b, 1, heads, 0.2)
+    d = H // heads
+    for i in range(heads):
+        blk = slice(i * d, (i + 1) * d)
+        one = gat.gat_layer_forward(ms, h, W[:, blk], a_s[blk], a_d[blk], b[blk], 1, 0.2)
+        assert np.array_equal(out[:, blk], one)
+    assert np.array_equal(gat.gat_layer_forward_heads(ms, h, W, a_s, a_d, b, 0, 1, 0.2), gat.gat_layer_forward(ms, h, W, a_s, a_d, b, 0, 0.2))
+    # heads differ: with different attention vectors two heads weight the same neighbours differently
+    same_w = np.concatenate([W[:, :d], W[:, :d]], axis=1)
+    two = gat.gat_layer_forward_heads(ms, h, same_w, np.concatenate([a_s[:d], 3 * a_s[:d]]), np.concatenate([a_d[:d], -a_d[:d]]),
+                                      np.zeros(2 * d), 0, 2, 0.2)
+    assert np.abs(two[:, :d] - two[:, d:]).max() > 1e-3
