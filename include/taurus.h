@@ -109,7 +109,10 @@ typedef struct {
   uint64_t seed;            /* seed of the neighbour-sampling hash                                         */
   int64_t host_evict_rows;  /* capacity (rows) of the pinned host store for evicted accumulators; 0 = none.
                                Must cover the rows evicted at once plus one chunk's victims (a chunk's victims
-                               leave before its reloads hand their host rows back); V - hub_count always suffices */
+                               leave before its reloads hand their host rows back); V - hub_count always suffices.
+                               The store is handed out in extents of up to 1 024 rows, one open extent per grid cell
+                               of chunk_sources sources (evicted rows are filed by the cell that will next need
+                               them): the library pins a few extents per cell more than this many rows */
   int64_t drain_rows;       /* capacity (rows) of the graduation buffer; must hold the completions of any one
                                pushed range as bounded by taurus_completion_bound (64-source granularity)  */
   int32_t flags;            /* TAURUS_FLAG_*                                                               */

@@ -277,7 +277,7 @@ static int init_impl(taurus_ctx* c, const taurus_graph* g, const taurus_model* m
     ALLOC(c->d_bk_off, c->n_buckets); ALLOC(c->d_bk_base, c->n_buckets);
     ALLOC(c->d_new_ext, (c->victim_capacity >> c->ext_shift) + c->n_buckets + 1);
     ALLOC(c->d_ext_ret[0], c->n_ext); ALLOC(c->d_ext_ret[1], c->n_ext);
-    ALLOC(c->d_xfer_list, c->pool_slots);   // one entry per need-list entry
+    ALLOC(c->d_xfer_list, std::min<long long>(c->pool_slots, c->touched_capacity));   // one entry per need-list entry: a chunk needs at most what it touches
     ALLOC(c->d_stage_out, (size_t)c->victim_capacity * c->Hmax);
     CU(cudaStreamCreateWithFlags(&c->xfer_stream, cudaStreamNonBlocking));
     CU(cudaEventCreateWithFlags(&c->moves_ready, cudaEventDisableTiming));
