@@ -1,9 +1,13 @@
 import os
 import sys
+import time
 
 import pytest
 
 sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+
+SESSION_START = time.time()      # the full-size tests look at the time the session has already used
 
 
 def pytest_configure(config):

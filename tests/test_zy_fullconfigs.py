@@ -4,7 +4,9 @@ All three run by default, late in the collection order (two to four minutes each
 125-145 GB of device memory); a machine with less prints why and skips.  'large' and 'sampled' run their first and
 last layer; 'stress' runs its last layer by default and its first one (512 input columns: the host needs two and a
 half minutes to generate the 551 GB of feature rows) as well with TAURUS_FULL_STRESS_LAYERS=all.  TAURUS_FULL_CONFIGS
-selects a subset: a comma-separated list of workload names, or "none".
+selects a subset: a comma-separated list of workload names, or "none".  A session that has TAURUS_SUITE_BUDGET_S
+seconds for the whole GPU suite (default 1 100) skips, with the reason printed, a workload that would not end inside it
+on a machine a quarter slower than the one these durations were measured on; 0 switches that guard off.
 
 At these sizes the full oracle is out of reach, so the checks are
   * output rows of a destination sample (random vertices + the largest hubs) against the oracle's pull-based
@@ -30,6 +32,7 @@ pytestmark = pytest.mark.gpu
 WANTED = [x for x in os.environ.get("TAURUS_FULL_CONFIGS", "large,sampled,stress").split(",") if x]
 HOST_GB = {"large": 110, "sampled": 130, "stress": 165}      # host memory (graph, check arrays, pinned evicted-row store)
 DEVICE_GB = {"large": 125, "sampled": 140, "stress": 145}
+EXPECT_S = {"large": 120, "sampled": 230, "stress": 170}      # measured durations of the default runs (stress: last layer only)
 
 
 def _oracle_rows(w, g, model, layer, dsts, ptr, src, eid):
@@ -63,6 +66,14 @@ def test_full_config(name):
         if host_gb < HOST_GB[base] or dev_gb < DEVICE_GB[base]:
             reason = "%s at full size needs %d GB of host and %d GB of device memory; %.0f and %.0f GB are free here" % (
                 base, HOST_GB[base], DEVICE_GB[base], host_gb, dev_gb)
+            print(reason)
+            pytest.skip(reason)
+
+        budget = float(os.environ.get("TAURUS_SUITE_BUDGET_S", "1100"))
+        import conftest
+        used = time.time() - conftest.SESSION_START
+        if budget > 0 and used + 1.25 * EXPECT_S[base] > budget:
+            reason = "%s at full size takes about %d s; the session has used %.0f s of its %d s" % (base, EXPECT_S[base], used, budget)
             print(reason)
             pytest.skip(reason)
 
