@@ -41,12 +41,13 @@ import taurus_gen as tg  # noqa: E402
 
 METRIC = "edges/sec per GNN layer (GTEPS)"
 
-# DRAM bytes (read + write) per accumulator-row reduction of the 256-float scatter_grouped_kernel instance, from the ncu
-# capture summarised in profiles/scatter_grouped_kernel_mid_1200k.md.  The figure belongs to the kernel source with
-# the digest below (sha256 of csrc/kernels_group.cu, first 16 hex digits); when the source has changed since the
-# capture the bench prints traffic = null instead of a stale number.
-SCATTER_TRAFFIC_PER_GROUP_BYTES = 2720.0
-SCATTER_CAPTURE_SOURCE = "19efb17de4f02d04"
+# DRAM bytes (read + write) of the 256-float scatter_grouped_kernel instance per algorithmic byte, from the ncu capture
+# summarised in profiles/scatter_grouped_kernel_mid_1200k.md (two launches: 2.691 and 2.721 GB measured against 2.143 and
+# 2.164 GB algorithmic).  The figure belongs to the kernel source with the digest below (sha256 of csrc/kernels_group.cu,
+# first 16 hex digits); when the source has changed since the capture the bench prints traffic = null instead of a
+# stale number.
+SCATTER_TRAFFIC_OVER_ALGORITHMIC = 1.257
+SCATTER_CAPTURE_SOURCE = "f25b718e2641c63c"
 
 
 def source_digest(name: str) -> str:
@@ -702,9 +703,9 @@ def run_full_pass(args, env, w):
     capture_valid = grouped and dom_w == 256 and source_digest("kernels_group.cu") == SCATTER_CAPTURE_SOURCE
     roofline = dict(bound="hbm", kernel=kname, achieved=achieved,
                     peak=pk["hbm_gbs"], unit="GB/s", frac=achieved / pk["hbm_gbs"], peak_source=pk["source"],
-                    traffic=SCATTER_TRAFFIC_PER_GROUP_BYTES * sum(groups_per_layer[l] for l in dom) / (len(dom) * len(chunks))
-                    if capture_valid else None,
-                    traffic_note=("ncu dram read+write per launch of the 256-float kernel, scaled by groups per launch "
+                    traffic=SCATTER_TRAFFIC_OVER_ALGORITHMIC * dom_bytes / (len(chunks) * len(dom)) if capture_valid else None,
+                    traffic_note=("ncu dram read+write per launch of the 256-float kernel on a 1.2 M-vertex instance, scaled by the "
+                                  "algorithmic bytes of a launch "
                                   "(profiles/scatter_grouped_kernel_mid_1200k.md)") if capture_valid else
                                  "no capture of this kernel source (profiles/scatter_grouped_kernel_mid_1200k.md names the source it measured)",
                     launches_per_step=len(chunks) * len(dom), avg_launch_ms=dom_ms / (len(chunks) * len(dom)),
@@ -781,7 +782,9 @@ def run_full_pass(args, env, w):
                             messages_per_step=msgs_per_step,
                             l2="inputs larger than L2 (accumulators %.1f GB)" % (w.pool_slots * 4 * max(w.dims[1:]) / 1e9),
                             parallelism="replicas only" if world > 1 else "1 gpu",
-                            layer_ms=[float(ph[:, l, :, :8].sum()) / args.steps for l in range(L)], phase_ms=phase_ms),
+                            layer_ms=[float(ph[:, l, :, :8].sum()) / args.steps for l in range(L)], phase_ms=phase_ms,
+                            phase_ms_per_layer=[dict(zip(PHASES, [round(float(x) / args.steps, 3) for x in ph[:, l].sum(axis=(0, 1))]))
+                                                for l in range(L)]),
                 clocks=clocks, roofline=roofline, e2e=e2e, cpu_baseline=cpu, gpu_launches=int(launches))
     for r in runs or []:
         r.destroy()

@@ -41,12 +41,15 @@ __global__ void gat_split_kernel(const float* __restrict__ PT, int ldpt, int n, 
 }
 
 // max over propagated in-edges (u -> v) of s_u, one warp per source row
+template <bool ONE>   // ONE: a single head, the source's scalar is read once per row
 __global__ void gat_edge_max_kernel(long long V, int heads, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
                                     const uint32_t* __restrict__ mask, const float* __restrict__ att_s, float* __restrict__ att_max) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    const float s1 = ONE ? att_s[u] : 0.f;
     for (long long e = row_ptr[u] + gl(); e < row_ptr[u + 1]; e += 32)
       if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) {
+        if (ONE) { atomic_max_float(&att_max[col[e]], s1); continue; }
         const size_t v = (size_t)col[e] * heads;
         for (int h = 0; h < heads; ++h) atomic_max_float(&att_max[v + h], att_s[(size_t)u * heads + h]);
       }
@@ -65,13 +68,21 @@ __global__ void gat_tm_kernel(long long V, const float* __restrict__ att_s, cons
   }
 }
 
+template <bool ONE>
 __global__ void gat_edge_sum_kernel(long long V, int heads, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
                                     const uint32_t* __restrict__ mask, const float* __restrict__ att_s,
                                     const float2* __restrict__ tm, float slope, float* __restrict__ z) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
+    const float s1 = ONE ? att_s[u] : 0.f;
     for (long long e = row_ptr[u] + gl(); e < row_ptr[u + 1]; e += 32)
       if (!mask || ((mask[e >> 5] >> (e & 31)) & 1u)) {
+        if (ONE) {
+          const int v1 = col[e];
+          const float2 x = tm[v1];
+          atomicAdd(&z[v1], __expf(lrelu(s1 + x.x, slope) - x.y));
+          continue;
+        }
         const size_t v = (size_t)col[e] * heads;
         for (int h = 0; h < heads; ++h) {
           const float2 x = tm[v + h];
@@ -130,9 +141,11 @@ void launch_gat_scores(taurus_ctx* c, int layer, const float* X, int ldx, int n,
 
 void launch_gat_attention(taurus_ctx* c, cudaStream_t st) {
   const int grid = c->sm_count * 8;
-  gat_edge_max_kernel<<<grid, 256, 0, st>>>(c->V, c->heads, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_max);
+  if (c->heads == 1) gat_edge_max_kernel<true><<<grid, 256, 0, st>>>(c->V, 1, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_max);
+  else gat_edge_max_kernel<false><<<grid, 256, 0, st>>>(c->V, c->heads, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_max);
   gat_tm_kernel<<<grid, 256, 0, st>>>(c->V * c->heads, c->d_att_s, c->d_att_t, c->d_att_max, c->leaky, c->d_att_tm, c->d_att_z);
-  gat_edge_sum_kernel<<<grid, 256, 0, st>>>(c->V, c->heads, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_tm, c->leaky, c->d_att_z);
+  if (c->heads == 1) gat_edge_sum_kernel<true><<<grid, 256, 0, st>>>(c->V, 1, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_tm, c->leaky, c->d_att_z);
+  else gat_edge_sum_kernel<false><<<grid, 256, 0, st>>>(c->V, c->heads, c->d_row_ptr, c->d_col, c->d_mask_cur, c->d_att_s, c->d_att_tm, c->leaky, c->d_att_z);
   c->launches += 3;
 }
 
