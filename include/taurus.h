@@ -449,7 +449,11 @@ int64_t taurus_launch_count(const taurus_ctx* ctx);
  * previous chunk's row transfers plus that chunk's finalise (bounded pools; else about zero), 4 slot hand-out (victims'
  * rows staged, new rows cleared), 5 scatter, 6 completion list, 7 the chunk's own finalise, 8 the chunk's row
  * transfers over the host link (evicted rows out, reloaded rows in; on the library's transfer stream, beside
- * k = 5, 6 of this chunk and k = 0..2 of the next); *out_pushes = pushes written (at most capacity_pushes). */
+ * k = 5, 6 of this chunk and k = 0..2 of the next); *out_pushes = pushes written (at most capacity_pushes).
+ * An event between two kernels costs about 2 us of the stream (twelve per push: 4-5 % of a pass whose pushes take half a
+ * millisecond); taurus_set_timing(ctx, 2) records only the two events around the scatter, and taurus_get_phase_ms then
+ * fills k = 5 and leaves the other columns 0.  on = 0 ends the window; another value is TAURUS_ERR_INVALID_ARG.  The
+ * call first enqueues the finalise of a chunk whose finalise was deferred (bounded pools), as the blocking calls do. */
 int taurus_set_timing(taurus_ctx* ctx, int32_t on);
 int taurus_get_phase_ms(taurus_ctx* ctx, float* out, int64_t capacity_pushes, int64_t* out_pushes);
 

@@ -418,8 +418,9 @@ class Context:
     def launch_count(self) -> int:
         return int(self._lib.taurus_launch_count(self._h))
 
-    def set_timing(self, on: bool):
-        self._check(self._lib.taurus_set_timing(self._h, 1 if on else 0), "taurus_set_timing")
+    def set_timing(self, on):
+        """False / 0: off; True / 1: events after every phase of a push; 2: events around the scatter only."""
+        self._check(self._lib.taurus_set_timing(self._h, int(on)), "taurus_set_timing")
 
     def get_phase_ms(self, capacity_pushes: int = 16384) -> np.ndarray:
         """float32 [pushes, 9] (ms per recorded push): copy-in, projection, classify + victim selection, wait for the

@@ -519,7 +519,7 @@ static int finish_chunk(taurus_ctx* c, cudaStream_t st) {
   const PendingChunk& p = *c->pend_chunk;
   const ChunkArgs& a = p.a;
   const int l = p.layer;
-  cudaEvent_t* pev = p.timed_index >= 0 ? &c->phase_ev[(size_t)p.timed_index * TAURUS_PUSH_EVENTS] : nullptr;
+  cudaEvent_t* pev = p.timed_index >= 0 && c->timing != 2 ? &c->phase_ev[(size_t)p.timed_index * TAURUS_PUSH_EVENTS] : nullptr;
   if (c->pipelined) {
     CU(cudaStreamWaitEvent(st, c->xfer_done, 0));   // reloaded partial sums have been added to the chunk's rows
     if (pev) cudaEventRecord(pev[8], st);           // (without transfers the finalise follows event 7 directly)
@@ -625,7 +625,8 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
     pev = &c->phase_ev[(size_t)c->timed_pushes * TAURUS_PUSH_EVENTS];
     c->timed_pushes += 1;
   }
-  const bool timing = pev != nullptr;
+  const bool scatter_timing = pev != nullptr;           // level 2 records the two events around the scatter only
+  const bool timing = pev != nullptr && c->timing != 2;
   if (timing) cudaEventRecord(pev[0], st);
   // S1: features to the device
   const float* X = nullptr;
@@ -682,7 +683,7 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   int run_rc = finish_chunk(c, st);
   if (timing && c->pipelined) cudaEventRecord(pev[4], st);
   launch_alloc(c, a, st);
-  if (timing) cudaEventRecord(pev[5], st);
+  if (scatter_timing) cudaEventRecord(pev[5], st);
   if (c->pipelined) {
     CU(cudaEventRecord(c->moves_ready, st));
     CU(cudaStreamWaitEvent(c->xfer_stream, c->moves_ready, 0));
@@ -694,12 +695,12 @@ static int push_core(taurus_ctx* c, int64_t src_begin, int64_t src_end, const fl
   // S5, S5', S6
   if (grouped) launch_scatter_grouped(c, a, st); else launch_scatter(c, a, st);
   if (xbuf >= 0 && x_in_use) { CU(cudaEventRecord(c->x_free[xbuf], st)); c->x_used[xbuf] = true; }   // the scatter read the staged rows in place
-  if (timing) cudaEventRecord(pev[6], st);
+  if (scatter_timing) cudaEventRecord(pev[6], st);
   launch_compact_done(c, a, st, c->pipelined);   // with transfers in flight the chunk record is written now, else by the commit after finalise
   if (timing) cudaEventRecord(pev[7], st);
   // S7: deferred behind the next chunk's select when rows cross the host link, else at once
   c->pend_chunk->a = a; c->pend_chunk->layer = l; c->pend_chunk->af = af; c->pend_chunk->bound = bound;
-  c->pend_chunk->timed_index = timing ? c->timed_pushes - 1 : -1;
+  c->pend_chunk->timed_index = scatter_timing ? c->timed_pushes - 1 : -1;
   c->pending = true;
   if (!c->pipelined) { int rc = finish_chunk(c, st); if (!run_rc) run_rc = rc; }
   CU(cudaGetLastError());
@@ -995,8 +996,11 @@ extern "C" int taurus_get_layer_plan(const taurus_ctx* c, int32_t layer, int32_t
 
 extern "C" int taurus_set_timing(taurus_ctx* c, int32_t on) {
   if (!c) return TAURUS_ERR_INVALID_ARG;
-  c->timing = on ? 1 : 0;
-  if (on) c->timed_pushes = 0;
+  if (on < 0 || on > 2) return TAURUS_ERR_INVALID_ARG;
+  CU(cudaSetDevice(c->device));
+  { int rc = finish_chunk(c, c->last_stream); if (rc) return rc; }   // a deferred finalise belongs to the level it was pushed under
+  c->timing = on;
+  if (on) { c->timed_pushes = 0; c->timed_level = on; }
   return TAURUS_OK;
 }
 
@@ -1016,7 +1020,7 @@ extern "C" int taurus_get_phase_ms(taurus_ctx* c, float* out, int64_t capacity_p
   for (long long p = 0; p < n; ++p)
     for (int i = 0; i < TAURUS_PHASES; ++i) {
       out[p * TAURUS_PHASES + i] = 0.f;
-      if (from[i] >= 0)
+      if (from[i] >= 0 && (c->timed_level == 1 || i == 5))
         CU(cudaEventElapsedTime(&out[p * TAURUS_PHASES + i], c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + from[i]],
                                 c->phase_ev[(size_t)p * TAURUS_PUSH_EVENTS + to[i]]));
     }

@@ -292,7 +292,8 @@ struct taurus_ctx {
   cudaStream_t last_stream = nullptr;
   cudaEvent_t order_event = nullptr;
   long long launches = 0;
-  int timing = 0;
+  int timing = 0;                      // 0 off, 1 every phase, 2 the scatter only
+  int timed_level = 1;                 // level of the recorded pushes
   std::vector<cudaEvent_t> phase_ev;   // TAURUS_PUSH_EVENTS events per timed push, created on demand
   long long timed_pushes = 0;          // pushes recorded since timing was switched on
   std::vector<std::vector<long long>> rank_cum_cache;   // per layer: rank_cum computed at the first layer_begin

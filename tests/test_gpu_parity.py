@@ -384,3 +384,45 @@ def test_finished_rows_leave_the_transform_complete(mode):
     w = replace(w, dims=(20, 100, 30, 50), pool_slots=18_000, hub_count=30)
     lib, _ = _full_check(w, dense_output=True)
     assert lib["stats"][0]["evictions"] > 0
+
+
+@pytest.mark.parametrize("bounded", [False, True])
+def test_phase_timing_levels(bounded):
+    """taurus_set_timing: level 1 fills every column of taurus_get_phase_ms, level 2 the scatter column only, and the
+    results of the pushes do not depend on the level."""
+    import torch
+    import paper_2607_17374_b200 as tb
+    from dataclasses import replace
+    w = replace(tg.scaled(tg.WORKLOADS["large"], 20_000, chunk=1024), dims=(64, 128), fanout=(0,),
+                pool_slots=12_000 if bounded else 20_000, hub_count=20)
+    g = tg.make_graph(w)
+    model = tg.make_model(w)
+    x = torch.from_numpy(tg.features(w.seed, 0, 0, g.V, w.dims[0])).cuda()
+    host_evict = g.V - w.hub_count if bounded else 0
+    ctx = tb.Context(g.V, g.E, g.row_ptr, g.col_idx, g.in_degree, w.mode, w.dims, model.W_neigh, model.W_self, model.bias, model.act,
+                     w.chunk, w.pool_slots, w.hub_count, w.fanout, w.seed, host_evict, 2 * g.V, w.gemm_mode, 0)
+    n_push = (g.V + w.chunk - 1) // w.chunk
+    outs = []
+    for level in (0, 1, 2):
+        out = torch.zeros((g.V, w.dims[1]), device="cuda")
+        ctx.layer_begin(0)
+        ctx.layer_set_dense_output(out, w.dims[1])
+        ctx.set_timing(level)
+        for s in range(0, g.V, w.chunk):
+            ctx.push_chunk(s, min(g.V, s + w.chunk), x[s:s + w.chunk])
+        ctx.layer_end()
+        outs.append(out.cpu().numpy())
+        if level:
+            ph = ctx.get_phase_ms()
+            ctx.set_timing(0)
+            assert ph.shape == (n_push, 9) and (ph >= 0).all()
+            assert (ph[:, 5] > 0).all()
+            if level == 2:
+                assert (np.delete(ph, 5, axis=1) == 0).all()
+            else:
+                assert (ph[:, [1, 2, 4, 6, 7]] > 0).all() and ((ph[:, 8] > 0).any() == bounded)
+    assert np.array_equal(outs[0], outs[1]) or np.allclose(outs[0], outs[1], rtol=1e-5, atol=1e-6)   # reductions may land in another order
+    assert np.allclose(outs[0], outs[2], rtol=1e-5, atol=1e-6)
+    with pytest.raises(tb.TaurusError):
+        ctx.set_timing(3)
+    ctx.destroy()
