@@ -803,9 +803,44 @@ def run_full_pass(args, env, w):
     return line
 
 
+# Host and device memory (GB) a replica of a full-size bounded-pool workload takes in this bench: the graph, the pinned
+# store of evicted rows (56 M rows of the timed layer's width) and the generator's temporaries; the pool, the grouped edge
+# order and the in-lists on the device.
+FULL_SIZE_NEEDS_GB = {"large": (90, 140), "sampled": (100, 150), "stress": (150, 150)}
+
+
+def fallback_reason(args, env, w):
+    """Why this box cannot hold the workload at full size (None when it can)."""
+    base = w.name.split("@")[0]
+    if args.vertices or args.pool_fraction > 0 or base not in FULL_SIZE_NEEDS_GB:
+        return None
+    host_need, dev_need = FULL_SIZE_NEEDS_GB[base]
+    host_free = 0.0
+    for ln in open("/proc/meminfo"):
+        if ln.startswith("MemAvailable:"):
+            host_free = int(ln.split()[1]) / 1e6
+    dev_free = env.torch.cuda.mem_get_info()[0] / 1e9
+    if host_free < host_need * env.world or dev_free < dev_need:
+        return ("'%s' at full size needs %d GB of host memory per replica (%d replicas) and %d GB of device memory; %.0f GB "
+                "and %.0f GB are free here" % (base, host_need, env.world, dev_need, host_free, dev_free))
+    return None
+
+
 def run_ours(args):
     env = Env()
     w = workload_of(args)
+    why = fallback_reason(args, env, w)
+    if max_over_ranks(0.0 if why is None else 1.0, env.world, env.dev) > 0 and why is None:   # every rank takes the same road
+        why = "another replica found too little memory for '%s' at full size" % w.name
+    if why is not None and args.secondary not in ("none", ""):
+        # the box cannot hold the configured workload: the secondary one becomes the line, and says so
+        w = workload_of(args, args.secondary)
+        line = run_windowed(args, env, w) if windowed(w) else run_full_pass(args, env, w)
+        line["config"]["fallback"] = why
+        if env.rank == 0:
+            print(json.dumps(line))
+        env.close()
+        return
     line = run_windowed(args, env, w) if windowed(w) else run_full_pass(args, env, w)
     if args.secondary not in ("none", "", w.name.split("@")[0]) and env.world == 1:
         import gc
