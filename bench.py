@@ -541,8 +541,10 @@ def run_windowed(args, env, w):
     free, total = torch.cuda.mem_get_info()
     # `roofline` is the kernel with the larger share of the step: the row transfers where the pool is short of the active
     # set (large, sampled), the scatter where few rows move (stress); the other one is kept beside it
+    # (a transfer launch that moves a few thousand rows is long only because its blocks wait for room on the SMs beside the
+    # scatter: it counts as the dominant kernel only when the link is busy with bytes, here a quarter of its peak)
     other = {}
-    if phase[8] >= phase[5]:
+    if phase[8] >= phase[5] and max(out_gbs, in_gbs) >= 0.25 * link["both_per_direction_gbs"]:
         other["roofline_hbm"] = roofline_hbm
     else:
         other["roofline_pcie"] = roofline
