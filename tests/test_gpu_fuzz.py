@@ -76,7 +76,10 @@ def random_config(seed):
     return w, g, kw
 
 
-@pytest.mark.parametrize("seed", range(int(os.environ.get("TAURUS_FUZZ_SEEDS", "32"))))   # more seeds: set TAURUS_FUZZ_SEEDS
+_FIRST = int(os.environ.get("TAURUS_FUZZ_FIRST", "0"))        # first seed of the sweep
+
+
+@pytest.mark.parametrize("seed", range(_FIRST, _FIRST + int(os.environ.get("TAURUS_FUZZ_SEEDS", "32"))))   # more seeds: set TAURUS_FUZZ_SEEDS
 def test_random_configuration(seed):
     w, g, kw = random_config(seed)
     print("config %d: %s V=%d E=%d mode=%d heads=%d dims=%s chunk=%d pool=%d hubs=%d fanout=%s %s" %
