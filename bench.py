@@ -109,6 +109,21 @@ def graph_of(args, w):
     return tg.make_graph(replace(w, chunk=base.chunk) if args.chunk > 0 else w)
 
 
+def plan_windows(n_chunks: int, K: int, W: int, window: int, prefill: int):
+    """Chunks per window and untimed prefill chunks of one layer pass that has to hold the prefill and W + K windows: the
+    where the pass is too short for what was asked, the prefill is cut to a quarter of it, then the window shrinks (a run with
+    many steps times shorter windows), then the prefill again."""
+    window, prefill = max(window, 1), max(prefill, 0)
+    if prefill + (W + K) * window > n_chunks:
+        prefill = min(prefill, n_chunks // 4)
+    while prefill + (W + K) * window > n_chunks and window > 1:
+        window -= 1
+    prefill = max(0, min(prefill, n_chunks - (W + K) * window))
+    if (W + K) * window > n_chunks:
+        raise SystemExit("workload too small for %d windows" % (W + K))
+    return window, prefill
+
+
 def windowed(w) -> bool:
     """Bounded pool: rows can be evicted, and a step is a window of chunks."""
     return w.pool_slots < w.V - w.hub_count
@@ -396,12 +411,7 @@ def run_windowed(args, env, w):
     l = timed_layers(args, w)[0]
     d_in, d_out = w.dims[l], w.dims[l + 1]
     K, W = max(args.steps, 1), max(args.warmup, 0)
-    window, prefill = max(args.window, 1), max(args.prefill, 0)
-    while prefill + (W + K) * window > len(chunks) and window > 1:
-        window -= 1
-    prefill = max(0, min(prefill, len(chunks) - (W + K) * window))
-    if (W + K) * window > len(chunks):
-        raise SystemExit("workload too small for %d windows" % (W + K))
+    window, prefill = plan_windows(len(chunks), K, W, args.window, args.prefill)
     cap = 3 * window * chunk                       # graduation buffer: drained once per window, earlier when it could overflow
     host_evict = min(V - w.hub_count, 56_000_000)   # rows evicted at once stay below this on the three bounded-pool workloads
     ctx = make_context(args, w, g, model, host_evict, cap)
@@ -811,17 +821,21 @@ def run_full_pass(args, env, w):
 FULL_SIZE_NEEDS_GB = {"large": (90, 140), "sampled": (100, 150), "stress": (150, 150)}
 
 
+def free_memory_gb(env):
+    host_free = 0.0
+    for ln in open("/proc/meminfo"):
+        if ln.startswith("MemAvailable:"):
+            host_free = int(ln.split()[1]) / 1e6
+    return host_free, env.torch.cuda.mem_get_info()[0] / 1e9
+
+
 def fallback_reason(args, env, w):
     """Why this box cannot hold the workload at full size (None when it can)."""
     base = w.name.split("@")[0]
     if args.vertices or args.pool_fraction > 0 or base not in FULL_SIZE_NEEDS_GB:
         return None
     host_need, dev_need = FULL_SIZE_NEEDS_GB[base]
-    host_free = 0.0
-    for ln in open("/proc/meminfo"):
-        if ln.startswith("MemAvailable:"):
-            host_free = int(ln.split()[1]) / 1e6
-    dev_free = env.torch.cuda.mem_get_info()[0] / 1e9
+    host_free, dev_free = free_memory_gb(env)
     if host_free < host_need * env.world or dev_free < dev_need:
         return ("'%s' at full size needs %d GB of host memory per replica (%d replicas) and %d GB of device memory; %.0f GB "
                 "and %.0f GB are free here" % (base, host_need, env.world, dev_need, host_free, dev_free))
