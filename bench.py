@@ -11,8 +11,8 @@ Workloads with a bounded pool ("large", "sampled", "stress"; a full pass takes t
 window of --window consecutive chunks of one layer pass in steady state.  The layer (--layer, default the first
 hidden-to-hidden layer) is begun, --prefill chunks fill the pool (untimed), then W warm-up windows and K timed
 windows follow in the same pass; every window ends with a drain of the rows it completed.  The layer's input rows
-are generated rows of the right width (the paper's convention of dummy inputs of matching dimensions for later
-layers, Sect. 4.2).  The full layer time is printed as an estimate from the timed windows, marked as such.
+are generated rows of the right width (as the paper feeds later layers, whose real inputs it cannot materialise, with
+stand-in rows of the same width, Sect. 4.2).  The full layer time is printed as an estimate from the timed windows, marked as such.
 
 The default run times "large" (the eviction-bound configuration) and then "mid" as a secondary entry in the same
 JSON line.  N > 1 (under torchrun): the path has no exchange step, so every rank runs an independent replica

@@ -196,7 +196,7 @@ int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const
 
 /*
  * GATConv in three sequential passes (GATConv paragraph of Sect. 3.9); contexts created with TAURUS_GAT, fp32
- * projection only.  One head or several (taurus_model.gat_heads: "the same procedure applies per head"; one pass over
+ * projection only.  One head or several (taurus_model.gat_heads: Sect. 3.9 runs the three passes once per head; here one pass over
  * the topology serves all heads, each head weighting its own block of columns).  Per head, with h' = h W,
  *     e_uv = LeakyReLU(att_src . h'_u + att_dst . h'_v),  alpha_uv = softmax over u in N(v) of e_uv,
  *     out_v = act(sum_{u in N(v)} alpha_uv h'_u + b),

@@ -10,7 +10,7 @@ The definition, pull-based and in fp64, one destination at a time:
 N(v) is the propagated in-multiset M(v) (all in-edges, or the sampled ones; a multi-edge counts once per
 copy) together with v itself: every vertex aggregates a self message (Sect. 3.8), so a vertex without
 in-edges keeps act(h'_v + b).  gat_layer_forward is one attention head; gat_layer_forward_heads applies the same
-procedure per head ("the same procedure applies per head", Sect. 3.9) to column blocks of W, a_src, a_dst and b and
+procedure per head (Sect. 3.9 treats several heads as independent repetitions) to column blocks of W, a_src, a_dst and b and
 concatenates the heads' outputs.
 
 Pins (tests/test_oracle_gat.py): two hand-worked examples (tests/golden/gat_example.txt), a dense masked

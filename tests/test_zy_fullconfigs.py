@@ -16,8 +16,8 @@ At these sizes the full oracle is out of reach, so the checks are
   * for sampled layers: the kept edge lists of the sampled destinations, bit-exact; the library's whole edge mask
     (one bit per CSR edge, all E of them) against the oracle's propagated-edge flags from its own full in-lists and
     its own sampler; and the per-chunk completion counts against the closed form over the sampled message sets.
-Each layer is run on its own generated input rows of the right width (the paper's convention of dummy inputs of
-matching dimensions for layers whose real input cannot be materialised, Sect. 4.2)."""
+Each layer is run on its own generated input rows of the right width (as the paper does for layers whose
+real input it cannot materialise: stand-in rows of the same width, Sect. 4.2)."""
 import os
 import time
 
