@@ -67,7 +67,7 @@ __global__ void af_gather_kernel(ChunkArgs a, float* __restrict__ A, long long r
       } else if (a.mode == TAURUS_GCN_SYM) {
         scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
       } else if (a.mode == TAURUS_GAT) {
-        scale = 1.0f / a.att_z[v];   // softmax normaliser
+        scale = (float)(1.0 / a.att_z[v]);   // softmax normaliser
       }
     }
     const int rows_here = n - i0 < per ? (int)(n - i0) : per;

@@ -58,20 +58,20 @@ __global__ void gat_edge_max_kernel(long long V, int heads, const long long* __r
 
 // tm[v] = (t_v, LeakyReLU(max_u s_u + t_v));  z[v] starts with the self term
 __global__ void gat_tm_kernel(long long V, const float* __restrict__ att_s, const float* __restrict__ att_t,
-                              const float* __restrict__ att_max, float slope, float2* __restrict__ tm, float* __restrict__ z) {   // V = vertices x heads
+                              const float* __restrict__ att_max, float slope, float2* __restrict__ tm, double* __restrict__ z) {   // V = vertices x heads
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < V; v += stride) {
     const float t = att_t[v];
     const float m = lrelu(att_max[v] + t, slope);
     tm[v] = make_float2(t, m);
-    z[v] = __expf(lrelu(att_s[v] + t, slope) - m);
+    z[v] = (double)__expf(lrelu(att_s[v] + t, slope) - m);
   }
 }
 
 template <bool ONE>
 __global__ void gat_edge_sum_kernel(long long V, int heads, const long long* __restrict__ row_ptr, const int32_t* __restrict__ col,
                                     const uint32_t* __restrict__ mask, const float* __restrict__ att_s,
-                                    const float2* __restrict__ tm, float slope, float* __restrict__ z) {
+                                    const float2* __restrict__ tm, float slope, double* __restrict__ z) {
   const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
   for (long long u = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < V; u += warps) {
     const float s1 = ONE ? att_s[u] : 0.f;
@@ -80,13 +80,13 @@ __global__ void gat_edge_sum_kernel(long long V, int heads, const long long* __r
         if (ONE) {
           const int v1 = col[e];
           const float2 x = tm[v1];
-          atomicAdd(&z[v1], __expf(lrelu(s1 + x.x, slope) - x.y));
+          atomicAdd(&z[v1], (double)__expf(lrelu(s1 + x.x, slope) - x.y));
           continue;
         }
         const size_t v = (size_t)col[e] * heads;
         for (int h = 0; h < heads; ++h) {
           const float2 x = tm[v + h];
-          atomicAdd(&z[v + h], __expf(lrelu(att_s[(size_t)u * heads + h] + x.x, slope) - x.y));
+          atomicAdd(&z[v + h], (double)__expf(lrelu(att_s[(size_t)u * heads + h] + x.x, slope) - x.y));
         }
       }
   }

@@ -484,7 +484,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
           const float2 tm = a.att_tm[vj];
           const float e = a.att_s[vj] + tm.x;
           ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
-          sc = a.att_z[vj];
+          sc = (float)a.att_z[vj];
         }
         if (!a.self_bias) sc = 0.f;             // aggregate-first: the bias is added after the transform
 #pragma unroll
@@ -495,7 +495,7 @@ scatter_grouped_kernel(ChunkArgs a, const int2* __restrict__ g_edge, const uint3
               const float2 tm = a.att_tm[at];
               const float e = a.att_s[at] + tm.x;
               ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
-              sc = a.self_bias ? a.att_z[at] : 0.f;
+              sc = a.self_bias ? (float)a.att_z[at] : 0.f;
             }
             float4 xx = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
             float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];

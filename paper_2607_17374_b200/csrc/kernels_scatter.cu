@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
                 const float2 tm = a.att_tm[sj];
                 const float e = a.att_s[sj] + tm.x;
                 ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
-                s = a.att_z[sj];
+                s = (float)a.att_z[sj];
               }
               if (!a.self_bias) s = 0.f;          // aggregate-first: the bias is added after the transform
 #pragma unroll
@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(256) scatter_kernel(ChunkArgs a) {
                     const float2 tm = a.att_tm[at];
                     const float e = a.att_s[at] + tm.x;
                     ps = __expf((e > 0.f ? e : a.leaky * e) - tm.y);
-                    s = a.self_bias ? a.att_z[at] : 0.f;
+                    s = a.self_bias ? (float)a.att_z[at] : 0.f;
                   }
                   float4 x = reinterpret_cast<const float4*>(p)[c4 + k * LPE];
                   float4 b = reinterpret_cast<const float4*>(a.bias)[c4 + k * LPE];

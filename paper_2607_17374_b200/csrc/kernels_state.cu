@@ -884,7 +884,7 @@ __global__ void finalise_kernel(ChunkArgs a) {
         } else if (a.mode == TAURUS_GCN_SYM) {
           scale = (float)(1.0 / sqrt((double)a.din[v] + 1.0));
         } else if (a.mode == TAURUS_GAT) {
-          scale = 1.0f / a.att_z[v];   // softmax normaliser
+          scale = (float)(1.0 / a.att_z[v]);   // softmax normaliser
         }                              // GIN: plain sum
         a.state[v] = TAURUS_COMPLETED;
         if (!a.dense_direct) a.grad_ids[base + mine] = v;
@@ -911,7 +911,7 @@ __global__ void finalise_kernel(ChunkArgs a) {
           if (k >= vec) continue;
           float4 y = x[q];
           float sk = sj;
-          if (a.mode == TAURUS_GAT && a.heads > 1) sk = 1.0f / a.att_z[(size_t)vj * a.heads + k / a.head_vec];   // normaliser of the column's head
+          if (a.mode == TAURUS_GAT && a.heads > 1) sk = (float)(1.0 / a.att_z[(size_t)vj * a.heads + k / a.head_vec]);   // normaliser of the column's head
           y.x *= sk; y.y *= sk; y.z *= sk; y.w *= sk;
           if (a.act) { y.x = fmaxf(y.x, 0.f); y.y = fmaxf(y.y, 0.f); y.z = fmaxf(y.z, 0.f); y.w = fmaxf(y.w, 0.f); }
           const int c0 = k << 2;

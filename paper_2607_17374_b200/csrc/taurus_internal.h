@@ -136,7 +136,7 @@ struct ChunkArgs {
   // GAT: per-vertex scalars from which every attention coefficient is recomputed
   const float* att_s;       // [V] att_src . h'_u
   const float2* att_tm;     // [V] (att_dst . h'_v, maximum score of v's neighbourhood)
-  const float* att_z;       // [V] softmax normaliser
+  const double* att_z;      // [V x heads] softmax normaliser (summed in double: a hub's sum has thousands of terms of very different size)
   float leaky;              // LeakyReLU slope
   int32_t heads;            // GAT: attention heads (the per-vertex scalars are [V x heads])
   int32_t head_vec;         // GAT: float4 per head (d_head / 4)
@@ -211,7 +211,7 @@ struct taurus_ctx {
   float* d_att_max = nullptr;   // [V] running maximum of att_src . h'_u over the neighbourhood
   float2* d_att_tm = nullptr;   // [V] (t, maximum score)
   float* d_att_w[TAURUS_MAX_LAYERS] = {nullptr};   // per layer: W att_src then W att_dst, dims[l] floats each (scores without the transformed rows)
-  float* d_att_z = nullptr;     // [V] normaliser
+  double* d_att_z = nullptr;    // [V x heads] normaliser
   long long gat_next_src = 0;   // next source taurus_gat_project_chunk expects
   bool gat_ready = false;       // taurus_gat_attention has run for this layer
   // aggregate-first layers

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 import taurus_gen as tg
-from gpu_harness import check_accounting, row_error, run_library, run_oracle
+from gpu_harness import check_accounting, forward_error, layer_on_input, row_error, run_library, run_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +55,30 @@ def test_gat_dense_output_mode_simt_projection():
     w = replace(w, mode=tg.GAT, dims=(100, 256, 47), fanout=(0, 0))
     _check(w, dense_output=True)
     _check(w, flags=2)                       # FFMA projection
+
+
+@pytest.mark.parametrize("flags", [0, 4])      # grouped scatter; CSR-order scatter
+def test_gat_destination_with_thousands_of_in_edges(flags):
+    """The softmax normaliser of a destination with thousands of in-edges sums positive terms that differ by many orders
+    of magnitude; added one by one in fp32 the small ones are lost (2e-4 of the sum at 8 000 in-edges, every output column
+    of the row too large by as much).  The library sums it in double precision: the hub's row stays at rounding level."""
+    w = tg.scaled(tg.WORKLOADS["stress"], 4_700, chunk=2048)
+    w = replace(w, mode=tg.GAT, dims=(33, 4), fanout=(0,), pool_slots=5_000, hub_count=1, gemm_mode=tg.GEMM_FP32, leaky_slope=0.0)
+    g = tg.make_graph(w)
+    hub = int(np.argmax(g.in_degree))
+    assert g.in_degree[hub] > 4000
+    model = tg.make_model(w, bias_scale=0.3)
+    model.att_src = [(a * 3).astype(np.float32) for a in model.att_src]
+    model.att_dst = [(a * 3).astype(np.float32) for a in model.att_dst]
+    x0 = tg.features(w.seed, 0, 0, g.V, w.dims[0])
+    lib = run_library(w, g, model, x0, flags=flags)
+    orc = run_oracle(w, g, model, x0)
+    ref, mag = layer_on_input(w, model, orc, 0, x0)
+    err = forward_error(lib["outs"][0], ref, mag)
+    hub_err = forward_error(lib["outs"][0][hub:hub + 1], ref[hub:hub + 1], mag[hub:hub + 1])
+    print("in-degree %d: forward error of the hub's row %.3e, of the layer %.3e" % (g.in_degree[hub], hub_err, err))
+    # the CSR-order kernels add the hub's 8 000 weighted rows one by one in fp32 (2e-5 here); the grouped order pre-sums them
+    assert err <= (TOL if flags else 5e-6), err
 
 
 def test_gat_several_heads_in_one_context():
