@@ -13,10 +13,13 @@ from gpu_harness import check_accounting, forward_error, layer_on_input, row_err
 pytestmark = pytest.mark.gpu
 
 
+_SCALE = int(os.environ.get("TAURUS_FUZZ_SCALE", "1"))      # multiplies the vertex counts drawn (400 .. 6 000)
+
+
 def random_config(seed):
     rng = np.random.default_rng(1000 + seed)
     base = ["tiny", "mid", "large", "stress"][int(rng.integers(0, 4))]
-    V = int(rng.integers(400, 6000))
+    V = int(rng.integers(400, 6000)) * _SCALE
     chunk = int(rng.choice([64, 100, 128, 257, 512, 1000, 2048]))
     w = tg.scaled(tg.WORKLOADS[base], V, chunk=chunk)
     L = int(rng.integers(1, 4))
