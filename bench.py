@@ -47,7 +47,7 @@ METRIC = "edges/sec per GNN layer (GTEPS)"
 # first 16 hex digits); when the source has changed since the capture the bench prints traffic = null instead of a
 # stale number.
 SCATTER_TRAFFIC_OVER_ALGORITHMIC = 1.257
-SCATTER_CAPTURE_SOURCE = "f25b718e2641c63c"
+SCATTER_CAPTURE_SOURCE = "85d27983976ae3e5"
 
 
 def source_digest(name: str) -> str:
