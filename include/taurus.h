@@ -191,6 +191,11 @@ int taurus_layer_begin(taurus_ctx* ctx, int32_t layer, void* cuda_stream);
  * valid and unchanged until that work has run (synchronise the stream, or drain).  Returns
  * TAURUS_ERR_DRAIN_FULL, before changing any state, when the vertices this chunk completes might not
  * fit the graduation buffer: drain and push the same chunk again.
+ * Where rows can be evicted (pool_slots < V - hub_count) the chunk's evicted and reloaded rows cross the host link on
+ * a stream of the library's own, beside the chunk's scatter and the next chunk's classification and victim
+ * selection; the chunk's finished rows are then finalised by the NEXT call on the context that needs them (the next
+ * push, a drain, taurus_layer_end, taurus_get_*): synchronising `cuda_stream` after a push does not by itself make that
+ * chunk's rows appear, a drain does.
  */
 int taurus_push_chunk(taurus_ctx* ctx, int64_t src_begin, int64_t src_end, const float* features, void* cuda_stream);
 
