@@ -70,8 +70,11 @@ def test_full_config(name):
             pytest.skip(reason)
 
         budget = float(os.environ.get("TAURUS_SUITE_BUDGET_S", "1100"))
-        import conftest
-        used = time.time() - conftest.SESSION_START
+        try:
+            import conftest
+            used = time.time() - conftest.SESSION_START
+        except (ImportError, AttributeError):      # another import mode: no session clock, no guard
+            used = 0.0
         if budget > 0 and used + 1.25 * EXPECT_S[base] > budget:
             reason = "%s at full size takes about %d s; the session has used %.0f s of its %d s" % (base, EXPECT_S[base], used, budget)
             print(reason)
